@@ -1,0 +1,227 @@
+"""Seeded synthetic inputs for the LQ-LoRA linear hot path.
+
+This module only *draws data*: weight-like matrices, low-rank factors, activations and
+per-matrix configuration tuples.  It holds none of the method's arithmetic (no codebook,
+no quantization, no dequantization, no layer product) and is the one module that both the
+CPU oracle's tests and the CUDA path's tests/bench import, so that both sides see the very
+same host buffers.
+
+All randomness comes from numpy's counter-based Philox generator keyed by an explicit
+seed; nothing depends on global state.  The seed rule is ``1000 * config + matrix_index``
+(config 1..5 as in the workload list below).
+
+Workloads (the real LLaMA-2 / RoBERTa weights are not available, so these seeded
+matrices of the real layer shapes stand in for them; weights of trained models are
+approximately Gaussian, Sec. 2.2 of the paper):
+
+  C1  1024x1024, N(0, 0.02^2), NF3/64/256, rank 64, X 512x1024
+  C2  4096x4096, planted rank-64 component + N(0, 0.02^2) noise, NF3/64/256,
+      M in {1, 16, 2048}; the matrix that is encoded is the residual W - L1 L2
+  C3  11008x4096 (gate, up) and 4096x11008 (down), Student-t(5) scaled to std 0.02,
+      NF4/64/256, M = 4096
+  C4  LLaMA-2-70B layer shapes, N(0, 0.02^2) with 0.1% entries x10, per-matrix mixed
+      configurations averaging about 2.75 bits, M in {1, 2048}
+  C5  8192x8192 N(0, 0.02^2), sweep of b0 x B0
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, List, Tuple
+
+import numpy as np
+
+RANK = 64
+
+
+@dataclass(frozen=True)
+class QuantConfig:
+    """The paper's configuration tuple c = (b0, b1, b2, B0, B1) (Sec. 3.2)."""
+
+    b0: int = 3
+    B0: int = 64
+    b1: int = 8
+    B1: int = 256
+    b2: int = 32
+
+    def as_tuple(self) -> Tuple[int, int, int, int, int]:
+        return (self.b0, self.B0, self.b1, self.B1, self.b2)
+
+
+def rng(seed: int) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=int(seed)))
+
+
+# ---------------------------------------------------------------------------------------
+# bf16 helpers for *inputs* (activations and low-rank factors are handed to both sides as
+# bf16 bit patterns; the value they carry is whatever these 16 bits decode to).
+# ---------------------------------------------------------------------------------------
+def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    """Round float32 to bfloat16 (nearest, ties to even); returns uint16 bit patterns."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    u = a.view(np.uint32).astype(np.uint64)
+    lsb = (u >> 16) & 1
+    u = u + 0x7FFF + lsb
+    return (u >> 16).astype(np.uint16)
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    b = np.ascontiguousarray(b, dtype=np.uint16)
+    return (b.astype(np.uint32) << 16).view(np.float32)
+
+
+# ---------------------------------------------------------------------------------------
+# matrices
+# ---------------------------------------------------------------------------------------
+def gaussian(seed: int, shape, std: float) -> np.ndarray:
+    g = rng(seed)
+    a = g.standard_normal(shape, dtype=np.float32)
+    a *= np.float32(std)
+    return a
+
+
+def student_t(seed: int, shape, nu: float, std: float) -> np.ndarray:
+    """Student-t(nu) entries rescaled so that the standard deviation is `std`."""
+    g = rng(seed)
+    z = g.standard_normal(shape, dtype=np.float32)
+    chi = g.chisquare(nu, size=shape).astype(np.float32)
+    t = z / np.sqrt(chi / np.float32(nu))
+    t *= np.float32(std / np.sqrt(nu / (nu - 2.0)))
+    return t.astype(np.float32)
+
+
+def gaussian_outliers(seed: int, shape, std: float, p: float, factor: float) -> np.ndarray:
+    g = rng(seed)
+    a = g.standard_normal(shape, dtype=np.float32)
+    a *= np.float32(std)
+    mask = g.random(shape, dtype=np.float32) < np.float32(p)
+    a[mask] *= np.float32(factor)
+    return a
+
+
+def lowrank_factors(seed: int, n: int, k: int, r: int = RANK, std: float = 0.01):
+    """L1 [n, r] and L2 [r, k] as bf16 bit patterns."""
+    g = rng(seed)
+    l1 = g.standard_normal((n, r), dtype=np.float32) * np.float32(std)
+    l2 = g.standard_normal((r, k), dtype=np.float32) * np.float32(std)
+    return f32_to_bf16_bits(l1), f32_to_bf16_bits(l2)
+
+
+def activations(seed: int, m: int, k: int, std: float = 1.0) -> np.ndarray:
+    """[m, k] activations (or output gradients) as bf16 bit patterns."""
+    g = rng(seed)
+    x = g.standard_normal((m, k), dtype=np.float32) * np.float32(std)
+    return f32_to_bf16_bits(x)
+
+
+def planted_lowrank_residual(seed: int, n: int, k: int, r: int = RANK,
+                             factor_std: float = 0.05, noise_std: float = 0.02):
+    """C2: W = L1 L2 + E with known factors; returns (R, L1_bits, L2_bits), R = W - L1 L2.
+
+    The factors are rounded to bf16 first and the product is formed from those rounded
+    values, so R is the residual with respect to exactly the factors the layer will use.
+    """
+    l1b, l2b = lowrank_factors(seed, n, k, r, std=factor_std)
+    l1 = bf16_bits_to_f32(l1b).astype(np.float64)
+    l2 = bf16_bits_to_f32(l2b).astype(np.float64)
+    p = (l1 @ l2).astype(np.float32)
+    e = gaussian(seed + 500, (n, k), noise_std)
+    w = p + e
+    return (w - p).astype(np.float32), l1b, l2b
+
+
+# ---------------------------------------------------------------------------------------
+# workload tables
+# ---------------------------------------------------------------------------------------
+@dataclass(frozen=True)
+class MatrixSpec:
+    name: str
+    N: int            # out_features
+    K: int            # in_features
+    cfg: QuantConfig
+    seed: int
+    kind: str         # gaussian | planted | student_t | outliers
+
+
+def storage_bits_formula(c: QuantConfig) -> float:
+    # only used to steer the C4 draw toward its bit budget; the tested implementation of
+    # the storage formula lives in the oracle and in the library.
+    return c.b0 + c.b1 / c.B0 + c.b2 / (c.B0 * c.B1)
+
+
+def config_c4_draw(seed: int = 4000) -> List[MatrixSpec]:
+    """LLaMA-2-70B layer: per-matrix configurations drawn from
+    b0 in {2,3,4} x B0 in {16,32,64,128} x B1 in {64,256} by seeded rejection sampling
+    until the parameter-weighted average storage lies in [2.70, 2.80] bits."""
+    shapes = [("q", 8192, 8192), ("k", 1024, 8192), ("v", 1024, 8192), ("o", 8192, 8192),
+              ("gate", 28672, 8192), ("up", 28672, 8192), ("down", 8192, 28672)]
+    g = rng(seed)
+    total = float(sum(n * k for _, n, k in shapes))
+    while True:
+        cfgs = [QuantConfig(b0=int(g.choice([2, 3, 4])), B0=int(g.choice([16, 32, 64, 128])),
+                            b1=8, B1=int(g.choice([64, 256])), b2=32) for _ in shapes]
+        avg = sum(storage_bits_formula(c) * n * k for c, (_, n, k) in zip(cfgs, shapes)) / total
+        if 2.70 <= avg <= 2.80:
+            break
+    return [MatrixSpec(nm, n, k, c, 4000 + i, "outliers")
+            for i, ((nm, n, k), c) in enumerate(zip(shapes, cfgs))]
+
+
+def workload(config: int) -> Dict:
+    """Matrix list and token counts of one of the five workloads."""
+    nf3 = QuantConfig(3, 64, 8, 256, 32)
+    nf4 = QuantConfig(4, 64, 8, 256, 32)
+    if config == 1:
+        return dict(matrices=[MatrixSpec("attn_proj", 1024, 1024, nf3, 1000, "gaussian")],
+                    Ms=[512], passes=("fwd",))
+    if config == 2:
+        return dict(matrices=[MatrixSpec("attn_proj", 4096, 4096, nf3, 2000, "planted")],
+                    Ms=[1, 16, 2048], passes=("fwd", "bwd"))
+    if config == 3:
+        return dict(matrices=[MatrixSpec("gate", 11008, 4096, nf4, 3000, "student_t"),
+                              MatrixSpec("up", 11008, 4096, nf4, 3001, "student_t"),
+                              MatrixSpec("down", 4096, 11008, nf4, 3002, "student_t")],
+                    Ms=[4096], passes=("fwd", "bwd"))
+    if config == 4:
+        return dict(matrices=config_c4_draw(), Ms=[1, 2048], passes=("fwd", "bwd"))
+    if config == 5:
+        mats = [MatrixSpec(f"b{b0}_B{B0}", 8192, 8192, QuantConfig(b0, B0, 8, 256, 32), 5000, "gaussian")
+                for b0 in (2, 3, 4, 8) for B0 in (16, 32, 64, 128, 256)]
+        return dict(matrices=mats, Ms=[1, 16, 128, 2048, 8192], passes=("fwd", "bwd", "encode"))
+    raise ValueError(f"unknown workload {config}")
+
+
+def make_matrix(spec: MatrixSpec):
+    """Returns (A, L1_bits, L2_bits): the fp32 matrix to encode and the bf16 factors."""
+    n, k = spec.N, spec.K
+    if spec.kind == "planted":
+        return planted_lowrank_residual(spec.seed, n, k)
+    if spec.kind == "gaussian":
+        a = gaussian(spec.seed, (n, k), 0.02)
+    elif spec.kind == "student_t":
+        a = student_t(spec.seed, (n, k), 5.0, 0.02)
+    elif spec.kind == "outliers":
+        a = gaussian_outliers(spec.seed, (n, k), 0.02, 0.001, 10.0)
+    else:
+        raise ValueError(spec.kind)
+    l1b, l2b = lowrank_factors(spec.seed + 700, n, k, RANK, 0.01)
+    return a, l1b, l2b
+
+
+def sample_rows(seed: int, m: int, count: int = 64, tile: int = 128) -> np.ndarray:
+    """Row indices for sampled parity at large M: first/last row, both sides of every
+    multiple of `tile` (while the budget lasts), the rest drawn at random."""
+    if m <= count:
+        return np.arange(m, dtype=np.int64)
+    chosen = [0, m - 1]
+    t = tile
+    while t < m and len(chosen) + 2 <= count // 2:
+        chosen += [t - 1, t]
+        t += tile
+    g = rng(seed)
+    rest = g.permutation(m)
+    for i in rest:
+        if len(chosen) >= count:
+            break
+        if int(i) not in chosen:
+            chosen.append(int(i))
+    return np.array(sorted(set(chosen)), dtype=np.int64)
