@@ -1,0 +1,177 @@
+/*
+ * lqlora.h -- C ABI of the B200 (sm_100a) LQ-LoRA linear-layer library.
+ *
+ * The layer (Sec. 2.1 and Sec. 3.1 of arXiv 2311.12023) keeps a pretrained matrix as a fixed
+ * quantized matrix Q plus a trainable rank-r product L1 L2 and computes X (Q + L1 L2).  This
+ * library stores matrices the way nn.Linear does, i.e. transposed with respect to the paper:
+ *
+ *     Q, W : [N = out_features, K = in_features]  row major
+ *     L1   : [N, r] bf16        L2 : [r, K] bf16
+ *     X    : [M, K] bf16        Y, dY : [M, N] bf16        dX : [M, K] bf16
+ *
+ *     forward          Y  = X deq(Q)^T + (X L2^T) L1^T
+ *     input gradient   dX = dY deq(Q)  + (dY L1) L2
+ *
+ * Q is produced by the NormalFloat double quantization of Sec. 2.2 / Sec. 3.2 with the
+ * configuration tuple c = (b0, b1, b2, B0, B1).
+ *
+ * General rules
+ *   - Every pointer named *_dev or documented as "device" is a CUDA device pointer owned by the
+ *     caller; the library never allocates or frees device memory and keeps no state besides
+ *     immutable code-book tables in constant memory (uploaded on first use per device).
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it and return without
+ *     synchronizing, unless stated otherwise.
+ *   - Every function returns an lqlora_status (0 = success, negative = error).  Arguments are
+ *     validated on the host before anything is launched; on error nothing has been enqueued.
+ *     No function throws, aborts or traps.
+ *   - Inputs must be finite.
+ *   - There is no CPU fallback: without a CUDA device every compute entry point returns
+ *     LQLORA_ERR_CUDA.
+ */
+#ifndef LQLORA_H_
+#define LQLORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LQLORA_OK = 0,
+    LQLORA_ERR_INVALID_CONFIG = -1,   /* b0 not in {2,3,4,8}; B0 not a power of two in [16,256];
+                                         B1 not a power of two in [16,4096]; b1 != 8; b2 != 32     */
+    LQLORA_ERR_INVALID_SHAPE = -2,    /* N, K, M <= 0; K % 64 != 0; K % B0 != 0; r % 16 != 0; r > 128 */
+    LQLORA_ERR_NULL_POINTER = -3,
+    LQLORA_ERR_MISALIGNED = -4,       /* a device pointer is not 16-byte aligned                    */
+    LQLORA_ERR_WORKSPACE_TOO_SMALL = -5,
+    LQLORA_ERR_CUDA = -6,             /* a CUDA runtime / driver call failed (no device, launch)   */
+    LQLORA_ERR_TIMEOUT = -7,          /* a bounded device-side wait expired (see lqlora_workspace_status) */
+    LQLORA_ERR_UNSUPPORTED = -8       /* valid arguments that this build has no kernel for          */
+} lqlora_status;
+
+/* Configuration tuple c = (b0, b1, b2, B0, B1) of Sec. 3.2. */
+typedef struct {
+    int b0;   /* bits of a NormalFloat code: 2, 3, 4 or 8                         */
+    int B0;   /* weights per first-level block (along K): 16, 32, 64, 128, 256    */
+    int b1;   /* bits of a quantized block scale: 8                               */
+    int B1;   /* blocks per second-level group (flattened row-major block order)  */
+    int b2;   /* bits of a second-level scale: 32 (fp32; cast(v, fp32) = v)       */
+} lqlora_config;
+
+/*
+ * A quantized matrix.  All three arrays are device memory owned by the caller, each 16-byte
+ * aligned, of the sizes lqlora_packed_sizes reports.
+ *
+ *   scale_codes  uint8 [N * K / B0]      s^_i, flattened row-major block order (block i covers
+ *                                        elements [i*B0, (i+1)*B0) of the row-major matrix)
+ *   scale2       fp32  [ceil(nblk / B1)] v_g = absmax of the block scales of group g
+ *   codes        packed b0-bit codes, exactly b0 bits per weight when N % 128 == 0 (rows are
+ *                padded to a multiple of 128 otherwise).  Layout ("tile-interleaved bitstream"):
+ *                  - the matrix is cut into tiles of 128 rows x 64 columns, stored one after the
+ *                    other in row-major tile order; a tile takes 1024*b0 bytes;
+ *                  - a tile is four slabs of 32 rows (rows 32q .. 32q+31, q = 0..3), 256*b0 bytes each;
+ *                  - inside a slab, the 64 columns form two groups g = 0, 1 of 32 columns; the 32
+ *                    codes of (row, g) are a little-endian bit string of 32*b0 bits (code j at bits
+ *                    [b0*j, b0*j + b0)), cut into b0 32-bit words w = 0..b0-1;
+ *                  - word w of (row, g) is the 32-bit word number (g*b0 + w)*32 + (row % 32) of the slab.
+ *                Consecutive 32-bit words of a slab therefore belong to consecutive rows, so a
+ *                warp reads or writes a slab with fully coalesced accesses and conflict-free
+ *                shared-memory accesses.  Use lqlora_unpack to obtain one code per byte.
+ */
+typedef struct {
+    void* codes;
+    uint8_t* scale_codes;
+    float* scale2;
+    int64_t N, K;
+    lqlora_config cfg;
+} lqlora_qmatrix;
+
+/* Storage cost in bits per parameter, Eq. (2) of Sec. 3.2: b0 + b1/B0 + b2/(B0*B1).  Pure host
+ * arithmetic.  Returns a negative value if cfg is NULL or invalid. */
+double lqlora_storage_bits_per_param(const lqlora_config* cfg);
+
+/* Sizes in bytes of the three arrays of an [N, K] quantized matrix and of the scratch that
+ * lqlora_encode needs.  Any output pointer may be NULL.  Host only.
+ * When N % 128 == 0 the three sizes add up to exactly N*K*Eq.(2)/8 bytes (scale2 rounded up to
+ * one fp32 per started group). */
+int lqlora_packed_sizes(int64_t N, int64_t K, const lqlora_config* cfg, size_t* code_bytes,
+                        size_t* scale_bytes, size_t* scale2_bytes, size_t* encode_workspace_bytes);
+
+/* The NormalFloat code book of Sec. 2.2 for b0 bits: 2^b0 ascending fp32 values in [-1, 1]
+ * (2^(b0-1) evenly spaced probabilities on [delta, 1/2], 2^(b0-1)+1 on [1/2, 1-delta],
+ * delta = (1/30 + 1/32)/2, Gaussian quantiles divided by the largest).  out_host: host memory,
+ * 2^b0 floats.  Host only. */
+int lqlora_nf_codebook(int b0, float* out_host);
+
+/*
+ * Quantize(A, c) of Sec. 3.2 (Quantize-NF, then Quantize-INT of the block absmax values, then
+ * cast to fp32) for A = W_dev, fp32 [N, K] row major, device memory.
+ *   s_i  = max |u_j| over block i (B0 consecutive elements along K);
+ *   c_j  = argmin_k |q~_k - fl32(u_j / s_i)|, the lower index on a tie; the code of 0 if s_i = 0;
+ *   v_g  = max s_i over group g (B1 consecutive blocks; the last group may be short);
+ *   s^_i = clamp(round_half_even(fl32(s_i / fl32(v_g / 127))), 0, 127); 0 if v_g = 0.
+ * out->N, K, cfg must be filled in and its three arrays allocated by the caller.
+ * workspace_dev: device scratch of at least encode_workspace_bytes (block absmax values in fp32).
+ * Errors: INVALID_CONFIG, INVALID_SHAPE, NULL_POINTER, MISALIGNED, WORKSPACE_TOO_SMALL, CUDA.
+ */
+int lqlora_encode(const float* W_dev, lqlora_qmatrix* out, void* workspace_dev,
+                  size_t workspace_bytes, void* stream);
+
+/* Parity / debug exports (not on the hot path).
+ * lqlora_unpack: one code per byte, codes_dev uint8 [N, K] row major (device).
+ * lqlora_dequant: "dequantization simply reverses this process" (Sec. 3.2):
+ *   s~_i = fl32(float(s^_i) * fl32(v_g / 127));  w~_j = fl32(q~[c_j] * s~_i)  -> deq32_dev fp32 [N, K];
+ *   deq16_dev = w~ rounded to bf16, nearest-even, [N, K] (the cast for bf16 training, App. A).
+ *   Either output may be NULL. */
+int lqlora_unpack(const lqlora_qmatrix* q, uint8_t* codes_dev, void* stream);
+int lqlora_dequant(const lqlora_qmatrix* q, float* deq32_dev, void* deq16_dev, void* stream);
+
+/* Bytes of device scratch lqlora_linear_fwd / lqlora_linear_bwd_input need for M rows.
+ * Returns 0 (and sets *bytes) or an error.  Host only. */
+int lqlora_linear_workspace_bytes(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M,
+                                  size_t* bytes);
+
+/*
+ * Forward of the layer, X (Q + L1 L2) of Sec. 2.1 / Sec. 3.1 in nn.Linear orientation:
+ *     Y[M, N] = X[M, K] deq16(Q)^T + bf16(X L2^T) L1^T
+ * bf16 operands, fp32 accumulation, bf16 output; Q is dequantized on the fly and never written
+ * to global memory.  r = 0 (L1 = L2 = NULL) computes the quantized part alone.
+ * All of Q's arrays, L1, L2, X, Y, workspace_dev: device, 16-byte aligned.
+ * The first 256 bytes of the workspace hold a status word (see lqlora_workspace_status); the rest
+ * is scratch for the rank-r intermediate and split-K partial sums.  Concurrent calls must use
+ * different workspaces.
+ * Errors: as lqlora_encode, plus UNSUPPORTED.
+ */
+int lqlora_linear_fwd(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r,
+                      const void* X_dev, int64_t M, void* Y_dev, void* workspace_dev,
+                      size_t workspace_bytes, void* stream);
+
+/*
+ * Input gradient of the same layer (only L1, L2 are trained, Q gets no gradient; Sec. 1, Sec. 2.1):
+ *     dX[M, K] = dY[M, N] deq16(Q) + bf16(dY L1) L2
+ * Same conventions as lqlora_linear_fwd.
+ */
+int lqlora_linear_bwd_input(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r,
+                            const void* dY_dev, int64_t M, void* dX_dev, void* workspace_dev,
+                            size_t workspace_bytes, void* stream);
+
+/* Synchronizes `stream`, reads the status word at the start of a linear workspace and returns it
+ * as an lqlora_status: LQLORA_OK, or LQLORA_ERR_TIMEOUT if a kernel gave up on a bounded wait
+ * (its output is then undefined).  The word is cleared by every linear call before it launches. */
+int lqlora_workspace_status(const void* workspace_dev, void* stream);
+
+/* Which kernel family the last dispatch of lqlora_linear_* would use for M rows:
+ * 0 = weight-streaming small-M kernel, 1 = tcgen05 tensor-core kernel.  Host only. */
+int lqlora_linear_path(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, int backward);
+
+/* Number of kernel launches the library has enqueued since it was loaded (for launch accounting). */
+int64_t lqlora_launch_count(void);
+
+const char* lqlora_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LQLORA_H_ */

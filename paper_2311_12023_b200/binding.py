@@ -1,0 +1,237 @@
+"""Thin Python binding of the C ABI declared in ``include/lqlora.h``.
+
+Argument marshalling only: every step of the path runs in the CUDA library.  torch is
+used for device memory and streams.  There is no fallback: if ``liblqlora.so`` is
+missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional, Tuple
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblqlora.so")
+
+EXPORTS = [
+    "lqlora_storage_bits_per_param", "lqlora_packed_sizes", "lqlora_nf_codebook", "lqlora_encode",
+    "lqlora_unpack", "lqlora_dequant", "lqlora_linear_workspace_bytes", "lqlora_linear_fwd",
+    "lqlora_linear_bwd_input", "lqlora_workspace_status", "lqlora_linear_path", "lqlora_launch_count",
+    "lqlora_status_string",
+]
+
+
+class LqloraError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+class CConfig(ctypes.Structure):
+    _fields_ = [("b0", ctypes.c_int), ("B0", ctypes.c_int), ("b1", ctypes.c_int), ("B1", ctypes.c_int),
+                ("b2", ctypes.c_int)]
+
+
+class CQMatrix(ctypes.Structure):
+    _fields_ = [("codes", ctypes.c_void_p), ("scale_codes", ctypes.c_void_p), ("scale2", ctypes.c_void_p),
+                ("N", ctypes.c_int64), ("K", ctypes.c_int64), ("cfg", CConfig)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the compiled library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2311_12023_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+        L.lqlora_storage_bits_per_param.argtypes = [ctypes.POINTER(CConfig)]
+        L.lqlora_storage_bits_per_param.restype = ctypes.c_double
+        L.lqlora_packed_sizes.argtypes = [i64, i64, ctypes.POINTER(CConfig)] + [ctypes.POINTER(sz)] * 4
+        L.lqlora_nf_codebook.argtypes = [ci, vp]
+        L.lqlora_encode.argtypes = [vp, ctypes.POINTER(CQMatrix), vp, sz, vp]
+        L.lqlora_unpack.argtypes = [ctypes.POINTER(CQMatrix), vp, vp]
+        L.lqlora_dequant.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, vp]
+        L.lqlora_linear_workspace_bytes.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ctypes.POINTER(sz)]
+        L.lqlora_linear_fwd.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, sz, vp]
+        L.lqlora_linear_bwd_input.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, sz, vp]
+        L.lqlora_workspace_status.argtypes = [vp, vp]
+        L.lqlora_linear_path.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ci]
+        L.lqlora_launch_count.restype = i64
+        L.lqlora_status_string.argtypes = [ci]
+        L.lqlora_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().lqlora_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise LqloraError(status, where)
+
+
+def _cfg(cfg) -> CConfig:
+    """cfg: anything with b0, B0, b1, B1, b2 attributes (e.g. inputs.QuantConfig)."""
+    return CConfig(int(cfg.b0), int(cfg.B0), int(cfg.b1), int(cfg.B1), int(cfg.b2))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+# ----------------------------------------------------------------------------- host-only calls
+def storage_bits_per_param(cfg) -> float:
+    c = _cfg(cfg)
+    return float(lib().lqlora_storage_bits_per_param(ctypes.byref(c)))
+
+
+def packed_sizes(N: int, K: int, cfg) -> Tuple[int, int, int, int]:
+    """(code_bytes, scale_bytes, scale2_bytes, encode_workspace_bytes)."""
+    c = _cfg(cfg)
+    out = [ctypes.c_size_t(0) for _ in range(4)]
+    _check(lib().lqlora_packed_sizes(N, K, ctypes.byref(c), *[ctypes.byref(o) for o in out]), "lqlora_packed_sizes")
+    return tuple(int(o.value) for o in out)
+
+
+def nf_codebook(b0: int) -> np.ndarray:
+    out = np.zeros(1 << b0, dtype=np.float32)
+    _check(lib().lqlora_nf_codebook(b0, out.ctypes.data_as(ctypes.c_void_p)), "lqlora_nf_codebook")
+    return out
+
+
+def linear_workspace_bytes(N: int, K: int, cfg, r: int, M: int) -> int:
+    c = _cfg(cfg)
+    out = ctypes.c_size_t(0)
+    _check(lib().lqlora_linear_workspace_bytes(N, K, ctypes.byref(c), r, M, ctypes.byref(out)),
+           "lqlora_linear_workspace_bytes")
+    return int(out.value)
+
+
+def linear_path(N: int, K: int, cfg, r: int, M: int, backward: bool) -> int:
+    c = _cfg(cfg)
+    return int(lib().lqlora_linear_path(N, K, ctypes.byref(c), r, M, int(backward)))
+
+
+def launch_count() -> int:
+    return int(lib().lqlora_launch_count())
+
+
+# ----------------------------------------------------------------------------- device calls
+@dataclass
+class QMatrix:
+    """Device arrays of one quantized matrix (owned here, as torch tensors)."""
+    codes: torch.Tensor        # uint8 buffer holding the packed code words
+    scale_codes: torch.Tensor  # uint8 [nblk]
+    scale2: torch.Tensor       # float32 [ngrp]
+    N: int
+    K: int
+    cfg: object
+
+    def cstruct(self) -> CQMatrix:
+        return CQMatrix(self.codes.data_ptr(), self.scale_codes.data_ptr(), self.scale2.data_ptr(),
+                        self.N, self.K, _cfg(self.cfg))
+
+    @property
+    def packed_bytes(self) -> int:
+        return self.codes.numel() + self.scale_codes.numel() + 4 * self.scale2.numel()
+
+
+def alloc_qmatrix(N: int, K: int, cfg, device="cuda") -> QMatrix:
+    cb, sb, s2b, _ = packed_sizes(N, K, cfg)
+    return QMatrix(torch.empty(cb, dtype=torch.uint8, device=device),
+                   torch.empty(sb, dtype=torch.uint8, device=device),
+                   torch.empty(s2b // 4, dtype=torch.float32, device=device), N, K, cfg)
+
+
+def encode(W: torch.Tensor, cfg, out: Optional[QMatrix] = None, workspace: Optional[torch.Tensor] = None) -> QMatrix:
+    """lqlora_encode: W fp32 [N, K] on the device -> packed codes, scale codes, second-level scales."""
+    assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous() and W.dim() == 2
+    N, K = W.shape
+    q = out if out is not None else alloc_qmatrix(N, K, cfg, W.device)
+    ws_bytes = packed_sizes(N, K, cfg)[3]
+    if workspace is None:
+        workspace = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=W.device)
+    cs = q.cstruct()
+    _check(lib().lqlora_encode(W.data_ptr(), ctypes.byref(cs), workspace.data_ptr(), workspace.numel(), _stream()),
+           "lqlora_encode")
+    return q
+
+
+def unpack(q: QMatrix) -> torch.Tensor:
+    out = torch.empty((q.N, q.K), dtype=torch.uint8, device=q.codes.device)
+    cs = q.cstruct()
+    _check(lib().lqlora_unpack(ctypes.byref(cs), out.data_ptr(), _stream()), "lqlora_unpack")
+    return out
+
+
+def dequant(q: QMatrix, want32: bool = True, want16: bool = True):
+    dev = q.codes.device
+    d32 = torch.empty((q.N, q.K), dtype=torch.float32, device=dev) if want32 else None
+    d16 = torch.empty((q.N, q.K), dtype=torch.bfloat16, device=dev) if want16 else None
+    cs = q.cstruct()
+    _check(lib().lqlora_dequant(ctypes.byref(cs), _ptr(d32), _ptr(d16), _stream()), "lqlora_dequant")
+    return d32, d16
+
+
+def alloc_workspace(q: QMatrix, r: int, M: int) -> torch.Tensor:
+    return torch.empty(linear_workspace_bytes(q.N, q.K, q.cfg, r, M), dtype=torch.uint8, device=q.codes.device)
+
+
+def _linear(fn, name, q, L1, L2, A, out_cols, out, workspace):
+    assert A.is_cuda and A.dtype == torch.bfloat16 and A.is_contiguous() and A.dim() == 2
+    M = A.shape[0]
+    r = 0 if L1 is None else L1.shape[1]
+    if r:
+        assert L1.dtype == torch.bfloat16 and L2.dtype == torch.bfloat16 and L1.is_contiguous() and L2.is_contiguous()
+        assert tuple(L1.shape) == (q.N, r) and tuple(L2.shape) == (r, q.K)
+    if out is None:
+        out = torch.empty((M, out_cols), dtype=torch.bfloat16, device=A.device)
+    if workspace is None:
+        workspace = alloc_workspace(q, r, M)
+    cs = q.cstruct()
+    _check(fn(ctypes.byref(cs), _ptr(L1), _ptr(L2), r, A.data_ptr(), M, out.data_ptr(), workspace.data_ptr(),
+              workspace.numel(), _stream()), name)
+    return out
+
+
+def linear_fwd(q: QMatrix, L1, L2, X: torch.Tensor, out=None, workspace=None) -> torch.Tensor:
+    """lqlora_linear_fwd: Y = X deq(Q)^T + (X L2^T) L1^T, bf16 [M, N]."""
+    assert X.shape[1] == q.K
+    return _linear(lib().lqlora_linear_fwd, "lqlora_linear_fwd", q, L1, L2, X, q.N, out, workspace)
+
+
+def linear_bwd_input(q: QMatrix, L1, L2, dY: torch.Tensor, out=None, workspace=None) -> torch.Tensor:
+    """lqlora_linear_bwd_input: dX = dY deq(Q) + (dY L1) L2, bf16 [M, K]."""
+    assert dY.shape[1] == q.N
+    return _linear(lib().lqlora_linear_bwd_input, "lqlora_linear_bwd_input", q, L1, L2, dY, q.K, out, workspace)
+
+
+def workspace_status(workspace: torch.Tensor) -> int:
+    return int(lib().lqlora_workspace_status(workspace.data_ptr(), _stream()))
+
+
+# ----------------------------------------------------------------------------- helpers for tests / bench
+def bf16_from_bits(bits: np.ndarray, device="cuda") -> torch.Tensor:
+    """uint16 bit patterns (host) -> bf16 tensor on the device, bit for bit."""
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(device)
+    return t.view(torch.bfloat16)
+
+
+def bits_from_bf16(t: torch.Tensor) -> np.ndarray:
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)

@@ -1,0 +1,193 @@
+// Quantize(A, c) of Sec. 3.2 on the GPU: block absmax, nearest NormalFloat code, bit packing,
+// 8-bit round-to-nearest quantization of the absmax values; plus the unpack / dequantize
+// exports used for parity checks.
+#pragma once
+
+#include "common.cuh"
+
+namespace lq {
+
+// ---------------------------------------------------------------------------------------
+// Nearest code by counting thresholds below x (thresholds ascending; a tie x == midpoint is
+// not "above", so it goes to the lower index).
+// ---------------------------------------------------------------------------------------
+template <int B>
+__device__ __forceinline__ uint32_t nearest_code(float x, const float* __restrict__ th_smem) {
+    if constexpr (B <= 4) {
+        uint32_t c = 0;
+#pragma unroll
+        for (int i = 0; i < (1 << B) - 1; ++i) c += (x > c_threshold[B == 2 ? 0 : B == 3 ? 1 : 2][i]) ? 1u : 0u;
+        return c;
+    } else {
+        uint32_t c = 0;
+#pragma unroll
+        for (int step = 128; step >= 1; step >>= 1)
+            if (x > th_smem[c + step - 1]) c += step;   // th_smem[255] = +inf, never exceeded
+        return c;
+    }
+}
+
+// One CTA: 32 rows x 256 columns.  Thread (row = tid % 32, grp = tid / 32) owns 32 consecutive
+// columns of one row: it finds the block absmax (with its neighbours through shared memory when
+// B0 > 32), the 32 codes, and writes the b0 words of its group to the packed slab.
+template <int B>
+__global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
+                                                           float* __restrict__ absmax, int N, int K, int B0, int logB0) {
+    __shared__ float red[8][33];
+    __shared__ float th8[256];
+    if constexpr (B == 8) {
+        th8[threadIdx.x] = c_threshold[3][threadIdx.x];
+    }
+    const int rl = threadIdx.x & 31, grp = threadIdx.x >> 5;
+    const int row = blockIdx.x * 32 + rl;
+    const int k0 = blockIdx.y * 256 + grp * 32;
+    const bool live = (k0 < K);
+    const bool real = live && (row < N);
+
+    float u[32];
+    if (real) {
+        const float4* src = reinterpret_cast<const float4*>(W + static_cast<size_t>(row) * K + k0);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float4 t = __ldg(src + i);
+            u[4 * i] = t.x; u[4 * i + 1] = t.y; u[4 * i + 2] = t.z; u[4 * i + 3] = t.w;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) u[i] = 0.0f;
+    }
+    // absmax of each 16-wide half
+    float m0 = 0.0f, m1 = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { m0 = fmaxf(m0, fabsf(u[i])); m1 = fmaxf(m1, fabsf(u[16 + i])); }
+    red[grp][rl] = fmaxf(m0, m1);
+    __syncthreads();
+
+    float s_lo, s_hi;   // block absmax for columns 0..15 and 16..31 of this thread's group
+    if (B0 == 16) { s_lo = m0; s_hi = m1; }
+    else if (B0 == 32) { s_lo = s_hi = fmaxf(m0, m1); }
+    else {
+        const int span = B0 >> 5, g0 = grp & ~(span - 1);
+        float m = 0.0f;
+        for (int i = 0; i < span; ++i) m = fmaxf(m, red[g0 + i][rl]);
+        s_lo = s_hi = m;
+    }
+    if (real) {
+        const int KB = K >> logB0;
+        if (B0 == 16) {
+            absmax[static_cast<size_t>(row) * KB + (k0 >> 4)] = s_lo;
+            absmax[static_cast<size_t>(row) * KB + (k0 >> 4) + 1] = s_hi;
+        } else if ((k0 & (B0 - 1)) == 0) {
+            absmax[static_cast<size_t>(row) * KB + (k0 >> logB0)] = s_lo;
+        }
+    }
+    if (!live) return;
+
+    constexpr uint32_t zero_code = (1u << (B - 1)) - 1u;
+    uint32_t words[B];
+#pragma unroll
+    for (int i = 0; i < B; ++i) words[i] = 0u;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const float s = (j < 16) ? s_lo : s_hi;
+        uint32_t c = zero_code;
+        if (s != 0.0f) c = nearest_code<B>(__fdiv_rn(u[j], s), th8);
+        const int p = B * j, wi = p >> 5, sh = p & 31;
+        words[wi] |= c << sh;
+        if (sh + B > 32) words[wi + 1] |= c >> (32 - sh);
+    }
+    uint32_t* dst = codes + slab_word_base(row, k0 >> 6, K >> 6, B);
+    const int g = (k0 >> 5) & 1;
+#pragma unroll
+    for (int w = 0; w < B; ++w) dst[slab_word_offset(row, g, w, B)] = words[w];
+}
+
+// One CTA per second-level group: v_g = max s_i, s^_i = clamp(rint(s_i / (v_g / 127)), 0, 127).
+__global__ void __launch_bounds__(256) encode_scales_kernel(const float* __restrict__ absmax, uint8_t* __restrict__ sc,
+                                                            float* __restrict__ v, long long nblk, int B1) {
+    __shared__ float red[8];
+    __shared__ float vmax;
+    const long long lo = static_cast<long long>(blockIdx.x) * B1;
+    const long long hi = (lo + B1 < nblk) ? lo + B1 : nblk;
+    float m = 0.0f;
+    for (long long i = lo + threadIdx.x; i < hi; i += blockDim.x) m = fmaxf(m, absmax[i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = red[0];
+        for (int i = 1; i < 8; ++i) t = fmaxf(t, red[i]);
+        vmax = t;
+        v[blockIdx.x] = t;
+    }
+    __syncthreads();
+    const float vg = vmax;
+    const float sigma = __fdiv_rn(vg, static_cast<float>(kScaleLevels));
+    for (long long i = lo + threadIdx.x; i < hi; i += blockDim.x) {
+        float c = 0.0f;
+        if (vg != 0.0f) {
+            c = rintf(__fdiv_rn(absmax[i], sigma));
+            c = fminf(fmaxf(c, 0.0f), static_cast<float>(kScaleLevels));
+        }
+        sc[i] = static_cast<uint8_t>(c);
+    }
+}
+
+// Thread per (row, 32-column group): unpack to one code per byte and / or dequantize.
+template <int B>
+__global__ void __launch_bounds__(256) export_kernel(QView q, uint8_t* __restrict__ codes_out, float* __restrict__ deq32,
+                                                     __nv_bfloat16* __restrict__ deq16) {
+    const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int groups_per_row = q.K >> 5;
+    // consecutive threads -> consecutive rows of one slab (coalesced packed reads)
+    const int rl = static_cast<int>(t & 31);
+    const long long rest = t >> 5;
+    const int grp = static_cast<int>(rest % groups_per_row);
+    const int row = static_cast<int>(rest / groups_per_row) * 32 + rl;
+    if (row >= q.N) return;
+    const int k0 = grp * 32;
+    const uint32_t* src = q.codes + slab_word_base(row, k0 >> 6, q.ktiles, B);
+    uint32_t w[B];
+#pragma unroll
+    for (int i = 0; i < B; ++i) w[i] = src[slab_word_offset(row, (k0 >> 5) & 1, i, B)];
+    const size_t out = static_cast<size_t>(row) * q.K + k0;
+    const float* cb = c_codebook[bits_index(B)];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const uint32_t c = extract_code<B>(w, j);
+        if (codes_out) codes_out[out + j] = static_cast<uint8_t>(c);
+        if (deq32 || deq16) {
+            const long long blk = static_cast<long long>(row) * q.KB + ((k0 + j) >> q.logB0);
+            const float st = block_scale(q.sc[blk], q.v[blk >> q.logB1]);
+            const float wv = __fmul_rn(cb[c], st);
+            if (deq32) deq32[out + j] = wv;
+            if (deq16) deq16[out + j] = __float2bfloat16_rn(wv);
+        }
+    }
+}
+
+template <int B>
+inline cudaError_t launch_encode(const float* W, const lqlora_qmatrix* out, float* absmax, cudaStream_t st) {
+    const int N = static_cast<int>(out->N), K = static_cast<int>(out->K);
+    const int Np = (N + kTileRows - 1) / kTileRows * kTileRows;
+    dim3 grid(Np / 32, (K + 255) / 256);
+    encode_codes_kernel<B><<<grid, 256, 0, st>>>(W, static_cast<uint32_t*>(out->codes), absmax, N, K, out->cfg.B0,
+                                                 ilog2(out->cfg.B0));
+    const long long nblk = static_cast<long long>(N) * K / out->cfg.B0;
+    const long long ngrp = (nblk + out->cfg.B1 - 1) / out->cfg.B1;
+    encode_scales_kernel<<<static_cast<unsigned>(ngrp), 256, 0, st>>>(absmax, out->scale_codes, out->scale2, nblk, out->cfg.B1);
+    count_launch(2);
+    return cudaGetLastError();
+}
+
+template <int B>
+inline cudaError_t launch_export(const QView& q, uint8_t* codes_out, float* deq32, void* deq16, cudaStream_t st) {
+    const long long total = static_cast<long long>((q.N + 31) / 32 * 32) * (q.K >> 5);
+    export_kernel<B><<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(q, codes_out, deq32,
+                                                                               static_cast<__nv_bfloat16*>(deq16));
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+}  // namespace lq

@@ -1,0 +1,108 @@
+// Shared declarations of the LQ-LoRA CUDA library: configuration checks, the packed-code
+// addressing rule, code-book tables and small device helpers.  Product code only; the CPU
+// oracle shares nothing with this file.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/lqlora.h"
+
+namespace lq {
+
+constexpr int kTileRows = 128;   // rows of a packed tile
+constexpr int kTileCols = 64;    // columns of a packed tile
+constexpr int kSlabRows = 32;    // rows of a slab (one warp's worth)
+constexpr int kScaleLevels = 127;  // 2^(b1-1) - 1 positive levels of the 8-bit RTN scale quantizer (Sec. 2.2)
+constexpr int kStatusBytes = 256;  // status word area at the start of a linear workspace
+
+// Index of a code width in the table arrays.
+__host__ __device__ inline int bits_index(int b0) { return b0 == 2 ? 0 : b0 == 3 ? 1 : b0 == 4 ? 2 : 3; }
+
+inline int ilog2(int x) { int l = 0; while ((1 << l) < x) ++l; return l; }
+inline bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+
+inline int check_config(const lqlora_config* c) {
+    if (!c) return LQLORA_ERR_NULL_POINTER;
+    if (!(c->b0 == 2 || c->b0 == 3 || c->b0 == 4 || c->b0 == 8)) return LQLORA_ERR_INVALID_CONFIG;
+    if (!is_pow2(c->B0) || c->B0 < 16 || c->B0 > 256) return LQLORA_ERR_INVALID_CONFIG;
+    if (!is_pow2(c->B1) || c->B1 < 16 || c->B1 > 4096) return LQLORA_ERR_INVALID_CONFIG;
+    if (c->b1 != 8 || c->b2 != 32) return LQLORA_ERR_INVALID_CONFIG;
+    return LQLORA_OK;
+}
+
+inline int check_shape(int64_t N, int64_t K, const lqlora_config* c) {
+    if (N <= 0 || K <= 0) return LQLORA_ERR_INVALID_SHAPE;
+    if (K % kTileCols != 0 || K % c->B0 != 0) return LQLORA_ERR_INVALID_SHAPE;
+    if (N > (int64_t(1) << 30) || K > (int64_t(1) << 30)) return LQLORA_ERR_INVALID_SHAPE;
+    return LQLORA_OK;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Device-side view of a quantized matrix.
+struct QView {
+    const uint32_t* codes;
+    const uint8_t* sc;     // s^ [N * KB]
+    const float* v;        // v  [ngrp]
+    int N, K;
+    int b0, B0, B1;
+    int logB0, logB1;
+    int KB;                // blocks per row  = K / B0
+    int ktiles;            // 64-column tiles per row = K / 64
+    int ntiles;            // 128-row tiles = ceil(N / 128)
+};
+
+inline QView make_view(const lqlora_qmatrix* q) {
+    QView v;
+    v.codes = static_cast<const uint32_t*>(q->codes);
+    v.sc = q->scale_codes;
+    v.v = q->scale2;
+    v.N = static_cast<int>(q->N);
+    v.K = static_cast<int>(q->K);
+    v.b0 = q->cfg.b0; v.B0 = q->cfg.B0; v.B1 = q->cfg.B1;
+    v.logB0 = ilog2(v.B0); v.logB1 = ilog2(v.B1);
+    v.KB = v.K / v.B0;
+    v.ktiles = v.K / kTileCols;
+    v.ntiles = (v.N + kTileRows - 1) / kTileRows;
+    return v;
+}
+
+// First 32-bit word of the slab holding (row, 64-column tile kt): tiles in row-major tile order,
+// four slabs of 32 rows per tile, 64*b0 words per slab.
+__host__ __device__ inline size_t slab_word_base(int row, int kt, int ktiles, int b0) {
+    const size_t tile = static_cast<size_t>(row >> 7) * ktiles + kt;
+    return (tile * 4 + ((row >> 5) & 3)) * static_cast<size_t>(64 * b0);
+}
+// Word w of the 32-code group g of `row` inside its slab.
+__host__ __device__ inline int slab_word_offset(int row, int g, int w, int b0) {
+    return (g * b0 + w) * 32 + (row & 31);
+}
+
+// Code j (0..31) of a group whose b0 words are in `w`: bits [b0*j, b0*j + b0) of the bit string.
+template <int B>
+__device__ __forceinline__ uint32_t extract_code(const uint32_t* w, int j) {
+    const int p = B * j;
+    const int wi = p >> 5, sh = p & 31;
+    if (sh + B <= 32) return (w[wi] >> sh) & ((1u << B) - 1u);
+    return __funnelshift_r(w[wi], w[wi + 1], sh) & ((1u << B) - 1u);
+}
+
+// s~ = fl32(float(s^) * fl32(v / 127))
+__device__ __forceinline__ float block_scale(uint8_t sc, float v) {
+    return __fmul_rn(static_cast<float>(sc), __fdiv_rn(v, static_cast<float>(kScaleLevels)));
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
+
+// Tables (index 0..3 for b0 = 2, 3, 4, 8): code book and the round-down fp32 midpoints between
+// neighbouring code-book entries (x > midpoint  <=>  x > threshold for fp32 x).
+__constant__ float c_codebook[4][256];
+__constant__ float c_threshold[4][256];
+
+int ensure_tables();                 // uploads the tables to the current device once; LQLORA_OK or error
+const float* host_codebook(int b0);  // 2^b0 floats
+void count_launch(int n = 1);
+
+}  // namespace lq

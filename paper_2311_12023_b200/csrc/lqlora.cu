@@ -1,0 +1,189 @@
+// C ABI of the LQ-LoRA library: argument validation, dispatch, launches.
+// Single translation unit: the kernels live in the headers included below.
+#include "../../include/lqlora.h"
+
+#include "common.cuh"
+#include "tables.cuh"
+#include "codec.cuh"
+#include "linear_small.cuh"
+#include "linear_tc.cuh"
+
+namespace lq {
+
+static int check_qmatrix(const lqlora_qmatrix* q) {
+    if (!q) return LQLORA_ERR_NULL_POINTER;
+    int rc = check_config(&q->cfg);
+    if (rc != LQLORA_OK) return rc;
+    rc = check_shape(q->N, q->K, &q->cfg);
+    if (rc != LQLORA_OK) return rc;
+    if (!q->codes || !q->scale_codes || !q->scale2) return LQLORA_ERR_NULL_POINTER;
+    if (!aligned16(q->codes) || !aligned16(q->scale_codes) || !aligned16(q->scale2)) return LQLORA_ERR_MISALIGNED;
+    return LQLORA_OK;
+}
+
+static int cuda_rc(cudaError_t e) {
+    if (e == cudaSuccess) return LQLORA_OK;
+    cudaGetLastError();
+    return LQLORA_ERR_CUDA;
+}
+
+static int check_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, int r, const void* A, int64_t M,
+                        void* out, void* ws, size_t ws_bytes, bool backward) {
+    int rc = check_qmatrix(q);
+    if (rc != LQLORA_OK) return rc;
+    if (M <= 0 || M > (int64_t(1) << 24)) return LQLORA_ERR_INVALID_SHAPE;
+    if (r < 0 || r > 128 || (r % 16) != 0) return LQLORA_ERR_INVALID_SHAPE;
+    if (!A || !out || !ws) return LQLORA_ERR_NULL_POINTER;
+    if (r > 0 && (!L1 || !L2)) return LQLORA_ERR_NULL_POINTER;
+    if (!aligned16(A) || !aligned16(out) || !aligned16(ws) || !aligned16(L1) || !aligned16(L2)) return LQLORA_ERR_MISALIGNED;
+    if ((backward ? q->N : q->K) % 8 != 0 || (backward ? q->K : q->N) % 8 != 0) {
+        // rows of X / Y must start on 16-byte boundaries for the vector loads and TMA
+        if (M > 1) return LQLORA_ERR_INVALID_SHAPE;
+    }
+    size_t need = 0;
+    rc = lqlora_linear_workspace_bytes(q->N, q->K, &q->cfg, r, M, &need);
+    if (rc != LQLORA_OK) return rc;
+    if (ws_bytes < need) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
+    return LQLORA_OK;
+}
+
+static int run_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, int r, const void* A, int64_t M,
+                      void* out, void* ws, size_t ws_bytes, void* stream, bool backward) {
+    int rc = check_linear(q, L1, L2, r, A, M, out, ws, ws_bytes, backward);
+    if (rc != LQLORA_OK) return rc;
+    rc = ensure_tables();
+    if (rc != LQLORA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const QView v = make_view(q);
+    if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) return cuda_rc(cudaGetLastError());
+    cudaError_t e = cudaSuccess;
+    if (tc_supported(v, r, M, backward)) {
+        return tc_launch(v, L1, L2, r, A, static_cast<int>(M), out, static_cast<char*>(ws), backward, st);
+    }
+    switch (v.b0) {
+        case 2: e = launch_small<2>(v, L1, L2, r, A, static_cast<int>(M), out, static_cast<char*>(ws), backward, st); break;
+        case 3: e = launch_small<3>(v, L1, L2, r, A, static_cast<int>(M), out, static_cast<char*>(ws), backward, st); break;
+        case 4: e = launch_small<4>(v, L1, L2, r, A, static_cast<int>(M), out, static_cast<char*>(ws), backward, st); break;
+        default: e = launch_small<8>(v, L1, L2, r, A, static_cast<int>(M), out, static_cast<char*>(ws), backward, st); break;
+    }
+    return cuda_rc(e);
+}
+
+}  // namespace lq
+
+extern "C" {
+
+int lqlora_encode(const float* W_dev, lqlora_qmatrix* out, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    using namespace lq;
+    if (!W_dev || !workspace_dev) return LQLORA_ERR_NULL_POINTER;
+    int rc = check_qmatrix(out);
+    if (rc != LQLORA_OK) return rc;
+    if (!aligned16(W_dev) || !aligned16(workspace_dev)) return LQLORA_ERR_MISALIGNED;
+    size_t need = 0;
+    lqlora_packed_sizes(out->N, out->K, &out->cfg, nullptr, nullptr, nullptr, &need);
+    if (workspace_bytes < need) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
+    rc = ensure_tables();
+    if (rc != LQLORA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* absmax = static_cast<float*>(workspace_dev);
+    cudaError_t e;
+    switch (out->cfg.b0) {
+        case 2: e = launch_encode<2>(W_dev, out, absmax, st); break;
+        case 3: e = launch_encode<3>(W_dev, out, absmax, st); break;
+        case 4: e = launch_encode<4>(W_dev, out, absmax, st); break;
+        default: e = launch_encode<8>(W_dev, out, absmax, st); break;
+    }
+    return cuda_rc(e);
+}
+
+int lqlora_unpack(const lqlora_qmatrix* q, uint8_t* codes_dev, void* stream) {
+    using namespace lq;
+    int rc = check_qmatrix(q);
+    if (rc != LQLORA_OK) return rc;
+    if (!codes_dev) return LQLORA_ERR_NULL_POINTER;
+    rc = ensure_tables();
+    if (rc != LQLORA_OK) return rc;
+    const QView v = make_view(q);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    switch (v.b0) {
+        case 2: e = launch_export<2>(v, codes_dev, nullptr, nullptr, st); break;
+        case 3: e = launch_export<3>(v, codes_dev, nullptr, nullptr, st); break;
+        case 4: e = launch_export<4>(v, codes_dev, nullptr, nullptr, st); break;
+        default: e = launch_export<8>(v, codes_dev, nullptr, nullptr, st); break;
+    }
+    return cuda_rc(e);
+}
+
+int lqlora_dequant(const lqlora_qmatrix* q, float* deq32_dev, void* deq16_dev, void* stream) {
+    using namespace lq;
+    int rc = check_qmatrix(q);
+    if (rc != LQLORA_OK) return rc;
+    if (!deq32_dev && !deq16_dev) return LQLORA_ERR_NULL_POINTER;
+    rc = ensure_tables();
+    if (rc != LQLORA_OK) return rc;
+    const QView v = make_view(q);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    switch (v.b0) {
+        case 2: e = launch_export<2>(v, nullptr, deq32_dev, deq16_dev, st); break;
+        case 3: e = launch_export<3>(v, nullptr, deq32_dev, deq16_dev, st); break;
+        case 4: e = launch_export<4>(v, nullptr, deq32_dev, deq16_dev, st); break;
+        default: e = launch_export<8>(v, nullptr, deq32_dev, deq16_dev, st); break;
+    }
+    return cuda_rc(e);
+}
+
+int lqlora_linear_workspace_bytes(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, size_t* bytes) {
+    using namespace lq;
+    int rc = check_config(cfg);
+    if (rc != LQLORA_OK) return rc;
+    rc = check_shape(N, K, cfg);
+    if (rc != LQLORA_OK) return rc;
+    if (M <= 0 || r < 0 || r > 128 || r % 16) return LQLORA_ERR_INVALID_SHAPE;
+    if (!bytes) return LQLORA_ERR_NULL_POINTER;
+    // the same workspace must serve forward and backward, small-M and tensor-core kernels
+    size_t need = 0;
+    for (int backward = 0; backward < 2; ++backward) {
+        const SmallPlan p = small_plan(N, K, r, M, backward != 0);
+        const size_t small = kStatusBytes + p.t_bytes + p.p_bytes;
+        const size_t tc = tc_workspace_bytes(N, K, r, M, backward != 0);
+        need = small > need ? small : need;
+        need = tc > need ? tc : need;
+    }
+    *bytes = need;
+    return LQLORA_OK;
+}
+
+int lqlora_linear_fwd(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r, const void* X_dev,
+                      int64_t M, void* Y_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    return lq::run_linear(q, L1_dev, L2_dev, r, X_dev, M, Y_dev, workspace_dev, workspace_bytes, stream, false);
+}
+
+int lqlora_linear_bwd_input(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r, const void* dY_dev,
+                            int64_t M, void* dX_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    return lq::run_linear(q, L1_dev, L2_dev, r, dY_dev, M, dX_dev, workspace_dev, workspace_bytes, stream, true);
+}
+
+int lqlora_workspace_status(const void* workspace_dev, void* stream) {
+    if (!workspace_dev) return LQLORA_ERR_NULL_POINTER;
+    int word = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, workspace_dev, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return LQLORA_ERR_CUDA;
+    }
+    return word == 0 ? LQLORA_OK : LQLORA_ERR_TIMEOUT;
+}
+
+int lqlora_linear_path(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, int backward) {
+    using namespace lq;
+    if (check_config(cfg) != LQLORA_OK || check_shape(N, K, cfg) != LQLORA_OK) return LQLORA_ERR_INVALID_CONFIG;
+    lqlora_qmatrix q{};
+    q.N = N; q.K = K; q.cfg = *cfg;
+    const QView v = make_view(&q);
+    return tc_supported(v, r, M, backward != 0) ? 1 : 0;
+}
+
+}  // extern "C"

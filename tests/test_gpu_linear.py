@@ -1,0 +1,138 @@
+"""Parity of lqlora_linear_fwd / lqlora_linear_bwd_input with the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2311_12023_b200 import binding, inputs
+from gpu_util import check_close, encode_both, to_np
+
+pytestmark = pytest.mark.gpu
+
+C = inputs.QuantConfig
+
+
+def run_case(A, l1b, l2b, cfg, M, seed, rows=None, passes=("fwd", "bwd")):
+    N, K = A.shape
+    q, ref = encode_both(A, cfg)
+    L1 = binding.bf16_from_bits(l1b) if l1b is not None else None
+    L2 = binding.bf16_from_bits(l2b) if l2b is not None else None
+    out = {}
+    if "fwd" in passes:
+        xb = inputs.activations(seed, M, K)
+        Y = binding.linear_fwd(q, L1, L2, binding.bf16_from_bits(xb))
+        torch.cuda.synchronize()
+        Yo = oracle.linear_fwd(ref["d32"], l1b, l2b, xb, rows)
+        got = to_np(Y) if rows is None else to_np(Y[torch.from_numpy(rows).cuda()])
+        out["fwd"] = check_close(got, Yo, f"Y M={M}")
+    if "bwd" in passes:
+        gb = inputs.activations(seed + 1, M, N)
+        dX = binding.linear_bwd_input(q, L1, L2, binding.bf16_from_bits(gb))
+        torch.cuda.synchronize()
+        dXo = oracle.linear_bwd_input(ref["d32"], l1b, l2b, gb, rows)
+        got = to_np(dX) if rows is None else to_np(dX[torch.from_numpy(rows).cuda()])
+        out["bwd"] = check_close(got, dXo, f"dX M={M}")
+    return out
+
+
+@pytest.mark.parametrize("b0,B0,B1", [(2, 16, 64), (3, 64, 256), (4, 32, 64), (4, 64, 256), (8, 128, 64), (3, 256, 256)])
+@pytest.mark.parametrize("M", [1, 5, 16, 33])
+def test_linear_small_shapes(b0, B0, B1, M):
+    N, K = 320, 768            # N not a multiple of 128; several column windows
+    A = inputs.gaussian(100 + b0, (N, K), 0.02)
+    l1b, l2b = inputs.lowrank_factors(101, N, K, 64, 0.01)
+    run_case(A, l1b, l2b, C(b0, B0, 8, B1, 32), M, seed=200 + M)
+
+
+@pytest.mark.parametrize("M", [128, 200, 384])
+@pytest.mark.parametrize("b0,B0", [(3, 64), (4, 64), (2, 16), (8, 32)])
+def test_linear_training_shapes(b0, B0, M):
+    N, K = 512, 1024
+    A = inputs.student_t(300 + b0, (N, K), 5.0, 0.02)
+    l1b, l2b = inputs.lowrank_factors(301, N, K, 64, 0.01)
+    run_case(A, l1b, l2b, C(b0, B0, 8, 256, 32), M, seed=400 + M)
+
+
+@pytest.mark.parametrize("M", [4, 256])
+def test_linear_without_lowrank_and_with_zero_weights(M):
+    N, K = 256, 512
+    cfg = C(4, 64, 8, 256, 32)
+    A = inputs.gaussian(7, (N, K), 0.02)
+    run_case(A, None, None, cfg, M, seed=8)                      # r = 0: quantized part alone
+    l1b, l2b = inputs.lowrank_factors(9, N, K, 32, 0.05)
+    run_case(np.zeros_like(A), l1b, l2b, cfg, M, seed=10)        # Q = 0: pure rank-32 product
+
+
+@pytest.mark.parametrize("M", [16, 256])
+def test_identity_rows_return_dequantized_columns(M):
+    """X = rows of the identity and L = 0: Y[m, :] must equal column m of deq16 exactly."""
+    N, K = 256, 256
+    cfg = C(3, 64, 8, 256, 32)
+    A = inputs.gaussian(11, (N, K), 0.02)
+    q, ref = encode_both(A, cfg)
+    X = torch.eye(K, dtype=torch.bfloat16, device="cuda")[:M].contiguous()
+    Y = binding.linear_fwd(q, None, None, X)
+    w16 = inputs.bf16_bits_to_f32(ref["d16"])
+    assert np.array_equal(to_np(Y), w16[:, :M].T)
+    G = torch.eye(N, dtype=torch.bfloat16, device="cuda")[:M].contiguous()
+    dX = binding.linear_bwd_input(q, None, None, G)
+    assert np.array_equal(to_np(dX), w16[:M, :])
+
+
+@pytest.mark.parametrize("M", [8, 192])
+def test_adjoint_identity_on_gpu(M):
+    """<dY, fwd(X)> = <bwd_input(dY), X> up to the bf16 rounding of the outputs."""
+    N, K = 384, 512
+    cfg = C(4, 64, 8, 256, 32)
+    A = inputs.gaussian(12, (N, K), 0.02)
+    l1b, l2b = inputs.lowrank_factors(13, N, K, 64, 0.02)
+    q, _ = encode_both(A, cfg)
+    L1, L2 = binding.bf16_from_bits(l1b), binding.bf16_from_bits(l2b)
+    X = binding.bf16_from_bits(inputs.activations(14, M, K))
+    G = binding.bf16_from_bits(inputs.activations(15, M, N))
+    Y = binding.linear_fwd(q, L1, L2, X).double()
+    dX = binding.linear_bwd_input(q, L1, L2, G).double()
+    lhs = (G.double() * Y).sum().item()
+    rhs = (dX * X.double()).sum().item()
+    scale = (G.double().norm() * Y.norm()).item()
+    assert abs(lhs - rhs) <= 2e-3 * scale
+
+
+def test_config1_forward():
+    w = inputs.workload(1)
+    spec = w["matrices"][0]
+    A, l1b, l2b = inputs.make_matrix(spec)
+    run_case(A, l1b, l2b, spec.cfg, 512, seed=1100, passes=("fwd",))
+
+
+@pytest.mark.parametrize("M", [1, 16, 2048])
+def test_config2_forward_and_backward(M):
+    spec = inputs.workload(2)["matrices"][0]
+    A, l1b, l2b = inputs.make_matrix(spec)
+    rows = inputs.sample_rows(2100 + M, M) if M > 512 else None
+    run_case(A, l1b, l2b, spec.cfg, M, seed=2200 + M, rows=rows)
+
+
+def test_config3_down_projection_sampled_rows():
+    spec = inputs.workload(3)["matrices"][2]          # 4096 x 11008
+    A, l1b, l2b = inputs.make_matrix(spec)
+    rows = inputs.sample_rows(3100, 4096, count=16)
+    run_case(A, l1b, l2b, spec.cfg, 4096, seed=3200, rows=rows)
+
+
+def test_config4_kv_projection_mixed_config():
+    spec = [s for s in inputs.workload(4)["matrices"] if s.name == "k"][0]    # 1024 x 8192
+    A, l1b, l2b = inputs.make_matrix(spec)
+    run_case(A, l1b, l2b, spec.cfg, 1, seed=4200)
+    rows = inputs.sample_rows(4100, 2048, count=16)
+    run_case(A, l1b, l2b, spec.cfg, 2048, seed=4300, rows=rows)
+
+
+def test_workspace_status_is_clean_after_a_call():
+    N, K, M = 256, 512, 8
+    cfg = C(3, 64, 8, 256, 32)
+    q, _ = encode_both(inputs.gaussian(1, (N, K), 0.02), cfg)
+    ws = binding.alloc_workspace(q, 0, M)
+    X = binding.bf16_from_bits(inputs.activations(2, M, K))
+    binding.linear_fwd(q, None, None, X, workspace=ws)
+    assert binding.workspace_status(ws) == 0
