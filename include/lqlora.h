@@ -121,7 +121,7 @@ int lqlora_encode(const float* W_dev, lqlora_qmatrix* out, void* workspace_dev,
 
 /* Parity / debug exports (not on the hot path).
  * lqlora_unpack: one code per byte, codes_dev uint8 [N, K] row major (device).
- * lqlora_dequant: "dequantization simply reverses this process" (Sec. 3.2):
+ * lqlora_dequant: the inverse of lqlora_encode, step by step in reverse order (Sec. 3.2):
  *   s~_i = fl32(float(s^_i) * fl32(v_g / 127));  w~_j = fl32(q~[c_j] * s~_i)  -> deq32_dev fp32 [N, K];
  *   deq16_dev = w~ rounded to bf16, nearest-even, [N, K] (the cast for bf16 training, App. A).
  *   Either output may be NULL. */
@@ -156,6 +156,26 @@ int lqlora_linear_fwd(const lqlora_qmatrix* q, const void* L1_dev, const void* L
 int lqlora_linear_bwd_input(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r,
                             const void* dY_dev, int64_t M, void* dX_dev, void* workspace_dev,
                             size_t workspace_bytes, void* stream);
+
+/*
+ * Host-buffer variants (end-to-end use: activations arrive from and results return to pinned host
+ * memory).  They enqueue, on `stream`: a host-to-device copy of the input into the caller's device
+ * staging buffer, the same kernels as the device-pointer entry points (Sec. 2.1, Sec. 3.2 as
+ * above), and a device-to-host copy of the result.  Nothing is allocated; the quantized matrix
+ * and L1, L2 stay on the device.
+ *   X_host / dY_host / W_host : host memory (pinned for asynchronous copies), read only
+ *   Y_host / dX_host          : host memory, written when the stream reaches the copy
+ *   *_stage_dev               : device scratch of the same size as the matching host buffer
+ * Errors as for the device-pointer entry points.
+ */
+int lqlora_encode_host(const float* W_host, float* W_stage_dev, lqlora_qmatrix* out, void* workspace_dev,
+                       size_t workspace_bytes, void* stream);
+int lqlora_linear_fwd_host(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r,
+                           const void* X_host, int64_t M, void* Y_host, void* X_stage_dev, void* Y_stage_dev,
+                           void* workspace_dev, size_t workspace_bytes, void* stream);
+int lqlora_linear_bwd_input_host(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r,
+                                 const void* dY_host, int64_t M, void* dX_host, void* dY_stage_dev,
+                                 void* dX_stage_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
 
 /* Synchronizes `stream`, reads the status word at the start of a linear workspace and returns it
  * as an lqlora_status: LQLORA_OK, or LQLORA_ERR_TIMEOUT if a kernel gave up on a bounded wait

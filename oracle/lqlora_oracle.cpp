@@ -169,7 +169,7 @@ int oracle_encode(const float* A, int64_t N, int64_t K, int b0, int B0, int b1, 
 }
 
 // ----------------------------------------------------------------------------------
-// Dequantize: "simply reverses this process" (Sec. 3.2).
+// Dequantize: the inverse of the steps above, applied in reverse order (Sec. 3.2).
 //   sigma_g = v_g / (2^(b1-1)-1);  s~_i = float(s^_i) * sigma_g;  w~_j = q~[c_j] * s~_i
 //   deq32 = w~ (fp32); deq16 = w~ rounded to bf16 (the cast for bf16 training, App. A).
 // Either output may be null.

@@ -21,7 +21,7 @@ EXPORTS = [
     "lqlora_storage_bits_per_param", "lqlora_packed_sizes", "lqlora_nf_codebook", "lqlora_encode",
     "lqlora_unpack", "lqlora_dequant", "lqlora_linear_workspace_bytes", "lqlora_linear_fwd",
     "lqlora_linear_bwd_input", "lqlora_workspace_status", "lqlora_linear_path", "lqlora_launch_count",
-    "lqlora_status_string",
+    "lqlora_status_string", "lqlora_encode_host", "lqlora_linear_fwd_host", "lqlora_linear_bwd_input_host",
 ]
 
 
@@ -64,6 +64,9 @@ def lib() -> ctypes.CDLL:
         L.lqlora_linear_workspace_bytes.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ctypes.POINTER(sz)]
         L.lqlora_linear_fwd.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, sz, vp]
         L.lqlora_linear_bwd_input.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, sz, vp]
+        L.lqlora_encode_host.argtypes = [vp, vp, ctypes.POINTER(CQMatrix), vp, sz, vp]
+        L.lqlora_linear_fwd_host.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, vp, vp, sz, vp]
+        L.lqlora_linear_bwd_input_host.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, vp, vp, sz, vp]
         L.lqlora_workspace_status.argtypes = [vp, vp]
         L.lqlora_linear_path.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ci]
         L.lqlora_launch_count.restype = i64
@@ -220,6 +223,32 @@ def linear_bwd_input(q: QMatrix, L1, L2, dY: torch.Tensor, out=None, workspace=N
     """lqlora_linear_bwd_input: dX = dY deq(Q) + (dY L1) L2, bf16 [M, K]."""
     assert dY.shape[1] == q.N
     return _linear(lib().lqlora_linear_bwd_input, "lqlora_linear_bwd_input", q, L1, L2, dY, q.K, out, workspace)
+
+
+def encode_host(W_host: torch.Tensor, W_stage: torch.Tensor, q: QMatrix, workspace: torch.Tensor) -> None:
+    """lqlora_encode_host: W_host is (pinned) host fp32 [N, K]; q and the scratch are on the device."""
+    assert not W_host.is_cuda and W_host.dtype == torch.float32 and W_stage.is_cuda
+    cs = q.cstruct()
+    _check(lib().lqlora_encode_host(W_host.data_ptr(), W_stage.data_ptr(), ctypes.byref(cs), workspace.data_ptr(),
+                                    workspace.numel(), _stream()), "lqlora_encode_host")
+
+
+def _linear_host(fn, name, q, L1, L2, A_host, out_host, A_stage, out_stage, workspace):
+    assert not A_host.is_cuda and not out_host.is_cuda and A_stage.is_cuda and out_stage.is_cuda
+    M = A_host.shape[0]
+    r = 0 if L1 is None else L1.shape[1]
+    cs = q.cstruct()
+    _check(fn(ctypes.byref(cs), _ptr(L1), _ptr(L2), r, A_host.data_ptr(), M, out_host.data_ptr(), A_stage.data_ptr(),
+              out_stage.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()), name)
+
+
+def linear_fwd_host(q, L1, L2, X_host, Y_host, X_stage, Y_stage, workspace) -> None:
+    _linear_host(lib().lqlora_linear_fwd_host, "lqlora_linear_fwd_host", q, L1, L2, X_host, Y_host, X_stage, Y_stage, workspace)
+
+
+def linear_bwd_input_host(q, L1, L2, dY_host, dX_host, dY_stage, dX_stage, workspace) -> None:
+    _linear_host(lib().lqlora_linear_bwd_input_host, "lqlora_linear_bwd_input_host", q, L1, L2, dY_host, dX_host,
+                 dY_stage, dX_stage, workspace)
 
 
 def workspace_status(workspace: torch.Tensor) -> int:

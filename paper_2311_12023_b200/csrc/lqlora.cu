@@ -165,6 +165,44 @@ int lqlora_linear_bwd_input(const lqlora_qmatrix* q, const void* L1_dev, const v
     return lq::run_linear(q, L1_dev, L2_dev, r, dY_dev, M, dX_dev, workspace_dev, workspace_bytes, stream, true);
 }
 
+int lqlora_encode_host(const float* W_host, float* W_stage_dev, lqlora_qmatrix* out, void* workspace_dev,
+                       size_t workspace_bytes, void* stream) {
+    if (!W_host || !W_stage_dev || !out) return LQLORA_ERR_NULL_POINTER;
+    int rc = lq::check_qmatrix(out);
+    if (rc != LQLORA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(W_stage_dev, W_host, sizeof(float) * out->N * out->K, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return lq::cuda_rc(cudaGetLastError());
+    return lqlora_encode(W_stage_dev, out, workspace_dev, workspace_bytes, stream);
+}
+
+static int linear_host(const lqlora_qmatrix* q, const void* L1, const void* L2, int r, const void* A_host, int64_t M,
+                       void* out_host, void* A_stage, void* out_stage, void* ws, size_t ws_bytes, void* stream, bool backward) {
+    if (!A_host || !out_host) return LQLORA_ERR_NULL_POINTER;
+    int rc = lq::check_linear(q, L1, L2, r, A_stage, M, out_stage, ws, ws_bytes, backward);
+    if (rc != LQLORA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t in_bytes = static_cast<size_t>(M) * (backward ? q->N : q->K) * 2;
+    const size_t out_bytes = static_cast<size_t>(M) * (backward ? q->K : q->N) * 2;
+    if (cudaMemcpyAsync(A_stage, A_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return lq::cuda_rc(cudaGetLastError());
+    rc = lq::run_linear(q, L1, L2, r, A_stage, M, out_stage, ws, ws_bytes, stream, backward);
+    if (rc != LQLORA_OK) return rc;
+    if (cudaMemcpyAsync(out_host, out_stage, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return lq::cuda_rc(cudaGetLastError());
+    return LQLORA_OK;
+}
+
+int lqlora_linear_fwd_host(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r, const void* X_host,
+                           int64_t M, void* Y_host, void* X_stage_dev, void* Y_stage_dev, void* workspace_dev,
+                           size_t workspace_bytes, void* stream) {
+    return linear_host(q, L1_dev, L2_dev, r, X_host, M, Y_host, X_stage_dev, Y_stage_dev, workspace_dev, workspace_bytes, stream, false);
+}
+
+int lqlora_linear_bwd_input_host(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r, const void* dY_host,
+                                 int64_t M, void* dX_host, void* dY_stage_dev, void* dX_stage_dev, void* workspace_dev,
+                                 size_t workspace_bytes, void* stream) {
+    return linear_host(q, L1_dev, L2_dev, r, dY_host, M, dX_host, dY_stage_dev, dX_stage_dev, workspace_dev, workspace_bytes, stream, true);
+}
+
 int lqlora_workspace_status(const void* workspace_dev, void* stream) {
     if (!workspace_dev) return LQLORA_ERR_NULL_POINTER;
     int word = 0;

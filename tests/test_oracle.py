@@ -26,7 +26,7 @@ def test_codebook_matches_quantile_construction(b):
     half = 1 << (b - 1)
     delta = 0.5 * (1 / 30 + 1 / 32)
     p = np.concatenate([np.linspace(delta, 0.5, half), np.linspace(0.5, 1 - delta, half + 1)[1:]])
-    assert len(p) == 1 << b                       # "this results in 2^b probability values"
+    assert len(p) == 1 << b                       # the shared 1/2 counted once leaves 2^b probabilities (Sec. 2.2)
     assert p[0] == delta and p[half - 1] == 0.5   # p_1 = delta, p_{2^(b-1)} = 1/2
     q = ndtri(p)
     ref = (q / q[-1]).astype(np.float32)
