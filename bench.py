@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the LQ-LoRA linear hot path on B200.
+
+One step = one pass of the whole hot path on the LLaMA-2-7B attention-projection workload
+(4096x4096, NF3, B0 = 64, B1 = 256, rank 64; seeded synthetic data):
+
+    encode(R)  ->  forward + input gradient at M = 2048 (training, tensor-core kernels)
+               ->  forward + input gradient at M = 16 and M = 1 (decode, weight-streaming kernels)
+
+`value` is the algorithmic TFLOP/s of the whole step: 2 M (N K + r K + N r) flop per linear
+call, summed over the six calls, divided by the device time of the step (CUDA events).  The
+JSON line also carries the per-phase figures (tensor TFLOP/s at M = 2048, packed-weight GB/s
+at M = 1 / 16, encode GB/s), the roofline of the dominant kernel, the end-to-end number
+through the host-buffer C ABI, and the CPU oracle timed on the host as a baseline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+With N > 1 (torchrun) every rank runs the same per-GPU workload on its own tokens (data
+parallel over tokens, no collective on the data path); time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2311_12023_b200 import inputs  # noqa: E402
+
+METRIC = "LQ-LoRA linear fwd/bwd TFLOP/s & packed-weight GB/s, % of B200 roofline"
+WORKLOAD = "llama2-7b attn-proj 4096x4096 NF3 B0=64 B1=256 r=64; encode + fwd/dX at M=2048,16,1"
+MS = (2048, 16, 1)
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+FALLBACK = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram bytes per forward launch of the tensor-core kernel at M = 2048 on this workload, from the
+# ncu capture summarised under profiles/ (None until a capture exists)
+TC_TRAFFIC_BYTES = None
+
+
+def linear_flops(M: int, N: int, K: int, r: int) -> float:
+    return 2.0 * M * (N * K + r * K + N * r)
+
+
+def packed_bytes(N: int, K: int, cfg) -> float:
+    return N * K * (cfg.b0 + cfg.b1 / cfg.B0 + cfg.b2 / (cfg.B0 * cfg.B1)) / 8.0
+
+
+def encode_bytes(N: int, K: int, cfg) -> float:
+    return 4.0 * N * K + packed_bytes(N, K, cfg)
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK), "fallback"
+
+
+# ------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------- reference arm
+def oracle_sample(spec, A, l1b, l2b, rows_large: int = 24):
+    """Times the CPU oracle on a bounded sample of the step; returns (flops_done, seconds, description)."""
+    import oracle
+    cfg = spec.cfg
+    N, K, r = spec.N, spec.K, inputs.RANK
+    t0 = time.perf_counter()
+    codes, _, sc, v = oracle.encode(A, cfg.b0, cfg.B0, cfg.b1, cfg.B1)
+    d32, _ = oracle.dequant(codes, sc, v, cfg.b0, cfg.B0, cfg.b1, cfg.B1)
+    flops = 0.0
+    for M in MS:
+        rows = inputs.sample_rows(900 + M, M, count=rows_large) if M > rows_large else None
+        nrows = M if rows is None else len(rows)
+        xb = inputs.activations(910 + M, M, K)
+        gb = inputs.activations(920 + M, M, N)
+        oracle.linear_fwd(d32, l1b, l2b, xb, rows)
+        oracle.linear_bwd_input(d32, l1b, l2b, gb, rows)
+        flops += 2 * linear_flops(nrows, N, K, r)
+    dt = time.perf_counter() - t0
+    desc = (f"encode+dequant of the full {N}x{K} matrix, then fwd and dX in fp64 on {rows_large} sampled rows "
+            f"of M=2048 and all rows of M=16 and M=1")
+    return flops, dt, desc
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    spec = inputs.workload(2)["matrices"][0]
+    A, l1b, l2b = inputs.make_matrix(spec)
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_sample(spec, A, l1b, l2b, rows_large=4)
+    times, flops = [], 0.0
+    for _ in range(args.steps):
+        flops, dt, desc = oracle_sample(spec, A, l1b, l2b, rows_large=64)
+        times.append(dt)
+    mean = sum(times) / len(times)
+    val = flops / mean / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "note": "each step is a bounded sample of the workload: " + desc},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------- device arm
+def shard_info():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def reduce_max(value: float, world: int, device=None) -> float:
+    """Max over ranks of a host scalar (identity when world == 1)."""
+    if world == 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def run_device(args):
+    import torch
+    from paper_2311_12023_b200 import binding
+
+    rank, world, local = shard_info()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    binding.lib()
+
+    spec = inputs.workload(2)["matrices"][0]
+    cfg, N, K, r = spec.cfg, spec.N, spec.K, inputs.RANK
+    # every rank draws its own tokens (seed offset by rank); the weights are replicated
+    A, l1b, l2b = inputs.make_matrix(spec)
+    W_host = torch.from_numpy(A).pin_memory()
+    W = W_host.to(dev)
+    L1, L2 = binding.bf16_from_bits(l1b, dev), binding.bf16_from_bits(l2b, dev)
+    q = binding.alloc_qmatrix(N, K, cfg, dev)
+    enc_ws = torch.empty(binding.packed_sizes(N, K, cfg)[3], dtype=torch.uint8, device=dev)
+    binding.encode(W, cfg, out=q, workspace=enc_ws)
+    torch.cuda.synchronize()
+
+    # cold copies of the packed matrix for the decode-sized calls: more than twice the L2 in total
+    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
+    ncopies = max(4, int(2.2 * l2_bytes / q.packed_bytes) + 1)
+    copies = [binding.QMatrix(q.codes.clone(), q.scale_codes.clone(), q.scale2.clone(), N, K, cfg) for _ in range(ncopies)]
+
+    X, G, Y, DX, WS, XH, GH, YH, DXH = {}, {}, {}, {}, {}, {}, {}, {}, {}
+    for M in MS:
+        XH[M] = torch.from_numpy(inputs.activations(7000 + 10 * rank + M, M, K).view(np.int16)).view(torch.bfloat16).pin_memory()
+        GH[M] = torch.from_numpy(inputs.activations(7500 + 10 * rank + M, M, N).view(np.int16)).view(torch.bfloat16).pin_memory()
+        X[M], G[M] = XH[M].to(dev), GH[M].to(dev)
+        Y[M] = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+        DX[M] = torch.empty((M, K), dtype=torch.bfloat16, device=dev)
+        YH[M] = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+        DXH[M] = torch.empty((M, K), dtype=torch.bfloat16).pin_memory()
+        WS[M] = binding.alloc_workspace(q, r, M)
+    flush = torch.empty(max(256 << 20, 2 * l2_bytes), dtype=torch.uint8, device=dev)
+
+    seg_names = ["encode"] + [f"{p}{M}" for M in MS for p in ("fwd", "bwd")]
+    nseg = len(seg_names)
+    copy_idx = [0]
+
+    def next_copy():
+        c = copies[copy_idx[0] % ncopies]
+        copy_idx[0] += 1
+        return c
+
+    def one_step(events=None):
+        """The whole hot path once, device-resident inputs.  events: list of nseg+1 CUDA events."""
+        if events:
+            events[0].record()
+        binding.encode(W, cfg, out=q, workspace=enc_ws)
+        i = 1
+        if events:
+            events[i].record()
+        for M in MS:
+            qq = q if M > 64 else next_copy()
+            binding.linear_fwd(qq, L1, L2, X[M], out=Y[M], workspace=WS[M])
+            i += 1
+            if events:
+                events[i].record()
+            qq = q if M > 64 else next_copy()
+            binding.linear_bwd_input(qq, L1, L2, G[M], out=DX[M], workspace=WS[M])
+            i += 1
+            if events:
+                events[i].record()
+
+    def one_step_host():
+        """Same step through the host-buffer C ABI: H2D of W, X, dY and D2H of Y, dX inside."""
+        binding.encode_host(W_host, W, q, enc_ws)
+        for M in MS:
+            qq = q if M > 64 else next_copy()
+            binding.linear_fwd_host(qq, L1, L2, XH[M], YH[M], X[M], Y[M], WS[M])
+            qq = q if M > 64 else next_copy()
+            binding.linear_bwd_input_host(qq, L1, L2, GH[M], DXH[M], G[M], DX[M], WS[M])
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        flush.fill_(1)
+        one_step()
+    torch.cuda.synchronize()
+    for M in MS:
+        st = binding.workspace_status(WS[M])
+        if st != 0:
+            raise SystemExit(f"kernel reported {binding.status_string(st)}")
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nseg + 1)] for _ in range(args.steps)]
+    launches0 = binding.launch_count()
+    barrier()
+    t_wall0 = time.perf_counter()
+    for s in range(args.steps):
+        flush.fill_(s & 0xFF)          # evict L2 between steps (untimed: outside the step's events)
+        one_step(evs[s])
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    launches = binding.launch_count() - launches0
+    seg_ms = np.zeros(nseg)
+    step_ms = []
+    for s in range(args.steps):
+        for i in range(nseg):
+            seg_ms[i] += evs[s][i].elapsed_time(evs[s][i + 1])
+        step_ms.append(evs[s][0].elapsed_time(evs[s][nseg]))
+    seg_ms /= args.steps
+    ms_step = reduce_max(sum(step_ms) / len(step_ms), world, dev)
+
+    # end to end through the host-buffer entry points
+    for _ in range(max(1, min(args.warmup, 3))):
+        one_step_host()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_steps = max(3, min(args.steps, 10))
+    e0.record()
+    for _ in range(e2e_steps):
+        one_step_host()
+    e1.record()
+    barrier()
+    e2e_ms = reduce_max(e0.elapsed_time(e1) / e2e_steps, world, dev)
+    clocks = sampler.stop() if rank == 0 else None
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    step_flops = sum(2 * linear_flops(M, N, K, r) for M in MS)
+    value = world * step_flops / (ms_step * 1e-3) / 1e12
+    pk, pk_kind = peaks()
+    seg = dict(zip(seg_names, seg_ms.tolist()))
+    pbytes = packed_bytes(N, K, cfg)
+    small_bytes = pbytes + 2 * r * (N + K)
+    breakdown = {
+        "encode": {"ms": seg["encode"], "GB/s": encode_bytes(N, K, cfg) / seg["encode"] / 1e6,
+                   "frac_of_hbm_" + pk_kind: encode_bytes(N, K, cfg) / seg["encode"] / 1e6 / pk["hbm_gbs"]},
+    }
+    for M in MS:
+        for ps in ("fwd", "bwd"):
+            ms = seg[f"{ps}{M}"]
+            ent = {"ms": ms, "TFLOP/s": linear_flops(M, N, K, r) / ms / 1e9}
+            if M > 64:
+                ent["frac_of_bf16_" + pk_kind] = ent["TFLOP/s"] / pk["bf16_tflops"]
+                ent["frac_of_bf16_nominal"] = ent["TFLOP/s"] / NOMINAL["bf16_tflops"]
+            else:
+                ent["packed_GB/s"] = pbytes / ms / 1e6
+                ent["frac_of_hbm_" + pk_kind] = ent["packed_GB/s"] / pk["hbm_gbs"]
+                ent["frac_of_hbm_nominal"] = ent["packed_GB/s"] / NOMINAL["hbm_gbs"]
+                ent["all_bytes_GB/s"] = (small_bytes + 2 * M * (N + K)) / ms / 1e6
+            breakdown[f"{ps}_M{M}"] = ent
+
+    # dominant kernel: the tensor-core linear (forward and input gradient at M = 2048)
+    tc_ms = 0.5 * (seg["fwd2048"] + seg["bwd2048"])
+    achieved = linear_flops(2048, N, K, r) / tc_ms / 1e9
+    roofline = {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / pk["bf16_tflops"], "traffic": TC_TRAFFIC_BYTES,
+                "kernel": "tc_linear_kernel (one lqlora_linear_fwd / lqlora_linear_bwd_input call at M=2048, "
+                          "including its rank-r pre-product launch)",
+                "peak_kind": pk_kind + " cuBLAS bf16 burst", "frac_of_nominal_2250": achieved / NOMINAL["bf16_tflops"]}
+
+    oflops, osec, odesc = oracle_sample(spec, A, l1b, l2b, rows_large=256)
+    import oracle
+    cpu = {"value": oflops / osec / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+           "sample": odesc, "seconds": osec}
+
+    h2d = W_host.numel() * 4 + sum(XH[M].numel() * 2 + GH[M].numel() * 2 for M in MS)
+    d2h = sum(YH[M].numel() * 2 + DXH[M].numel() * 2 for M in MS)
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "N": N, "K": K, "rank": r, "M": list(MS), "quant": list(cfg.as_tuple()),
+                   "parallelism": f"dp{world} over tokens, weights replicated, no collective",
+                   "l2": "flushed between steps by a 256 MiB device write outside the timed events; decode-sized "
+                         f"calls rotate over {ncopies} cold copies of the packed matrix",
+                   "wall_ms_per_step_incl_flush": t_wall / args.steps * 1e3},
+        "clocks": clocks,
+        "e2e": {"value": world * step_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "breakdown": breakdown,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_device(args)
+
+
+if __name__ == "__main__":
+    main()

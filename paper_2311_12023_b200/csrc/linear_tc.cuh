@@ -4,9 +4,9 @@
 // elements:
 //   - a producer thread issues a TMA tile load of the bf16 activations (128-byte swizzle) and
 //     bulk copies of the packed code slabs into shared memory;
-//   - eight dequantization warps unpack the codes, multiply by the block scale in fp32, round to
+//   - sixteen dequantization warps unpack the codes, multiply by the block scale in fp32, round to
 //     bf16 and write the weight tile into shared memory in the 128-byte-swizzled layout that the
-//     tensor core reads (one thread = one weight row);
+//     tensor core reads (one thread = 32 weights of one row);
 //   - one thread issues tcgen05.mma (M = 128, N = 256, K = 16) with fp32 accumulators in tensor
 //     memory and commits the stage back to the producer.
 // The rank-r term is folded in as extra contraction steps whose two operands come by TMA
@@ -32,7 +32,7 @@ namespace tc {
 
 constexpr int BK = 64;
 constexpr int BN = 256;
-constexpr int kDeqWarps = 8;
+constexpr int kDeqWarps = 16;
 constexpr int kThreads = (2 + kDeqWarps) * 32;
 constexpr int kBBytes = BN * 128;            // bf16 weight tile of one step
 constexpr long long kWaitCycles = 4000000000LL;   // about two seconds
@@ -149,52 +149,100 @@ __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, const Ctl& c
 }
 
 // ------------------------------------------------------------------------------------ dequantization
-// One thread dequantizes 64 consecutive weights of one row (two groups of 32 codes) and writes
-// them as eight 16-byte chunks of a 128-byte row, chunk index XOR (row % 8).
+// Look-up tables in shared memory.  For 2- and 3-bit codes a table entry holds the fp32 code-book
+// values of TWO neighbouring codes (index = both codes, 2*b0 bits) and is fetched with one 64-bit
+// load; for 4- and 8-bit codes an entry is one fp32 value.  Entries are replicated per lane
+// (16 copies of the 8-byte entries, 32 copies of the 4-byte entries of the 4-bit table) so that
+// the loads of a warp never conflict; the 8-bit table (1 KB) is not replicated.
+template <int B> struct Lut {
+    static constexpr bool kPair = (B <= 3);
+    static constexpr int kIdxBits = kPair ? 2 * B : B;
+    static constexpr int kShift = (B <= 4) ? 7 : 2;                 // log2(bytes between consecutive entries)
+    static constexpr int kBytes = (1 << kIdxBits) << kShift;
+    static constexpr uint32_t kMask = ((1u << kIdxBits) - 1u) << kShift;
+};
+
 template <int B>
-__device__ __forceinline__ void dequant_row(const uint32_t* __restrict__ slab, int lane, const float* __restrict__ cb,
-                                            const float (&scale)[4], uint8_t* __restrict__ out_row, int row_in_8) {
-#pragma unroll
-    for (int g = 0; g < 2; ++g) {
-        uint32_t w[B + 1];
-#pragma unroll
-        for (int i = 0; i < B; ++i) w[i] = slab[(g * B + i) * 32 + lane];
-        w[B] = 0u;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            uint32_t packed[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int j = c * 8 + e * 2;
-                const uint32_t c0 = extract_code<B>(w, j), c1 = extract_code<B>(w, j + 1);
-                float q0, q1;
-                if constexpr (B <= 4) { q0 = cb[c0 * 32 + lane]; q1 = cb[c1 * 32 + lane]; }
-                else { q0 = cb[c0]; q1 = cb[c1]; }
-                const float s = scale[g * 2 + (c >> 1)];
-                const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(q0, s), __fmul_rn(q1, s));
-                packed[e] = *reinterpret_cast<const uint32_t*>(&h);
-            }
-            const int chunk = (g * 4 + c) ^ row_in_8;
-            *reinterpret_cast<uint4*>(out_row + chunk * 16) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+__device__ __forceinline__ void fill_lut(uint8_t* lut, int tid, int nthreads) {
+    const float* cb = c_codebook[bits_index(B)];
+    if constexpr (Lut<B>::kPair) {
+        float2* t = reinterpret_cast<float2*>(lut);
+        for (int i = tid; i < (1 << (2 * B)) * 16; i += nthreads) {
+            const int idx = i >> 4;
+            t[i] = make_float2(cb[idx & ((1 << B) - 1)], cb[idx >> B]);
         }
+    } else if constexpr (B == 4) {
+        float* t = reinterpret_cast<float*>(lut);
+        for (int i = tid; i < 16 * 32; i += nthreads) t[i] = cb[i >> 5];
+    } else {
+        float* t = reinterpret_cast<float*>(lut);
+        for (int i = tid; i < 256; i += nthreads) t[i] = cb[i];
     }
 }
 
-// Block scales s~ of the four 16-column quarters of (row, columns k .. k+63).
-__device__ __forceinline__ void load_scales(const QView& q, int row, int k, float (&scale)[4]) {
-    if (row >= q.N || k >= q.K) { scale[0] = scale[1] = scale[2] = scale[3] = 0.0f; return; }
-    const long long blk = static_cast<long long>(row) * q.KB + (k >> q.logB0);
-    if (q.B0 >= 64) {
-        const float s = block_scale(q.sc[blk], q.v[blk >> q.logB1]);
-        scale[0] = scale[1] = scale[2] = scale[3] = s;
-    } else if (q.B0 == 32) {
-        const float s0 = block_scale(q.sc[blk], q.v[blk >> q.logB1]);
-        const float s1 = block_scale(q.sc[blk + 1], q.v[(blk + 1) >> q.logB1]);
-        scale[0] = scale[1] = s0; scale[2] = scale[3] = s1;
-    } else {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) scale[i] = block_scale(q.sc[blk + i], q.v[(blk + i) >> q.logB1]);
+// Byte offset into the table of the entry whose index starts at bit `pos` of the little-endian bit
+// string w[0..B-1] (w[B] = 0), already OR-ed with the lane's replica offset.
+template <int B>
+__device__ __forceinline__ uint32_t lut_offset(const uint32_t (&w)[B + 1], int pos, uint32_t lane_off) {
+    constexpr int S = Lut<B>::kShift;
+    uint32_t x;
+    if (pos < S) x = w[0] << (S - pos);
+    else {
+        const int q = pos - S, wi = q >> 5, sh = q & 31;
+        x = (sh + Lut<B>::kIdxBits + S <= 32) ? (w[wi] >> sh) : __funnelshift_r(w[wi], w[wi + 1], sh);
     }
+    return (x & Lut<B>::kMask) | lane_off;
+}
+
+// One thread dequantizes the 32 consecutive weights of one (row, group) -- b0 words of the slab --
+// and writes them as four 16-byte chunks of the row's 128 bytes; `dst` is the row start, `xr` is
+// (row % 8) * 16, chunk c of the row lives at byte offset (c * 16) ^ xr.
+template <int B>
+__device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ slab_words, int g, int lane, const uint8_t* __restrict__ lut,
+                                              uint32_t lane_off, float s_lo, float s_hi, uint8_t* __restrict__ dst, uint32_t xr) {
+    uint32_t w[B + 1];
+#pragma unroll
+    for (int i = 0; i < B; ++i) w[i] = slab_words[(g * B + i) * 32 + lane];
+    w[B] = 0u;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const float s = (c < 2) ? s_lo : s_hi;
+        uint32_t packed[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int j = c * 8 + e * 2;           // first code of the pair
+            float q0, q1;
+            if constexpr (Lut<B>::kPair) {
+                const float2 qq = *reinterpret_cast<const float2*>(lut + lut_offset<B>(w, B * j, lane_off));
+                q0 = qq.x; q1 = qq.y;
+            } else {
+                q0 = *reinterpret_cast<const float*>(lut + lut_offset<B>(w, B * j, lane_off));
+                q1 = *reinterpret_cast<const float*>(lut + lut_offset<B>(w, B * (j + 1), lane_off));
+            }
+            const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(q0, s), __fmul_rn(q1, s));
+            packed[e] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        *reinterpret_cast<uint4*>(dst + ((((g * 4 + c) << 4)) ^ xr)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    }
+}
+
+// Raw scale data of the 32 weights (row, k .. k+31): the one or two 8-bit scale codes and the
+// second-level scale of their group (B1 >= 16 blocks, so both codes share it).
+struct RawScale { uint32_t sc; float v; };
+__device__ __forceinline__ RawScale fetch_scale(const QView& q, int row, int k) {
+    RawScale r{0u, 0.0f};
+    if (row < q.N && k < q.K) {
+        const long long blk = static_cast<long long>(row) * q.KB + (k >> q.logB0);
+        r.sc = (q.B0 == 16) ? static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(q.sc + blk)) : static_cast<uint32_t>(q.sc[blk]);
+        r.v = q.v[blk >> q.logB1];
+    }
+    return r;
+}
+// s~ = fl32(float(s^) * fl32(v / 127)); the quotient is recomputed only when v changes.
+__device__ __forceinline__ void make_scales(const QView& q, const RawScale& r, float& v_cached, float& sigma, float& s_lo, float& s_hi) {
+    if (r.v != v_cached) { v_cached = r.v; sigma = __fdiv_rn(r.v, static_cast<float>(kScaleLevels)); }
+    s_lo = __fmul_rn(static_cast<float>(r.sc & 0xFFu), sigma);
+    s_hi = (q.B0 == 16) ? __fmul_rn(static_cast<float>(r.sc >> 8), sigma) : s_lo;
 }
 
 // ------------------------------------------------------------------------------------ kernel
@@ -205,15 +253,15 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     constexpr int A_BYTES = MH * 128 * 128;
     constexpr int P_BYTES = 2048 * B;
     constexpr int STAGE = A_BYTES + kBBytes + P_BYTES;
-    constexpr int CB_FLOATS = (B <= 4) ? (1 << B) * 32 : 256;
+    constexpr int LUT_BYTES = Lut<B>::kBytes;
     constexpr uint32_t TMEM_COLS = MH * BN;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* tail = base + static_cast<size_t>(p.stages) * STAGE;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);            // full_tma[8], full_b[8], empty[8], acc_full, drain
-    float* cb = reinterpret_cast<float*>(tail + 256);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 256 + CB_FLOATS * 4);
+    uint8_t* lut = tail + 256;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 256 + LUT_BYTES);
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -234,8 +282,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         *abort_s = 0;
         fence_barrier_init();
     }
-    for (int i = threadIdx.x; i < CB_FLOATS; i += kThreads)
-        cb[i] = (B <= 4) ? c_codebook[bits_index(B)][i >> 5] : c_codebook[3][i];
+    fill_lut<B>(lut, threadIdx.x, kThreads);
     if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), TMEM_COLS); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
@@ -337,52 +384,55 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ dequantization warps, then epilogue
+        // warp dw handles slab (dw / 2) of the step's packed data and the 32-column group (dw % 2);
+        // one thread = one row of that slab.
         const int dw = warp - 2;
-        const uint32_t* slab_off = nullptr;
-        int row_local, row_sub;   // row inside the B tile / inside its 128-byte-row sub-tile
+        const int slab_i = dw >> 1, g = dw & 1;
+        int row_local;            // row inside the 128-byte-row (sub-)tile of the B operand
         uint32_t b_off;           // byte offset of this thread's row inside the B tile
-        if (!BWD) { row_local = dw * 32 + lane; row_sub = row_local; b_off = row_local * 128; }
-        else { row_local = (dw & 1) * 32 + lane; row_sub = row_local; b_off = (dw >> 1) * 8192 + row_local * 128; }
-        (void)slab_off;
-        float scale[4];
+        if (!BWD) { row_local = slab_i * 32 + lane; b_off = row_local * 128; }
+        else { row_local = (slab_i & 1) * 32 + lane; b_off = (slab_i >> 1) * 8192 + row_local * 128; }
+        const uint32_t xr = (row_local & 7) << 4;
+        const uint32_t lane_off = Lut<B>::kPair ? (lane & 15) * 8 : (B == 4 ? lane * 4 : 0);
+        // scale of step `st`: forward  (row c0 + row_local, columns st*64 + 32 g ..),
+        //                     backward (row st*64 + row_local, columns c0 + 64*(slab_i/2) + 32 g ..)
+        auto fetch = [&](int st) {
+            return BWD ? fetch_scale(p.q, st * BK + row_local, c0 + (slab_i >> 1) * 64 + g * 32)
+                       : fetch_scale(p.q, c0 + row_local, st * BK + g * 32);
+        };
+        float v_cached = -1.0f, sigma = 0.0f, s_lo = 0.0f, s_hi = 0.0f;
+        RawScale r1{0u, 0.0f}, r2{0u, 0.0f};
         if (p.steps_q > 0) {
-            if (!BWD) load_scales(p.q, c0 + row_local, 0, scale);
-            else load_scales(p.q, row_local, c0 + (dw >> 1) * 64, scale);
+            make_scales(p.q, fetch(0), v_cached, sigma, s_lo, s_hi);
+            if (p.steps_q > 1) r1 = fetch(1);
         }
         bool ok = true;
         for (int step = 0; step < total && ok; ++step) {
             const int s = step % p.stages;
             const uint32_t ph = (step / p.stages) & 1;
+            if (step + 2 < p.steps_q) r2 = fetch(step + 2);      // lands two steps before it is needed
             ok = wait(full_tma(s), ph, ctl, 4);
             if (!ok) break;
             if (step < p.steps_q) {
                 uint8_t* st = base + static_cast<size_t>(s) * STAGE;
-                const uint32_t* slab = reinterpret_cast<const uint32_t*>(st + A_BYTES + kBBytes) + dw * (64 * B);
-                float next[4];
-                if (step + 1 < p.steps_q) {     // prefetch the next step's scales before the ALU work
-                    if (!BWD) load_scales(p.q, c0 + row_local, (step + 1) * BK, next);
-                    else load_scales(p.q, (step + 1) * BK + row_local, c0 + (dw >> 1) * 64, next);
-                }
-                dequant_row<B>(slab, lane, cb, scale, st + A_BYTES + b_off, row_sub & 7);
-                if (step + 1 < p.steps_q) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) scale[i] = next[i];
-                }
+                const uint32_t* slab = reinterpret_cast<const uint32_t*>(st + A_BYTES + kBBytes) + slab_i * (64 * B);
+                dequant_group<B>(slab, g, lane, lut, lane_off, s_lo, s_hi, st + A_BYTES + b_off, xr);
                 fence_proxy_async();            // make the generic-proxy stores visible to the tensor core
+                if (step + 1 < p.steps_q) { make_scales(p.q, r1, v_cached, sigma, s_lo, s_hi); r1 = r2; }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(full_b(s));
         }
-        // epilogue: warp reads its quarter of the 128 accumulator lanes, half of the 256 columns
+        // epilogue: warp reads its quarter of the 128 accumulator lanes and 64 of the 256 columns
         if (ok && wait(acc_full, 0, ctl, 5)) {
             tc_fence_after();
-            const int quarter = warp & 3, colhalf = dw >> 2;
+            const int quarter = warp & 3, colq = dw >> 2;
 #pragma unroll 1
             for (int h = 0; h < MH; ++h) {
                 const int m = m0 + h * 128 + quarter * 32 + lane;
 #pragma unroll 1
-                for (int cc = 0; cc < 4; ++cc) {
-                    const int col = colhalf * 128 + cc * 32;
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int col = colq * 64 + cc * 32;
                     uint32_t v[32];
                     tmem_ld32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + h * BN + col, v);
                     tmem_ld_wait();
@@ -409,6 +459,166 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
+}
+
+
+// ------------------------------------------------------------------------------------ rank-r pre-product
+// T = bf16(A F) with a short output width (r <= 128):  forward  T = X L2^T  (F = L2 [r, K], K-major B operand),
+// backward T = dY L1 (F = L1 [N, r], MN-major B operand).  Grid = (row tiles of 128, splits of the
+// contraction).  Each CTA accumulates its part in tensor memory and stores it as an fp32 partial tile;
+// the CTA that arrives last on the tile's counter adds the partial tiles in a fixed order and writes bf16.
+struct PreParams {
+    float* partial;        // [nsplit][M][rp] fp32
+    __nv_bfloat16* T;      // [M][r]
+    int* counters;         // one per row tile, zeroed before the launch
+    int* status;
+    int M, r, rp;          // rp = r rounded up to 64 (MMA N)
+    int steps;             // contraction steps of 64 in total
+    int steps_per_split;
+    int stages;
+};
+
+template <bool BWD>
+__global__ void __launch_bounds__(192, 1)
+tc_lowrank_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const PreParams p) {
+    constexpr int A_BYTES = 16384;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int b_bytes = p.rp * 128;
+    const int stage_bytes = A_BYTES + b_bytes;
+    uint8_t* tail = base + static_cast<size_t>(p.stages) * stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);      // full[8], empty[8], acc_full, drain
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 160);
+    volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* last_s = reinterpret_cast<volatile int*>(tmem_slot + 2);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * 128;
+    const int split = blockIdx.y, nsplit = gridDim.y;
+    const int s_lo = split * p.steps_per_split;
+    const int s_hi = min(p.steps, s_lo + p.steps_per_split);
+    const int total = s_hi - s_lo;
+    const Ctl ctl{abort_s, p.status};
+    const uint32_t tmem_cols = (p.rp <= 64) ? 64u : 128u;
+
+    auto full = [&](int s) { return smem_u32(bars + s); };
+    auto empty = [&](int s) { return smem_u32(bars + 8 + s); };
+    const uint32_t acc_full = smem_u32(bars + 16), drain = smem_u32(bars + 17);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        mbar_init(acc_full, 1);
+        mbar_init(drain, 1);
+        *abort_s = 0;
+        *last_s = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), tmem_cols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int i = 0; i < total; ++i) {
+                const int s = i % p.stages;
+                const uint32_t ph = (i / p.stages) & 1;
+                if (!wait(empty(s), ph ^ 1, ctl, 11)) break;
+                const uint32_t a_dst = smem_u32(base + static_cast<size_t>(s) * stage_bytes), b_dst = a_dst + A_BYTES;
+                const int c = (s_lo + i) * BK;
+                mbar_expect_tx(full(s), A_BYTES + b_bytes);
+                tma_load_2d(a_dst, &tmA, c, m0, full(s));
+                if (!BWD) tma_load_2d(b_dst, &tmB, c, 0, full(s));                       // [rp rows of L2] x 64 columns
+                else for (int t = 0; t < p.rp / 64; ++t) tma_load_2d(b_dst + t * 8192, &tmB, t * 64, c, full(s));  // 64 rows of L1
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((BWD ? 1u : 0u) << 16) |
+                                   (static_cast<uint32_t>(p.rp >> 3) << 17) | (static_cast<uint32_t>(128 >> 4) << 24);
+            bool ok = true;
+            for (int i = 0; i < total && ok; ++i) {
+                const int s = i % p.stages;
+                const uint32_t ph = (i / p.stages) & 1;
+                ok = wait(full(s), ph, ctl, 12);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_src = smem_u32(base + static_cast<size_t>(s) * stage_bytes), b_src = a_src + A_BYTES;
+#pragma unroll
+                for (int k16 = 0; k16 < 4; ++k16) {
+                    const uint64_t adesc = make_desc(a_src + k16 * 32, 16, 1024);
+                    const uint64_t bdesc = BWD ? make_desc(b_src + k16 * 2048, 8192, 1024) : make_desc(b_src + k16 * 32, 16, 1024);
+                    tc_mma(tmem, adesc, bdesc, idesc, (i > 0 || k16 > 0) ? 1u : 0u);
+                }
+                tc_commit(empty(s));
+            }
+            if (ok) tc_commit(acc_full);
+            else {
+                tc_commit(drain);
+                const long long t0 = clock64();
+                while (!mbar_try_wait(drain, 0) && clock64() - t0 < 20000000LL) {}
+            }
+        }
+        __syncwarp();
+    } else {
+        // epilogue warps 2..5: TMEM lane quarter = warp % 4
+        const int quarter = warp & 3;
+        const int m = m0 + quarter * 32 + lane;
+        const bool ok = (total > 0) ? wait(acc_full, 0, ctl, 13) : true;
+        if (ok) {
+            tc_fence_after();
+            for (int col = 0; col < p.rp; col += 32) {
+                uint32_t v[32];
+                if (total > 0) { tmem_ld32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + col, v); tmem_ld_wait(); }
+                else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = 0u;
+                }
+                if (m < p.M) {
+                    float4* dst = reinterpret_cast<float4*>(p.partial + (static_cast<size_t>(split) * p.M + m) * p.rp + col);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                             __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+                }
+            }
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 64) {
+                const int old = atomicAdd(p.counters + blockIdx.x, 1);
+                *last_s = (old == nsplit - 1) ? 1 : 0;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (*last_s) {
+                __threadfence();
+                if (m < p.M) {
+                    for (int col = 0; col < p.r; col += 8) {
+                        float acc[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
+                        for (int z = 0; z < nsplit; ++z) {
+                            const float4* src = reinterpret_cast<const float4*>(p.partial + (static_cast<size_t>(z) * p.M + m) * p.rp + col);
+                            const float4 a = __ldcg(src), b = __ldcg(src + 1);
+                            acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+                            acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+                        }
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const __nv_bfloat162 hh = __floats2bfloat162_rn(acc[2 * e], acc[2 * e + 1]);
+                            w[e] = *reinterpret_cast<const uint32_t*>(&hh);
+                        }
+                        *reinterpret_cast<uint4*>(p.T + static_cast<size_t>(m) * p.r + col) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, tmem_cols);
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -448,7 +658,7 @@ constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA
 template <int B, int MH>
 constexpr int stage_bytes() { return MH * 16384 + kBBytes + 2048 * B; }
 template <int B>
-constexpr int tail_bytes() { return 256 + ((B <= 4) ? (1 << B) * 32 : 256) * 4 + 64; }
+constexpr int tail_bytes() { return 256 + Lut<B>::kBytes + 64; }
 
 template <int B, bool BWD, int MH>
 inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, Params p, cudaStream_t st) {
@@ -473,6 +683,50 @@ inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUten
     return LQLORA_OK;
 }
 
+
+struct PrePlan {
+    int mtiles, nsplit, steps, steps_per_split, rp;
+    size_t counters_bytes, partial_bytes, t_bytes;
+};
+
+inline PrePlan pre_plan(int64_t C, int r, int64_t M) {
+    PrePlan pl;
+    pl.mtiles = static_cast<int>((M + 127) / 128);
+    pl.steps = static_cast<int>((C + BK - 1) / BK);
+    int want = (148 + pl.mtiles - 1) / pl.mtiles;
+    if (want > pl.steps / 2) want = pl.steps / 2;
+    if (want < 1) want = 1;
+    if (want > 32) want = 32;
+    pl.steps_per_split = (pl.steps + want - 1) / want;
+    pl.nsplit = (pl.steps + pl.steps_per_split - 1) / pl.steps_per_split;
+    pl.rp = (r <= 64) ? 64 : 128;
+    pl.counters_bytes = round_up(static_cast<size_t>(pl.mtiles) * 4, 256);
+    pl.partial_bytes = round_up(static_cast<size_t>(pl.nsplit) * M * pl.rp * 4, 256);
+    pl.t_bytes = round_up(static_cast<size_t>(M) * (r > 0 ? r : 1) * 2, 256);
+    return pl;
+}
+
+template <bool BWD>
+inline int launch_pre(const CUtensorMap& tA, const CUtensorMap& tB, PreParams p, int mtiles, int nsplit, cudaStream_t st) {
+    const int stage = 16384 + p.rp * 128;
+    int stages = (kSmemLimit - 1024 - 256) / stage;
+    if (stages > 8) stages = 8;
+    p.stages = stages;
+    const int smem = 1024 + stages * stage + 256;
+    auto kern = tc_lowrank_kernel<BWD>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
+            cudaGetLastError();
+            return LQLORA_ERR_CUDA;
+        }
+        attr_done = true;
+    }
+    kern<<<dim3(mtiles, nsplit), 192, smem, st>>>(tA, tB, p);
+    count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? LQLORA_OK : LQLORA_ERR_CUDA;
+}
+
 template <int B>
 inline int launch_b(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, const Params& p, bool bwd, int mh,
                     cudaStream_t st) {
@@ -493,25 +747,34 @@ inline bool tc_supported(const QView& q, int r, int64_t M, bool backward) {
 }
 
 inline size_t tc_workspace_bytes(int64_t N, int64_t K, int r, int64_t M, bool backward) {
-    (void)N; (void)K; (void)backward;
-    return kStatusBytes + round_up(static_cast<size_t>(M) * (r > 0 ? r : 1) * 2, 256);
+    const tc::PrePlan pl = tc::pre_plan(backward ? N : K, r, M);
+    return kStatusBytes + pl.counters_bytes + pl.t_bytes + (r > 0 ? pl.partial_bytes : 0);
 }
 
 inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, const void* A, int M, void* out, char* ws,
                      bool backward, cudaStream_t st) {
     using namespace tc;
-    __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes);
-    const __nv_bfloat16* a = static_cast<const __nv_bfloat16*>(A);
     const int C = backward ? q.N : q.K;              // contraction length
-    if (r > 0) {
-        if (!backward) lowrank_pre_kernel<<<M, 256, 0, st>>>(a, static_cast<const __nv_bfloat16*>(L2), T, q.K, r, q.K, 1);
-        else lowrank_pre_kernel<<<M, 256, 0, st>>>(a, static_cast<const __nv_bfloat16*>(L1), T, q.N, r, 1, r);
-        count_launch(1);
-    }
+    const PrePlan pl = pre_plan(C, r, M);
+    // workspace: [status][row-tile counters][T bf16][fp32 partial tiles]; status and counters were zeroed by the caller
+    int* counters = reinterpret_cast<int*>(ws + kStatusBytes);
+    __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + pl.counters_bytes);
+    float* partial = reinterpret_cast<float*>(ws + kStatusBytes + pl.counters_bytes + pl.t_bytes);
     const int mh = (M > 128) ? 2 : 1;
     CUtensorMap tA, tA2, tB2;
     if (!make_map(&tA, A, M, C, mh * 128)) return LQLORA_ERR_CUDA;
     if (r > 0) {
+        // rank-r pre-product on the tensor cores: T = X L2^T (forward) or dY L1 (backward)
+        CUtensorMap tPA, tPB;
+        if (!make_map(&tPA, A, M, C, 128)) return LQLORA_ERR_CUDA;
+        const bool okp = backward ? make_map(&tPB, L1, q.N, r, 64) : make_map(&tPB, L2, r, q.K, pl.rp);
+        if (!okp) return LQLORA_ERR_CUDA;
+        PreParams pp;
+        pp.partial = partial; pp.T = T; pp.counters = counters; pp.status = reinterpret_cast<int*>(ws);
+        pp.M = M; pp.r = r; pp.rp = pl.rp; pp.steps = pl.steps; pp.steps_per_split = pl.steps_per_split; pp.stages = 0;
+        const int rc = backward ? launch_pre<true>(tPA, tPB, pp, pl.mtiles, pl.nsplit, st)
+                                : launch_pre<false>(tPA, tPB, pp, pl.mtiles, pl.nsplit, st);
+        if (rc != LQLORA_OK) return rc;
         if (!make_map(&tA2, T, M, r, mh * 128)) return LQLORA_ERR_CUDA;
         const bool okb = backward ? make_map(&tB2, L2, r, q.K, 64) : make_map(&tB2, L1, q.N, r, 256);
         if (!okb) return LQLORA_ERR_CUDA;

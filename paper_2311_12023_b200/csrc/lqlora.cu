@@ -55,9 +55,11 @@ static int run_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, i
     if (rc != LQLORA_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const QView v = make_view(q);
-    if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) return cuda_rc(cudaGetLastError());
+    const bool use_tc = tc_supported(v, r, M, backward);
+    const size_t zero_bytes = kStatusBytes + (use_tc ? tc::pre_plan(backward ? v.N : v.K, r, M).counters_bytes : 0);
+    if (cudaMemsetAsync(ws, 0, zero_bytes, st) != cudaSuccess) return cuda_rc(cudaGetLastError());
     cudaError_t e = cudaSuccess;
-    if (tc_supported(v, r, M, backward)) {
+    if (use_tc) {
         return tc_launch(v, L1, L2, r, A, static_cast<int>(M), out, static_cast<char*>(ws), backward, st);
     }
     switch (v.b0) {
