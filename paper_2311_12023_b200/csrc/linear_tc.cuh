@@ -593,24 +593,45 @@ tc_lowrank_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (*last_s) {
                 __threadfence();
-                if (m < p.M) {
-                    for (int col = 0; col < p.r; col += 8) {
-                        float acc[8];
+                // coalesced reduction of the nsplit partial tiles: thread -> 4 columns, rows strided
+                const int t = threadIdx.x - 64;
+                const int groups = p.rp >> 2;                 // float4 groups per row: 16 or 32
+                const int cg = t % groups, rstep = 128 / groups;
+                const size_t zstride = static_cast<size_t>(p.M) * p.rp;
+                // four rows at a time so that up to 32 loads are in flight per thread
+                for (int rr = t / groups; rr < 128; rr += 4 * rstep) {
+                    float4 acc[4];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
-                        for (int z = 0; z < nsplit; ++z) {
-                            const float4* src = reinterpret_cast<const float4*>(p.partial + (static_cast<size_t>(z) * p.M + m) * p.rp + col);
-                            const float4 a = __ldcg(src), b = __ldcg(src + 1);
-                            acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
-                            acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
-                        }
-                        uint32_t w[4];
+                    for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int z0 = 0; z0 < nsplit; z0 += 8) {
+                        float4 v[4][8];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const __nv_bfloat162 hh = __floats2bfloat162_rn(acc[2 * e], acc[2 * e + 1]);
-                            w[e] = *reinterpret_cast<const uint32_t*>(&hh);
+                        for (int u = 0; u < 4; ++u) {
+                            const int row = m0 + rr + u * rstep;
+                            const float* src = p.partial + static_cast<size_t>(row) * p.rp + cg * 4;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                v[u][i] = (z0 + i < nsplit && row < p.M && rr + u * rstep < 128)
+                                              ? __ldcg(reinterpret_cast<const float4*>(src + (z0 + i) * zstride))
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
                         }
-                        *reinterpret_cast<uint4*>(p.T + static_cast<size_t>(m) * p.r + col) = make_uint4(w[0], w[1], w[2], w[3]);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                acc[u].x += v[u][i].x; acc[u].y += v[u][i].y; acc[u].z += v[u][i].z; acc[u].w += v[u][i].w;
+                            }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int row = m0 + rr + u * rstep;
+                        if (row < p.M && rr + u * rstep < 128 && cg * 4 < p.r) {
+                            const __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[u].x, acc[u].y), h1 = __floats2bfloat162_rn(acc[u].z, acc[u].w);
+                            uint2 o;
+                            o.x = *reinterpret_cast<const uint32_t*>(&h0);
+                            o.y = *reinterpret_cast<const uint32_t*>(&h1);
+                            *reinterpret_cast<uint2*>(p.T + static_cast<size_t>(row) * p.r + cg * 4) = o;
+                        }
                     }
                 }
             }
@@ -693,7 +714,7 @@ inline PrePlan pre_plan(int64_t C, int r, int64_t M) {
     PrePlan pl;
     pl.mtiles = static_cast<int>((M + 127) / 128);
     pl.steps = static_cast<int>((C + BK - 1) / BK);
-    int want = (148 + pl.mtiles - 1) / pl.mtiles;
+    int want = 148 / pl.mtiles;                 // one wave of CTAs
     if (want > pl.steps / 2) want = pl.steps / 2;
     if (want < 1) want = 1;
     if (want > 32) want = 32;
