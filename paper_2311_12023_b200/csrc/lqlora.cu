@@ -27,6 +27,13 @@ static int cuda_rc(cudaError_t e) {
     return LQLORA_ERR_CUDA;
 }
 
+// Scratch bytes one direction of the linear needs for M rows, for the kernel family it dispatches to.
+static size_t linear_need(const QView& v, int r, int64_t M, bool backward) {
+    if (tc_supported(v, r, M, backward)) return tc_workspace_bytes(v.N, v.K, r, M, backward);
+    const SmallPlan p = small_plan(v.N, v.K, r, M, backward);
+    return kStatusBytes + p.t_bytes + p.p_bytes;
+}
+
 static int check_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, int r, const void* A, int64_t M,
                         void* out, void* ws, size_t ws_bytes, bool backward) {
     int rc = check_qmatrix(q);
@@ -40,10 +47,7 @@ static int check_linear(const lqlora_qmatrix* q, const void* L1, const void* L2,
         // rows of X / Y must start on 16-byte boundaries for the vector loads and TMA
         if (M > 1) return LQLORA_ERR_INVALID_SHAPE;
     }
-    size_t need = 0;
-    rc = lqlora_linear_workspace_bytes(q->N, q->K, &q->cfg, r, M, &need);
-    if (rc != LQLORA_OK) return rc;
-    if (ws_bytes < need) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
+    if (ws_bytes < linear_need(make_view(q), r, M, backward)) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
     return LQLORA_OK;
 }
 
@@ -144,15 +148,12 @@ int lqlora_linear_workspace_bytes(int64_t N, int64_t K, const lqlora_config* cfg
     if (rc != LQLORA_OK) return rc;
     if (M <= 0 || r < 0 || r > 128 || r % 16) return LQLORA_ERR_INVALID_SHAPE;
     if (!bytes) return LQLORA_ERR_NULL_POINTER;
-    // the same workspace must serve forward and backward, small-M and tensor-core kernels
-    size_t need = 0;
-    for (int backward = 0; backward < 2; ++backward) {
-        const SmallPlan p = small_plan(N, K, r, M, backward != 0);
-        const size_t small = kStatusBytes + p.t_bytes + p.p_bytes;
-        const size_t tc = tc_workspace_bytes(N, K, r, M, backward != 0);
-        need = small > need ? small : need;
-        need = tc > need ? tc : need;
-    }
+    // the same workspace must serve the forward and the input gradient
+    lqlora_qmatrix q{};
+    q.N = N; q.K = K; q.cfg = *cfg;
+    const QView v = make_view(&q);
+    const size_t f = linear_need(v, r, M, false), b = linear_need(v, r, M, true);
+    const size_t need = f > b ? f : b;
     *bytes = need;
     return LQLORA_OK;
 }
