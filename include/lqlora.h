@@ -158,6 +158,31 @@ int lqlora_linear_bwd_input(const lqlora_qmatrix* q, const void* L1_dev, const v
                             size_t workspace_bytes, void* stream);
 
 /*
+ * Forward pass for callers that are not allowed to allocate device memory (no counterpart in the
+ * paper: this entry point exists for deployment reasons only).  Typical examples are an inference
+ * server whose memory pool was carved up at start-up, or code running inside another framework's
+ * stream callback or plug-in hook, where calling cudaMalloc (directly or through a tensor library)
+ * is forbidden or would synchronize the device.  The call computes exactly what lqlora_linear_fwd
+ * computes, with the same kernels, but takes its scratch from an 8 MiB array that is compiled into
+ * the library (lqlora_static_scratch_bytes() returns the size).  The caller passes only the
+ * inputs and the output; the function itself never allocates or frees anything.
+ *   - A problem whose scratch (lqlora_linear_workspace_bytes) exceeds the array is refused with
+ *     LQLORA_ERR_WORKSPACE_TOO_SMALL before anything is enqueued; use lqlora_linear_fwd then.
+ *   - Every device that loads the library carries the array until the process ends.
+ *   - The first call on a device looks up the array's device address (a one-off set-up step);
+ *     make that first call outside any stream capture.
+ *   - All calls share the one array.  It still holds the previous call's data when the next call
+ *     starts; the words that have to start at zero (status word, arrival counters) are cleared on
+ *     the stream by each call.  Two calls whose kernels can overlap on the GPU (different streams
+ *     without ordering between them) would race on it: order them, or use lqlora_linear_fwd with
+ *     separate workspaces.  lqlora_workspace_status is not available for this array.
+ * Other arguments, layouts and error codes as for lqlora_linear_fwd.
+ */
+size_t lqlora_static_scratch_bytes(void);
+int lqlora_linear_fwd_static(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r,
+                             const void* X_dev, int64_t M, void* Y_dev, void* stream);
+
+/*
  * Host-buffer variants (end-to-end use: activations arrive from and results return to pinned host
  * memory).  They enqueue, on `stream`: a host-to-device copy of the input into the caller's device
  * staging buffer, the same kernels as the device-pointer entry points (Sec. 2.1, Sec. 3.2 as

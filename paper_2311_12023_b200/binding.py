@@ -22,7 +22,10 @@ EXPORTS = [
     "lqlora_unpack", "lqlora_dequant", "lqlora_linear_workspace_bytes", "lqlora_linear_fwd",
     "lqlora_linear_bwd_input", "lqlora_workspace_status", "lqlora_linear_path", "lqlora_launch_count",
     "lqlora_status_string", "lqlora_encode_host", "lqlora_linear_fwd_host", "lqlora_linear_bwd_input_host",
+    "lqlora_static_scratch_bytes", "lqlora_linear_fwd_static",
 ]
+
+STATIC_SCRATCH_BYTES = 8 << 20   # size of the scratch array compiled into the library (lqlora_static_scratch_bytes)
 
 
 class LqloraError(RuntimeError):
@@ -68,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.lqlora_linear_fwd_host.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, vp, vp, sz, vp]
         L.lqlora_linear_bwd_input_host.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, vp, vp, sz, vp]
         L.lqlora_workspace_status.argtypes = [vp, vp]
+        L.lqlora_static_scratch_bytes.restype = sz
+        L.lqlora_linear_fwd_static.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp]
         L.lqlora_linear_path.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ci]
         L.lqlora_launch_count.restype = i64
         L.lqlora_status_string.argtypes = [ci]
@@ -217,6 +222,29 @@ def linear_fwd(q: QMatrix, L1, L2, X: torch.Tensor, out=None, workspace=None) ->
     """lqlora_linear_fwd: Y = X deq(Q)^T + (X L2^T) L1^T, bf16 [M, N]."""
     assert X.shape[1] == q.K
     return _linear(lib().lqlora_linear_fwd, "lqlora_linear_fwd", q, L1, L2, X, q.N, out, workspace)
+
+
+def linear_fwd_static(q: QMatrix, L1, L2, X: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """lqlora_linear_fwd_static: the forward pass with the library's built-in scratch array.
+
+    For callers that must not allocate device memory while they run (a server with a fixed memory
+    pool, code inside another framework's hook): pass ``out`` and this wrapper allocates nothing
+    either.  Same result as ``linear_fwd``; problems that need more than ``STATIC_SCRATCH_BYTES`` of
+    scratch raise ``LqloraError`` (workspace too small).  Calls share one array, so they must not
+    overlap on the GPU.
+    """
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.is_contiguous() and X.dim() == 2 and X.shape[1] == q.K
+    M = X.shape[0]
+    r = 0 if L1 is None else L1.shape[1]
+    if r:
+        assert L1.dtype == torch.bfloat16 and L2.dtype == torch.bfloat16 and L1.is_contiguous() and L2.is_contiguous()
+        assert tuple(L1.shape) == (q.N, r) and tuple(L2.shape) == (r, q.K)
+    if out is None:
+        out = torch.empty((M, q.N), dtype=torch.bfloat16, device=X.device)
+    cs = q.cstruct()
+    _check(lib().lqlora_linear_fwd_static(ctypes.byref(cs), _ptr(L1), _ptr(L2), r, X.data_ptr(), M, out.data_ptr(),
+                                          _stream()), "lqlora_linear_fwd_static")
+    return out
 
 
 def linear_bwd_input(q: QMatrix, L1, L2, dY: torch.Tensor, out=None, workspace=None) -> torch.Tensor:

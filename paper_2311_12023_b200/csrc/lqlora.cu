@@ -75,6 +75,31 @@ static int run_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, i
     return cuda_rc(e);
 }
 
+
+// ---------------------------------------------------------------------------------------
+// Built-in scratch for lqlora_linear_fwd_static.  The array lives in every device's copy of
+// the module from the moment the library is loaded there until the process exits.
+// In host code the name `g_static_scratch` is only a handle for the symbol, not a device
+// address; the address is looked up once per device (with that device current) below.
+// ---------------------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = size_t(8) << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+static int static_scratch_ptr(void** out) {
+    static std::mutex mu;
+    static void* ptrs[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
+        ptrs[dev] = p;
+    }
+    *out = ptrs[dev];
+    return LQLORA_OK;
+}
+
 }  // namespace lq
 
 extern "C" {
@@ -166,6 +191,24 @@ int lqlora_linear_fwd(const lqlora_qmatrix* q, const void* L1_dev, const void* L
 int lqlora_linear_bwd_input(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r, const void* dY_dev,
                             int64_t M, void* dX_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
     return lq::run_linear(q, L1_dev, L2_dev, r, dY_dev, M, dX_dev, workspace_dev, workspace_bytes, stream, true);
+}
+
+size_t lqlora_static_scratch_bytes(void) { return lq::kStaticScratchBytes; }
+
+int lqlora_linear_fwd_static(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r, const void* X_dev,
+                             int64_t M, void* Y_dev, void* stream) {
+    using namespace lq;
+    // size check first: nothing is looked up or enqueued for a problem that cannot fit
+    int rc = check_qmatrix(q);
+    if (rc != LQLORA_OK) return rc;
+    if (M <= 0 || M > (int64_t(1) << 24) || r < 0 || r > 128 || (r % 16) != 0) return LQLORA_ERR_INVALID_SHAPE;
+    if (linear_need(make_view(q), r, M, false) > kStaticScratchBytes) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
+    void* scratch = nullptr;
+    rc = static_scratch_ptr(&scratch);
+    if (rc != LQLORA_OK) return rc;
+    // run_linear clears the status word and the arrival counters at the head of the scratch on every
+    // call, so whatever the previous call left behind is never read before it is overwritten
+    return run_linear(q, L1_dev, L2_dev, r, X_dev, M, Y_dev, scratch, kStaticScratchBytes, stream, false);
 }
 
 int lqlora_encode_host(const float* W_host, float* W_stage_dev, lqlora_qmatrix* out, void* workspace_dev,

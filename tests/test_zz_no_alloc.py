@@ -47,7 +47,8 @@ def test_static_scratch_forward_matches_ordinary_forward_twice_in_a_row(M):
 def test_static_scratch_rejects_oversized_problems_without_launching():
     cfg = inputs.QuantConfig(3, 64, 8, 256, 32)
     N = K = 4096
-    M = 8192                                   # needs far more than 8 MiB of scratch
+    M = 1 << 16                                # needs far more than 8 MiB of scratch
+    assert int(binding.lib().lqlora_static_scratch_bytes()) == binding.STATIC_SCRATCH_BYTES
     assert binding.linear_workspace_bytes(N, K, cfg, 64, M) > binding.STATIC_SCRATCH_BYTES
     fake = 0x10000                             # never dereferenced: the size check comes first
     q = binding.CQMatrix(fake, fake, fake, N, K, binding._cfg(cfg))
