@@ -92,9 +92,7 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
         const float s = (j < 16) ? s_lo : s_hi;
         uint32_t c = zero_code;
         if (s != 0.0f) c = nearest_code<B>(__fdiv_rn(u[j], s), th8);
-        const int p = B * j, wi = p >> 5, sh = p & 31;
-        words[wi] |= c << sh;
-        if (sh + B > 32) words[wi + 1] |= c >> (32 - sh);
+        deposit_code<B>(words, j, c);
     }
     uint32_t* dst = codes + slab_word_base(row, k0 >> 6, K >> 6, B);
     const int g = (k0 >> 5) & 1;

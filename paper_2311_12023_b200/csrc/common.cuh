@@ -80,13 +80,41 @@ __host__ __device__ inline int slab_word_offset(int row, int g, int w, int b0) {
     return (g * b0 + w) * 32 + (row & 31);
 }
 
-// Code j (0..31) of a group whose b0 words are in `w`: bits [b0*j, b0*j + b0) of the bit string.
+// Bit layout of the 32 codes c[0..31] of one (row, 32-column group) inside its b0 words.  Every
+// word is a string of eight 4-bit fields ("selectors") so that a byte-permute instruction can use
+// it directly as a table index for eight weights:
+//   b0 = 4: word w holds codes 8w .. 8w+7, code 8w+i in field i (bits [4i, 4i+4));
+//   b0 = 3: word w (0..2) holds code 8w+i in the low three bits of field i; the top bit of field i
+//           of word w is bit w of code 24+i;
+//   b0 = 2: word w (0..1) holds code 16w+i in the low two bits of field i and code 16w+8+i in its
+//           high two bits;
+//   b0 = 8: word w holds codes 4w .. 4w+3, one per byte.
 template <int B>
-__device__ __forceinline__ uint32_t extract_code(const uint32_t* w, int j) {
-    const int p = B * j;
-    const int wi = p >> 5, sh = p & 31;
-    if (sh + B <= 32) return (w[wi] >> sh) & ((1u << B) - 1u);
-    return __funnelshift_r(w[wi], w[wi + 1], sh) & ((1u << B) - 1u);
+__host__ __device__ __forceinline__ void deposit_code(uint32_t* w, int j, uint32_t c) {
+    if constexpr (B == 4) w[j >> 3] |= c << (4 * (j & 7));
+    else if constexpr (B == 8) w[j >> 2] |= c << (8 * (j & 3));
+    else if constexpr (B == 2) w[j >> 4] |= c << (4 * (j & 7) + 2 * ((j >> 3) & 1));
+    else {
+        if (j < 24) w[j >> 3] |= c << (4 * (j & 7));
+        else {
+            const int i = j - 24;
+            w[0] |= (c & 1u) << (4 * i + 3);
+            w[1] |= ((c >> 1) & 1u) << (4 * i + 3);
+            w[2] |= ((c >> 2) & 1u) << (4 * i + 3);
+        }
+    }
+}
+// Code j (0..31) of a group whose b0 words are in `w`.
+template <int B>
+__host__ __device__ __forceinline__ uint32_t extract_code(const uint32_t* w, int j) {
+    if constexpr (B == 4) return (w[j >> 3] >> (4 * (j & 7))) & 15u;
+    else if constexpr (B == 8) return (w[j >> 2] >> (8 * (j & 3))) & 255u;
+    else if constexpr (B == 2) return (w[j >> 4] >> (4 * (j & 7) + 2 * ((j >> 3) & 1))) & 3u;
+    else {
+        if (j < 24) return (w[j >> 3] >> (4 * (j & 7))) & 7u;
+        const int sh = 4 * (j - 24) + 3;
+        return ((w[0] >> sh) & 1u) | (((w[1] >> sh) & 1u) << 1) | (((w[2] >> sh) & 1u) << 2);
+    }
 }
 
 // s~ = fl32(float(s^) * fl32(v / 127))

@@ -149,80 +149,96 @@ __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, const Ctl& c
 }
 
 // ------------------------------------------------------------------------------------ dequantization
-// Look-up tables in shared memory.  For 2- and 3-bit codes a table entry holds the fp32 code-book
-// values of TWO neighbouring codes (index = both codes, 2*b0 bits) and is fetched with one 64-bit
-// load; for 4- and 8-bit codes an entry is one fp32 value.  Entries are replicated per lane
-// (16 copies of the 8-byte entries, 32 copies of the 4-byte entries of the 4-bit table) so that
-// the loads of a warp never conflict; the 8-bit table (1 KB) is not replicated.
-template <int B> struct Lut {
-    static constexpr bool kPair = (B <= 3);
-    static constexpr int kIdxBits = kPair ? 2 * B : B;
-    static constexpr int kShift = (B <= 4) ? 7 : 2;                 // log2(bytes between consecutive entries)
-    static constexpr int kBytes = (1 << kIdxBits) << kShift;
-    static constexpr uint32_t kMask = ((1u << kIdxBits) - 1u) << kShift;
-};
-
-template <int B>
-__device__ __forceinline__ void fill_lut(uint8_t* lut, int tid, int nthreads) {
-    const float* cb = c_codebook[bits_index(B)];
-    if constexpr (Lut<B>::kPair) {
-        float2* t = reinterpret_cast<float2*>(lut);
-        for (int i = tid; i < (1 << (2 * B)) * 16; i += nthreads) {
-            const int idx = i >> 4;
-            t[i] = make_float2(cb[idx & ((1 << B) - 1)], cb[idx >> B]);
-        }
-    } else if constexpr (B == 4) {
-        float* t = reinterpret_cast<float*>(lut);
-        for (int i = tid; i < 16 * 32; i += nthreads) t[i] = cb[i >> 5];
-    } else {
-        float* t = reinterpret_cast<float*>(lut);
-        for (int i = tid; i < 256; i += nthreads) t[i] = cb[i];
-    }
+// The 2^b0 products fl32(q~[c] * s~) of one block, rounded to bf16, are kept in registers as a
+// byte table: lo[] holds the low bytes, hi[] the high bytes, four entries per register.  One
+// byte-permute with a selector word (four 4-bit table indices) then fetches four low bytes, a
+// second one the four high bytes, and two more interleave them into two bf16 pairs.  The results
+// are the same bits as rounding each fp32 product on its own.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
 }
 
-// Byte offset into the table of the entry whose index starts at bit `pos` of the little-endian bit
-// string w[0..B-1] (w[B] = 0), already OR-ed with the lane's replica offset.
-template <int B>
-__device__ __forceinline__ uint32_t lut_offset(const uint32_t (&w)[B + 1], int pos, uint32_t lane_off) {
-    constexpr int S = Lut<B>::kShift;
-    uint32_t x;
-    if (pos < S) x = w[0] << (S - pos);
-    else {
-        const int q = pos - S, wi = q >> 5, sh = q & 31;
-        x = (sh + Lut<B>::kIdxBits + S <= 32) ? (w[wi] >> sh) : __funnelshift_r(w[wi], w[wi + 1], sh);
+template <int B> struct BlockTable {
+    static constexpr int kRegs = (B == 2) ? 1 : (B == 3) ? 2 : 4;
+    uint32_t lo[kRegs], hi[kRegs];
+    __device__ __forceinline__ void build(float s) {
+        const float* cb = c_codebook[bits_index(B)];
+        uint32_t e[(1 << B) / 2];
+#pragma unroll
+        for (int i = 0; i < (1 << B) / 2; ++i) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(cb[2 * i], s), __fmul_rn(cb[2 * i + 1], s));
+            e[i] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+#pragma unroll
+        for (int j = 0; j < kRegs; ++j) {
+            lo[j] = prmt(e[2 * j], e[2 * j + 1], 0x6420u);
+            hi[j] = prmt(e[2 * j], e[2 * j + 1], 0x7531u);
+        }
     }
-    return (x & Lut<B>::kMask) | lane_off;
+    // four weights from the four indices in the low 16 bits of `sel` (sel2: second-level selector, 4-bit codes only)
+    __device__ __forceinline__ void lookup4(uint32_t sel, uint32_t sel2, uint32_t& out0, uint32_t& out1) const {
+        uint32_t l, h;
+        if constexpr (B == 2) { l = prmt(lo[0], 0u, sel); h = prmt(hi[0], 0u, sel); }
+        else if constexpr (B == 3) { l = prmt(lo[0], lo[1], sel); h = prmt(hi[0], hi[1], sel); }
+        else {
+            l = prmt(prmt(lo[0], lo[1], sel), prmt(lo[2], lo[3], sel), sel2);
+            h = prmt(prmt(hi[0], hi[1], sel), prmt(hi[2], hi[3], sel), sel2);
+        }
+        out0 = prmt(l, h, 0x5140u);
+        out1 = prmt(l, h, 0x7362u);
+    }
+};
+
+// Selector word (eight 4-bit indices) of chunk c (columns 8c .. 8c+7 of the group) from the group's words.
+template <int B>
+__device__ __forceinline__ uint32_t chunk_selector(const uint32_t (&w)[B], int c) {
+    if constexpr (B == 4) return w[c];
+    else if constexpr (B == 2) return (c & 1) ? ((w[c >> 1] >> 2) & 0x33333333u) : (w[c >> 1] & 0x33333333u);
+    else {
+        if (c < 3) return w[c] & 0x77777777u;
+        return ((w[0] >> 3) & 0x11111111u) | ((w[1] >> 2) & 0x22222222u) | ((w[2] >> 1) & 0x44444444u);
+    }
 }
 
 // One thread dequantizes the 32 consecutive weights of one (row, group) -- b0 words of the slab --
 // and writes them as four 16-byte chunks of the row's 128 bytes; `dst` is the row start, `xr` is
 // (row % 8) * 16, chunk c of the row lives at byte offset (c * 16) ^ xr.
 template <int B>
-__device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ slab_words, int g, int lane, const uint8_t* __restrict__ lut,
-                                              uint32_t lane_off, float s_lo, float s_hi, uint8_t* __restrict__ dst, uint32_t xr) {
-    uint32_t w[B + 1];
+__device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ slab_words, int g, int lane, const float* __restrict__ lut8,
+                                              float s_lo, float s_hi, bool two_scales, uint8_t* __restrict__ dst, uint32_t xr) {
+    uint32_t w[B];
 #pragma unroll
     for (int i = 0; i < B; ++i) w[i] = slab_words[(g * B + i) * 32 + lane];
-    w[B] = 0u;
+    if constexpr (B == 8) {
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        const float s = (c < 2) ? s_lo : s_hi;
-        uint32_t packed[4];
+        for (int c = 0; c < 4; ++c) {
+            const float s = (c < 2) ? s_lo : s_hi;
+            uint32_t packed[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int j = c * 8 + e * 2;           // first code of the pair
-            float q0, q1;
-            if constexpr (Lut<B>::kPair) {
-                const float2 qq = *reinterpret_cast<const float2*>(lut + lut_offset<B>(w, B * j, lane_off));
-                q0 = qq.x; q1 = qq.y;
-            } else {
-                q0 = *reinterpret_cast<const float*>(lut + lut_offset<B>(w, B * j, lane_off));
-                q1 = *reinterpret_cast<const float*>(lut + lut_offset<B>(w, B * (j + 1), lane_off));
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t ww = w[2 * c + (e >> 1)] >> (16 * (e & 1));
+                const float q0 = lut8[ww & 255u], q1 = lut8[(ww >> 8) & 255u];
+                const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(q0, s), __fmul_rn(q1, s));
+                packed[e] = *reinterpret_cast<const uint32_t*>(&h);
             }
-            const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(q0, s), __fmul_rn(q1, s));
-            packed[e] = *reinterpret_cast<const uint32_t*>(&h);
+            *reinterpret_cast<uint4*>(dst + ((((g * 4 + c) << 4)) ^ xr)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
         }
-        *reinterpret_cast<uint4*>(dst + ((((g * 4 + c) << 4)) ^ xr)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    } else {
+        BlockTable<B> tab;
+        tab.build(s_lo);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (c == 2 && two_scales) tab.build(s_hi);
+            const uint32_t sel = chunk_selector<B>(w, c);
+            uint32_t selA = sel, selB = 0u;
+            if constexpr (B == 4) { selA = sel & 0x77777777u; selB = ((sel >> 1) & 0x44444444u) | 0x32103210u; }
+            uint32_t o[4];
+            tab.lookup4(selA, selB, o[0], o[1]);
+            tab.lookup4(selA >> 16, selB >> 16, o[2], o[3]);
+            *reinterpret_cast<uint4*>(dst + ((((g * 4 + c) << 4)) ^ xr)) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
     }
 }
 
@@ -233,8 +249,8 @@ __device__ __forceinline__ RawScale fetch_scale(const QView& q, int row, int k) 
     RawScale r{0u, 0.0f};
     if (row < q.N && k < q.K) {
         const long long blk = static_cast<long long>(row) * q.KB + (k >> q.logB0);
-        r.sc = (q.B0 == 16) ? static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(q.sc + blk)) : static_cast<uint32_t>(q.sc[blk]);
-        r.v = q.v[blk >> q.logB1];
+        r.sc = (q.B0 == 16) ? static_cast<uint32_t>(__ldg(reinterpret_cast<const uint16_t*>(q.sc + blk))) : static_cast<uint32_t>(__ldg(q.sc + blk));
+        r.v = __ldg(q.v + (blk >> q.logB1));
     }
     return r;
 }
@@ -246,22 +262,30 @@ __device__ __forceinline__ void make_scales(const QView& q, const RawScale& r, f
 }
 
 // ------------------------------------------------------------------------------------ kernel
+// Shared memory: [activation ring: SA x A_BYTES][weight ring: 2 x 32 KB][packed ring: SA x 2048*b0]
+// [barriers][8-bit look-up table].  The activation / packed-code ring runs several steps ahead of
+// the tensor core (it hides the latency of global memory); the dequantized weight ring needs two
+// stages only (one being read by the tensor core, one being written).
+constexpr int kBStages = 2;
+
 template <int B, bool BWD, int MH>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA2,
                  const __grid_constant__ CUtensorMap tmB2, const Params p) {
     constexpr int A_BYTES = MH * 128 * 128;
     constexpr int P_BYTES = 2048 * B;
-    constexpr int STAGE = A_BYTES + kBBytes + P_BYTES;
-    constexpr int LUT_BYTES = Lut<B>::kBytes;
     constexpr uint32_t TMEM_COLS = MH * BN;
+    const int SA = p.stages;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    uint8_t* tail = base + static_cast<size_t>(p.stages) * STAGE;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);            // full_tma[8], full_b[8], empty[8], acc_full, drain
-    uint8_t* lut = tail + 256;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 256 + LUT_BYTES);
+    uint8_t* a_ring = base;
+    uint8_t* b_ring = a_ring + static_cast<size_t>(SA) * A_BYTES;
+    uint8_t* p_ring = b_ring + kBStages * kBBytes;
+    uint8_t* tail = p_ring + static_cast<size_t>(SA) * P_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);   // full_a[8], empty_a[8], full_b[2], empty_b[2], acc_full, drain
+    float* lut8 = reinterpret_cast<float*>(tail + 256);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 256 + (B == 8 ? 1024 : 0));
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -270,19 +294,23 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int total = p.steps_q + p.steps_d;
     const Ctl ctl{abort_s, p.status};
 
-    auto full_tma = [&](int s) { return smem_u32(bars + s); };
-    auto full_b = [&](int s) { return smem_u32(bars + 8 + s); };
-    auto empty = [&](int s) { return smem_u32(bars + 16 + s); };
-    const uint32_t acc_full = smem_u32(bars + 24), drain = smem_u32(bars + 25);
+    auto full_a = [&](int s) { return smem_u32(bars + s); };
+    auto empty_a = [&](int s) { return smem_u32(bars + 8 + s); };
+    auto full_b = [&](int s) { return smem_u32(bars + 16 + s); };
+    auto empty_b = [&](int s) { return smem_u32(bars + 18 + s); };
+    const uint32_t acc_full = smem_u32(bars + 20), drain = smem_u32(bars + 21);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) { mbar_init(full_tma(s), 1); mbar_init(full_b(s), kDeqWarps); mbar_init(empty(s), 1); }
+        for (int s = 0; s < SA; ++s) { mbar_init(full_a(s), 1); mbar_init(empty_a(s), 1); }
+        for (int s = 0; s < kBStages; ++s) { mbar_init(full_b(s), kDeqWarps); mbar_init(empty_b(s), 1); }
         mbar_init(acc_full, 1);
         mbar_init(drain, 1);
         *abort_s = 0;
         fence_barrier_init();
     }
-    fill_lut<B>(lut, threadIdx.x, kThreads);
+    if constexpr (B == 8) {
+        for (int i = threadIdx.x; i < 256; i += kThreads) lut8[i] = c_codebook[3][i];
+    }
     if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), TMEM_COLS); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
@@ -290,60 +318,47 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t tmem = *tmem_slot;
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ producer
+        // ------------------------------------------------------------------ producer: activations + packed codes
         if (lane == 0) {
+            const uint8_t* codes = reinterpret_cast<const uint8_t*>(p.q.codes);
             for (int step = 0; step < total; ++step) {
-                const int s = step % p.stages;
-                const uint32_t ph = (step / p.stages) & 1;
-                if (!wait(empty(s), ph ^ 1, ctl, 1)) break;
-                uint8_t* st = base + static_cast<size_t>(s) * STAGE;
-                const uint32_t a_dst = smem_u32(st), b_dst = a_dst + A_BYTES, p_dst = b_dst + kBBytes;
+                const int s = step % SA;
+                const uint32_t ph = (step / SA) & 1;
+                if (!wait(empty_a(s), ph ^ 1, ctl, 1)) break;
+                const uint32_t a_dst = smem_u32(a_ring + static_cast<size_t>(s) * A_BYTES);
+                const uint32_t p_dst = smem_u32(p_ring + static_cast<size_t>(s) * P_BYTES);
                 if (step < p.steps_q) {
-                    const uint8_t* codes = reinterpret_cast<const uint8_t*>(p.q.codes);
-                    uint32_t bytes = A_BYTES;
                     if (!BWD) {
                         int nt_have = 0;
                         for (int t = 0; t < 2; ++t) if ((c0 >> 7) + t < p.q.ntiles) ++nt_have;
-                        bytes += nt_have * 1024 * B;
-                        mbar_expect_tx(full_tma(s), bytes);
-                        tma_load_2d(a_dst, &tmA, step * BK, m0, full_tma(s));
+                        mbar_expect_tx(full_a(s), A_BYTES + nt_have * 1024 * B);
+                        tma_load_2d(a_dst, &tmA, step * BK, m0, full_a(s));
                         for (int t = 0; t < nt_have; ++t) {
                             const size_t tile = static_cast<size_t>((c0 >> 7) + t) * p.q.ktiles + step;
-                            bulk_load(p_dst + t * 1024 * B, codes + tile * (1024 * B), 1024 * B, full_tma(s));
+                            bulk_load(p_dst + t * 1024 * B, codes + tile * (1024 * B), 1024 * B, full_a(s));
                         }
                     } else {
                         const int nn0 = step * BK;
                         int kt_have = 0;
                         for (int t = 0; t < 4; ++t) if ((c0 >> 6) + t < p.q.ktiles) ++kt_have;
-                        bytes += kt_have * 512 * B;
-                        mbar_expect_tx(full_tma(s), bytes);
-                        tma_load_2d(a_dst, &tmA, nn0, m0, full_tma(s));
+                        mbar_expect_tx(full_a(s), A_BYTES + kt_have * 512 * B);
+                        tma_load_2d(a_dst, &tmA, nn0, m0, full_a(s));
                         for (int t = 0; t < kt_have; ++t) {
                             const size_t tile = static_cast<size_t>(nn0 >> 7) * p.q.ktiles + (c0 >> 6) + t;
                             bulk_load(p_dst + t * 512 * B, codes + tile * (1024 * B) + ((nn0 >> 6) & 1) * (512 * B), 512 * B,
-                                      full_tma(s));
+                                      full_a(s));
                         }
                     }
                 } else {
-                    const int d = step - p.steps_q;
-                    if (!BWD) {
-                        mbar_expect_tx(full_tma(s), A_BYTES + kBBytes);
-                        tma_load_2d(a_dst, &tmA2, d * BK, m0, full_tma(s));
-                        tma_load_2d(b_dst, &tmB2, d * BK, c0, full_tma(s));
-                    } else {
-                        int kt_have = 0;
-                        for (int t = 0; t < 4; ++t) if (c0 + t * 64 < p.out_cols) ++kt_have;
-                        mbar_expect_tx(full_tma(s), A_BYTES + kt_have * 8192);
-                        tma_load_2d(a_dst, &tmA2, d * BK, m0, full_tma(s));
-                        for (int t = 0; t < kt_have; ++t) tma_load_2d(b_dst + t * 8192, &tmB2, c0 + t * 64, d * BK, full_tma(s));
-                    }
+                    mbar_expect_tx(full_a(s), A_BYTES);
+                    tma_load_2d(a_dst, &tmA2, (step - p.steps_q) * BK, m0, full_a(s));
                 }
             }
             if (*abort_s) {
                 // let copies that are still in flight land before the CTA exits (bounded)
-                for (int s = 0; s < p.stages; ++s) {
+                for (int s = 0; s < SA; ++s) {
                     const long long t0 = clock64();
-                    while (!mbar_try_wait(full_tma(s), 0) && !mbar_try_wait(full_tma(s), 1) && clock64() - t0 < 20000000LL) {}
+                    while (!mbar_try_wait(full_a(s), 0) && !mbar_try_wait(full_a(s), 1) && clock64() - t0 < 20000000LL) {}
                 }
             }
         }
@@ -355,12 +370,12 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                        (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(128 >> 4) << 24);
             bool ok = true;
             for (int step = 0; step < total && ok; ++step) {
-                const int s = step % p.stages;
-                const uint32_t ph = (step / p.stages) & 1;
-                ok = wait(full_tma(s), ph, ctl, 2) && wait(full_b(s), ph, ctl, 3);
+                const int sa = step % SA, sb = step % kBStages;
+                ok = wait(full_a(sa), (step / SA) & 1, ctl, 2) && wait(full_b(sb), (step / kBStages) & 1, ctl, 3);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t a_src = smem_u32(base + static_cast<size_t>(s) * STAGE), b_src = a_src + A_BYTES;
+                const uint32_t a_src = smem_u32(a_ring + static_cast<size_t>(sa) * A_BYTES);
+                const uint32_t b_src = smem_u32(b_ring + static_cast<size_t>(sb) * kBBytes);
 #pragma unroll
                 for (int h = 0; h < MH; ++h) {
 #pragma unroll
@@ -371,7 +386,8 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         tc_mma(tmem + h * BN, adesc, bdesc, idesc, (step > 0 || k16 > 0) ? 1u : 0u);
                     }
                 }
-                tc_commit(empty(s));
+                tc_commit(empty_a(sa));
+                tc_commit(empty_b(sb));
             }
             if (ok) {
                 tc_commit(acc_full);
@@ -393,35 +409,57 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (!BWD) { row_local = slab_i * 32 + lane; b_off = row_local * 128; }
         else { row_local = (slab_i & 1) * 32 + lane; b_off = (slab_i >> 1) * 8192 + row_local * 128; }
         const uint32_t xr = (row_local & 7) << 4;
-        const uint32_t lane_off = Lut<B>::kPair ? (lane & 15) * 8 : (B == 4 ? lane * 4 : 0);
+        const bool two_scales = (p.q.B0 == 16);
         // scale of step `st`: forward  (row c0 + row_local, columns st*64 + 32 g ..),
         //                     backward (row st*64 + row_local, columns c0 + 64*(slab_i/2) + 32 g ..)
         auto fetch = [&](int st) {
             return BWD ? fetch_scale(p.q, st * BK + row_local, c0 + (slab_i >> 1) * 64 + g * 32)
                        : fetch_scale(p.q, c0 + row_local, st * BK + g * 32);
         };
+        // the raw scale data are fetched four steps before they are needed
         float v_cached = -1.0f, sigma = 0.0f, s_lo = 0.0f, s_hi = 0.0f;
-        RawScale r1{0u, 0.0f}, r2{0u, 0.0f};
-        if (p.steps_q > 0) {
-            make_scales(p.q, fetch(0), v_cached, sigma, s_lo, s_hi);
-            if (p.steps_q > 1) r1 = fetch(1);
-        }
+        RawScale r0{0u, 0.0f}, r1 = r0, r2 = r0, r3 = r0;
+        if (p.steps_q > 0) r0 = fetch(0);
+        if (p.steps_q > 1) r1 = fetch(1);
+        if (p.steps_q > 2) r2 = fetch(2);
+        if (p.steps_q > 3) r3 = fetch(3);
         bool ok = true;
         for (int step = 0; step < total && ok; ++step) {
-            const int s = step % p.stages;
-            const uint32_t ph = (step / p.stages) & 1;
-            if (step + 2 < p.steps_q) r2 = fetch(step + 2);      // lands two steps before it is needed
-            ok = wait(full_tma(s), ph, ctl, 4);
+            const int sa = step % SA, sb = step % kBStages;
+            RawScale r4{0u, 0.0f};
+            if (step + 4 < p.steps_q) r4 = fetch(step + 4);
+            ok = wait(empty_b(sb), ((step / kBStages) & 1) ^ 1, ctl, 6);
             if (!ok) break;
+            uint8_t* b_dst = b_ring + static_cast<size_t>(sb) * kBBytes;
             if (step < p.steps_q) {
-                uint8_t* st = base + static_cast<size_t>(s) * STAGE;
-                const uint32_t* slab = reinterpret_cast<const uint32_t*>(st + A_BYTES + kBBytes) + slab_i * (64 * B);
-                dequant_group<B>(slab, g, lane, lut, lane_off, s_lo, s_hi, st + A_BYTES + b_off, xr);
+                make_scales(p.q, r0, v_cached, sigma, s_lo, s_hi);
+                r0 = r1; r1 = r2; r2 = r3; r3 = r4;
+                ok = wait(full_a(sa), (step / SA) & 1, ctl, 4);
+                if (!ok) break;
+                const uint32_t* slab = reinterpret_cast<const uint32_t*>(p_ring + static_cast<size_t>(sa) * P_BYTES) + slab_i * (64 * B);
+                dequant_group<B>(slab, g, lane, lut8, s_lo, s_hi, two_scales, b_dst + b_off, xr);
                 fence_proxy_async();            // make the generic-proxy stores visible to the tensor core
-                if (step + 1 < p.steps_q) { make_scales(p.q, r1, v_cached, sigma, s_lo, s_hi); r1 = r2; }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full_b(sb));
+            } else if (dw == 0) {
+                // rank-r step: the second operand ([L1 | ..] rows or L2 rows) comes by TMA into the weight ring
+                if (lane == 0) {
+                    const int d = step - p.steps_q;
+                    const uint32_t dst = smem_u32(b_dst);
+                    if (!BWD) {
+                        mbar_expect_tx(full_b(sb), kBBytes);
+                        tma_load_2d(dst, &tmB2, d * BK, c0, full_b(sb));
+                    } else {
+                        int kt_have = 0;
+                        for (int t = 0; t < 4; ++t) if (c0 + t * 64 < p.out_cols) ++kt_have;
+                        mbar_expect_tx(full_b(sb), kt_have * 8192);
+                        for (int t = 0; t < kt_have; ++t) tma_load_2d(dst + t * 8192, &tmB2, c0 + t * 64, d * BK, full_b(sb));
+                    }
+                }
+                __syncwarp();
+            } else {
+                if (lane == 0) mbar_arrive(full_b(sb));
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(full_b(s));
         }
         // epilogue: warp reads its quarter of the 128 accumulator lanes and 64 of the 256 columns
         if (ok && wait(acc_full, 0, ctl, 5)) {
@@ -677,17 +715,18 @@ inline bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t 
 constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA
 
 template <int B, int MH>
-constexpr int stage_bytes() { return MH * 16384 + kBBytes + 2048 * B; }
+constexpr int stage_bytes() { return MH * 16384 + 2048 * B; }        // one stage of the activation + packed-code ring
 template <int B>
-constexpr int tail_bytes() { return 256 + Lut<B>::kBytes + 64; }
+constexpr int tail_bytes() { return 256 + (B == 8 ? 1024 : 0) + 64; }
+constexpr int kFixedBytes = 1024 + kBStages * kBBytes;               // alignment slack + dequantized weight ring
 
 template <int B, bool BWD, int MH>
 inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, Params p, cudaStream_t st) {
-    int stages = (kSmemLimit - 1024 - tail_bytes<B>()) / stage_bytes<B, MH>();
+    int stages = (kSmemLimit - kFixedBytes - tail_bytes<B>()) / stage_bytes<B, MH>();
     if (stages > 8) stages = 8;
     if (stages < 2) return LQLORA_ERR_UNSUPPORTED;
     p.stages = stages;
-    const int smem = 1024 + stages * stage_bytes<B, MH>() + tail_bytes<B>();
+    const int smem = kFixedBytes + stages * stage_bytes<B, MH>() + tail_bytes<B>();
     auto kern = tc_linear_kernel<B, BWD, MH>;
     static bool attr_done = false;
     if (!attr_done) {
