@@ -202,15 +202,17 @@ __device__ __forceinline__ uint32_t chunk_selector(const uint32_t (&w)[B], int c
     }
 }
 
-// One thread dequantizes the 32 consecutive weights of one (row, group) -- b0 words of the slab --
-// and writes them as four 16-byte chunks of the row's 128 bytes; `dst` is the row start, `xr` is
-// (row % 8) * 16, chunk c of the row lives at byte offset (c * 16) ^ xr.
+// One thread dequantizes the 32 consecutive weights of one (row, group) -- b0 words of the slab,
+// `words` pointing at the thread's first word, the others 32 words apart -- and writes them as four
+// 16-byte chunks of the row's 128 bytes; `dst` is the row start, `goff` the byte offset of the group
+// in the row (0 or 64), `xr` is (row % 8) * 16; a chunk at byte offset o of the row lives at o ^ xr.
 template <int B>
-__device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ slab_words, int g, int lane, const float* __restrict__ lut8,
-                                              float s_lo, float s_hi, bool two_scales, uint8_t* __restrict__ dst, uint32_t xr) {
+__device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ words, float s_lo, float s_hi, bool two_scales,
+                                              uint8_t* __restrict__ dst, uint32_t goff, uint32_t xr, const float* __restrict__ lut8) {
     uint32_t w[B];
 #pragma unroll
-    for (int i = 0; i < B; ++i) w[i] = slab_words[(g * B + i) * 32 + lane];
+    for (int i = 0; i < B; ++i) w[i] = words[i * 32];
+    const uint32_t x = (goff ^ xr);          // chunk c sits at this offset with bits 4, 5 flipped by c
     if constexpr (B == 8) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -223,7 +225,7 @@ __device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ slab_
                 const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(q0, s), __fmul_rn(q1, s));
                 packed[e] = *reinterpret_cast<const uint32_t*>(&h);
             }
-            *reinterpret_cast<uint4*>(dst + ((((g * 4 + c) << 4)) ^ xr)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            *reinterpret_cast<uint4*>(dst + (x ^ (c << 4))) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
         }
     } else {
         BlockTable<B> tab;
@@ -237,7 +239,7 @@ __device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ slab_
             uint32_t o[4];
             tab.lookup4(selA, selB, o[0], o[1]);
             tab.lookup4(selA >> 16, selB >> 16, o[2], o[3]);
-            *reinterpret_cast<uint4*>(dst + ((((g * 4 + c) << 4)) ^ xr)) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(dst + (x ^ (c << 4))) = make_uint4(o[0], o[1], o[2], o[3]);
         }
     }
 }
@@ -245,15 +247,6 @@ __device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ slab_
 // Raw scale data of the 32 weights (row, k .. k+31): the one or two 8-bit scale codes and the
 // second-level scale of their group (B1 >= 16 blocks, so both codes share it).
 struct RawScale { uint32_t sc; float v; };
-__device__ __forceinline__ RawScale fetch_scale(const QView& q, int row, int k) {
-    RawScale r{0u, 0.0f};
-    if (row < q.N && k < q.K) {
-        const long long blk = static_cast<long long>(row) * q.KB + (k >> q.logB0);
-        r.sc = (q.B0 == 16) ? static_cast<uint32_t>(__ldg(reinterpret_cast<const uint16_t*>(q.sc + blk))) : static_cast<uint32_t>(__ldg(q.sc + blk));
-        r.v = __ldg(q.v + (blk >> q.logB1));
-    }
-    return r;
-}
 // s~ = fl32(float(s^) * fl32(v / 127)); the quotient is recomputed only when v changes.
 __device__ __forceinline__ void make_scales(const QView& q, const RawScale& r, float& v_cached, float& sigma, float& s_lo, float& s_hi) {
     if (r.v != v_cached) { v_cached = r.v; sigma = __fdiv_rn(r.v, static_cast<float>(kScaleLevels)); }
@@ -266,7 +259,30 @@ __device__ __forceinline__ void make_scales(const QView& q, const RawScale& r, f
 // [barriers][8-bit look-up table].  The activation / packed-code ring runs several steps ahead of
 // the tensor core (it hides the latency of global memory); the dequantized weight ring needs two
 // stages only (one being read by the tensor core, one being written).
-constexpr int kBStages = 2;
+constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA
+// stages of the dequantized weight ring: three, so that the dequantization of a step may start two
+// tensor-core steps before its result is needed (two for 8-bit codes, whose packed data leave less room)
+template <int B, int MH>
+__host__ __device__ constexpr int b_stages() { return (B == 8 && MH == 2) ? 2 : 3; }
+
+template <int B, int MH>
+__host__ __device__ constexpr int stage_bytes() { return MH * 16384 + 2048 * B; }        // one stage of the activation + packed-code ring
+template <int B>
+__host__ __device__ constexpr int tail_bytes() { return 256 + (B == 8 ? 1024 : 0) + 64; }
+template <int B, int MH>
+__host__ __device__ constexpr int fixed_bytes() { return 1024 + b_stages<B, MH>() * kBBytes; }   // alignment slack + weight ring
+template <int B, int MH>
+__host__ __device__ constexpr int ring_stages() {
+    const int s = (kSmemLimit - fixed_bytes<B, MH>() - tail_bytes<B>()) / stage_bytes<B, MH>();
+    return s > 6 ? 6 : s;
+}
+
+// Ring position that advances without divisions: stage index and the parity of the current pass.
+template <int S> struct RingPos {
+    int s = 0;
+    uint32_t ph = 0;
+    __device__ __forceinline__ void advance() { if (++s == S) { s = 0; ph ^= 1u; } }
+};
 
 template <int B, bool BWD, int MH>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -275,7 +291,8 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     constexpr int A_BYTES = MH * 128 * 128;
     constexpr int P_BYTES = 2048 * B;
     constexpr uint32_t TMEM_COLS = MH * BN;
-    const int SA = p.stages;
+    constexpr int SA = ring_stages<B, MH>();
+    constexpr int kBStages = b_stages<B, MH>();
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -283,7 +300,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     uint8_t* b_ring = a_ring + static_cast<size_t>(SA) * A_BYTES;
     uint8_t* p_ring = b_ring + kBStages * kBBytes;
     uint8_t* tail = p_ring + static_cast<size_t>(SA) * P_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);   // full_a[8], empty_a[8], full_b[2], empty_b[2], acc_full, drain
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);   // full_a[8], empty_a[8], full_b[4], empty_b[4], acc_full, drain
     float* lut8 = reinterpret_cast<float*>(tail + 256);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 256 + (B == 8 ? 1024 : 0));
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -297,8 +314,8 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     auto full_a = [&](int s) { return smem_u32(bars + s); };
     auto empty_a = [&](int s) { return smem_u32(bars + 8 + s); };
     auto full_b = [&](int s) { return smem_u32(bars + 16 + s); };
-    auto empty_b = [&](int s) { return smem_u32(bars + 18 + s); };
-    const uint32_t acc_full = smem_u32(bars + 20), drain = smem_u32(bars + 21);
+    auto empty_b = [&](int s) { return smem_u32(bars + 20 + s); };
+    const uint32_t acc_full = smem_u32(bars + 24), drain = smem_u32(bars + 25);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < SA; ++s) { mbar_init(full_a(s), 1); mbar_init(empty_a(s), 1); }
@@ -321,12 +338,12 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ------------------------------------------------------------------ producer: activations + packed codes
         if (lane == 0) {
             const uint8_t* codes = reinterpret_cast<const uint8_t*>(p.q.codes);
-            for (int step = 0; step < total; ++step) {
-                const int s = step % SA;
-                const uint32_t ph = (step / SA) & 1;
-                if (!wait(empty_a(s), ph ^ 1, ctl, 1)) break;
-                const uint32_t a_dst = smem_u32(a_ring + static_cast<size_t>(s) * A_BYTES);
-                const uint32_t p_dst = smem_u32(p_ring + static_cast<size_t>(s) * P_BYTES);
+            RingPos<SA> ra;
+            for (int step = 0; step < total; ++step, ra.advance()) {
+                const int s = ra.s;
+                if (!wait(empty_a(s), ra.ph ^ 1, ctl, 1)) break;
+                const uint32_t a_dst = smem_u32(a_ring) + s * A_BYTES;
+                const uint32_t p_dst = smem_u32(p_ring) + s * P_BYTES;
                 if (step < p.steps_q) {
                     if (!BWD) {
                         int nt_have = 0;
@@ -369,13 +386,15 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((BWD ? 1u : 0u) << 16) |
                                        (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(128 >> 4) << 24);
             bool ok = true;
-            for (int step = 0; step < total && ok; ++step) {
-                const int sa = step % SA, sb = step % kBStages;
-                ok = wait(full_a(sa), (step / SA) & 1, ctl, 2) && wait(full_b(sb), (step / kBStages) & 1, ctl, 3);
+            RingPos<SA> ra;
+            RingPos<kBStages> rb;
+            for (int step = 0; step < total && ok; ++step, ra.advance(), rb.advance()) {
+                const int sa = ra.s, sb = rb.s;
+                ok = wait(full_a(sa), ra.ph, ctl, 2) && wait(full_b(sb), rb.ph, ctl, 3);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t a_src = smem_u32(a_ring + static_cast<size_t>(sa) * A_BYTES);
-                const uint32_t b_src = smem_u32(b_ring + static_cast<size_t>(sb) * kBBytes);
+                const uint32_t a_src = smem_u32(a_ring) + sa * A_BYTES;
+                const uint32_t b_src = smem_u32(b_ring) + sb * kBBytes;
 #pragma unroll
                 for (int h = 0; h < MH; ++h) {
 #pragma unroll
@@ -410,55 +429,76 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         else { row_local = (slab_i & 1) * 32 + lane; b_off = (slab_i >> 1) * 8192 + row_local * 128; }
         const uint32_t xr = (row_local & 7) << 4;
         const bool two_scales = (p.q.B0 == 16);
-        // scale of step `st`: forward  (row c0 + row_local, columns st*64 + 32 g ..),
-        //                     backward (row st*64 + row_local, columns c0 + 64*(slab_i/2) + 32 g ..)
+        // block index of the scale of step `st` (32-bit: the host checks that N*K/B0 fits):
+        //   forward  (row c0 + row_local, columns st*64 + 32 g ..), backward (row st*64 + row_local, columns c0 + 64*(slab_i/2) + 32 g ..)
+        const int my_row = BWD ? row_local : c0 + row_local;
+        const int my_col = BWD ? c0 + (slab_i >> 1) * 64 + g * 32 : g * 32;
+        const bool col_ok = my_col < p.q.K;
+        const uint32_t blk0 = static_cast<uint32_t>(my_row) * p.q.KB + (BWD ? (my_col >> p.q.logB0) : 0);
+        const uint32_t row_stride = static_cast<uint32_t>(BK) * p.q.KB;
+        const uint8_t* __restrict__ scp = p.q.sc;
+        const float* __restrict__ vp = p.q.v;
+        const int logB0 = p.q.logB0, logB1 = p.q.logB1;
         auto fetch = [&](int st) {
-            return BWD ? fetch_scale(p.q, st * BK + row_local, c0 + (slab_i >> 1) * 64 + g * 32)
-                       : fetch_scale(p.q, c0 + row_local, st * BK + g * 32);
+            RawScale r{0u, 0.0f};
+            const int row = BWD ? st * BK + my_row : my_row;
+            if (row < p.q.N && col_ok) {
+                const uint32_t blk = BWD ? blk0 + st * row_stride : blk0 + ((st * BK + my_col) >> logB0);
+                r.sc = two_scales ? static_cast<uint32_t>(__ldg(reinterpret_cast<const uint16_t*>(scp + blk))) : static_cast<uint32_t>(__ldg(scp + blk));
+                r.v = __ldg(vp + (blk >> logB1));
+            }
+            return r;
         };
-        // the raw scale data are fetched four steps before they are needed
+        // The raw scale data of step s + 4 are requested right after those of step s have been used,
+        // into the same slot; the loop is unrolled by four so that the slots are fixed registers and
+        // no instruction touches a slot while its load is in flight.
         float v_cached = -1.0f, sigma = 0.0f, s_lo = 0.0f, s_hi = 0.0f;
-        RawScale r0{0u, 0.0f}, r1 = r0, r2 = r0, r3 = r0;
-        if (p.steps_q > 0) r0 = fetch(0);
-        if (p.steps_q > 1) r1 = fetch(1);
-        if (p.steps_q > 2) r2 = fetch(2);
-        if (p.steps_q > 3) r3 = fetch(3);
+        RawScale slot[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) slot[u] = (u < p.steps_q) ? fetch(u) : RawScale{0u, 0.0f};
+        const uint32_t* __restrict__ my_slab = reinterpret_cast<const uint32_t*>(p_ring) + slab_i * (64 * B) + g * (B * 32) + lane;
+        uint8_t* my_b = b_ring + b_off;
         bool ok = true;
-        for (int step = 0; step < total && ok; ++step) {
-            const int sa = step % SA, sb = step % kBStages;
-            RawScale r4{0u, 0.0f};
-            if (step + 4 < p.steps_q) r4 = fetch(step + 4);
-            ok = wait(empty_b(sb), ((step / kBStages) & 1) ^ 1, ctl, 6);
-            if (!ok) break;
-            uint8_t* b_dst = b_ring + static_cast<size_t>(sb) * kBBytes;
-            if (step < p.steps_q) {
-                make_scales(p.q, r0, v_cached, sigma, s_lo, s_hi);
-                r0 = r1; r1 = r2; r2 = r3; r3 = r4;
-                ok = wait(full_a(sa), (step / SA) & 1, ctl, 4);
+        RingPos<SA> ra;
+        RingPos<kBStages> rb;
+        for (int step4 = 0; step4 < total && ok; step4 += 4) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int step = step4 + u;
+                if (step >= total || !ok) break;
+                const int sa = ra.s, sb = rb.s;
+                ok = wait(empty_b(sb), rb.ph ^ 1, ctl, 6);
                 if (!ok) break;
-                const uint32_t* slab = reinterpret_cast<const uint32_t*>(p_ring + static_cast<size_t>(sa) * P_BYTES) + slab_i * (64 * B);
-                dequant_group<B>(slab, g, lane, lut8, s_lo, s_hi, two_scales, b_dst + b_off, xr);
-                fence_proxy_async();            // make the generic-proxy stores visible to the tensor core
-                __syncwarp();
-                if (lane == 0) mbar_arrive(full_b(sb));
-            } else if (dw == 0) {
-                // rank-r step: the second operand ([L1 | ..] rows or L2 rows) comes by TMA into the weight ring
-                if (lane == 0) {
-                    const int d = step - p.steps_q;
-                    const uint32_t dst = smem_u32(b_dst);
-                    if (!BWD) {
-                        mbar_expect_tx(full_b(sb), kBBytes);
-                        tma_load_2d(dst, &tmB2, d * BK, c0, full_b(sb));
-                    } else {
-                        int kt_have = 0;
-                        for (int t = 0; t < 4; ++t) if (c0 + t * 64 < p.out_cols) ++kt_have;
-                        mbar_expect_tx(full_b(sb), kt_have * 8192);
-                        for (int t = 0; t < kt_have; ++t) tma_load_2d(dst + t * 8192, &tmB2, c0 + t * 64, d * BK, full_b(sb));
+                if (step < p.steps_q) {
+                    make_scales(p.q, slot[u], v_cached, sigma, s_lo, s_hi);
+                    if (step + 4 < p.steps_q) slot[u] = fetch(step + 4);
+                    ok = wait(full_a(sa), ra.ph, ctl, 4);
+                    if (!ok) break;
+                    dequant_group<B>(my_slab + sa * (P_BYTES / 4), s_lo, s_hi, two_scales, my_b + sb * kBBytes, g << 6, xr, lut8);
+                    fence_proxy_async();            // make the generic-proxy stores visible to the tensor core
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(full_b(sb));
+                } else if (dw == 0) {
+                    // rank-r step: the second operand ([L1 | ..] rows or L2 rows) comes by TMA into the weight ring
+                    if (lane == 0) {
+                        const int d = step - p.steps_q;
+                        const uint32_t dst = smem_u32(b_ring) + sb * kBBytes;
+                        if (!BWD) {
+                            mbar_expect_tx(full_b(sb), kBBytes);
+                            tma_load_2d(dst, &tmB2, d * BK, c0, full_b(sb));
+                        } else {
+                            int kt_have = 0;
+                            for (int t = 0; t < 4; ++t) if (c0 + t * 64 < p.out_cols) ++kt_have;
+                            mbar_expect_tx(full_b(sb), kt_have * 8192);
+                            for (int t = 0; t < kt_have; ++t) tma_load_2d(dst + t * 8192, &tmB2, c0 + t * 64, d * BK, full_b(sb));
+                        }
                     }
+                    __syncwarp();
+                } else {
+                    if (lane == 0) mbar_arrive(full_b(sb));
                 }
-                __syncwarp();
-            } else {
-                if (lane == 0) mbar_arrive(full_b(sb));
+                ra.advance();
+                rb.advance();
             }
         }
         // epilogue: warp reads its quarter of the 128 accumulator lanes and 64 of the 256 columns
@@ -712,21 +752,13 @@ inline bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr int kSmemLimit = 232448;   // 227 KB of dynamic shared memory per CTA
-
-template <int B, int MH>
-constexpr int stage_bytes() { return MH * 16384 + 2048 * B; }        // one stage of the activation + packed-code ring
-template <int B>
-constexpr int tail_bytes() { return 256 + (B == 8 ? 1024 : 0) + 64; }
-constexpr int kFixedBytes = 1024 + kBStages * kBBytes;               // alignment slack + dequantized weight ring
-
 template <int B, bool BWD, int MH>
 inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, Params p, cudaStream_t st) {
-    int stages = (kSmemLimit - kFixedBytes - tail_bytes<B>()) / stage_bytes<B, MH>();
-    if (stages > 8) stages = 8;
-    if (stages < 2) return LQLORA_ERR_UNSUPPORTED;
+    constexpr int stages = ring_stages<B, MH>();
+    static_assert(stages >= 2, "activation ring too shallow");
     p.stages = stages;
-    const int smem = kFixedBytes + stages * stage_bytes<B, MH>() + tail_bytes<B>();
+    constexpr int smem = fixed_bytes<B, MH>() + stages * stage_bytes<B, MH>() + tail_bytes<B>();
+    static_assert(smem <= kSmemLimit, "shared memory budget exceeded");
     auto kern = tc_linear_kernel<B, BWD, MH>;
     static bool attr_done = false;
     if (!attr_done) {
@@ -802,6 +834,7 @@ inline bool tc_supported(const QView& q, int r, int64_t M, bool backward) {
     (void)r;
     if (M < kTcMinRows) return false;
     if (q.N % 8 != 0 || q.K % 8 != 0) return false;
+    if (static_cast<long long>(q.N) * q.KB >= (1LL << 31)) return false;   // block indices are 32-bit in the kernel
     (void)backward;
     return true;
 }
