@@ -71,6 +71,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -112,6 +113,12 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may
+// start while its predecessor in the stream still runs; pdl_wait() blocks until that predecessor
+// has completed and its memory is visible, pdl_launch_dependents() lets the successor start early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -367,6 +374,13 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         }
                     }
                 } else {
+                    if (step == p.steps_q) {
+                        // the rank-r intermediate is written by the preceding kernel, which may still be
+                        // running (programmatic dependent launch): wait for it, then order this thread's
+                        // bulk-copy reads after what it wrote
+                        pdl_wait();
+                        fence_proxy_async_all();
+                    }
                     mbar_expect_tx(full_a(s), A_BYTES);
                     tma_load_2d(a_dst, &tmA2, (step - p.steps_q) * BK, m0, full_a(s));
                 }
@@ -570,6 +584,7 @@ tc_lowrank_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* last_s = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
+    pdl_launch_dependents();      // the linear kernel behind this one needs T only in its last steps
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * 128;
     const int split = blockIdx.y, nsplit = gridDim.y;
@@ -768,10 +783,19 @@ inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUten
         }
         attr_done = true;
     }
-    dim3 grid((p.M + MH * 128 - 1) / (MH * 128), (p.out_cols + BN - 1) / BN);
-    kern<<<grid, kThreads, smem, st>>>(tA, tA2, tB2, p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((p.M + MH * 128 - 1) / (MH * 128), (p.out_cols + BN - 1) / BN);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (p.steps_d > 0) ? 1 : 0;      // overlap with the rank-r pre-product kernel in front of it
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA, tA2, tB2, p);
     count_launch(1);
-    if (cudaGetLastError() != cudaSuccess) return LQLORA_ERR_CUDA;
+    if (e != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
     return LQLORA_OK;
 }
 
@@ -781,14 +805,34 @@ struct PrePlan {
     size_t counters_bytes, partial_bytes, t_bytes;
 };
 
-inline PrePlan pre_plan(int64_t C, int r, int64_t M) {
+// Number of SMs of the current device (148 on B200; also the answer when no device is present).
+inline int sm_count() {
+    static const int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+            cudaGetLastError();
+            v = 148;
+        }
+        return v;
+    }();
+    return n;
+}
+
+// C = contraction length, out_cols = width of the output of the linear kernel that follows.
+inline PrePlan pre_plan(int64_t C, int r, int64_t M, int64_t out_cols) {
     PrePlan pl;
     pl.mtiles = static_cast<int>((M + 127) / 128);
     pl.steps = static_cast<int>((C + BK - 1) / BK);
-    int want = 148 / pl.mtiles;                 // one wave of CTAs
+    // The pre-product runs beside the linear kernel that follows it (programmatic dependent launch):
+    // give it the SMs that the last wave of that kernel leaves idle, and at least one CTA per row tile.
+    const int mh = (M > 128) ? 2 : 1;
+    const long long main_ctas = ((M + mh * 128 - 1) / (mh * 128)) * ((out_cols + BN - 1) / BN);
+    const int sms = sm_count();
+    const int idle = static_cast<int>((sms - main_ctas % sms) % sms);
+    int want = idle / pl.mtiles;
     if (want > pl.steps / 2) want = pl.steps / 2;
-    if (want < 1) want = 1;
     if (want > 32) want = 32;
+    if (want < 1) want = 1;
     pl.steps_per_split = (pl.steps + want - 1) / want;
     pl.nsplit = (pl.steps + pl.steps_per_split - 1) / pl.steps_per_split;
     pl.rp = (r <= 64) ? 64 : 128;
@@ -840,7 +884,7 @@ inline bool tc_supported(const QView& q, int r, int64_t M, bool backward) {
 }
 
 inline size_t tc_workspace_bytes(int64_t N, int64_t K, int r, int64_t M, bool backward) {
-    const tc::PrePlan pl = tc::pre_plan(backward ? N : K, r, M);
+    const tc::PrePlan pl = tc::pre_plan(backward ? N : K, r, M, backward ? K : N);
     return kStatusBytes + pl.counters_bytes + pl.t_bytes + (r > 0 ? pl.partial_bytes : 0);
 }
 
@@ -848,7 +892,7 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
                      bool backward, cudaStream_t st) {
     using namespace tc;
     const int C = backward ? q.N : q.K;              // contraction length
-    const PrePlan pl = pre_plan(C, r, M);
+    const PrePlan pl = pre_plan(C, r, M, backward ? q.K : q.N);
     // workspace: [status][row-tile counters][T bf16][fp32 partial tiles]; status and counters were zeroed by the caller
     int* counters = reinterpret_cast<int*>(ws + kStatusBytes);
     __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + pl.counters_bytes);

@@ -60,7 +60,7 @@ static int run_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, i
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const QView v = make_view(q);
     const bool use_tc = tc_supported(v, r, M, backward);
-    const size_t zero_bytes = kStatusBytes + (use_tc ? tc::pre_plan(backward ? v.N : v.K, r, M).counters_bytes : 0);
+    const size_t zero_bytes = kStatusBytes + (use_tc ? tc::pre_plan(backward ? v.N : v.K, r, M, backward ? v.K : v.N).counters_bytes : 0);
     if (cudaMemsetAsync(ws, 0, zero_bytes, st) != cudaSuccess) return cuda_rc(cudaGetLastError());
     cudaError_t e = cudaSuccess;
     if (use_tc) {
