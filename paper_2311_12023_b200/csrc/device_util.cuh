@@ -49,6 +49,32 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+constexpr long long kWaitCycles = 4000000000LL;   // about two seconds
+
+// Bounded wait.  Returns false when the wait was abandoned (another thread aborted, or time ran out).
+struct Ctl {
+    volatile int* abort_s;
+    int* status_g;
+};
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const Ctl& c, int where) {
+    const long long t0 = clock64();
+    for (int it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63) == 63) {
+            if (*c.abort_s) return false;
+            if (clock64() - t0 > kWaitCycles) {
+                *c.abort_s = 1;
+                atomicCAS(c.status_g, 0, where);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, const Ctl& c, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return wait_slow(bar, parity, c, where);
+}
+
 // ------------------------------------------------------------------------------------ dequantization tables
 // The 2^b0 products fl32(q~[c] * s~) of one block, rounded to bf16, are kept in registers as a
 // byte table: lo[] holds the low bytes, hi[] the high bytes, four entries per register.  One

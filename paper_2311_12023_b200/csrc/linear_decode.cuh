@@ -1,0 +1,527 @@
+// Forward pass for decode-sized inputs (M <= 16 rows of X): the packed matrix is streamed once.
+//
+//   - One CTA owns a tile row of Q (128 rows) and a slice of K; the K slices of a tile row form a
+//     thread-block cluster and are added up through distributed shared memory, so there is no
+//     workspace of partial sums and nothing to zero.
+//   - A producer thread streams the packed tiles of the CTA (they are contiguous in memory) into a
+//     shared-memory ring with bulk copies; eight consumer warps dequantize them in registers with
+//     the byte-table method (bf16 bits identical to the exported dequantized weights) and feed
+//     mma.sync m16n8k16 (weights = the 16-row operand, tokens = the 8-column operand, fp32 accumulators).
+//     The contraction index is permuted so that a thread supplies 4 consecutive weights of one row per MMA
+//     and reads the matching 4 activations with one 128-bit load per 8 columns.
+//   - Block scales s~ of the CTA's rows and columns are computed once into shared memory.
+//   - The rank-r intermediate T = X L2^T comes from a small kernel launched in front of this one; the two
+//     overlap (programmatic dependent launch) and T is only read in the epilogue, which adds T L1^T.
+#pragma once
+
+#include "common.cuh"
+#include "device_util.cuh"
+
+namespace lq {
+namespace dec {
+using namespace dev;
+
+constexpr int kConsumerWarps = 8;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kStageTiles = 8;              // 64-column tiles per ring stage (four windows of 128 columns)
+constexpr int kSmemLimit = 232448;
+
+template <int B> __host__ __device__ constexpr int stage_bytes() { return kStageTiles * 1024 * B; }
+// NT = number of 8-token groups (1: M <= 8, two CTAs per SM; 2: M <= 16, one CTA per SM)
+template <int B, int NT> __host__ __device__ constexpr int num_stages() { return (B == 8) ? 2 : (NT == 2 ? 4 : 2); }
+
+struct Params {
+    QView q;
+    const __nv_bfloat16* X;    // [M][K]
+    const __nv_bfloat16* T;    // [M][r], written by the kernel in front of this one (r > 0)
+    const __nv_bfloat16* L1;   // [N][r]
+    __nv_bfloat16* Y;          // [M][N]
+    int* status;
+    int M, r;
+    int S;                     // K slices per tile row = cluster size
+    int tiles_per_split;       // 64-column tiles per CTA (even)
+    int nkb_cap;               // capacity of the scale table in blocks
+};
+
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank) {
+    uint32_t ra;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ uint32_t pick(const uint4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
+__device__ __forceinline__ float pickf(const float4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
+
+// The 32 weights of one (row, group) as sixteen bf16 pairs: o[c][e] holds columns 8c + 2e, 8c + 2e + 1.
+template <int B>
+__device__ __forceinline__ void dequant_row32(const uint32_t (&w)[B], float s_lo, float s_hi, bool two_scales,
+                                              uint32_t (&o)[4][4], const float* __restrict__ lut8) {
+    if constexpr (B == 8) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const float s = (c < 2) ? s_lo : s_hi;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t ww = w[2 * c + (e >> 1)] >> (16 * (e & 1));
+                const float q0 = lut8[ww & 255u], q1 = lut8[(ww >> 8) & 255u];
+                const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(q0, s), __fmul_rn(q1, s));
+                o[c][e] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+        }
+    } else {
+        BlockTable<B> tab;
+        tab.build(s_lo);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (c == 2 && two_scales) tab.build(s_hi);
+            const uint32_t sel = chunk_selector<B>(w, c);
+            uint32_t selA = sel, selB = 0u;
+            if constexpr (B == 4) { selA = sel & 0x77777777u; selB = ((sel >> 1) & 0x44444444u) | 0x32103210u; }
+            tab.lookup4(selA, selB, o[c][0], o[c][1]);
+            tab.lookup4(selA >> 16, selB >> 16, o[c][2], o[c][3]);
+        }
+    }
+}
+
+template <int B, int NT>
+__global__ void __launch_bounds__(kThreads, (NT == 1 && B != 8) ? 2 : 1)
+decode_fwd_kernel(const Params p) {
+    constexpr int NS = num_stages<B, NT>();
+    constexpr int STAGE = stage_bytes<B>();
+    constexpr int MT = 8 * NT;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
+    uint8_t* ring = base;
+    float* part = reinterpret_cast<float*>(ring + NS * STAGE);        // [128][MT] partial sums of this CTA
+    float* lut8 = part + 128 * MT;                                     // 256 floats (8-bit codes only)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(lut8 + (B == 8 ? 256 : 0));   // full[NS], empty[NS]
+    volatile int* abort_s = reinterpret_cast<volatile int*>(bars + 2 * NS);
+    float* stab = reinterpret_cast<float*>(bars + 2 * NS + 2);         // [nkb][128] block scales s~
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile_row = blockIdx.x;
+    const int split = blockIdx.y;
+    const QView& q = p.q;
+    const int kt0 = split * p.tiles_per_split;
+    const int kt1 = min(q.ktiles, kt0 + p.tiles_per_split);
+    const int ntiles_cta = max(0, kt1 - kt0);
+    const int nstage_total = (ntiles_cta + kStageTiles - 1) / kStageTiles;
+    const Ctl ctl{abort_s, p.status};
+
+    auto full = [&](int s) { return smem_u32(bars + s); };
+    auto empty = [&](int s) { return smem_u32(bars + NS + s); };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), kConsumerWarps); }
+        *abort_s = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+
+    const uint8_t* codes = reinterpret_cast<const uint8_t*>(q.codes) +
+                           (static_cast<size_t>(tile_row) * q.ktiles + kt0) * (1024 * B);
+    auto issue_stage = [&](int it) {
+        const int s = it % NS;
+        const int nt = min(kStageTiles, ntiles_cta - it * kStageTiles);
+        mbar_expect_tx(full(s), nt * 1024 * B);
+        bulk_load(smem_u32(ring + s * STAGE), codes + static_cast<size_t>(it) * STAGE, nt * 1024 * B, full(s));
+    };
+    if (warp == kConsumerWarps && lane == 0) {
+        for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it);
+    }
+
+    // block scales of the CTA's rows and columns: s~ = fl32(float(s^) * fl32(v / 127)), 0 for rows past N
+    const int kb_first = (kt0 * kTileCols) >> q.logB0;
+    const int nkb = (ntiles_cta > 0) ? (((kt1 * kTileCols - 1) >> q.logB0) - kb_first + 1) : 0;
+    for (int idx = threadIdx.x; idx < nkb * 128; idx += kThreads) {
+        const int row = idx / nkb, kb = idx - row * nkb;
+        const int grow = tile_row * 128 + row;
+        float val = 0.0f;
+        if (grow < q.N) {
+            const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first + kb;
+            val = block_scale(__ldg(q.sc + blk), __ldg(q.v + (blk >> q.logB1)));
+        }
+        stab[kb * 128 + row] = val;
+    }
+    if constexpr (B == 8) {
+        for (int i = threadIdx.x; i < 256; i += kThreads) lut8[i] = c_codebook[3][i];
+    }
+    __syncthreads();
+
+    float acc[2][2][NT][4];
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < 2; ++b)
+#pragma unroll
+            for (int c = 0; c < NT; ++c)
+#pragma unroll
+                for (int d = 0; d < 4; ++d) acc[a][b][c][d] = 0.0f;
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            for (int it = NS; it < nstage_total; ++it) {
+                const int s = it % NS;
+                if (!wait(empty(s), ((it / NS) & 1) ^ 1, ctl, 21)) break;
+                issue_stage(it);
+            }
+            if (*abort_s) {
+                for (int s = 0; s < NS; ++s) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(full(s), 0) && !mbar_try_wait(full(s), 1) && clock64() - t0 < 20000000LL) {}
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ consumers
+        const int gid = lane >> 2, t = lane & 3;
+        const int win_slot = warp & 3, half = warp >> 2;
+        const bool two_scales = (q.B0 == 16);
+        bool ok = true;
+        for (int it = 0; it < nstage_total && ok; ++it) {
+            const int s = it % NS;
+            ok = wait(full(s), (it / NS) & 1, ctl, 22);
+            if (!ok) break;
+            const int tiles_here = min(kStageTiles, ntiles_cta - it * kStageTiles);
+            if (2 * win_slot < tiles_here) {
+                const int tile_in_stage = 2 * win_slot + (t >> 1);
+                const bool kt_ok = tile_in_stage < tiles_here;
+                const int col0 = (kt0 + it * kStageTiles + tile_in_stage) * kTileCols + (t & 1) * 32;
+                uint4 x[NT][4];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int m = nt * 8 + gid;
+                    if (m < p.M && kt_ok) {
+                        const uint4* xp = reinterpret_cast<const uint4*>(p.X + static_cast<size_t>(m) * q.K + col0);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) x[nt][c] = __ldg(xp + c);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) x[nt][c] = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+                const uint32_t* tile = reinterpret_cast<const uint32_t*>(ring + s * STAGE) + (kt_ok ? tile_in_stage : 0) * (256 * B);
+                const int kb = kt_ok ? ((col0 >> q.logB0) - kb_first) : 0;
+#pragma unroll
+                for (int sl = 0; sl < 2; ++sl) {
+                    const int slab = 2 * half + sl;
+                    const uint32_t* sp = tile + slab * (64 * B) + (t & 1) * (B * 32) + 4 * gid;
+                    uint4 w4[B];
+#pragma unroll
+                    for (int i = 0; i < B; ++i) w4[i] = *reinterpret_cast<const uint4*>(sp + i * 32);
+                    float4 sc_lo = *reinterpret_cast<const float4*>(stab + kb * 128 + slab * 32 + 4 * gid);
+                    float4 sc_hi = sc_lo;
+                    if (two_scales) sc_hi = *reinterpret_cast<const float4*>(stab + (kb + 1) * 128 + slab * 32 + 4 * gid);
+                    if (!kt_ok) { sc_lo = make_float4(0.f, 0.f, 0.f, 0.f); sc_hi = sc_lo; }
+#pragma unroll
+                    for (int set = 0; set < 2; ++set) {
+                        uint32_t oa[4][4], ob[4][4];
+                        {
+                            uint32_t w[B];
+#pragma unroll
+                            for (int i = 0; i < B; ++i) w[i] = pick(w4[i], 2 * set);
+                            dequant_row32<B>(w, pickf(sc_lo, 2 * set), pickf(sc_hi, 2 * set), two_scales, oa, lut8);
+#pragma unroll
+                            for (int i = 0; i < B; ++i) w[i] = pick(w4[i], 2 * set + 1);
+                            dequant_row32<B>(w, pickf(sc_lo, 2 * set + 1), pickf(sc_hi, 2 * set + 1), two_scales, ob, lut8);
+                        }
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) {
+                                mma16816(acc[sl][set][nt], oa[c][0], ob[c][0], oa[c][1], ob[c][1], x[nt][c].x, x[nt][c].y);
+                                mma16816(acc[sl][set][nt], oa[c][2], ob[c][2], oa[c][3], ob[c][3], x[nt][c].z, x[nt][c].w);
+                            }
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty(s));
+        }
+    }
+
+    // ---------------------------------------------------------------------- reduction over the K windows of the CTA
+    // acc[sl][set][nt][e]: row (2 half + sl) * 32 + 4 gid + 2 set + (e >> 1), token nt * 8 + 2 t + (e & 1)
+    for (int round = 0; round < 4; ++round) {
+        if (warp < kConsumerWarps && (warp & 3) == round) {
+            const int gid = lane >> 2, t = lane & 3, half = warp >> 2;
+#pragma unroll
+            for (int sl = 0; sl < 2; ++sl)
+#pragma unroll
+                for (int set = 0; set < 2; ++set)
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int row = (2 * half + sl) * 32 + 4 * gid + 2 * set + (e >> 1);
+                            const int tok = nt * 8 + 2 * t + (e & 1);
+                            float* dst = part + row * MT + tok;
+                            *dst = (round == 0) ? acc[sl][set][nt][e] : *dst + acc[sl][set][nt][e];
+                        }
+        }
+        __syncthreads();
+    }
+
+    // ---------------------------------------------------------------------- reduction over the K slices (cluster), rank-r term, store
+    cluster_sync_all();
+    const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
+    const int rows_share = 128 / p.S;
+    const int row_lo = static_cast<int>(rank) * rows_share;
+    if (p.r > 0) pdl_wait();          // T is written by the kernel launched in front of this one
+    const uint32_t part_addr = smem_u32(part);
+    for (int o = threadIdx.x; o < rows_share * p.M; o += kThreads) {
+        const int m = o / rows_share, rl = o - m * rows_share;
+        const int row = row_lo + rl;
+        const int n = tile_row * 128 + row;
+        if (n >= q.N) continue;
+        float sum = 0.0f;
+        for (int rk = 0; rk < p.S; ++rk) sum += ld_dsmem_f32(part_addr + static_cast<uint32_t>(row * MT + m) * 4u, static_cast<uint32_t>(rk));
+        if (p.r > 0) {
+            const uint4* l1 = reinterpret_cast<const uint4*>(p.L1 + static_cast<size_t>(n) * p.r);
+            const uint4* tt = reinterpret_cast<const uint4*>(p.T + static_cast<size_t>(m) * p.r);
+            float lr = 0.0f;
+            for (int j = 0; j < p.r / 8; ++j) {
+                const uint4 a = __ldg(l1 + j), b = tt[j];
+                const uint32_t aa[4] = {a.x, a.y, a.z, a.w}, bb[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    lr = fmaf(__uint_as_float(aa[e] << 16), __uint_as_float(bb[e] << 16), lr);
+                    lr = fmaf(__uint_as_float(aa[e] & 0xffff0000u), __uint_as_float(bb[e] & 0xffff0000u), lr);
+                }
+            }
+            sum += lr;
+        }
+        p.Y[static_cast<size_t>(m) * q.N + n] = __float2bfloat16_rn(sum);
+    }
+    cluster_sync_all();               // shared memory of this CTA may be read by its peers until here
+}
+
+// ------------------------------------------------------------------------------------ rank-r pre-product for few rows
+// T[m][j] = bf16( sum_c A[m][c] * F(j, c) ) for m < M <= 16, j < r <= 128:
+//   forward  A = X [M][K],  F(j, c) = L2[j][c]   (T = X L2^T)
+//   backward A = dY [M][N], F(j, c) = L1[c][j]   (T = dY L1)
+// One cluster of CTAs; each CTA sums a slice of the contraction, the slices are added through
+// distributed shared memory by rank 0.  Thread = (column j, one of four contraction phases).
+struct PreParams {
+    const __nv_bfloat16* A;
+    const __nv_bfloat16* F;
+    __nv_bfloat16* T;
+    int* status;       // cleared here: this kernel is the first of a call
+    int M, C, r;
+    int chunk;         // contraction elements per CTA (multiple of 32)
+    int nranks;
+};
+
+template <bool BWD>
+__global__ void __launch_bounds__(256) decode_pre_kernel(const PreParams p) {
+    __shared__ float red[4][16][64];
+    __shared__ float part[16][128];
+    pdl_launch_dependents();
+    if (blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0;
+    const int jl = threadIdx.x & 63, ph = threadIdx.x >> 6;
+    const int c_lo = blockIdx.x * p.chunk;
+    const int c_hi = min(p.C, c_lo + p.chunk);
+    for (int jb = 0; jb < p.r; jb += 64) {
+        const int j = jb + jl;
+        float acc[16];
+#pragma unroll
+        for (int m = 0; m < 16; ++m) acc[m] = 0.0f;
+        if (j < p.r) {
+            for (int c = c_lo + ph * 8; c < c_hi; c += 32) {
+                float f[8];
+                if (!BWD) {
+                    const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.F + static_cast<size_t>(j) * p.C + c));
+                    const uint32_t vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) { f[2 * e] = __uint_as_float(vv[e] << 16); f[2 * e + 1] = __uint_as_float(vv[e] & 0xffff0000u); }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) f[e] = (c + e < c_hi) ? __bfloat162float(p.F[static_cast<size_t>(c + e) * p.r + j]) : 0.0f;
+                }
+#pragma unroll
+                for (int m = 0; m < 16; ++m) {
+                    if (m < p.M) {
+                        const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.A + static_cast<size_t>(m) * p.C + c));
+                        const uint32_t vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            acc[m] = fmaf(__uint_as_float(vv[e] << 16), f[2 * e], acc[m]);
+                            acc[m] = fmaf(__uint_as_float(vv[e] & 0xffff0000u), f[2 * e + 1], acc[m]);
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < 16; ++m) red[ph][m][jl] = acc[m];
+        __syncthreads();
+        for (int o = threadIdx.x; o < 16 * 64; o += 256) {
+            const int m = o >> 6, jj = o & 63;
+            part[m][jb + jj] = red[0][m][jj] + red[1][m][jj] + red[2][m][jj] + red[3][m][jj];
+        }
+        __syncthreads();
+    }
+    cluster_sync_all();
+    if (p.nranks == 1 || cluster_ctarank() == 0) {
+        const uint32_t part_addr = smem_u32(&part[0][0]);
+        for (int o = threadIdx.x; o < p.M * p.r; o += 256) {
+            const int m = o / p.r, j = o - m * p.r;
+            float sum = 0.0f;
+            for (int rk = 0; rk < p.nranks; ++rk) sum += ld_dsmem_f32(part_addr + static_cast<uint32_t>(m * 128 + j) * 4u, static_cast<uint32_t>(rk));
+            p.T[o] = __float2bfloat16_rn(sum);
+        }
+    }
+    cluster_sync_all();
+}
+
+// ------------------------------------------------------------------------------------ host side
+struct Plan {
+    bool ok;
+    int NT, S, tiles_per_split, nkb_cap, tile_rows;
+    size_t smem;
+};
+
+template <int B, int NT>
+inline size_t smem_bytes(int nkb_cap) {
+    return 128 + static_cast<size_t>(num_stages<B, NT>()) * stage_bytes<B>() + 128 * 8 * NT * 4 + (B == 8 ? 1024 : 0) +
+           (2 * num_stages<B, NT>() + 2) * 8 + static_cast<size_t>(nkb_cap) * 512;
+}
+
+inline int sm_count_cached() {
+    static const int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+            cudaGetLastError();
+            v = 148;
+        }
+        return v;
+    }();
+    return n;
+}
+
+template <int B>
+inline Plan make_plan(const QView& q, int M) {
+    Plan pl{};
+    pl.NT = (M <= 8) ? 1 : 2;
+    pl.tile_rows = q.ntiles;
+    const int per_sm = (pl.NT == 1 && B != 8) ? 2 : 1;
+    const int slots = sm_count_cached() * per_sm;
+    const size_t limit = (per_sm == 2) ? 113 * 1024 : kSmemLimit;
+    int S = 1;
+    while (S < 8 && pl.tile_rows * (2 * S) <= slots && q.ktiles / (2 * S) >= 2) S *= 2;
+    for (;; S *= 2) {
+        int tps = (q.ktiles + S - 1) / S;
+        tps += tps & 1;
+        const int nkb_cap = ((tps * kTileCols) >> q.logB0) + 2;
+        const size_t smem = (pl.NT == 1) ? smem_bytes<B, 1>(nkb_cap) : smem_bytes<B, 2>(nkb_cap);
+        if (smem <= limit || (per_sm == 2 && S == 8 && smem <= static_cast<size_t>(kSmemLimit))) {
+            pl.ok = true; pl.S = S; pl.tiles_per_split = tps; pl.nkb_cap = nkb_cap; pl.smem = smem;
+            return pl;
+        }
+        if (S >= 8) break;
+    }
+    pl.ok = false;
+    return pl;
+}
+
+inline bool supported(const QView& q, int64_t M) {
+    if (M > 16 || q.K % 8 != 0) return false;
+    if (static_cast<long long>(q.N) * q.KB >= (1LL << 31)) return false;
+    switch (q.b0) {
+        case 2: return make_plan<2>(q, static_cast<int>(M)).ok;
+        case 3: return make_plan<3>(q, static_cast<int>(M)).ok;
+        case 4: return make_plan<4>(q, static_cast<int>(M)).ok;
+        default: return make_plan<8>(q, static_cast<int>(M)).ok;
+    }
+}
+
+// Launches the pre-product kernel for few rows (both directions use it).
+template <bool BWD>
+inline cudaError_t launch_pre(const __nv_bfloat16* A, const __nv_bfloat16* F, __nv_bfloat16* T, int* status, int M, int C, int r,
+                              cudaStream_t st) {
+    PreParams pp;
+    pp.A = A; pp.F = F; pp.T = T; pp.status = status; pp.M = M; pp.C = C; pp.r = r;
+    int nranks = 8;
+    while (nranks > 1 && C / nranks < 256) nranks >>= 1;
+    int chunk = (C + nranks - 1) / nranks;
+    chunk = (chunk + 31) / 32 * 32;
+    pp.chunk = chunk; pp.nranks = nranks;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(nranks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = nranks; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    count_launch(1);
+    return cudaLaunchKernelEx(&cfg, decode_pre_kernel<BWD>, pp);
+}
+
+template <int B, int NT>
+inline cudaError_t launch_fwd_nt(const Params& p, const Plan& pl, bool after_pre, cudaStream_t st) {
+    auto kern = decode_fwd_kernel<B, NT>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(pl.tile_rows, pl.S);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = pl.S; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_pre ? 2 : 1;
+    count_launch(1);
+    return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+// Forward for M <= 16.  ws: [status 256 B][T bf16].  When r > 0 the pre-product kernel clears the status
+// word; otherwise the caller has cleared it.
+template <int B>
+inline cudaError_t launch_fwd(const QView& q, const void* L1, const void* L2, int r, const void* X, int M, void* Y, char* ws,
+                              cudaStream_t st) {
+    const Plan pl = make_plan<B>(q, M);
+    Params p;
+    p.q = q;
+    p.X = static_cast<const __nv_bfloat16*>(X);
+    p.T = reinterpret_cast<const __nv_bfloat16*>(ws + kStatusBytes);
+    p.L1 = static_cast<const __nv_bfloat16*>(L1);
+    p.Y = static_cast<__nv_bfloat16*>(Y);
+    p.status = reinterpret_cast<int*>(ws);
+    p.M = M; p.r = r; p.S = pl.S; p.tiles_per_split = pl.tiles_per_split; p.nkb_cap = pl.nkb_cap;
+    if (r > 0) {
+        cudaError_t e = launch_pre<false>(p.X, static_cast<const __nv_bfloat16*>(L2), reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes),
+                                          p.status, M, q.K, r, st);
+        if (e != cudaSuccess) return e;
+    }
+    return (pl.NT == 1) ? launch_fwd_nt<B, 1>(p, pl, r > 0, st) : launch_fwd_nt<B, 2>(p, pl, r > 0, st);
+}
+
+}  // namespace dec
+}  // namespace lq

@@ -4,6 +4,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "linear_decode.cuh"
 
 namespace lq {
 
@@ -259,7 +260,15 @@ inline cudaError_t launch_small(const QView& q, const void* L1, const void* L2, 
             static_cast<__nv_bfloat16*>(out), M, q.N, r, r, 1);
         launches += 2;
     } else {
-        if (r > 0) { lowrank_pre_kernel<<<M, 256, 0, st>>>(a, l1, T, q.N, r, 1, r); ++launches; }
+        if (r > 0) {
+            if (M <= 16 && q.N % 8 == 0) {
+                const cudaError_t e = dec::launch_pre<true>(a, l1, T, reinterpret_cast<int*>(ws), M, q.N, r, st);
+                if (e != cudaSuccess) return e;
+            } else {
+                lowrank_pre_kernel<<<M, 256, 0, st>>>(a, l1, T, q.N, r, 1, r);
+                ++launches;
+            }
+        }
         constexpr int MT = 2;
         dim3 grid(((q.K + 127) / 128 + 3) / 4, p.splits, (M + MT - 1) / MT);
         small_bwd_kernel<B, MT><<<grid, 128, 0, st>>>(q, a, P, M, p.per_split);

@@ -37,7 +37,6 @@ constexpr int BN = 256;
 constexpr int kDeqWarps = 16;
 constexpr int kThreads = (2 + kDeqWarps) * 32;
 constexpr int kBBytes = BN * 128;            // bf16 weight tile of one step
-constexpr long long kWaitCycles = 4000000000LL;   // about two seconds
 
 struct Params {
     QView q;
@@ -92,30 +91,6 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     d |= static_cast<uint64_t>(1) << 46;
     d |= static_cast<uint64_t>(2) << 61;
     return d;
-}
-
-// Bounded wait.  Returns false when the wait was abandoned (another thread aborted, or time ran out).
-struct Ctl {
-    volatile int* abort_s;
-    int* status_g;
-};
-__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const Ctl& c, int where) {
-    const long long t0 = clock64();
-    for (int it = 0;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63) == 63) {
-            if (*c.abort_s) return false;
-            if (clock64() - t0 > kWaitCycles) {
-                *c.abort_s = 1;
-                atomicCAS(c.status_g, 0, where);
-                return false;
-            }
-        }
-    }
-}
-__device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, const Ctl& c, int where) {
-    if (mbar_try_wait(bar, parity)) return true;
-    return wait_slow(bar, parity, c, where);
 }
 
 // ------------------------------------------------------------------------------------ dequantization
