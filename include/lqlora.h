@@ -73,9 +73,15 @@ typedef struct {
  *                    other in row-major tile order; a tile takes 1024*b0 bytes;
  *                  - a tile is four slabs of 32 rows (rows 32q .. 32q+31, q = 0..3), 256*b0 bytes each;
  *                  - inside a slab, the 64 columns form two groups g = 0, 1 of 32 columns; the 32
- *                    codes of (row, g) are a little-endian bit string of 32*b0 bits (code j at bits
- *                    [b0*j, b0*j + b0)), cut into b0 32-bit words w = 0..b0-1;
- *                  - word w of (row, g) is the 32-bit word number (g*b0 + w)*32 + (row % 32) of the slab.
+ *                    codes c[0..31] of (row, g) take b0 32-bit words w = 0..b0-1, each a string of
+ *                    eight 4-bit fields (for b0 = 8: four bytes):
+ *                      b0 = 4: field i of word w = c[8w+i];
+ *                      b0 = 3: low three bits of field i of word w (w < 3) = c[8w+i], top bit = bit w of c[24+i];
+ *                      b0 = 2: low two bits of field i of word w = c[16w+i], high two bits = c[16w+8+i];
+ *                      b0 = 8: byte i of word w = c[4w+i];
+ *                  - word w of (row, g) in tile column kt is the 32-bit word number
+ *                    (g*b0 + w)*32 + ((row + 8*g + 16*(kt % 2)) % 32) of the slab (the rows of a word plane
+ *                    are rotated per group and per tile column to spread shared-memory banks).
  *                Consecutive 32-bit words of a slab therefore belong to consecutive rows, so a
  *                warp reads or writes a slab with fully coalesced accesses and conflict-free
  *                shared-memory accesses.  Use lqlora_unpack to obtain one code per byte.

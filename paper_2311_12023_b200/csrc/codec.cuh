@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
     uint32_t* dst = codes + slab_word_base(row, k0 >> 6, K >> 6, B);
     const int g = (k0 >> 5) & 1;
 #pragma unroll
-    for (int w = 0; w < B; ++w) dst[slab_word_offset(row, g, w, B)] = words[w];
+    for (int w = 0; w < B; ++w) dst[slab_word_offset(row, g, w, B, k0 >> 6)] = words[w];
 }
 
 // One CTA per second-level group: v_g = max s_i, s^_i = clamp(rint(s_i / (v_g / 127)), 0, 127).
@@ -148,7 +148,7 @@ __global__ void __launch_bounds__(256) export_kernel(QView q, uint8_t* __restric
     const uint32_t* src = q.codes + slab_word_base(row, k0 >> 6, q.ktiles, B);
     uint32_t w[B];
 #pragma unroll
-    for (int i = 0; i < B; ++i) w[i] = src[slab_word_offset(row, (k0 >> 5) & 1, i, B)];
+    for (int i = 0; i < B; ++i) w[i] = src[slab_word_offset(row, (k0 >> 5) & 1, i, B, k0 >> 6)];
     const size_t out = static_cast<size_t>(row) * q.K + k0;
     const float* cb = c_codebook[bits_index(B)];
 #pragma unroll

@@ -75,9 +75,13 @@ __host__ __device__ inline size_t slab_word_base(int row, int kt, int ktiles, in
     const size_t tile = static_cast<size_t>(row >> 7) * ktiles + kt;
     return (tile * 4 + ((row >> 5) & 3)) * static_cast<size_t>(64 * b0);
 }
-// Word w of the 32-code group g of `row` inside its slab.
-__host__ __device__ inline int slab_word_offset(int row, int g, int w, int b0) {
-    return (g * b0 + w) * 32 + (row & 31);
+// Word w of the 32-code group g of `row` inside the slab of 64-column tile kt.  The 32 rows of a word
+// plane are rotated by 8 g + 16 (kt % 2) positions, so that threads that read the same four rows from
+// the two groups of two neighbouring tiles (the access pattern of the decode kernels) hit different
+// shared-memory banks; a rotation by a multiple of four keeps aligned groups of four rows together.
+__host__ __device__ inline int slab_row_slot(int row, int g, int kt) { return (row + 8 * g + 16 * (kt & 1)) & 31; }
+__host__ __device__ inline int slab_word_offset(int row, int g, int w, int b0, int kt) {
+    return (g * b0 + w) * 32 + slab_row_slot(row, g, kt);
 }
 
 // Bit layout of the 32 codes c[0..31] of one (row, 32-column group) inside its b0 words.  Every

@@ -25,6 +25,7 @@ constexpr int kConsumerWarps = 8;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kStageTiles = 8;              // 64-column tiles per ring stage (four windows of 128 columns)
 constexpr int kSmemLimit = 232448;
+constexpr int kStabStride = 136;            // floats per block column of the scale table (128 rows + padding against bank conflicts)
 
 template <int B> __host__ __device__ constexpr int stage_bytes() { return kStageTiles * 1024 * B; }
 // NT = number of 8-token groups (1: M <= 8, two CTAs per SM; 2: M <= 16, one CTA per SM)
@@ -66,8 +67,8 @@ __device__ __forceinline__ uint32_t pick(const uint4& v, int i) { return i == 0 
 __device__ __forceinline__ float pickf(const float4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
 
 // The 32 weights of one (row, group) as sixteen bf16 pairs: o[c][e] holds columns 8c + 2e, 8c + 2e + 1.
-template <int B>
-__device__ __forceinline__ void dequant_row32(const uint32_t (&w)[B], float s_lo, float s_hi, bool two_scales,
+template <int B, bool TWO>
+__device__ __forceinline__ void dequant_row32(const uint32_t (&w)[B], float s_lo, float s_hi,
                                               uint32_t (&o)[4][4], const float* __restrict__ lut8) {
     if constexpr (B == 8) {
 #pragma unroll
@@ -86,7 +87,7 @@ __device__ __forceinline__ void dequant_row32(const uint32_t (&w)[B], float s_lo
         tab.build(s_lo);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            if (c == 2 && two_scales) tab.build(s_hi);
+            if (TWO && c == 2) tab.build(s_hi);
             const uint32_t sel = chunk_selector<B>(w, c);
             uint32_t selA = sel, selB = 0u;
             if constexpr (B == 4) { selA = sel & 0x77777777u; selB = ((sel >> 1) & 0x44444444u) | 0x32103210u; }
@@ -96,7 +97,7 @@ __device__ __forceinline__ void dequant_row32(const uint32_t (&w)[B], float s_lo
     }
 }
 
-template <int B, int NT>
+template <int B, int NT, bool TWO>
 __global__ void __launch_bounds__(kThreads, (NT == 1 && B != 8) ? 2 : 1)
 decode_fwd_kernel(const Params p) {
     constexpr int NS = num_stages<B, NT>();
@@ -106,11 +107,11 @@ decode_fwd_kernel(const Params p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
     uint8_t* ring = base;
-    float* part = reinterpret_cast<float*>(ring + NS * STAGE);        // [128][MT] partial sums of this CTA
+    float* part = reinterpret_cast<float*>(ring + NS * STAGE);        // 128 x MT partial sums of this CTA, fragment order
     float* lut8 = part + 128 * MT;                                     // 256 floats (8-bit codes only)
     uint64_t* bars = reinterpret_cast<uint64_t*>(lut8 + (B == 8 ? 256 : 0));   // full[NS], empty[NS]
     volatile int* abort_s = reinterpret_cast<volatile int*>(bars + 2 * NS);
-    float* stab = reinterpret_cast<float*>(bars + 2 * NS + 2);         // [nkb][128] block scales s~
+    float* stab = reinterpret_cast<float*>(bars + 2 * NS + 2);         // [nkb][kStabStride] block scales s~
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile_row = blockIdx.x;
@@ -147,15 +148,29 @@ decode_fwd_kernel(const Params p) {
     // block scales of the CTA's rows and columns: s~ = fl32(float(s^) * fl32(v / 127)), 0 for rows past N
     const int kb_first = (kt0 * kTileCols) >> q.logB0;
     const int nkb = (ntiles_cta > 0) ? (((kt1 * kTileCols - 1) >> q.logB0) - kb_first + 1) : 0;
-    for (int idx = threadIdx.x; idx < nkb * 128; idx += kThreads) {
-        const int row = idx / nkb, kb = idx - row * nkb;
-        const int grow = tile_row * 128 + row;
-        float val = 0.0f;
-        if (grow < q.N) {
-            const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first + kb;
-            val = block_scale(__ldg(q.sc + blk), __ldg(q.v + (blk >> q.logB1)));
+    // (four elements per thread and pass, all loads requested before the first is used)
+    for (int e0 = threadIdx.x; e0 < nkb * 128; e0 += 4 * kThreads) {
+        uint32_t sc8[4];
+        float v[4];
+        int slot[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int e = e0 + u * kThreads;
+            sc8[u] = 0u; v[u] = 0.0f; slot[u] = -1;
+            if (e < nkb * 128) {
+                const int row = e / nkb, kb = e - row * nkb;
+                const int grow = tile_row * 128 + row;
+                slot[u] = kb * kStabStride + row;
+                if (grow < q.N) {
+                    const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first + kb;
+                    sc8[u] = __ldg(q.sc + blk);
+                    v[u] = __ldg(q.v + (blk >> q.logB1));
+                }
+            }
         }
-        stab[kb * 128 + row] = val;
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (slot[u] >= 0) stab[slot[u]] = block_scale(static_cast<uint8_t>(sc8[u]), v[u]);
     }
     if constexpr (B == 8) {
         for (int i = threadIdx.x; i < 256; i += kThreads) lut8[i] = c_codebook[3][i];
@@ -177,6 +192,7 @@ decode_fwd_kernel(const Params p) {
         if (lane == 0) {
             for (int it = NS; it < nstage_total; ++it) {
                 const int s = it % NS;
+                while (!mbar_try_wait(empty(s), ((it / NS) & 1) ^ 1) && !*abort_s) __nanosleep(200);   // leave the issue slots to the consumers
                 if (!wait(empty(s), ((it / NS) & 1) ^ 1, ctl, 21)) break;
                 issue_stage(it);
             }
@@ -192,42 +208,43 @@ decode_fwd_kernel(const Params p) {
         // ------------------------------------------------------------------ consumers
         const int gid = lane >> 2, t = lane & 3;
         const int win_slot = warp & 3, half = warp >> 2;
-        const bool two_scales = (q.B0 == 16);
         bool ok = true;
         for (int it = 0; it < nstage_total && ok; ++it) {
             const int s = it % NS;
+            const int tiles_here = min(kStageTiles, ntiles_cta - it * kStageTiles);
+            const bool active = 2 * win_slot < tiles_here;
+            const int tile_in_stage = 2 * win_slot + (t >> 1);
+            const bool kt_ok = tile_in_stage < tiles_here;
+            const int col0 = (kt0 + it * kStageTiles + tile_in_stage) * kTileCols + (t & 1) * 32;
+            // the activations of the window do not depend on the packed data: request them before waiting
+            uint4 x[NT][4];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const int m = nt * 8 + gid;
+                if (active && m < p.M && kt_ok) {
+                    const uint4* xp = reinterpret_cast<const uint4*>(p.X + static_cast<size_t>(m) * q.K + col0);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) x[nt][c] = __ldg(xp + c);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) x[nt][c] = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
             ok = wait(full(s), (it / NS) & 1, ctl, 22);
             if (!ok) break;
-            const int tiles_here = min(kStageTiles, ntiles_cta - it * kStageTiles);
-            if (2 * win_slot < tiles_here) {
-                const int tile_in_stage = 2 * win_slot + (t >> 1);
-                const bool kt_ok = tile_in_stage < tiles_here;
-                const int col0 = (kt0 + it * kStageTiles + tile_in_stage) * kTileCols + (t & 1) * 32;
-                uint4 x[NT][4];
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const int m = nt * 8 + gid;
-                    if (m < p.M && kt_ok) {
-                        const uint4* xp = reinterpret_cast<const uint4*>(p.X + static_cast<size_t>(m) * q.K + col0);
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) x[nt][c] = __ldg(xp + c);
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) x[nt][c] = make_uint4(0u, 0u, 0u, 0u);
-                    }
-                }
+            if (active) {
                 const uint32_t* tile = reinterpret_cast<const uint32_t*>(ring + s * STAGE) + (kt_ok ? tile_in_stage : 0) * (256 * B);
                 const int kb = kt_ok ? ((col0 >> q.logB0) - kb_first) : 0;
 #pragma unroll
                 for (int sl = 0; sl < 2; ++sl) {
                     const int slab = 2 * half + sl;
-                    const uint32_t* sp = tile + slab * (64 * B) + (t & 1) * (B * 32) + 4 * gid;
+                    const uint32_t* sp = tile + slab * (64 * B) + (t & 1) * (B * 32) + slab_row_slot(4 * gid, t & 1, tile_in_stage);
                     uint4 w4[B];
 #pragma unroll
                     for (int i = 0; i < B; ++i) w4[i] = *reinterpret_cast<const uint4*>(sp + i * 32);
-                    float4 sc_lo = *reinterpret_cast<const float4*>(stab + kb * 128 + slab * 32 + 4 * gid);
+                    float4 sc_lo = *reinterpret_cast<const float4*>(stab + kb * kStabStride + slab * 32 + 4 * gid);
                     float4 sc_hi = sc_lo;
-                    if (two_scales) sc_hi = *reinterpret_cast<const float4*>(stab + (kb + 1) * 128 + slab * 32 + 4 * gid);
+                    if (TWO) sc_hi = *reinterpret_cast<const float4*>(stab + (kb + 1) * kStabStride + slab * 32 + 4 * gid);
                     if (!kt_ok) { sc_lo = make_float4(0.f, 0.f, 0.f, 0.f); sc_hi = sc_lo; }
 #pragma unroll
                     for (int set = 0; set < 2; ++set) {
@@ -236,10 +253,10 @@ decode_fwd_kernel(const Params p) {
                             uint32_t w[B];
 #pragma unroll
                             for (int i = 0; i < B; ++i) w[i] = pick(w4[i], 2 * set);
-                            dequant_row32<B>(w, pickf(sc_lo, 2 * set), pickf(sc_hi, 2 * set), two_scales, oa, lut8);
+                            dequant_row32<B, TWO>(w, pickf(sc_lo, 2 * set), pickf(sc_hi, 2 * set), oa, lut8);
 #pragma unroll
                             for (int i = 0; i < B; ++i) w[i] = pick(w4[i], 2 * set + 1);
-                            dequant_row32<B>(w, pickf(sc_lo, 2 * set + 1), pickf(sc_hi, 2 * set + 1), two_scales, ob, lut8);
+                            dequant_row32<B, TWO>(w, pickf(sc_lo, 2 * set + 1), pickf(sc_hi, 2 * set + 1), ob, lut8);
                         }
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
@@ -258,57 +275,71 @@ decode_fwd_kernel(const Params p) {
     }
 
     // ---------------------------------------------------------------------- reduction over the K windows of the CTA
-    // acc[sl][set][nt][e]: row (2 half + sl) * 32 + 4 gid + 2 set + (e >> 1), token nt * 8 + 2 t + (e & 1)
-    for (int round = 0; round < 4; ++round) {
-        if (warp < kConsumerWarps && (warp & 3) == round) {
-            const int gid = lane >> 2, t = lane & 3, half = warp >> 2;
+    // Every consumer warp writes its accumulators, in fragment order, to its own region of the (now
+    // idle) ring; then the four warps that cover the same rows are added into `part`, still in
+    // fragment order:  part[(half * 16 NT + k) * 32 + lane],  k = ((sl * 2 + set) * NT + nt) * 4 + e,
+    // which is row (2 half + sl) * 32 + 4 gid + 2 set + (e >> 1) and token nt * 8 + 2 t + (e & 1).
+    constexpr int KF = 16 * NT;
+    float* red = reinterpret_cast<float*>(ring);
+    __syncthreads();                      // all stages consumed: the ring is free
+    if (warp < kConsumerWarps) {
 #pragma unroll
-            for (int sl = 0; sl < 2; ++sl)
+        for (int sl = 0; sl < 2; ++sl)
 #pragma unroll
-                for (int set = 0; set < 2; ++set)
+            for (int set = 0; set < 2; ++set)
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt)
+                for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int row = (2 * half + sl) * 32 + 4 * gid + 2 * set + (e >> 1);
-                            const int tok = nt * 8 + 2 * t + (e & 1);
-                            float* dst = part + row * MT + tok;
-                            *dst = (round == 0) ? acc[sl][set][nt][e] : *dst + acc[sl][set][nt][e];
-                        }
-        }
-        __syncthreads();
+                    for (int e = 0; e < 4; ++e)
+                        red[(warp * KF + ((sl * 2 + set) * NT + nt) * 4 + e) * 32 + lane] = acc[sl][set][nt][e];
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < 2 * KF * 32; idx += kThreads) {
+        const int half = idx / (KF * 32), rest = idx - half * (KF * 32);
+        const float* src = red + (half * 4 * KF) * 32 + rest;
+        part[idx] = (src[0] + src[KF * 32]) + (src[2 * KF * 32] + src[3 * KF * 32]);
     }
 
     // ---------------------------------------------------------------------- reduction over the K slices (cluster), rank-r term, store
+    // Eight lanes per output: lane `sub` fetches the partial sum of cluster rank `sub` and multiplies
+    // eight (sixteen for r > 64) elements of the rank-r term; a shuffle tree adds the eight lanes.
     cluster_sync_all();
     const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
     const int rows_share = 128 / p.S;
     const int row_lo = static_cast<int>(rank) * rows_share;
     if (p.r > 0) pdl_wait();          // T is written by the kernel launched in front of this one
     const uint32_t part_addr = smem_u32(part);
-    for (int o = threadIdx.x; o < rows_share * p.M; o += kThreads) {
-        const int m = o / rows_share, rl = o - m * rows_share;
+    const int sub = threadIdx.x & 7;
+    const int n_out = rows_share * p.M;
+    for (int o0 = (threadIdx.x >> 3) & ~3; o0 < n_out; o0 += (kThreads >> 3) & ~3) {
+        const int o = o0 + ((threadIdx.x >> 3) & 3);       // a warp handles four consecutive outputs
+        const bool live = o < n_out;
+        const int m = live ? o / rows_share : 0, rl = live ? o - m * rows_share : 0;
         const int row = row_lo + rl;
         const int n = tile_row * 128 + row;
-        if (n >= q.N) continue;
         float sum = 0.0f;
-        for (int rk = 0; rk < p.S; ++rk) sum += ld_dsmem_f32(part_addr + static_cast<uint32_t>(row * MT + m) * 4u, static_cast<uint32_t>(rk));
-        if (p.r > 0) {
-            const uint4* l1 = reinterpret_cast<const uint4*>(p.L1 + static_cast<size_t>(n) * p.r);
-            const uint4* tt = reinterpret_cast<const uint4*>(p.T + static_cast<size_t>(m) * p.r);
-            float lr = 0.0f;
-            for (int j = 0; j < p.r / 8; ++j) {
-                const uint4 a = __ldg(l1 + j), b = tt[j];
+        if (live && sub < p.S) {
+            const int half = row >> 6, sl = (row >> 5) & 1, r32 = row & 31;
+            const int k = (((sl * 2 + ((r32 >> 1) & 1)) * NT + (m >> 3)) * 4) + (r32 & 1) * 2 + (m & 1);
+            const int ln = (r32 >> 2) * 4 + ((m & 7) >> 1);
+            sum = ld_dsmem_f32(part_addr + static_cast<uint32_t>((half * KF + k) * 32 + ln) * 4u, static_cast<uint32_t>(sub));
+        }
+        if (live && p.r > 0 && n < q.N) {
+            for (int j = sub; j < p.r / 8; j += 8) {
+                const uint4 a = __ldg(reinterpret_cast<const uint4*>(p.L1 + static_cast<size_t>(n) * p.r) + j);
+                const uint4 b = *(reinterpret_cast<const uint4*>(p.T + static_cast<size_t>(m) * p.r) + j);
                 const uint32_t aa[4] = {a.x, a.y, a.z, a.w}, bb[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    lr = fmaf(__uint_as_float(aa[e] << 16), __uint_as_float(bb[e] << 16), lr);
-                    lr = fmaf(__uint_as_float(aa[e] & 0xffff0000u), __uint_as_float(bb[e] & 0xffff0000u), lr);
+                    sum = fmaf(__uint_as_float(aa[e] << 16), __uint_as_float(bb[e] << 16), sum);
+                    sum = fmaf(__uint_as_float(aa[e] & 0xffff0000u), __uint_as_float(bb[e] & 0xffff0000u), sum);
                 }
             }
-            sum += lr;
         }
-        p.Y[static_cast<size_t>(m) * q.N + n] = __float2bfloat16_rn(sum);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+        if (live && sub == 0 && n < q.N) p.Y[static_cast<size_t>(m) * q.N + n] = __float2bfloat16_rn(sum);
     }
     cluster_sync_all();               // shared memory of this CTA may be read by its peers until here
 }
@@ -325,67 +356,101 @@ struct PreParams {
     __nv_bfloat16* T;
     int* status;       // cleared here: this kernel is the first of a call
     int M, C, r;
-    int chunk;         // contraction elements per CTA (multiple of 32)
+    int chunk;         // contraction elements per CTA (multiple of 64)
     int nranks;
 };
 
-template <bool BWD>
-__global__ void __launch_bounds__(256) decode_pre_kernel(const PreParams p) {
-    __shared__ float red[4][16][64];
-    __shared__ float part[16][128];
+constexpr int kPreThreads = 512;      // 64 columns j x 8 contraction phases
+
+// Dynamic shared memory: [A slice: 16 rows x chunk bf16][red: 8 x 16 x 64 fp32][part: 16 x 128 fp32]
+// MP = M rounded up to a power of two: the row loops are unrolled to MP so that the code stays small for M = 1.
+template <bool BWD, int MP>
+__global__ void __launch_bounds__(kPreThreads) decode_pre_kernel(const PreParams p) {
+    extern __shared__ uint8_t pre_smem[];
+    __nv_bfloat16* as = reinterpret_cast<__nv_bfloat16*>(pre_smem);
+    float* red = reinterpret_cast<float*>(pre_smem + static_cast<size_t>(16) * p.chunk * 2);
+    float* part = red + 8 * 16 * 64;
     pdl_launch_dependents();
     if (blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0;
     const int jl = threadIdx.x & 63, ph = threadIdx.x >> 6;
     const int c_lo = blockIdx.x * p.chunk;
     const int c_hi = min(p.C, c_lo + p.chunk);
+    // stage the CTA's slice of A (rows past M and columns past the end read as zero)
+    const int vec_per_row = p.chunk >> 3;
+    for (int i = threadIdx.x; i < MP * vec_per_row; i += kPreThreads) {
+        const int m = i / vec_per_row, v = i - m * vec_per_row;
+        const int c = c_lo + v * 8;
+        uint4 val = make_uint4(0u, 0u, 0u, 0u);
+        if (m < p.M && c < c_hi) val = __ldg(reinterpret_cast<const uint4*>(p.A + static_cast<size_t>(m) * p.C + c));
+        *reinterpret_cast<uint4*>(as + static_cast<size_t>(m) * p.chunk + v * 8) = val;
+    }
+    __syncthreads();
+    const int span = p.chunk >> 3;                 // contraction elements per phase (multiple of 8)
     for (int jb = 0; jb < p.r; jb += 64) {
         const int j = jb + jl;
-        float acc[16];
+        float acc[MP];
 #pragma unroll
-        for (int m = 0; m < 16; ++m) acc[m] = 0.0f;
+        for (int m = 0; m < MP; ++m) acc[m] = 0.0f;
         if (j < p.r) {
-            for (int c = c_lo + ph * 8; c < c_hi; c += 32) {
-                float f[8];
-                if (!BWD) {
-                    const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.F + static_cast<size_t>(j) * p.C + c));
-                    const uint32_t vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll 1
+            for (int cc = ph * span; cc < (ph + 1) * span; cc += 64) {
+                // eight vectors of eight factors, all requested before the first is used
+                float f[8][8];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) { f[2 * e] = __uint_as_float(vv[e] << 16); f[2 * e + 1] = __uint_as_float(vv[e] & 0xffff0000u); }
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) f[e] = (c + e < c_hi) ? __bfloat162float(p.F[static_cast<size_t>(c + e) * p.r + j]) : 0.0f;
-                }
-#pragma unroll
-                for (int m = 0; m < 16; ++m) {
-                    if (m < p.M) {
-                        const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.A + static_cast<size_t>(m) * p.C + c));
+                for (int u = 0; u < 8; ++u) {
+                    const int c = c_lo + cc + u * 8;
+                    const bool in = (cc + u * 8 < (ph + 1) * span) && (c < c_hi);
+                    if (!BWD) {
+                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                        if (in) v = __ldg(reinterpret_cast<const uint4*>(p.F + static_cast<size_t>(j) * p.C + c));
                         const uint32_t vv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            acc[m] = fmaf(__uint_as_float(vv[e] << 16), f[2 * e], acc[m]);
-                            acc[m] = fmaf(__uint_as_float(vv[e] & 0xffff0000u), f[2 * e + 1], acc[m]);
+                        for (int e = 0; e < 4; ++e) { f[u][2 * e] = __uint_as_float(vv[e] << 16); f[u][2 * e + 1] = __uint_as_float(vv[e] & 0xffff0000u); }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) f[u][e] = in ? __bfloat162float(p.F[static_cast<size_t>(c + e) * p.r + j]) : 0.0f;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (cc + u * 8 < (ph + 1) * span) {
+#pragma unroll
+                        for (int m = 0; m < MP; ++m) {
+                            if (m < p.M) {
+                                const uint4 v = *reinterpret_cast<const uint4*>(as + static_cast<size_t>(m) * p.chunk + cc + u * 8);
+                                const uint32_t vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    acc[m] = fmaf(__uint_as_float(vv[e] << 16), f[u][2 * e], acc[m]);
+                                    acc[m] = fmaf(__uint_as_float(vv[e] & 0xffff0000u), f[u][2 * e + 1], acc[m]);
+                                }
+                            }
                         }
                     }
                 }
             }
         }
 #pragma unroll
-        for (int m = 0; m < 16; ++m) red[ph][m][jl] = acc[m];
+        for (int m = 0; m < MP; ++m) red[(ph * 16 + m) * 64 + jl] = acc[m];
         __syncthreads();
-        for (int o = threadIdx.x; o < 16 * 64; o += 256) {
-            const int m = o >> 6, jj = o & 63;
-            part[m][jb + jj] = red[0][m][jj] + red[1][m][jj] + red[2][m][jj] + red[3][m][jj];
+        for (int o = threadIdx.x; o < MP * 64; o += kPreThreads) {
+            float sum = 0.0f;
+#pragma unroll
+            for (int q8 = 0; q8 < 8; ++q8) sum += red[q8 * 16 * 64 + o];
+            part[(o >> 6) * 128 + jb + (o & 63)] = sum;
         }
         __syncthreads();
     }
     cluster_sync_all();
     if (p.nranks == 1 || cluster_ctarank() == 0) {
-        const uint32_t part_addr = smem_u32(&part[0][0]);
-        for (int o = threadIdx.x; o < p.M * p.r; o += 256) {
+        const uint32_t part_addr = smem_u32(part);
+        for (int o = threadIdx.x; o < p.M * p.r; o += kPreThreads) {
             const int m = o / p.r, j = o - m * p.r;
-            float sum = 0.0f;
-            for (int rk = 0; rk < p.nranks; ++rk) sum += ld_dsmem_f32(part_addr + static_cast<uint32_t>(m * 128 + j) * 4u, static_cast<uint32_t>(rk));
-            p.T[o] = __float2bfloat16_rn(sum);
+            float v[8];
+#pragma unroll
+            for (int rk = 0; rk < 8; ++rk)
+                v[rk] = (rk < p.nranks) ? ld_dsmem_f32(part_addr + static_cast<uint32_t>(m * 128 + j) * 4u, static_cast<uint32_t>(rk)) : 0.0f;
+            p.T[o] = __float2bfloat16_rn(((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7])));
         }
     }
     cluster_sync_all();
@@ -401,7 +466,7 @@ struct Plan {
 template <int B, int NT>
 inline size_t smem_bytes(int nkb_cap) {
     return 128 + static_cast<size_t>(num_stages<B, NT>()) * stage_bytes<B>() + 128 * 8 * NT * 4 + (B == 8 ? 1024 : 0) +
-           (2 * num_stages<B, NT>() + 2) * 8 + static_cast<size_t>(nkb_cap) * 512;
+           (2 * num_stages<B, NT>() + 2) * 8 + static_cast<size_t>(nkb_cap) * (kStabStride * 4);
 }
 
 inline int sm_count_cached() {
@@ -442,7 +507,7 @@ inline Plan make_plan(const QView& q, int M) {
 }
 
 inline bool supported(const QView& q, int64_t M) {
-    if (M > 16 || q.K % 8 != 0) return false;
+    if (M > 16 || q.K % 8 != 0 || q.K > 49152) return false;   // the pre-product stages K / 8 columns of X per CTA
     if (static_cast<long long>(q.N) * q.KB >= (1LL << 31)) return false;
     switch (q.b0) {
         case 2: return make_plan<2>(q, static_cast<int>(M)).ok;
@@ -459,13 +524,32 @@ inline cudaError_t launch_pre(const __nv_bfloat16* A, const __nv_bfloat16* F, __
     PreParams pp;
     pp.A = A; pp.F = F; pp.T = T; pp.status = status; pp.M = M; pp.C = C; pp.r = r;
     int nranks = 8;
-    while (nranks > 1 && C / nranks < 256) nranks >>= 1;
+    while (nranks > 1 && C / nranks < 512) nranks >>= 1;
     int chunk = (C + nranks - 1) / nranks;
-    chunk = (chunk + 31) / 32 * 32;
+    chunk = (chunk + 63) / 64 * 64;
     pp.chunk = chunk; pp.nranks = nranks;
+    const size_t smem = static_cast<size_t>(16) * chunk * 2 + (8 * 16 * 64 + 16 * 128) * sizeof(float);
+    if (smem > static_cast<size_t>(kSmemLimit)) return cudaErrorInvalidValue;
+    void (*kern)(PreParams) = decode_pre_kernel<BWD, 16>;
+    if (M <= 1) kern = decode_pre_kernel<BWD, 1>;
+    else if (M <= 2) kern = decode_pre_kernel<BWD, 2>;
+    else if (M <= 4) kern = decode_pre_kernel<BWD, 4>;
+    else if (M <= 8) kern = decode_pre_kernel<BWD, 8>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaSuccess;
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_pre_kernel<BWD, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_pre_kernel<BWD, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_pre_kernel<BWD, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_pre_kernel<BWD, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_pre_kernel<BWD, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(nranks);
-    cfg.blockDim = dim3(256);
+    cfg.blockDim = dim3(kPreThreads);
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -473,12 +557,12 @@ inline cudaError_t launch_pre(const __nv_bfloat16* A, const __nv_bfloat16* F, __
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     count_launch(1);
-    return cudaLaunchKernelEx(&cfg, decode_pre_kernel<BWD>, pp);
+    return cudaLaunchKernelEx(&cfg, kern, pp);
 }
 
-template <int B, int NT>
+template <int B, int NT, bool TWO>
 inline cudaError_t launch_fwd_nt(const Params& p, const Plan& pl, bool after_pre, cudaStream_t st) {
-    auto kern = decode_fwd_kernel<B, NT>;
+    auto kern = decode_fwd_kernel<B, NT, TWO>;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
@@ -520,7 +604,8 @@ inline cudaError_t launch_fwd(const QView& q, const void* L1, const void* L2, in
                                           p.status, M, q.K, r, st);
         if (e != cudaSuccess) return e;
     }
-    return (pl.NT == 1) ? launch_fwd_nt<B, 1>(p, pl, r > 0, st) : launch_fwd_nt<B, 2>(p, pl, r > 0, st);
+    if (q.B0 == 16) return (pl.NT == 1) ? launch_fwd_nt<B, 1, true>(p, pl, r > 0, st) : launch_fwd_nt<B, 2, true>(p, pl, r > 0, st);
+    return (pl.NT == 1) ? launch_fwd_nt<B, 1, false>(p, pl, r > 0, st) : launch_fwd_nt<B, 2, false>(p, pl, r > 0, st);
 }
 
 }  // namespace dec

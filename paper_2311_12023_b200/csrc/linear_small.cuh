@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(128) small_fwd_kernel(QView q, const __nv_bflo
         if (kbase >= q.K) continue;          // K is a multiple of 64: the last window may be half empty
         const uint32_t* slab = q.codes + slab_word_base(rowgroup * 32, kbase >> 6, q.ktiles, B);
         uint4 w[B];
-        load_group4<B>(slab, (kbase >> 5) & 1, 4 * rq, w);
+        load_group4<B>(slab, (kbase >> 5) & 1, slab_row_slot(4 * rq, (kbase >> 5) & 1, kbase >> 6), w);
         // activations of this lane's 32 columns
         float x[MT][32];
 #pragma unroll
@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(128) small_bwd_kernel(QView q, const __nv_bflo
     for (int rg = g_lo; rg < g_hi && kact; ++rg) {
         const uint32_t* slab = q.codes + slab_word_base(rg * 32, kbase >> 6, q.ktiles, B);
         uint4 w[B];
-        load_group4<B>(slab, (kbase >> 5) & 1, 4 * rq, w);
+        load_group4<B>(slab, (kbase >> 5) & 1, slab_row_slot(4 * rq, (kbase >> 5) & 1, kbase >> 6), w);
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             const int row = rg * 32 + 4 * rq + r;
@@ -261,7 +261,7 @@ inline cudaError_t launch_small(const QView& q, const void* L1, const void* L2, 
         launches += 2;
     } else {
         if (r > 0) {
-            if (M <= 16 && q.N % 8 == 0) {
+            if (M <= 16 && q.N % 8 == 0 && q.N <= 49152) {
                 const cudaError_t e = dec::launch_pre<true>(a, l1, T, reinterpret_cast<int*>(ws), M, q.N, r, st);
                 if (e != cudaSuccess) return e;
             } else {

@@ -355,7 +355,11 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         RawScale slot[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) slot[u] = (u < p.steps_q) ? fetch(u) : RawScale{0u, 0.0f};
-        const uint32_t* __restrict__ my_slab = reinterpret_cast<const uint32_t*>(p_ring) + slab_i * (64 * B) + g * (B * 32) + lane;
+        // word plane slot of this thread's row: rotated by 8 g + 16 (tile column % 2), see slab_row_slot();
+        // forward: the tile column is the step index, backward: it is fixed per thread
+        const uint32_t* __restrict__ slab_base = reinterpret_cast<const uint32_t*>(p_ring) + slab_i * (64 * B) + g * (B * 32);
+        const int slot_even = slab_row_slot(lane, g, BWD ? ((c0 >> 6) + (slab_i >> 1)) : 0);
+        const int slot_odd = BWD ? slot_even : slab_row_slot(lane, g, 1);
         uint8_t* my_b = b_ring + b_off;
         bool ok = true;
         RingPos<SA> ra;
@@ -373,7 +377,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (step + 4 < p.steps_q) slot[u] = fetch(step + 4);
                     ok = wait(full_a(sa), ra.ph, ctl, 4);
                     if (!ok) break;
-                    dequant_group<B>(my_slab + sa * (P_BYTES / 4), s_lo, s_hi, two_scales, my_b + sb * kBBytes, g << 6, xr, lut8);
+                    dequant_group<B>(slab_base + sa * (P_BYTES / 4) + ((step & 1) ? slot_odd : slot_even), s_lo, s_hi, two_scales, my_b + sb * kBBytes, g << 6, xr, lut8);
                     fence_proxy_async();            // make the generic-proxy stores visible to the tensor core
                     __syncwarp();
                     if (lane == 0) mbar_arrive(full_b(sb));
