@@ -356,7 +356,7 @@ struct PreParams {
     __nv_bfloat16* T;
     int* status;       // cleared here: this kernel is the first of a call
     int M, C, r;
-    int chunk;         // contraction elements per CTA (multiple of 64)
+    int chunk;         // contraction elements per CTA (multiple of 512)
     int nranks;
 };
 
@@ -388,9 +388,10 @@ __global__ void __launch_bounds__(kPreThreads) decode_pre_kernel(const PreParams
     const int span = p.chunk >> 3;                 // contraction elements per phase (multiple of 8)
     for (int jb = 0; jb < p.r; jb += 64) {
         const int j = jb + jl;
-        float acc[MP];
-#pragma unroll
-        for (int m = 0; m < MP; ++m) acc[m] = 0.0f;
+        // this thread's slots of `red` hold its sums; the row loop is not unrolled (small code: the kernel
+        // runs once per SM, so instruction fetch is part of its latency)
+#pragma unroll 1
+        for (int m = 0; m < MP; ++m) red[(ph * 16 + m) * 64 + jl] = 0.0f;
         if (j < p.r) {
 #pragma unroll 1
             for (int cc = ph * span; cc < (ph + 1) * span; cc += 64) {
@@ -411,27 +412,24 @@ __global__ void __launch_bounds__(kPreThreads) decode_pre_kernel(const PreParams
                         for (int e = 0; e < 8; ++e) f[u][e] = in ? __bfloat162float(p.F[static_cast<size_t>(c + e) * p.r + j]) : 0.0f;
                     }
                 }
+#pragma unroll 1
+                for (int m = 0; m < p.M; ++m) {
+                    float acc = 0.0f;
+                    const __nv_bfloat16* arow = as + static_cast<size_t>(m) * p.chunk + cc;
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (cc + u * 8 < (ph + 1) * span) {
+                    for (int u = 0; u < 8; ++u) {
+                        const uint4 v = *reinterpret_cast<const uint4*>(arow + u * 8);
+                        const uint32_t vv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-                        for (int m = 0; m < MP; ++m) {
-                            if (m < p.M) {
-                                const uint4 v = *reinterpret_cast<const uint4*>(as + static_cast<size_t>(m) * p.chunk + cc + u * 8);
-                                const uint32_t vv[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    acc[m] = fmaf(__uint_as_float(vv[e] << 16), f[u][2 * e], acc[m]);
-                                    acc[m] = fmaf(__uint_as_float(vv[e] & 0xffff0000u), f[u][2 * e + 1], acc[m]);
-                                }
-                            }
+                        for (int e = 0; e < 4; ++e) {
+                            acc = fmaf(__uint_as_float(vv[e] << 16), f[u][2 * e], acc);
+                            acc = fmaf(__uint_as_float(vv[e] & 0xffff0000u), f[u][2 * e + 1], acc);
                         }
                     }
+                    red[(ph * 16 + m) * 64 + jl] += acc;
                 }
             }
         }
-#pragma unroll
-        for (int m = 0; m < MP; ++m) red[(ph * 16 + m) * 64 + jl] = acc[m];
         __syncthreads();
         for (int o = threadIdx.x; o < MP * 64; o += kPreThreads) {
             float sum = 0.0f;
@@ -507,7 +505,7 @@ inline Plan make_plan(const QView& q, int M) {
 }
 
 inline bool supported(const QView& q, int64_t M) {
-    if (M > 16 || q.K % 8 != 0 || q.K > 49152) return false;   // the pre-product stages K / 8 columns of X per CTA
+    if (M > 16 || q.K % 8 != 0 || q.K > 40960) return false;   // the pre-product stages K / 8 columns of X per CTA
     if (static_cast<long long>(q.N) * q.KB >= (1LL << 31)) return false;
     switch (q.b0) {
         case 2: return make_plan<2>(q, static_cast<int>(M)).ok;
@@ -526,7 +524,7 @@ inline cudaError_t launch_pre(const __nv_bfloat16* A, const __nv_bfloat16* F, __
     int nranks = 8;
     while (nranks > 1 && C / nranks < 512) nranks >>= 1;
     int chunk = (C + nranks - 1) / nranks;
-    chunk = (chunk + 63) / 64 * 64;
+    chunk = (chunk + 511) / 512 * 512;      // every one of the eight phases then covers whole groups of 64 columns
     pp.chunk = chunk; pp.nranks = nranks;
     const size_t smem = static_cast<size_t>(16) * chunk * 2 + (8 * 16 * 64 + 16 * 128) * sizeof(float);
     if (smem > static_cast<size_t>(kSmemLimit)) return cudaErrorInvalidValue;
