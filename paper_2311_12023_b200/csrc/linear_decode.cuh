@@ -356,99 +356,99 @@ struct PreParams {
     __nv_bfloat16* T;
     int* status;       // cleared here: this kernel is the first of a call
     int M, C, r;
-    int chunk;         // contraction elements per CTA (multiple of 512)
+    int chunk;         // contraction elements per CTA (multiple of 8)
     int nranks;
 };
 
-constexpr int kPreThreads = 512;      // 64 columns j x 8 contraction phases
+constexpr int kPreThreads = 512;      // 16 columns j x 32 contraction phases
+constexpr int kPreJ = 16;             // columns of T per CTA
+constexpr int kPrePhases = kPreThreads / kPreJ;
 
-// Dynamic shared memory: [A slice: 16 rows x chunk bf16][red: 8 x 16 x 64 fp32][part: 16 x 128 fp32]
-// MP = M rounded up to a power of two: the row loops are unrolled to MP so that the code stays small for M = 1.
+// Grid (ranks, r / 16), cluster (ranks, 1, 1): a cluster computes 16 columns of T, each of its CTAs over a slice
+// of the contraction.  Dynamic shared memory: [A slice: MP rows x chunk bf16][red: 32 x 16 x 16 fp32][part: 16 x 16 fp32]
+// MP = M rounded up to a power of two (rows staged).
 template <bool BWD, int MP>
 __global__ void __launch_bounds__(kPreThreads) decode_pre_kernel(const PreParams p) {
     extern __shared__ uint8_t pre_smem[];
     __nv_bfloat16* as = reinterpret_cast<__nv_bfloat16*>(pre_smem);
-    float* red = reinterpret_cast<float*>(pre_smem + static_cast<size_t>(16) * p.chunk * 2);
-    float* part = red + 8 * 16 * 64;
+    float* red = reinterpret_cast<float*>(pre_smem + static_cast<size_t>(MP) * p.chunk * 2);
+    float* part = red + kPrePhases * 16 * kPreJ;
     pdl_launch_dependents();
-    if (blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0;
-    const int jl = threadIdx.x & 63, ph = threadIdx.x >> 6;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.status = 0;
+    const int jl = threadIdx.x & (kPreJ - 1), ph = threadIdx.x / kPreJ;
+    const int j = blockIdx.y * kPreJ + jl;
     const int c_lo = blockIdx.x * p.chunk;
     const int c_hi = min(p.C, c_lo + p.chunk);
     // stage the CTA's slice of A (rows past M and columns past the end read as zero)
-    const int vec_per_row = p.chunk >> 3;
-    for (int i = threadIdx.x; i < MP * vec_per_row; i += kPreThreads) {
-        const int m = i / vec_per_row, v = i - m * vec_per_row;
+    const int nvec = p.chunk >> 3;
+    for (int i = threadIdx.x; i < MP * nvec; i += kPreThreads) {
+        const int m = i / nvec, v = i - m * nvec;
         const int c = c_lo + v * 8;
         uint4 val = make_uint4(0u, 0u, 0u, 0u);
         if (m < p.M && c < c_hi) val = __ldg(reinterpret_cast<const uint4*>(p.A + static_cast<size_t>(m) * p.C + c));
         *reinterpret_cast<uint4*>(as + static_cast<size_t>(m) * p.chunk + v * 8) = val;
     }
+#pragma unroll 1
+    for (int m = 0; m < 16; ++m) red[(ph * 16 + m) * kPreJ + jl] = 0.0f;
     __syncthreads();
-    const int span = p.chunk >> 3;                 // contraction elements per phase (multiple of 8)
-    for (int jb = 0; jb < p.r; jb += 64) {
-        const int j = jb + jl;
-        // this thread's slots of `red` hold its sums; the row loop is not unrolled (small code: the kernel
-        // runs once per SM, so instruction fetch is part of its latency)
+    if (j < p.r) {
+        // vectors of eight contraction elements, phase ph takes vectors ph, ph + 32, ...; four are in flight at a time
 #pragma unroll 1
-        for (int m = 0; m < MP; ++m) red[(ph * 16 + m) * 64 + jl] = 0.0f;
-        if (j < p.r) {
-#pragma unroll 1
-            for (int cc = ph * span; cc < (ph + 1) * span; cc += 64) {
-                // eight vectors of eight factors, all requested before the first is used
-                float f[8][8];
+        for (int v0 = ph; v0 < nvec; v0 += 4 * kPrePhases) {
+            float f[4][8];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int c = c_lo + cc + u * 8;
-                    const bool in = (cc + u * 8 < (ph + 1) * span) && (c < c_hi);
-                    if (!BWD) {
-                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                        if (in) v = __ldg(reinterpret_cast<const uint4*>(p.F + static_cast<size_t>(j) * p.C + c));
-                        const uint32_t vv[4] = {v.x, v.y, v.z, v.w};
+            for (int u = 0; u < 4; ++u) {
+                const int v = v0 + u * kPrePhases;
+                const int c = c_lo + v * 8;
+                const bool in = (v < nvec) && (c < c_hi);
+                if (!BWD) {
+                    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+                    if (in) w = __ldg(reinterpret_cast<const uint4*>(p.F + static_cast<size_t>(j) * p.C + c));
+                    const uint32_t vv[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) { f[u][2 * e] = __uint_as_float(vv[e] << 16); f[u][2 * e + 1] = __uint_as_float(vv[e] & 0xffff0000u); }
-                    } else {
+                    for (int e = 0; e < 4; ++e) { f[u][2 * e] = __uint_as_float(vv[e] << 16); f[u][2 * e + 1] = __uint_as_float(vv[e] & 0xffff0000u); }
+                } else {
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) f[u][e] = in ? __bfloat162float(p.F[static_cast<size_t>(c + e) * p.r + j]) : 0.0f;
-                    }
-                }
-#pragma unroll 1
-                for (int m = 0; m < p.M; ++m) {
-                    float acc = 0.0f;
-                    const __nv_bfloat16* arow = as + static_cast<size_t>(m) * p.chunk + cc;
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const uint4 v = *reinterpret_cast<const uint4*>(arow + u * 8);
-                        const uint32_t vv[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            acc = fmaf(__uint_as_float(vv[e] << 16), f[u][2 * e], acc);
-                            acc = fmaf(__uint_as_float(vv[e] & 0xffff0000u), f[u][2 * e + 1], acc);
-                        }
-                    }
-                    red[(ph * 16 + m) * 64 + jl] += acc;
+                    for (int e = 0; e < 8; ++e) f[u][e] = in ? __bfloat162float(p.F[static_cast<size_t>(c + e) * p.r + j]) : 0.0f;
                 }
             }
-        }
-        __syncthreads();
-        for (int o = threadIdx.x; o < MP * 64; o += kPreThreads) {
-            float sum = 0.0f;
+#pragma unroll 1
+            for (int m = 0; m < p.M; ++m) {
+                float acc = 0.0f;
 #pragma unroll
-            for (int q8 = 0; q8 < 8; ++q8) sum += red[q8 * 16 * 64 + o];
-            part[(o >> 6) * 128 + jb + (o & 63)] = sum;
+                for (int u = 0; u < 4; ++u) {
+                    const int v = min(v0 + u * kPrePhases, nvec - 1);      // past the end: factors are zero
+                    const uint4 w = *reinterpret_cast<const uint4*>(as + static_cast<size_t>(m) * p.chunk + v * 8);
+                    const uint32_t vv[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        acc = fmaf(__uint_as_float(vv[e] << 16), f[u][2 * e], acc);
+                        acc = fmaf(__uint_as_float(vv[e] & 0xffff0000u), f[u][2 * e + 1], acc);
+                    }
+                }
+                red[(ph * 16 + m) * kPreJ + jl] += acc;
+            }
         }
-        __syncthreads();
+    }
+    __syncthreads();
+    if (threadIdx.x < 16 * kPreJ) {
+        float sum = 0.0f;
+#pragma unroll 8
+        for (int q8 = 0; q8 < kPrePhases; ++q8) sum += red[q8 * 16 * kPreJ + threadIdx.x];
+        part[threadIdx.x] = sum;          // part[m * 16 + jl]
     }
     cluster_sync_all();
     if (p.nranks == 1 || cluster_ctarank() == 0) {
         const uint32_t part_addr = smem_u32(part);
-        for (int o = threadIdx.x; o < p.M * p.r; o += kPreThreads) {
-            const int m = o / p.r, j = o - m * p.r;
-            float v[8];
+        if (threadIdx.x < 16 * kPreJ) {
+            const int m = threadIdx.x / kPreJ, jj = blockIdx.y * kPreJ + (threadIdx.x & (kPreJ - 1));
+            if (m < p.M && jj < p.r) {
+                float v[8];
 #pragma unroll
-            for (int rk = 0; rk < 8; ++rk)
-                v[rk] = (rk < p.nranks) ? ld_dsmem_f32(part_addr + static_cast<uint32_t>(m * 128 + j) * 4u, static_cast<uint32_t>(rk)) : 0.0f;
-            p.T[o] = __float2bfloat16_rn(((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7])));
+                for (int rk = 0; rk < 8; ++rk)
+                    v[rk] = (rk < p.nranks) ? ld_dsmem_f32(part_addr + static_cast<uint32_t>(threadIdx.x) * 4u, static_cast<uint32_t>(rk)) : 0.0f;
+                p.T[static_cast<size_t>(m) * p.r + jj] = __float2bfloat16_rn(((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7])));
+            }
         }
     }
     cluster_sync_all();
@@ -524,9 +524,10 @@ inline cudaError_t launch_pre(const __nv_bfloat16* A, const __nv_bfloat16* F, __
     int nranks = 8;
     while (nranks > 1 && C / nranks < 512) nranks >>= 1;
     int chunk = (C + nranks - 1) / nranks;
-    chunk = (chunk + 511) / 512 * 512;      // every one of the eight phases then covers whole groups of 64 columns
+    chunk = (chunk + 7) / 8 * 8;
     pp.chunk = chunk; pp.nranks = nranks;
-    const size_t smem = static_cast<size_t>(16) * chunk * 2 + (8 * 16 * 64 + 16 * 128) * sizeof(float);
+    const int MP = M <= 1 ? 1 : M <= 2 ? 2 : M <= 4 ? 4 : M <= 8 ? 8 : 16;
+    const size_t smem = static_cast<size_t>(MP) * chunk * 2 + (kPrePhases * 16 * kPreJ + 16 * kPreJ) * sizeof(float);
     if (smem > static_cast<size_t>(kSmemLimit)) return cudaErrorInvalidValue;
     void (*kern)(PreParams) = decode_pre_kernel<BWD, 16>;
     if (M <= 1) kern = decode_pre_kernel<BWD, 1>;
@@ -545,7 +546,7 @@ inline cudaError_t launch_pre(const __nv_bfloat16* A, const __nv_bfloat16* F, __
         attr_done = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(nranks);
+    cfg.gridDim = dim3(nranks, (r + kPreJ - 1) / kPreJ);
     cfg.blockDim = dim3(kPreThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
