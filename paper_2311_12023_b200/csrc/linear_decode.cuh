@@ -27,8 +27,10 @@ constexpr int kStageTiles = 8;              // 64-column tiles per ring stage (f
 constexpr int kSmemLimit = 232448;
 constexpr int kStabStride = 136;            // floats per block column of the scale table (128 rows + padding against bank conflicts)
 
-template <int B> __host__ __device__ constexpr int stage_bytes() { return kStageTiles * 1024 * B; }
+constexpr int kXRowBytes = kStageTiles * kTileCols * 2 + 16;   // one token's activations of a stage, padded
+// A ring stage: the packed tiles, then the activations of the stage's 512 columns for 8 NT token rows.
 // NT = number of 8-token groups (1: M <= 8, two CTAs per SM; 2: M <= 16, one CTA per SM)
+template <int B, int NT> __host__ __device__ constexpr int stage_bytes() { return kStageTiles * 1024 * B + 8 * NT * kXRowBytes; }
 template <int B, int NT> __host__ __device__ constexpr int num_stages() { return (B == 8) ? 2 : (NT == 2 ? 4 : 2); }
 
 struct Params {
@@ -66,34 +68,24 @@ __device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank
 __device__ __forceinline__ uint32_t pick(const uint4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
 __device__ __forceinline__ float pickf(const float4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
 
-// The 32 weights of one (row, group) as sixteen bf16 pairs: o[c][e] holds columns 8c + 2e, 8c + 2e + 1.
-template <int B, bool TWO>
-__device__ __forceinline__ void dequant_row32(const uint32_t (&w)[B], float s_lo, float s_hi,
-                                              uint32_t (&o)[4][4], const float* __restrict__ lut8) {
+// Chunk c (columns 8c .. 8c+7) of one (row, group) as four bf16 pairs: o[e] holds columns 8c + 2e, 8c + 2e + 1.
+template <int B>
+__device__ __forceinline__ void dequant_chunk(const uint32_t (&w)[B], int c, const BlockTable<B>& tab, float s,
+                                              uint32_t (&o)[4], const float* __restrict__ lut8) {
     if constexpr (B == 8) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const float s = (c < 2) ? s_lo : s_hi;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const uint32_t ww = w[2 * c + (e >> 1)] >> (16 * (e & 1));
-                const float q0 = lut8[ww & 255u], q1 = lut8[(ww >> 8) & 255u];
-                const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(q0, s), __fmul_rn(q1, s));
-                o[c][e] = *reinterpret_cast<const uint32_t*>(&h);
-            }
+        for (int e = 0; e < 4; ++e) {
+            const uint32_t ww = w[2 * c + (e >> 1)] >> (16 * (e & 1));
+            const float q0 = lut8[ww & 255u], q1 = lut8[(ww >> 8) & 255u];
+            const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(q0, s), __fmul_rn(q1, s));
+            o[e] = *reinterpret_cast<const uint32_t*>(&h);
         }
     } else {
-        BlockTable<B> tab;
-        tab.build(s_lo);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            if (TWO && c == 2) tab.build(s_hi);
-            const uint32_t sel = chunk_selector<B>(w, c);
-            uint32_t selA = sel, selB = 0u;
-            if constexpr (B == 4) { selA = sel & 0x77777777u; selB = ((sel >> 1) & 0x44444444u) | 0x32103210u; }
-            tab.lookup4(selA, selB, o[c][0], o[c][1]);
-            tab.lookup4(selA >> 16, selB >> 16, o[c][2], o[c][3]);
-        }
+        const uint32_t sel = chunk_selector<B>(w, c);
+        uint32_t selA = sel, selB = 0u;
+        if constexpr (B == 4) { selA = sel & 0x77777777u; selB = ((sel >> 1) & 0x44444444u) | 0x32103210u; }
+        tab.lookup4(selA, selB, o[0], o[1]);
+        tab.lookup4(selA >> 16, selB >> 16, o[2], o[3]);
     }
 }
 
@@ -101,7 +93,8 @@ template <int B, int NT, bool TWO>
 __global__ void __launch_bounds__(kThreads, (NT == 1 && B != 8) ? 2 : 1)
 decode_fwd_kernel(const Params p) {
     constexpr int NS = num_stages<B, NT>();
-    constexpr int STAGE = stage_bytes<B>();
+    constexpr int STAGE = stage_bytes<B, NT>();
+    constexpr int XOFF = kStageTiles * 1024 * B;      // activations inside a stage
     constexpr int MT = 8 * NT;
 
     extern __shared__ uint8_t smem_raw[];
@@ -138,8 +131,12 @@ decode_fwd_kernel(const Params p) {
     auto issue_stage = [&](int it) {
         const int s = it % NS;
         const int nt = min(kStageTiles, ntiles_cta - it * kStageTiles);
-        mbar_expect_tx(full(s), nt * 1024 * B);
-        bulk_load(smem_u32(ring + s * STAGE), codes + static_cast<size_t>(it) * STAGE, nt * 1024 * B, full(s));
+        const uint32_t dst = smem_u32(ring + s * STAGE);
+        mbar_expect_tx(full(s), nt * 1024 * B + p.M * nt * (kTileCols * 2));
+        bulk_load(dst, codes + static_cast<size_t>(it) * (kStageTiles * 1024 * B), nt * 1024 * B, full(s));
+        const __nv_bfloat16* xsrc = p.X + static_cast<size_t>(kt0 + it * kStageTiles) * kTileCols;
+        for (int m = 0; m < p.M; ++m)
+            bulk_load(dst + XOFF + m * kXRowBytes, xsrc + static_cast<size_t>(m) * q.K, nt * (kTileCols * 2), full(s));
     };
     if (warp == kConsumerWarps && lane == 0) {
         for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it);
@@ -148,6 +145,46 @@ decode_fwd_kernel(const Params p) {
     // block scales of the CTA's rows and columns: s~ = fl32(float(s^) * fl32(v / 127)), 0 for rows past N
     const int kb_first = (kt0 * kTileCols) >> q.logB0;
     const int nkb = (ntiles_cta > 0) ? (((kt1 * kTileCols - 1) >> q.logB0) - kb_first + 1) : 0;
+    const bool vec16 = (q.KB % 16 == 0) && (nkb % 16 == 0) && (kb_first % 16 == 0);
+    if (vec16) {
+        // sixteen scale codes per load; they lie in at most two second-level groups (B1 >= 16)
+        const int nvec = nkb >> 4;
+        for (int e0 = threadIdx.x; e0 < nvec * 128; e0 += 2 * kThreads) {
+            uint4 sc16[2];
+            float v0[2], v1[2];
+            int rowv[2], kbv[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int e = e0 + u * kThreads;
+                sc16[u] = make_uint4(0u, 0u, 0u, 0u); v0[u] = v1[u] = 0.0f; rowv[u] = -1; kbv[u] = 0;
+                if (e < nvec * 128) {
+                    const int row = e / nvec, kv = e - row * nvec;
+                    const int grow = tile_row * 128 + row;
+                    rowv[u] = row; kbv[u] = kv * 16;
+                    if (grow < q.N) {
+                        const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first + kv * 16;
+                        sc16[u] = __ldg(reinterpret_cast<const uint4*>(q.sc + blk));
+                        v0[u] = __ldg(q.v + (blk >> q.logB1));
+                        v1[u] = __ldg(q.v + ((blk + 15) >> q.logB1));
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                if (rowv[u] < 0) continue;
+                const int grow = tile_row * 128 + rowv[u];
+                const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first + kbv[u];
+                const uint32_t g0 = blk >> q.logB1;
+                const uint32_t words[4] = {sc16[u].x, sc16[u].y, sc16[u].z, sc16[u].w};
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const uint32_t code = (words[i >> 2] >> (8 * (i & 3))) & 255u;
+                    const float vv = (((blk + i) >> q.logB1) == g0) ? v0[u] : v1[u];
+                    stab[(kbv[u] + i) * kStabStride + rowv[u]] = block_scale(static_cast<uint8_t>(code), vv);
+                }
+            }
+        }
+    } else {
     // (four elements per thread and pass, all loads requested before the first is used)
     for (int e0 = threadIdx.x; e0 < nkb * 128; e0 += 4 * kThreads) {
         uint32_t sc8[4];
@@ -171,6 +208,7 @@ decode_fwd_kernel(const Params p) {
 #pragma unroll
         for (int u = 0; u < 4; ++u)
             if (slot[u] >= 0) stab[slot[u]] = block_scale(static_cast<uint8_t>(sc8[u]), v[u]);
+    }
     }
     if constexpr (B == 8) {
         for (int i = threadIdx.x; i < 256; i += kThreads) lut8[i] = c_codebook[3][i];
@@ -216,25 +254,25 @@ decode_fwd_kernel(const Params p) {
             const int tile_in_stage = 2 * win_slot + (t >> 1);
             const bool kt_ok = tile_in_stage < tiles_here;
             const int col0 = (kt0 + it * kStageTiles + tile_in_stage) * kTileCols + (t & 1) * 32;
-            // the activations of the window do not depend on the packed data: request them before waiting
-            uint4 x[NT][4];
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                const int m = nt * 8 + gid;
-                if (active && m < p.M && kt_ok) {
-                    const uint4* xp = reinterpret_cast<const uint4*>(p.X + static_cast<size_t>(m) * q.K + col0);
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) x[nt][c] = __ldg(xp + c);
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) x[nt][c] = make_uint4(0u, 0u, 0u, 0u);
-                }
-            }
             ok = wait(full(s), (it / NS) & 1, ctl, 22);
             if (!ok) break;
             if (active) {
                 const uint32_t* tile = reinterpret_cast<const uint32_t*>(ring + s * STAGE) + (kt_ok ? tile_in_stage : 0) * (256 * B);
                 const int kb = kt_ok ? ((col0 >> q.logB0) - kb_first) : 0;
+                // activations of this thread's 32 columns (token rows past M and missing tiles read as zero)
+                uint4 x[NT][4];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int m = nt * 8 + gid;
+                    if (m < p.M && kt_ok) {
+                        const uint4* xp = reinterpret_cast<const uint4*>(ring + s * STAGE + XOFF + m * kXRowBytes + (tile_in_stage * kTileCols + (t & 1) * 32) * 2);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) x[nt][c] = xp[c];
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) x[nt][c] = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
 #pragma unroll
                 for (int sl = 0; sl < 2; ++sl) {
                     const int slab = 2 * half + sl;
@@ -248,22 +286,27 @@ decode_fwd_kernel(const Params p) {
                     if (!kt_ok) { sc_lo = make_float4(0.f, 0.f, 0.f, 0.f); sc_hi = sc_lo; }
 #pragma unroll
                     for (int set = 0; set < 2; ++set) {
-                        uint32_t oa[4][4], ob[4][4];
-                        {
-                            uint32_t w[B];
+                        // rows a = 2 set, b = 2 set + 1 of the thread's four; the two MMAs of a chunk are issued right
+                        // after its eight weights are ready, so consecutive MMAs on one accumulator are spaced out
+                        uint32_t wa[B], wb[B];
 #pragma unroll
-                            for (int i = 0; i < B; ++i) w[i] = pick(w4[i], 2 * set);
-                            dequant_row32<B, TWO>(w, pickf(sc_lo, 2 * set), pickf(sc_hi, 2 * set), oa, lut8);
-#pragma unroll
-                            for (int i = 0; i < B; ++i) w[i] = pick(w4[i], 2 * set + 1);
-                            dequant_row32<B, TWO>(w, pickf(sc_lo, 2 * set + 1), pickf(sc_hi, 2 * set + 1), ob, lut8);
-                        }
+                        for (int i = 0; i < B; ++i) { wa[i] = pick(w4[i], 2 * set); wb[i] = pick(w4[i], 2 * set + 1); }
+                        const float sa_lo = pickf(sc_lo, 2 * set), sb_lo = pickf(sc_lo, 2 * set + 1);
+                        const float sa_hi = pickf(sc_hi, 2 * set), sb_hi = pickf(sc_hi, 2 * set + 1);
+                        BlockTable<B> ta, tb;
+                        if constexpr (B != 8) { ta.build(sa_lo); tb.build(sb_lo); }
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
+                            if constexpr (B != 8) {
+                                if (TWO && c == 2) { ta.build(sa_hi); tb.build(sb_hi); }
+                            }
+                            uint32_t oa[4], ob[4];
+                            dequant_chunk<B>(wa, c, ta, (TWO && c >= 2) ? sa_hi : sa_lo, oa, lut8);
+                            dequant_chunk<B>(wb, c, tb, (TWO && c >= 2) ? sb_hi : sb_lo, ob, lut8);
 #pragma unroll
                             for (int nt = 0; nt < NT; ++nt) {
-                                mma16816(acc[sl][set][nt], oa[c][0], ob[c][0], oa[c][1], ob[c][1], x[nt][c].x, x[nt][c].y);
-                                mma16816(acc[sl][set][nt], oa[c][2], ob[c][2], oa[c][3], ob[c][3], x[nt][c].z, x[nt][c].w);
+                                mma16816(acc[sl][set][nt], oa[0], ob[0], oa[1], ob[1], x[nt][c].x, x[nt][c].y);
+                                mma16816(acc[sl][set][nt], oa[2], ob[2], oa[3], ob[3], x[nt][c].z, x[nt][c].w);
                             }
                         }
                     }
@@ -463,7 +506,7 @@ struct Plan {
 
 template <int B, int NT>
 inline size_t smem_bytes(int nkb_cap) {
-    return 128 + static_cast<size_t>(num_stages<B, NT>()) * stage_bytes<B>() + 128 * 8 * NT * 4 + (B == 8 ? 1024 : 0) +
+    return 128 + static_cast<size_t>(num_stages<B, NT>()) * stage_bytes<B, NT>() + 128 * 8 * NT * 4 + (B == 8 ? 1024 : 0) +
            (2 * num_stages<B, NT>() + 2) * 8 + static_cast<size_t>(nkb_cap) * (kStabStride * 4);
 }
 
