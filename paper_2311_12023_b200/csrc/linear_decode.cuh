@@ -387,6 +387,295 @@ decode_fwd_kernel(const Params p) {
     cluster_sync_all();               // shared memory of this CTA may be read by its peers until here
 }
 
+// ------------------------------------------------------------------------------------ input gradient for few rows
+// dX[m][k] = sum_n dY[m][n] deq16(Q)[n][k] + sum_j T'[m][j] L2[j][k],  M <= 16.
+// One CTA owns a window of 256 columns of Q (four 64-column tiles) and a slice of the rows; the row slices
+// of a window form a cluster.  A ring stage holds two tile rows (256 rows x 256 columns of packed codes,
+// two contiguous pieces) and the matching 256 entries of every dY row.  Work item of a warp: 16 rows x 256
+// columns; lane (gid, t) holds rows 4t .. 4t+3 and the 32-column group gid.  The contraction runs over
+// rows, so the tensor-core operand needs pairs (W[n][k], W[n+1][k]): the byte-table look-ups of two rows
+// are merged by two more byte-permute stages (three permutes per two weights instead of two).
+// mma.sync m16n8k16: 16 columns x 16 rows (weights) times 16 rows x 8 tokens (dY).
+struct BwdParams {
+    QView q;
+    const __nv_bfloat16* dY;   // [M][N]
+    const __nv_bfloat16* T;    // [M][r] = dY L1, written by the kernel in front of this one (r > 0)
+    const __nv_bfloat16* L2;   // [r][K]
+    __nv_bfloat16* dX;         // [M][K]
+    int* status;
+    int M, r;
+    int S;                     // row slices per column window = cluster size
+    int trows_per_split;       // tile rows (128 rows) per CTA, even
+    int rows_stride;           // floats per block column of the scale table
+};
+
+constexpr int kBwdStageRows = 256;
+constexpr int kBwdYRowBytes = kBwdStageRows * 2 + 16;
+template <int B, int NT> __host__ __device__ constexpr int bwd_stage_bytes() { return 8 * 1024 * B + 8 * NT * kBwdYRowBytes; }
+template <int B> __host__ __device__ constexpr int bwd_stages() { return (B == 8) ? 2 : 3; }
+
+template <int B, int NT, bool TWO>
+__global__ void __launch_bounds__(kThreads, 1)
+decode_bwd_kernel(const BwdParams p) {
+    constexpr int NS = bwd_stages<B>();
+    constexpr int STAGE = bwd_stage_bytes<B, NT>();
+    constexpr int YOFF = 8 * 1024 * B;
+    constexpr int KF = 64 * NT;            // accumulator registers per thread
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
+    uint8_t* ring = base;
+    float* part = reinterpret_cast<float*>(ring + NS * STAGE);        // KF x 32 partial sums, fragment order
+    float* lut8 = part + KF * 32;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(lut8 + (B == 8 ? 256 : 0));
+    volatile int* abort_s = reinterpret_cast<volatile int*>(bars + 2 * NS);
+    float* stab = reinterpret_cast<float*>(bars + 2 * NS + 2);         // [nkb][rows_stride] block scales s~
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const QView& q = p.q;
+    const int cw = blockIdx.x, split = blockIdx.y;
+    const int kt_first = 4 * cw;
+    const int ncol_tiles = min(4, q.ktiles - kt_first);
+    const int tr0 = split * p.trows_per_split;
+    const int tr1 = min(q.ntiles, tr0 + p.trows_per_split);
+    const int ntr_cta = max(0, tr1 - tr0);
+    const int nstage_total = (ntr_cta + 1) >> 1;
+    const Ctl ctl{abort_s, p.status};
+
+    auto full = [&](int s) { return smem_u32(bars + s); };
+    auto empty = [&](int s) { return smem_u32(bars + NS + s); };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), kConsumerWarps); }
+        *abort_s = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+
+    const uint8_t* codes = reinterpret_cast<const uint8_t*>(q.codes);
+    auto issue_stage = [&](int it) {
+        const int s = it % NS;
+        const int ntr = min(2, ntr_cta - 2 * it);
+        const uint32_t dst = smem_u32(ring + s * STAGE);
+        const int row0 = (tr0 + 2 * it) * 128;
+        const int nrows = min(ntr * 128, q.N - row0);             // entries of dY that exist (a multiple of 8)
+        mbar_expect_tx(full(s), ntr * ncol_tiles * 1024 * B + p.M * nrows * 2);
+        for (int j = 0; j < ntr; ++j)
+            bulk_load(dst + j * (4 * 1024 * B), codes + (static_cast<size_t>(tr0 + 2 * it + j) * q.ktiles + kt_first) * (1024 * B),
+                      ncol_tiles * 1024 * B, full(s));
+        for (int m = 0; m < p.M; ++m)
+            bulk_load(dst + YOFF + m * kBwdYRowBytes, p.dY + static_cast<size_t>(m) * q.N + row0, nrows * 2, full(s));
+    };
+    if (warp == kConsumerWarps && lane == 0) {
+        for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it);
+    }
+
+    // block scales of the CTA's rows and its (at most 256) columns
+    const int col_first = kt_first * kTileCols;
+    const int kb_first = col_first >> q.logB0;
+    const int nkb = (((col_first + ncol_tiles * kTileCols - 1) >> q.logB0) - kb_first) + 1;
+    const int nrows_cta = ntr_cta * 128;
+    for (int e0 = threadIdx.x; e0 < nkb * nrows_cta; e0 += 4 * kThreads) {
+        uint32_t sc8[4];
+        float v[4];
+        int slot[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int e = e0 + u * kThreads;
+            sc8[u] = 0u; v[u] = 0.0f; slot[u] = -1;
+            if (e < nkb * nrows_cta) {
+                const int row = e / nkb, kb = e - row * nkb;
+                const int grow = tr0 * 128 + row;
+                slot[u] = kb * p.rows_stride + row;
+                if (grow < q.N) {
+                    const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first + kb;
+                    sc8[u] = __ldg(q.sc + blk);
+                    v[u] = __ldg(q.v + (blk >> q.logB1));
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (slot[u] >= 0) stab[slot[u]] = block_scale(static_cast<uint8_t>(sc8[u]), v[u]);
+    }
+    if constexpr (B == 8) {
+        for (int i = threadIdx.x; i < 256; i += kThreads) lut8[i] = c_codebook[3][i];
+    }
+    __syncthreads();
+
+    // acc[mm][nt][e]: mm = chunk * 4 + half * 2 + pair -> columns cA = 8 chunk + 4 half + 2 pair (e < 2) and cA + 1 (e >= 2)
+    // of the thread's group; token nt * 8 + 2 t + (e & 1)
+    float acc[16][NT][4];
+#pragma unroll
+    for (int a = 0; a < 16; ++a)
+#pragma unroll
+        for (int b = 0; b < NT; ++b)
+#pragma unroll
+            for (int d = 0; d < 4; ++d) acc[a][b][d] = 0.0f;
+
+    if (warp == kConsumerWarps) {
+        if (lane == 0) {
+            for (int it = NS; it < nstage_total; ++it) {
+                const int s = it % NS;
+                while (!mbar_try_wait(empty(s), ((it / NS) & 1) ^ 1) && !*abort_s) __nanosleep(200);
+                if (!wait(empty(s), ((it / NS) & 1) ^ 1, ctl, 31)) break;
+                issue_stage(it);
+            }
+            if (*abort_s) {
+                for (int s = 0; s < NS; ++s) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(full(s), 0) && !mbar_try_wait(full(s), 1) && clock64() - t0 < 20000000LL) {}
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        const int gid = lane >> 2, t = lane & 3;
+        const int ctile = gid >> 1, grp = gid & 1;
+        const bool col_ok = ctile < ncol_tiles;
+        const int kb = col_ok ? (((col_first + ctile * kTileCols + grp * 32) >> q.logB0) - kb_first) : 0;
+        bool ok = true;
+        for (int it = 0; it < nstage_total && ok; ++it) {
+            const int s = it % NS;
+            const int ntr = min(2, ntr_cta - 2 * it);
+            ok = wait(full(s), (it / NS) & 1, ctl, 32);
+            if (!ok) break;
+            const uint8_t* stage = ring + s * STAGE;
+#pragma unroll 1
+            for (int ii = 0; ii < 2; ++ii) {
+                const int item = warp * 2 + ii;                 // 0..15: tile row j, half-slab hs
+                const int j = item >> 3, hs = item & 7;
+                if (j >= ntr) continue;
+                const int slab = hs >> 1, row_in_tile = slab * 32 + (hs & 1) * 16 + 4 * t;
+                const int row_local = (2 * it + j) * 128 + row_in_tile;       // within the CTA's rows
+                const bool row_ok = tr0 * 128 + row_local < q.N;
+                const uint32_t* sp = reinterpret_cast<const uint32_t*>(stage) + (j * 4 + (col_ok ? ctile : 0)) * (256 * B) + slab * (64 * B) +
+                                     grp * (B * 32) + slab_row_slot((hs & 1) * 16 + 4 * t, grp, ctile);
+                uint4 w4[B];
+#pragma unroll
+                for (int i = 0; i < B; ++i) w4[i] = *reinterpret_cast<const uint4*>(sp + i * 32);
+                float4 sc_lo = *reinterpret_cast<const float4*>(stab + kb * p.rows_stride + row_local);
+                float4 sc_hi = sc_lo;
+                if (TWO) sc_hi = *reinterpret_cast<const float4*>(stab + (kb + 1) * p.rows_stride + row_local);
+                if (!col_ok) { sc_lo = make_float4(0.f, 0.f, 0.f, 0.f); sc_hi = sc_lo; }
+                // dY of the four rows for this lane's token(s)
+                uint32_t y0[NT], y1[NT];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int m = nt * 8 + gid;
+                    y0[nt] = 0u; y1[nt] = 0u;
+                    if (m < p.M && row_ok) {
+                        const uint2 yy = *reinterpret_cast<const uint2*>(stage + YOFF + m * kBwdYRowBytes + (j * 128 + row_in_tile) * 2);
+                        y0[nt] = yy.x; y1[nt] = yy.y;
+                    }
+                }
+                uint32_t w[4][B];
+#pragma unroll
+                for (int rr = 0; rr < 4; ++rr)
+#pragma unroll
+                    for (int i = 0; i < B; ++i) w[rr][i] = pick(w4[i], rr);
+                BlockTable<B> tab[4];
+                if constexpr (B != 8) {
+#pragma unroll
+                    for (int rr = 0; rr < 4; ++rr) tab[rr].build(pickf(sc_lo, rr));
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if constexpr (B != 8) {
+                        if (TWO && c == 2) {
+#pragma unroll
+                            for (int rr = 0; rr < 4; ++rr) tab[rr].build(pickf(sc_hi, rr));
+                        }
+                    }
+                    uint32_t o[4][4];      // o[row][e]: columns 8c + 2e, 8c + 2e + 1 of the row
+#pragma unroll
+                    for (int rr = 0; rr < 4; ++rr) dequant_chunk<B>(w[rr], c, tab[rr], pickf((TWO && c >= 2) ? sc_hi : sc_lo, rr), o[rr], lut8);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        // columns cA = 8c + 2e, cB = cA + 1: pairs along the rows
+                        const uint32_t a0 = prmt(o[0][e], o[1][e], 0x5410u), a1 = prmt(o[0][e], o[1][e], 0x7632u);
+                        const uint32_t a2 = prmt(o[2][e], o[3][e], 0x5410u), a3 = prmt(o[2][e], o[3][e], 0x7632u);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) mma16816(acc[c * 4 + e][nt], a0, a1, a2, a3, y0[nt], y1[nt]);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty(s));
+        }
+    }
+
+    // ---------------------------------------------------------------------- sum over the eight warps (they all cover the same columns)
+    // tree: the upper half of the active warps writes its accumulators to the idle ring, the lower half adds them
+    float* red = reinterpret_cast<float*>(ring);
+    static_assert(4 * KF * 32 * 4 <= NS * STAGE, "reduction buffer must fit into the ring");
+    __syncthreads();
+    for (int active = kConsumerWarps; active > 1; active >>= 1) {
+        const int hw = active >> 1;
+        if (warp >= hw && warp < active) {
+#pragma unroll
+            for (int mm = 0; mm < 16; ++mm)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) red[(((warp - hw) * 16 + mm) * NT + nt) * 128 + e * 32 + lane] = acc[mm][nt][e];
+        }
+        __syncthreads();
+        if (warp < hw) {
+#pragma unroll
+            for (int mm = 0; mm < 16; ++mm)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[mm][nt][e] += red[((warp * 16 + mm) * NT + nt) * 128 + e * 32 + lane];
+        }
+        __syncthreads();
+    }
+    if (warp == 0) {
+#pragma unroll
+        for (int mm = 0; mm < 16; ++mm)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) part[((mm * NT + nt) * 4 + e) * 32 + lane] = acc[mm][nt][e];
+    }
+    __syncthreads();
+
+    // ---------------------------------------------------------------------- sum over the row slices (cluster), rank-r term, store
+    cluster_sync_all();
+    const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
+    const int cols_share = 256 / p.S;
+    const int col_lo = static_cast<int>(rank) * cols_share;
+    if (p.r > 0) pdl_wait();
+    const uint32_t part_addr = smem_u32(part);
+    const int sub = threadIdx.x & 7;
+    const int n_out = cols_share * p.M;
+    for (int o0 = (threadIdx.x >> 3) & ~3; o0 < n_out; o0 += (kThreads >> 3) & ~3) {
+        const int o = o0 + ((threadIdx.x >> 3) & 3);
+        const bool live = o < n_out;
+        const int m = live ? o / cols_share : 0, cl = live ? o - m * cols_share : 0;
+        const int col_local = col_lo + cl;                    // 0..255 inside the window
+        const int kcol = col_first + col_local;
+        float sum = 0.0f;
+        if (live && sub < p.S) {
+            const int g8 = col_local >> 5, cc = col_local & 31;
+            const int mm = (cc >> 3) * 4 + ((cc >> 1) & 3);
+            const int e = (cc & 1) * 2 + (m & 1);
+            const int ln = g8 * 4 + ((m & 7) >> 1);
+            sum = ld_dsmem_f32(part_addr + static_cast<uint32_t>(((mm * NT + (m >> 3)) * 4 + e) * 32 + ln) * 4u, static_cast<uint32_t>(sub));
+        }
+        if (live && p.r > 0 && kcol < q.K) {
+            for (int jj = sub; jj < p.r; jj += 8)
+                sum = fmaf(__bfloat162float(p.T[static_cast<size_t>(m) * p.r + jj]), __bfloat162float(p.L2[static_cast<size_t>(jj) * q.K + kcol]), sum);
+        }
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+        if (live && sub == 0 && kcol < q.K) p.dX[static_cast<size_t>(m) * q.K + kcol] = __float2bfloat16_rn(sum);
+    }
+    cluster_sync_all();
+}
+
 // ------------------------------------------------------------------------------------ rank-r pre-product for few rows
 // T[m][j] = bf16( sum_c A[m][c] * F(j, c) ) for m < M <= 16, j < r <= 128:
 //   forward  A = X [M][K],  F(j, c) = L2[j][c]   (T = X L2^T)
@@ -648,6 +937,134 @@ inline cudaError_t launch_fwd(const QView& q, const void* L1, const void* L2, in
     }
     if (q.B0 == 16) return (pl.NT == 1) ? launch_fwd_nt<B, 1, true>(p, pl, r > 0, st) : launch_fwd_nt<B, 2, true>(p, pl, r > 0, st);
     return (pl.NT == 1) ? launch_fwd_nt<B, 1, false>(p, pl, r > 0, st) : launch_fwd_nt<B, 2, false>(p, pl, r > 0, st);
+}
+
+// Number of clusters of the given launch configuration that can be resident at the same time (0 on error).
+template <typename Kern>
+inline int max_active_clusters(Kern kern, int threads, size_t smem, int cluster_y) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1, cluster_y);
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = cluster_y; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    // the answer depends on (kernel, shared memory, cluster size) only: keep the last few per kernel
+    struct Entry { size_t smem; int cy, n; };
+    static Entry cache[8] = {};
+    static int used = 0;
+    for (int i = 0; i < used; ++i)
+        if (cache[i].smem == smem && cache[i].cy == cluster_y) return cache[i].n;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+    cache[used % 8] = Entry{smem, cluster_y, n};
+    if (used < 8) ++used;
+    return n;
+}
+
+struct BwdPlan {
+    bool ok;
+    int NT, S, trows_per_split, rows_stride, nwin;
+    size_t smem;
+};
+
+// Plan for a given number of row slices S (a power of two <= 8); ok = false when it does not fit.
+template <int B>
+inline BwdPlan make_bwd_plan_s(const QView& q, int M, int S) {
+    BwdPlan pl{};
+    pl.NT = (M <= 8) ? 1 : 2;
+    pl.nwin = (q.ktiles + 3) / 4;
+    int trps = (q.ntiles + S - 1) / S;
+    trps += trps & 1;
+    const int rows_stride = trps * 128 + 8;
+    const int nkb_cap = (256 >> q.logB0) + 2;
+    const size_t stage = (pl.NT == 1) ? bwd_stage_bytes<B, 1>() : bwd_stage_bytes<B, 2>();
+    const size_t smem = 128 + bwd_stages<B>() * stage + 64 * pl.NT * 32 * 4 + (B == 8 ? 1024 : 0) + (2 * bwd_stages<B>() + 2) * 8 +
+                        static_cast<size_t>(nkb_cap) * rows_stride * 4;
+    pl.ok = smem <= static_cast<size_t>(kSmemLimit) && (S == 1 || q.ntiles / S >= 1);
+    pl.S = S; pl.trows_per_split = trps; pl.rows_stride = rows_stride; pl.smem = smem;
+    return pl;
+}
+
+// Default plan (used for the support check): the largest S that fits.
+template <int B>
+inline BwdPlan make_bwd_plan(const QView& q, int M) {
+    for (int S = 8; S >= 1; S >>= 1) {
+        const BwdPlan pl = make_bwd_plan_s<B>(q, M, S);
+        if (pl.ok) return pl;
+    }
+    BwdPlan none{};
+    return none;
+}
+
+inline bool bwd_supported(const QView& q, int64_t M) {
+    if (M > 16 || q.N % 8 != 0 || q.K % 8 != 0 || q.N > 40960) return false;
+    if (static_cast<long long>(q.N) * q.KB >= (1LL << 31)) return false;
+    switch (q.b0) {
+        case 2: return make_bwd_plan<2>(q, static_cast<int>(M)).ok;
+        case 3: return make_bwd_plan<3>(q, static_cast<int>(M)).ok;
+        case 4: return make_bwd_plan<4>(q, static_cast<int>(M)).ok;
+        default: return make_bwd_plan<8>(q, static_cast<int>(M)).ok;
+    }
+}
+
+template <int B, int NT, bool TWO>
+inline cudaError_t launch_bwd_nt(BwdParams p, const QView& q, int M, bool after_pre, cudaStream_t st) {
+    auto kern = decode_bwd_kernel<B, NT, TWO>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    // the most row slices whose clusters are all resident at once; failing that, the fewest slices that fit
+    BwdPlan pl{};
+    for (int S = 8; S >= 1; S >>= 1) {
+        const BwdPlan c = make_bwd_plan_s<B>(q, M, S);
+        if (!c.ok) continue;
+        pl = c;
+        if (S == 1 || c.nwin <= max_active_clusters(kern, kThreads, c.smem, S)) break;
+    }
+    if (!pl.ok) return cudaErrorInvalidValue;
+    p.S = pl.S; p.trows_per_split = pl.trows_per_split; p.rows_stride = pl.rows_stride;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(pl.nwin, pl.S);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = pl.S; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_pre ? 2 : 1;
+    count_launch(1);
+    return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+// Input gradient for M <= 16.  ws: [status 256 B][T' bf16]; same status-word convention as launch_fwd.
+template <int B>
+inline cudaError_t launch_bwd(const QView& q, const void* L1, const void* L2, int r, const void* dY, int M, void* dX, char* ws,
+                              cudaStream_t st) {
+    BwdParams p;
+    p.q = q;
+    p.dY = static_cast<const __nv_bfloat16*>(dY);
+    p.T = reinterpret_cast<const __nv_bfloat16*>(ws + kStatusBytes);
+    p.L2 = static_cast<const __nv_bfloat16*>(L2);
+    p.dX = static_cast<__nv_bfloat16*>(dX);
+    p.status = reinterpret_cast<int*>(ws);
+    p.M = M; p.r = r; p.S = 1; p.trows_per_split = 0; p.rows_stride = 0;
+    const int NT = (M <= 8) ? 1 : 2;
+    if (r > 0) {
+        cudaError_t e = launch_pre<true>(p.dY, static_cast<const __nv_bfloat16*>(L1), reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes),
+                                         p.status, M, q.N, r, st);
+        if (e != cudaSuccess) return e;
+    }
+    if (q.B0 == 16) return (NT == 1) ? launch_bwd_nt<B, 1, true>(p, q, M, r > 0, st) : launch_bwd_nt<B, 2, true>(p, q, M, r > 0, st);
+    return (NT == 1) ? launch_bwd_nt<B, 1, false>(p, q, M, r > 0, st) : launch_bwd_nt<B, 2, false>(p, q, M, r > 0, st);
 }
 
 }  // namespace dec

@@ -61,7 +61,7 @@ static int run_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, i
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const QView v = make_view(q);
     const bool use_tc = tc_supported(v, r, M, backward);
-    const bool use_decode = !use_tc && !backward && dec::supported(v, M);
+    const bool use_decode = !use_tc && (backward ? dec::bwd_supported(v, M) : dec::supported(v, M));
     if (!(use_decode && r > 0)) {      // the decode path's first kernel clears the status word itself
         const size_t zero_bytes = kStatusBytes + (use_tc ? tc::pre_plan(backward ? v.N : v.K, r, M, backward ? v.K : v.N).counters_bytes : 0);
         if (cudaMemsetAsync(ws, 0, zero_bytes, st) != cudaSuccess) return cuda_rc(cudaGetLastError());
@@ -71,11 +71,22 @@ static int run_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, i
         return tc_launch(v, L1, L2, r, A, static_cast<int>(M), out, static_cast<char*>(ws), backward, st);
     }
     if (use_decode) {
-        switch (v.b0) {
-            case 2: e = dec::launch_fwd<2>(v, L1, L2, r, A, static_cast<int>(M), out, static_cast<char*>(ws), st); break;
-            case 3: e = dec::launch_fwd<3>(v, L1, L2, r, A, static_cast<int>(M), out, static_cast<char*>(ws), st); break;
-            case 4: e = dec::launch_fwd<4>(v, L1, L2, r, A, static_cast<int>(M), out, static_cast<char*>(ws), st); break;
-            default: e = dec::launch_fwd<8>(v, L1, L2, r, A, static_cast<int>(M), out, static_cast<char*>(ws), st); break;
+        char* w = static_cast<char*>(ws);
+        const int m = static_cast<int>(M);
+        if (!backward) {
+            switch (v.b0) {
+                case 2: e = dec::launch_fwd<2>(v, L1, L2, r, A, m, out, w, st); break;
+                case 3: e = dec::launch_fwd<3>(v, L1, L2, r, A, m, out, w, st); break;
+                case 4: e = dec::launch_fwd<4>(v, L1, L2, r, A, m, out, w, st); break;
+                default: e = dec::launch_fwd<8>(v, L1, L2, r, A, m, out, w, st); break;
+            }
+        } else {
+            switch (v.b0) {
+                case 2: e = dec::launch_bwd<2>(v, L1, L2, r, A, m, out, w, st); break;
+                case 3: e = dec::launch_bwd<3>(v, L1, L2, r, A, m, out, w, st); break;
+                case 4: e = dec::launch_bwd<4>(v, L1, L2, r, A, m, out, w, st); break;
+                default: e = dec::launch_bwd<8>(v, L1, L2, r, A, m, out, w, st); break;
+            }
         }
         return cuda_rc(e);
     }
