@@ -760,6 +760,11 @@ inline int launch_b(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtenso
 }
 
 }  // namespace tc
+}  // namespace lq
+
+#include "linear_tc2.cuh"
+
+namespace lq {
 
 constexpr int kTcMinRows = 33;   // fewer rows go to the weight-streaming kernels
 
@@ -787,8 +792,9 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
     __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + pl.counters_bytes);
     float* partial = reinterpret_cast<float*>(ws + kStatusBytes + pl.counters_bytes + pl.t_bytes);
     const int mh = (M > 128) ? 2 : 1;
+    const bool pair = M > 256;            // CTA pairs (cta_group::2) on [512, 256] tiles; boxes of 128 rows
     CUtensorMap tA, tA2, tB2;
-    if (!make_map(&tA, A, M, C, mh * 128)) return LQLORA_ERR_CUDA;
+    if (!make_map(&tA, A, M, C, pair ? 128 : mh * 128)) return LQLORA_ERR_CUDA;
     if (r > 0) {
         // rank-r pre-product on the tensor cores: T = X L2^T (forward) or dY L1 (backward)
         CUtensorMap tPA, tPB;
@@ -801,8 +807,8 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
         const int rc = backward ? launch_pre<true>(tPA, tPB, pp, pl.mtiles, pl.nsplit, st)
                                 : launch_pre<false>(tPA, tPB, pp, pl.mtiles, pl.nsplit, st);
         if (rc != LQLORA_OK) return rc;
-        if (!make_map(&tA2, T, M, r, mh * 128)) return LQLORA_ERR_CUDA;
-        const bool okb = backward ? make_map(&tB2, L2, r, q.K, 64) : make_map(&tB2, L1, q.N, r, 256);
+        if (!make_map(&tA2, T, M, r, pair ? 128 : mh * 128)) return LQLORA_ERR_CUDA;
+        const bool okb = backward ? make_map(&tB2, L2, r, q.K, 64) : make_map(&tB2, L1, q.N, r, pair ? 128 : 256);
         if (!okb) return LQLORA_ERR_CUDA;
     } else {
         tA2 = tA; tB2 = tA;
@@ -816,6 +822,14 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
     p.steps_q = (C + BK - 1) / BK;
     p.steps_d = (r + BK - 1) / BK;
     p.stages = 0;
+    if (pair) {
+        switch (q.b0) {
+            case 2: return backward ? launch_pair<2, true>(tA, tA2, tB2, p, st) : launch_pair<2, false>(tA, tA2, tB2, p, st);
+            case 3: return backward ? launch_pair<3, true>(tA, tA2, tB2, p, st) : launch_pair<3, false>(tA, tA2, tB2, p, st);
+            case 4: return backward ? launch_pair<4, true>(tA, tA2, tB2, p, st) : launch_pair<4, false>(tA, tA2, tB2, p, st);
+            default: return backward ? launch_pair<8, true>(tA, tA2, tB2, p, st) : launch_pair<8, false>(tA, tA2, tB2, p, st);
+        }
+    }
     switch (q.b0) {
         case 2: return launch_b<2>(tA, tA2, tB2, p, backward, mh, st);
         case 3: return launch_b<3>(tA, tA2, tB2, p, backward, mh, st);
