@@ -42,9 +42,10 @@ WORKLOAD = "llama2-7b attn-proj 4096x4096 NF3 B0=64 B1=256 r=64; encode + fwd/dX
 MS = (2048, 16, 1)
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 FALLBACK = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram bytes per forward launch of the tensor-core kernel at M = 2048 on this workload, from the
-# ncu capture summarised under profiles/ (None until a capture exists)
-TC_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum per forward launch of tc_pair_linear_kernel<3, 0> at M = 2048 on this
+# workload (profiles/kernels_c2_4096_nf3_ncu_full.txt): the operands are read once (X 16.8 MB + packed 6.6 MB +
+# factors), the output stays in L2 during the capture
+TC_TRAFFIC_BYTES = 24198144
 
 
 def linear_flops(M: int, N: int, K: int, r: int) -> float:
@@ -425,7 +426,7 @@ def run_device(args):
     achieved = linear_flops(2048, N, K, r) / tc_ms / 1e9
     roofline = {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": achieved / pk["bf16_tflops"], "traffic": TC_TRAFFIC_BYTES,
-                "kernel": "tc_linear_kernel (mean of lqlora_linear_fwd and lqlora_linear_bwd_input at M=2048, launched back to "
+                "kernel": "tc_pair_linear_kernel (mean of lqlora_linear_fwd and lqlora_linear_bwd_input at M=2048, launched back to "
                           f"back over {nrot} rotating activation buffers larger than L2; the rank-r pre-product kernel runs "
                           "beside it on the SMs its last wave leaves idle)",
                 "ms_per_launch": tc_ms,
