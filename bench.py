@@ -462,13 +462,95 @@ def run_device(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Sweep of one 8192 x 8192 matrix (b0 x B0 x M): encode GB/s, forward / input-gradient throughput and the
+    fraction of the binding roofline per point, as a text table on stdout (not the one-line contract)."""
+    import torch
+    from paper_2311_12023_b200 import binding
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    pk, pk_kind = peaks()
+    N = K = 8192
+    r = inputs.RANK
+    W = torch.from_numpy(inputs.gaussian(5000, (N, K), 0.02)).to(dev)
+    l1b, l2b = inputs.lowrank_factors(5700, N, K, r, 0.01)
+    L1, L2 = binding.bf16_from_bits(l1b, dev), binding.bf16_from_bits(l2b, dev)
+    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
+    Ms = [int(m) for m in args.sweep_ms.split(",")]
+    print(f"# sweep on one {N}x{K} matrix, rank {r}; peaks ({pk_kind}): HBM {pk['hbm_gbs']:.0f} GB/s, bf16 {pk['bf16_tflops']:.0f} TFLOP/s")
+    print("# M <= 16: packed-weight GB/s and fraction of HBM peak (calls replayed as a CUDA graph over cold copies);")
+    print("# M >= 128: algorithmic TFLOP/s and fraction of the bf16 peak (back to back over rotating activation buffers)")
+    print(f"{'b0':>3} {'B0':>4} {'bits':>6} {'enc GB/s':>9} {'enc frac':>8} " + " ".join(f"{'fwd M=' + str(m):>12} {'frac':>6} {'bwd M=' + str(m):>12} {'frac':>6}" for m in Ms))
+
+    def timed(fn, count):
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / count
+
+    for b0 in (2, 3, 4, 8):
+        for B0 in (16, 32, 64, 128, 256):
+            cfg = inputs.QuantConfig(b0, B0, 8, 256, 32)
+            q = binding.alloc_qmatrix(N, K, cfg, dev)
+            enc_ws = torch.empty(binding.packed_sizes(N, K, cfg)[3], dtype=torch.uint8, device=dev)
+            enc_ms = timed(lambda: [binding.encode(W, cfg, out=q, workspace=enc_ws) for _ in range(3)], 3)
+            enc_gbs = encode_bytes(N, K, cfg) / enc_ms / 1e6
+            pbytes = packed_bytes(N, K, cfg)
+            ncopies = max(2, int(2.2 * l2_bytes / q.packed_bytes) + 1)
+            copies = [binding.QMatrix(q.codes.clone(), q.scale_codes.clone(), q.scale2.clone(), N, K, cfg) for _ in range(ncopies)]
+            cells = []
+            for M in Ms:
+                X = binding.bf16_from_bits(inputs.activations(5200 + M, M, K), dev)
+                G = binding.bf16_from_bits(inputs.activations(5300 + M, M, N), dev)
+                ws = binding.alloc_workspace(q, r, M)
+                for bwd in (False, True):
+                    fn = binding.linear_bwd_input if bwd else binding.linear_fwd
+                    A = G if bwd else X
+                    if M <= 16:
+                        out = torch.empty((M, K if bwd else N), dtype=torch.bfloat16, device=dev)
+
+                        def body():
+                            for c in copies:
+                                fn(c, L1, L2, A, out=out, workspace=ws)
+                        body()
+                        torch.cuda.synchronize()
+                        g = torch.cuda.CUDAGraph()
+                        with torch.cuda.graph(g):
+                            body()
+                        ms = timed(g.replay, ncopies)
+                        val = pbytes / ms / 1e6
+                        cells.append(f"{val:9.0f}GB/s {val / pk['hbm_gbs']:6.3f}")
+                    else:
+                        nrot = max(2, int(1.1 * l2_bytes / (M * (N + K) * 2)) + 1) if M < 8192 else 2
+                        As = [A.clone() for _ in range(nrot)]
+                        outs = [torch.empty((M, K if bwd else N), dtype=torch.bfloat16, device=dev) for _ in range(nrot)]
+                        reps = max(2, min(4 * nrot, 16))
+                        ms = timed(lambda: [fn(q, L1, L2, As[i % nrot], out=outs[i % nrot], workspace=ws) for i in range(reps)], reps)
+                        val = linear_flops(M, N, K, r) / ms / 1e9
+                        cells.append(f"{val:8.0f}TF/s {val / pk['bf16_tflops']:6.3f}")
+                        del As, outs
+            bits = cfg.b0 + cfg.b1 / cfg.B0 + cfg.b2 / (cfg.B0 * cfg.B1)
+            print(f"{b0:>3} {B0:>4} {bits:6.3f} {enc_gbs:9.0f} {enc_gbs / pk['hbm_gbs']:8.3f} " + " ".join(cells), flush=True)
+            del copies, q
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sweep", action="store_true", help="print the b0 x B0 x M table of the 8192 x 8192 sweep instead")
+    ap.add_argument("--sweep-ms", default="1,16,128,2048,8192")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)

@@ -128,6 +128,50 @@ def test_config4_kv_projection_mixed_config():
     run_case(A, l1b, l2b, spec.cfg, 2048, seed=4300, rows=rows)
 
 
+def test_config3_gate_projection_sampled_rows():
+    spec = inputs.workload(3)["matrices"][0]          # 11008 x 4096, Student-t, NF4
+    A, l1b, l2b = inputs.make_matrix(spec)
+    rows = inputs.sample_rows(3300, 4096, count=16)
+    run_case(A, l1b, l2b, spec.cfg, 4096, seed=3400, rows=rows)
+
+
+def test_config4_query_projection_mixed_config():
+    spec = [s for s in inputs.workload(4)["matrices"] if s.name == "q"][0]    # 8192 x 8192, drawn config
+    A, l1b, l2b = inputs.make_matrix(spec)
+    run_case(A, l1b, l2b, spec.cfg, 1, seed=4400)
+    rows = inputs.sample_rows(4500, 2048, count=16)
+    run_case(A, l1b, l2b, spec.cfg, 2048, seed=4600, rows=rows)
+
+
+@pytest.mark.parametrize("name,M", [("gate", 1), ("down", 2048)])
+def test_config4_mlp_projections_largest_shapes(name, M):
+    spec = [s for s in inputs.workload(4)["matrices"] if s.name == name][0]   # 28672 x 8192 / 8192 x 28672
+    A, l1b, l2b = inputs.make_matrix(spec)
+    rows = inputs.sample_rows(4700, M, count=8) if M > 16 else None
+    run_case(A, l1b, l2b, spec.cfg, M, seed=4800 + M, rows=rows)
+
+
+@pytest.mark.parametrize("b0,B0", [(2, 16), (4, 128), (8, 256)])
+def test_config5_sweep_points(b0, B0):
+    """Points of the 8192 x 8192 sweep at every kind of M: decode kernels, one-CTA and CTA-pair tensor-core kernels."""
+    A = inputs.gaussian(5000, (8192, 8192), 0.02)
+    l1b, l2b = inputs.lowrank_factors(5700, 8192, 8192, 64, 0.01)
+    cfg = C(b0, B0, 8, 256, 32)
+    N, K = A.shape
+    q, ref = encode_both(A, cfg)
+    L1, L2 = binding.bf16_from_bits(l1b), binding.bf16_from_bits(l2b)
+    for M in (1, 16, 128, 2048):
+        rows = inputs.sample_rows(5100 + M, M, count=8) if M > 16 else None
+        xb = inputs.activations(5200 + M, M, K)
+        gb = inputs.activations(5300 + M, M, N)
+        Y = binding.linear_fwd(q, L1, L2, binding.bf16_from_bits(xb))
+        dX = binding.linear_bwd_input(q, L1, L2, binding.bf16_from_bits(gb))
+        torch.cuda.synchronize()
+        sel = slice(None) if rows is None else torch.from_numpy(rows).cuda()
+        check_close(to_np(Y[sel]), oracle.linear_fwd(ref["d32"], l1b, l2b, xb, rows), f"Y b0={b0} B0={B0} M={M}")
+        check_close(to_np(dX[sel]), oracle.linear_bwd_input(ref["d32"], l1b, l2b, gb, rows), f"dX b0={b0} B0={B0} M={M}")
+
+
 def test_workspace_status_is_clean_after_a_call():
     N, K, M = 256, 512, 8
     cfg = C(3, 64, 8, 256, 32)
