@@ -31,7 +31,7 @@ constexpr int kXRowBytes = kStageTiles * kTileCols * 2 + 16;   // one token's ac
 // A ring stage: the packed tiles, then the activations of the stage's 512 columns for 8 NT token rows.
 // NT = number of 8-token groups (1: M <= 8, two CTAs per SM; 2: M <= 16, one CTA per SM)
 template <int B, int NT> __host__ __device__ constexpr int stage_bytes() { return kStageTiles * 1024 * B + 8 * NT * kXRowBytes; }
-template <int B, int NT> __host__ __device__ constexpr int num_stages() { return (B == 8) ? 2 : (NT == 2 ? 4 : 2); }
+template <int B, int NT> __host__ __device__ constexpr int num_stages() { return (B == 8) ? 2 : (NT == 2 ? (B == 4 ? 3 : 4) : 2); }
 
 struct Params {
     QView q;

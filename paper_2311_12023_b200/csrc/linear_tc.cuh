@@ -200,7 +200,12 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * (MH * 128);
     const int c0 = blockIdx.y * BN;          // first output column: n0 (forward) or k0 (backward)
-    const int total = p.steps_q + p.steps_d;
+    // split of the contraction over the CTAs of a cluster (gridDim.z of them); the rank-r steps go to split 0
+    const int nsplit = gridDim.z, split = blockIdx.z;
+    const int per_split = (p.steps_q + nsplit - 1) / nsplit;
+    const int q_lo = min(p.steps_q, split * per_split);
+    const int nq = min(p.steps_q, q_lo + per_split) - q_lo;       // dequantized steps of this CTA
+    const int total = nq + (split == 0 ? p.steps_d : 0);
     const Ctl ctl{abort_s, p.status};
 
     auto full_a = [&](int s) { return smem_u32(bars + s); };
@@ -225,6 +230,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    bool acc_ok = false;          // this thread saw the accumulators complete (dequantization warps only)
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer: activations + packed codes
@@ -236,18 +242,19 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (!wait(empty_a(s), ra.ph ^ 1, ctl, 1)) break;
                 const uint32_t a_dst = smem_u32(a_ring) + s * A_BYTES;
                 const uint32_t p_dst = smem_u32(p_ring) + s * P_BYTES;
-                if (step < p.steps_q) {
+                if (step < nq) {
+                    const int qs = q_lo + step;                  // step index in the whole contraction
                     if (!BWD) {
                         int nt_have = 0;
                         for (int t = 0; t < 2; ++t) if ((c0 >> 7) + t < p.q.ntiles) ++nt_have;
                         mbar_expect_tx(full_a(s), A_BYTES + nt_have * 1024 * B);
-                        tma_load_2d(a_dst, &tmA, step * BK, m0, full_a(s));
+                        tma_load_2d(a_dst, &tmA, qs * BK, m0, full_a(s));
                         for (int t = 0; t < nt_have; ++t) {
-                            const size_t tile = static_cast<size_t>((c0 >> 7) + t) * p.q.ktiles + step;
+                            const size_t tile = static_cast<size_t>((c0 >> 7) + t) * p.q.ktiles + qs;
                             bulk_load(p_dst + t * 1024 * B, codes + tile * (1024 * B), 1024 * B, full_a(s));
                         }
                     } else {
-                        const int nn0 = step * BK;
+                        const int nn0 = qs * BK;
                         int kt_have = 0;
                         for (int t = 0; t < 4; ++t) if ((c0 >> 6) + t < p.q.ktiles) ++kt_have;
                         mbar_expect_tx(full_a(s), A_BYTES + kt_have * 512 * B);
@@ -259,7 +266,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         }
                     }
                 } else {
-                    if (step == p.steps_q) {
+                    if (step == nq) {
                         // the rank-r intermediate is written by the preceding kernel, which may still be
                         // running (programmatic dependent launch): wait for it, then order this thread's
                         // bulk-copy reads after what it wrote
@@ -267,7 +274,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         fence_proxy_async_all();
                     }
                     mbar_expect_tx(full_a(s), A_BYTES);
-                    tma_load_2d(a_dst, &tmA2, (step - p.steps_q) * BK, m0, full_a(s));
+                    tma_load_2d(a_dst, &tmA2, (step - nq) * BK, m0, full_a(s));
                 }
             }
             if (*abort_s) {
@@ -354,7 +361,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         float v_cached = -1.0f, sigma = 0.0f, s_lo = 0.0f, s_hi = 0.0f;
         RawScale slot[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) slot[u] = (u < p.steps_q) ? fetch(u) : RawScale{0u, 0.0f};
+        for (int u = 0; u < 4; ++u) slot[u] = (u < nq) ? fetch(q_lo + u) : RawScale{0u, 0.0f};
         // word plane slot of this thread's row: rotated by 8 g + 16 (tile column % 2), see slab_row_slot();
         // forward: the tile column is the step index, backward: it is fixed per thread
         const uint32_t* __restrict__ slab_base = reinterpret_cast<const uint32_t*>(p_ring) + slab_i * (64 * B) + g * (B * 32);
@@ -372,19 +379,19 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int sa = ra.s, sb = rb.s;
                 ok = wait(empty_b(sb), rb.ph ^ 1, ctl, 6);
                 if (!ok) break;
-                if (step < p.steps_q) {
+                if (step < nq) {
                     make_scales(p.q, slot[u], v_cached, sigma, s_lo, s_hi);
-                    if (step + 4 < p.steps_q) slot[u] = fetch(step + 4);
+                    if (step + 4 < nq) slot[u] = fetch(q_lo + step + 4);
                     ok = wait(full_a(sa), ra.ph, ctl, 4);
                     if (!ok) break;
-                    dequant_group<B>(slab_base + sa * (P_BYTES / 4) + ((step & 1) ? slot_odd : slot_even), s_lo, s_hi, two_scales, my_b + sb * kBBytes, g << 6, xr, lut8);
+                    dequant_group<B>(slab_base + sa * (P_BYTES / 4) + (((q_lo + step) & 1) ? slot_odd : slot_even), s_lo, s_hi, two_scales, my_b + sb * kBBytes, g << 6, xr, lut8);
                     fence_proxy_async();            // make the generic-proxy stores visible to the tensor core
                     __syncwarp();
                     if (lane == 0) mbar_arrive(full_b(sb));
                 } else if (dw == 0) {
                     // rank-r step: the second operand ([L1 | ..] rows or L2 rows) comes by TMA into the weight ring
                     if (lane == 0) {
-                        const int d = step - p.steps_q;
+                        const int d = step - nq;
                         const uint32_t dst = smem_u32(b_ring) + sb * kBBytes;
                         if (!BWD) {
                             mbar_expect_tx(full_b(sb), kBBytes);
@@ -405,7 +412,8 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
         }
         // epilogue: warp reads its quarter of the 128 accumulator lanes and 64 of the 256 columns
-        if (ok && wait(acc_full, 0, ctl, 5)) {
+        acc_ok = ok && wait(acc_full, 0, ctl, 5);
+        if (acc_ok && nsplit == 1) {
             tc_fence_after();
             const int quarter = warp & 3, colq = dw >> 2;
 #pragma unroll 1
@@ -435,6 +443,59 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                 }
             }
+        }
+    }
+    if (nsplit > 1) {
+        // ------------------------------------------------------------------ sum over the splits of the contraction
+        // Every CTA of the cluster writes its accumulator tile (fp32, [256 columns][128 rows]) over the idle
+        // rings; CTA `split` then adds the 256 / nsplit columns it owns from all CTAs through distributed
+        // shared memory, rounds to bf16 and stores.  The barriers are executed by all threads of all CTAs,
+        // whatever happened before (a CTA that gave up on a wait still takes part; its output is undefined
+        // and the status word says so).
+        float* accbuf = reinterpret_cast<float*>(base);
+        const uint32_t accbuf_addr = smem_u32(accbuf);
+        const int cols_share = BN / nsplit, col_lo = split * cols_share;
+#pragma unroll 1
+        for (int h = 0; h < MH; ++h) {
+            if (warp >= 2 && acc_ok) {
+                tc_fence_after();
+                const int dw = warp - 2, quarter = warp & 3, colq = dw >> 2;
+#pragma unroll 1
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int col = colq * 64 + cc * 32;
+                    uint32_t v[32];
+                    tmem_ld32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + h * BN + col, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) accbuf[(col + i) * 128 + quarter * 32 + lane] = __uint_as_float(v[i]);
+                }
+            }
+            __syncthreads();
+            dec::cluster_sync_all();
+            for (int item = threadIdx.x; item < 128 * (cols_share / 8); item += kThreads) {
+                const int row = item & 127, cg = item >> 7;
+                const int m = m0 + h * 128 + row;
+                const int col = col_lo + cg * 8;
+                float sum[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) sum[i] = 0.0f;
+                for (int rk = 0; rk < nsplit; ++rk) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        sum[i] += dec::ld_dsmem_f32(accbuf_addr + static_cast<uint32_t>((col + i) * 128 + row) * 4u, static_cast<uint32_t>(rk));
+                }
+                if (m < p.M && c0 + col < p.out_cols) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const __nv_bfloat162 hh = __floats2bfloat162_rn(sum[2 * e], sum[2 * e + 1]);
+                        w[e] = *reinterpret_cast<const uint32_t*>(&hh);
+                    }
+                    *reinterpret_cast<uint4*>(p.out + static_cast<size_t>(m) * p.out_cols + c0 + col) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+            __syncthreads();
+            dec::cluster_sync_all();           // the buffers may be overwritten (next half) or released (exit) only now
         }
     }
     tc_fence_before();
@@ -657,7 +718,7 @@ inline bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t 
 }
 
 template <int B, bool BWD, int MH>
-inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, Params p, cudaStream_t st) {
+inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, Params p, int ksplit, cudaStream_t st) {
     constexpr int stages = ring_stages<B, MH>();
     static_assert(stages >= 2, "activation ring too shallow");
     p.stages = stages;
@@ -673,21 +734,34 @@ inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUten
         attr_done = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((p.M + MH * 128 - 1) / (MH * 128), (p.out_cols + BN - 1) / BN);
+    cfg.gridDim = dim3((p.M + MH * 128 - 1) / (MH * 128), (p.out_cols + BN - 1) / BN, ksplit);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;      // the splits of the contraction of one tile form a cluster
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = ksplit;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = (p.steps_d > 0) ? 1 : 0;      // overlap with the rank-r pre-product kernel in front of it
+    cfg.numAttrs = (p.steps_d > 0) ? 2 : 1;      // overlap with the rank-r pre-product kernel in front of it
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA, tA2, tB2, p);
     count_launch(1);
     if (e != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
     return LQLORA_OK;
 }
 
+
+// Splits of the contraction for the one-CTA kernel (M <= 256): few output tiles would leave most SMs idle, so
+// the contraction of a tile is divided over a cluster of up to eight CTAs (each keeps at least eight steps).
+inline int tc_ksplit(int64_t M, int64_t out_cols, int steps_q, int sms) {
+    if (M > 256) return 1;
+    const int mh = (M > 128) ? 2 : 1;
+    const long long tiles = ((M + mh * 128 - 1) / (mh * 128)) * ((out_cols + BN - 1) / BN);
+    int ks = 1;
+    while (ks < 8 && tiles * (2 * ks) <= sms && steps_q / (2 * ks) >= 8) ks *= 2;
+    return ks;
+}
 
 struct PrePlan {
     int mtiles, nsplit, steps, steps_per_split, rp;
@@ -715,8 +789,8 @@ inline PrePlan pre_plan(int64_t C, int r, int64_t M, int64_t out_cols) {
     // The pre-product runs beside the linear kernel that follows it (programmatic dependent launch):
     // give it the SMs that the last wave of that kernel leaves idle, and at least one CTA per row tile.
     const int mh = (M > 128) ? 2 : 1;
-    const long long main_ctas = ((M + mh * 128 - 1) / (mh * 128)) * ((out_cols + BN - 1) / BN);
     const int sms = sm_count();
+    const long long main_ctas = ((M + mh * 128 - 1) / (mh * 128)) * ((out_cols + BN - 1) / BN) * tc_ksplit(M, out_cols, pl.steps, sms);
     const int idle = static_cast<int>((sms - main_ctas % sms) % sms);
     int want = idle / pl.mtiles;
     if (want > pl.steps / 2) want = pl.steps / 2;
@@ -754,9 +828,9 @@ inline int launch_pre(const CUtensorMap& tA, const CUtensorMap& tB, PreParams p,
 
 template <int B>
 inline int launch_b(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, const Params& p, bool bwd, int mh,
-                    cudaStream_t st) {
-    if (!bwd) return mh == 2 ? launch_one<B, false, 2>(tA, tA2, tB2, p, st) : launch_one<B, false, 1>(tA, tA2, tB2, p, st);
-    return mh == 2 ? launch_one<B, true, 2>(tA, tA2, tB2, p, st) : launch_one<B, true, 1>(tA, tA2, tB2, p, st);
+                    int ksplit, cudaStream_t st) {
+    if (!bwd) return mh == 2 ? launch_one<B, false, 2>(tA, tA2, tB2, p, ksplit, st) : launch_one<B, false, 1>(tA, tA2, tB2, p, ksplit, st);
+    return mh == 2 ? launch_one<B, true, 2>(tA, tA2, tB2, p, ksplit, st) : launch_one<B, true, 1>(tA, tA2, tB2, p, ksplit, st);
 }
 
 }  // namespace tc
@@ -830,11 +904,12 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
             default: return backward ? launch_pair<8, true>(tA, tA2, tB2, p, st) : launch_pair<8, false>(tA, tA2, tB2, p, st);
         }
     }
+    const int ksplit = tc_ksplit(M, p.out_cols, p.steps_q, sm_count());
     switch (q.b0) {
-        case 2: return launch_b<2>(tA, tA2, tB2, p, backward, mh, st);
-        case 3: return launch_b<3>(tA, tA2, tB2, p, backward, mh, st);
-        case 4: return launch_b<4>(tA, tA2, tB2, p, backward, mh, st);
-        default: return launch_b<8>(tA, tA2, tB2, p, backward, mh, st);
+        case 2: return launch_b<2>(tA, tA2, tB2, p, backward, mh, ksplit, st);
+        case 3: return launch_b<3>(tA, tA2, tB2, p, backward, mh, ksplit, st);
+        case 4: return launch_b<4>(tA, tA2, tB2, p, backward, mh, ksplit, st);
+        default: return launch_b<8>(tA, tA2, tB2, p, backward, mh, ksplit, st);
     }
 }
 
