@@ -217,6 +217,13 @@ int lqlora_workspace_status(const void* workspace_dev, void* stream);
  * 0 = weight-streaming small-M kernel, 1 = tcgen05 tensor-core kernel.  Host only. */
 int lqlora_linear_path(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, int backward);
 
+/* lqlora_encode finds the nearest code (Sec. 2.2: c_j = argmin_k |q~_k - u_j / s_i|) with a bin table over [-1, 1]:
+ * every bin holds at most one decision threshold (the midpoint of two neighbouring code-book entries), and inputs
+ * closer than 1e-6 to a threshold are decided with the exact IEEE quotient.  This returns the smallest distance
+ * between a threshold and a bin edge for the b0-bit table; it must exceed that 1e-6 by a wide margin for the
+ * fast and the exact route to agree (checked by the host tests).  Negative for an invalid b0.  Host only. */
+double lqlora_encode_search_clearance(int b0);
+
 /* Number of kernel launches the library has enqueued since it was loaded (for launch accounting). */
 int64_t lqlora_launch_count(void);
 

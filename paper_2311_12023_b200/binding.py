@@ -22,7 +22,7 @@ EXPORTS = [
     "lqlora_unpack", "lqlora_dequant", "lqlora_linear_workspace_bytes", "lqlora_linear_fwd",
     "lqlora_linear_bwd_input", "lqlora_workspace_status", "lqlora_linear_path", "lqlora_launch_count",
     "lqlora_status_string", "lqlora_encode_host", "lqlora_linear_fwd_host", "lqlora_linear_bwd_input_host",
-    "lqlora_static_scratch_bytes", "lqlora_linear_fwd_static",
+    "lqlora_static_scratch_bytes", "lqlora_linear_fwd_static", "lqlora_encode_search_clearance",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20   # size of the scratch array compiled into the library (lqlora_static_scratch_bytes)
@@ -72,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.lqlora_linear_bwd_input_host.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, vp, vp, sz, vp]
         L.lqlora_workspace_status.argtypes = [vp, vp]
         L.lqlora_static_scratch_bytes.restype = sz
+        L.lqlora_encode_search_clearance.argtypes = [ci]
+        L.lqlora_encode_search_clearance.restype = ctypes.c_double
         L.lqlora_linear_fwd_static.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp]
         L.lqlora_linear_path.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ci]
         L.lqlora_launch_count.restype = i64

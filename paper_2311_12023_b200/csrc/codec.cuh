@@ -35,9 +35,20 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
                                                            float* __restrict__ absmax, int N, int K, int B0, int logB0) {
     __shared__ float red[8][33];
     __shared__ float th8[256];
+    __shared__ float2 bins[kMaxBins + 1];        // (threshold of the bin or +inf, number of thresholds below the bin)
     if constexpr (B == 8) {
         th8[threadIdx.x] = c_threshold[3][threadIdx.x];
     }
+    // the bin table pays off for 4- and 8-bit codes (15 / 255 thresholds); 2- and 3-bit codes compare directly
+    constexpr bool kUseBins = (B >= 4);
+    const int nb = kUseBins ? c_nbins[bits_index(B)] : 0;
+    if constexpr (kUseBins) {
+        for (int i = threadIdx.x; i <= nb; i += 256) {
+            const BinEntry e = c_bins[bits_index(B)][i];
+            bins[i] = make_float2(e.thr, __int_as_float(e.base));
+        }
+    }
+    const float bin_scale = 0.5f * static_cast<float>(nb);
     const int rl = threadIdx.x & 31, grp = threadIdx.x >> 5;
     const int row = blockIdx.x * 32 + rl;
     const int k0 = blockIdx.y * 256 + grp * 32;
@@ -87,11 +98,31 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
     uint32_t words[B];
 #pragma unroll
     for (int i = 0; i < B; ++i) words[i] = 0u;
+    // Fast search: x^ = u * fl(1/s) is within 2 ulp of the quotient fl(u/s) that defines the code; the bin of x^
+    // holds at most one threshold, and the code is the number of thresholds below the bin plus (x^ > threshold).
+    // When x^ comes within 1e-6 of that threshold (or is not a number in [-1, 1]: zero, subnormal or huge block
+    // maxima) the decision is taken exactly, with the IEEE quotient and the full search.  No threshold lies that
+    // close to a bin edge (the bin count is chosen on the host for the largest clearance), so the two routes agree.
+    const float r_lo = (s_lo != 0.0f) ? __fdiv_rn(1.0f, s_lo) : 0.0f;
+    const float r_hi = (s_hi != 0.0f) ? __fdiv_rn(1.0f, s_hi) : 0.0f;
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
         const float s = (j < 16) ? s_lo : s_hi;
-        uint32_t c = zero_code;
-        if (s != 0.0f) c = nearest_code<B>(__fdiv_rn(u[j], s), th8);
+        if constexpr (!kUseBins) {
+            uint32_t c = zero_code;
+            if (s != 0.0f) c = nearest_code<B>(__fdiv_rn(u[j], s), th8);
+            deposit_code<B>(words, j, c);
+            continue;
+        }
+        const float xh = u[j] * ((j < 16) ? r_lo : r_hi);
+        int k = __float2int_rd(fmaf(xh, bin_scale, bin_scale));
+        k = min(max(k, 0), nb);
+        const float2 e = bins[k];
+        uint32_t c = static_cast<uint32_t>(__float_as_int(e.y)) + ((xh > e.x) ? 1u : 0u);
+        if (!(fabsf(xh - e.x) > 1e-6f) || !(fabsf(xh) <= 1.001f)) {
+            c = zero_code;
+            if (s != 0.0f) c = nearest_code<B>(__fdiv_rn(u[j], s), th8);
+        }
         deposit_code<B>(words, j, c);
     }
     uint32_t* dst = codes + slab_word_base(row, k0 >> 6, K >> 6, B);

@@ -133,6 +133,14 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_
 __constant__ float c_codebook[4][256];
 __constant__ float c_threshold[4][256];
 
+// Bin table for the nearest-code search of the encoder: [-1, 1] is cut into `nb` equal bins chosen so that every
+// bin holds at most one threshold and no threshold lies near a bin edge.  Entry k = (threshold in the bin or +inf,
+// number of thresholds below the bin); entry nb serves x slightly above 1.
+constexpr int kMaxBins = 1280;
+struct BinEntry { float thr; int base; };
+__constant__ BinEntry c_bins[4][kMaxBins + 1];
+__constant__ int c_nbins[4];
+
 int ensure_tables();                 // uploads the tables to the current device once; LQLORA_OK or error
 const float* host_codebook(int b0);  // 2^b0 floats
 void count_launch(int n = 1);

@@ -33,6 +33,44 @@ inline double gauss_quantile(double p) {
 struct HostTables {
     float codebook[4][256];
     float threshold[4][256];
+    BinEntry bins[4][kMaxBins + 1];
+    int nbins[4];
+    // Bin count for `n - 1` thresholds: the candidate with the largest distance between any threshold and any
+    // bin edge among those with at most one threshold per bin.
+    void build_bins(int t, int n) {
+        const int lo = (n <= 16) ? 48 : 1000, hi = (n <= 16) ? 96 : kMaxBins;
+        int best_nb = 0;
+        double best_clear = -1.0;
+        for (int nb = lo; nb <= hi; ++nb) {
+            double clear = 1e9;
+            bool ok = true;
+            int prev_bin = -1;
+            for (int i = 0; i + 1 < n && ok; ++i) {
+                const double pos = (static_cast<double>(threshold[t][i]) + 1.0) * 0.5 * nb;
+                const int b = static_cast<int>(std::floor(pos));
+                if (b == prev_bin) ok = false;
+                prev_bin = b;
+                const double d = std::fmin(pos - std::floor(pos), std::ceil(pos) - pos) * 2.0 / nb;
+                clear = std::fmin(clear, d);
+            }
+            if (ok && clear > best_clear) { best_clear = clear; best_nb = nb; }
+        }
+        nbins[t] = best_nb;
+        for (int k = 0; k <= kMaxBins; ++k) { bins[t][k].thr = INFINITY; bins[t][k].base = n - 1; }
+        int below = 0;
+        for (int k = 0; k < best_nb; ++k) {
+            bins[t][k].base = below;
+            bins[t][k].thr = INFINITY;
+            while (below + 1 < n) {
+                const double pos = (static_cast<double>(threshold[t][below]) + 1.0) * 0.5 * best_nb;
+                if (static_cast<int>(std::floor(pos)) != k) break;
+                bins[t][k].thr = threshold[t][below];
+                ++below;
+            }
+        }
+        bin_clearance[t] = best_clear;
+    }
+    double bin_clearance[4];
     HostTables() {
         const int bits[4] = {2, 3, 4, 8};
         const double delta = 0.5 * (1.0 / 30.0 + 1.0 / 32.0);
@@ -55,6 +93,7 @@ struct HostTables {
                 if (static_cast<double>(th) > mid) th = std::nextafterf(th, -INFINITY);
                 threshold[t][i] = th;                       // largest fp32 <= midpoint
             }
+            build_bins(t, n);
         }
     }
 };
@@ -77,7 +116,9 @@ int ensure_tables() {
     if (done[dev]) return LQLORA_OK;
     const detail::HostTables& t = detail::host_tables();
     if (cudaMemcpyToSymbol(c_codebook, t.codebook, sizeof(t.codebook)) != cudaSuccess ||
-        cudaMemcpyToSymbol(c_threshold, t.threshold, sizeof(t.threshold)) != cudaSuccess) {
+        cudaMemcpyToSymbol(c_threshold, t.threshold, sizeof(t.threshold)) != cudaSuccess ||
+        cudaMemcpyToSymbol(c_bins, t.bins, sizeof(t.bins)) != cudaSuccess ||
+        cudaMemcpyToSymbol(c_nbins, t.nbins, sizeof(t.nbins)) != cudaSuccess) {
         cudaGetLastError();
         return LQLORA_ERR_CUDA;
     }
@@ -120,6 +161,11 @@ int lqlora_nf_codebook(int b0, float* out_host) {
     const float* cb = lq::host_codebook(b0);
     for (int i = 0; i < (1 << b0); ++i) out_host[i] = cb[i];
     return LQLORA_OK;
+}
+
+double lqlora_encode_search_clearance(int b0) {
+    if (!(b0 == 2 || b0 == 3 || b0 == 4 || b0 == 8)) return -1.0;
+    return lq::detail::host_tables().bin_clearance[lq::bits_index(b0)];
 }
 
 int64_t lqlora_launch_count(void) { return lq::g_launches.load(std::memory_order_relaxed); }

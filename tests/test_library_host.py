@@ -41,6 +41,12 @@ def test_library_codebook_is_bit_identical_to_oracle(binding, b):
     assert np.array_equal(binding.nf_codebook(b), oracle.nf_codebook(b))
 
 
+@pytest.mark.parametrize("b", [2, 3, 4, 8])
+def test_encoder_bin_table_keeps_thresholds_away_from_bin_edges(binding, b):
+    # the fast nearest-code search is exact only if no threshold sits within its 1e-6 guard band of a bin edge
+    assert binding.lib().lqlora_encode_search_clearance(b) >= 1e-5
+
+
 def test_storage_formula_and_packed_sizes(binding):
     for b0 in (2, 3, 4, 8):
         for B0 in (16, 32, 64, 128, 256):
