@@ -897,11 +897,13 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
     p.steps_d = (r + BK - 1) / BK;
     p.stages = 0;
     if (pair) {
+        CUtensorMap tOut;         // output as boxes of 32 rows x 64 columns
+        if (!make_map(&tOut, out, M, p.out_cols, 32)) return LQLORA_ERR_CUDA;
         switch (q.b0) {
-            case 2: return backward ? launch_pair<2, true>(tA, tA2, tB2, p, st) : launch_pair<2, false>(tA, tA2, tB2, p, st);
-            case 3: return backward ? launch_pair<3, true>(tA, tA2, tB2, p, st) : launch_pair<3, false>(tA, tA2, tB2, p, st);
-            case 4: return backward ? launch_pair<4, true>(tA, tA2, tB2, p, st) : launch_pair<4, false>(tA, tA2, tB2, p, st);
-            default: return backward ? launch_pair<8, true>(tA, tA2, tB2, p, st) : launch_pair<8, false>(tA, tA2, tB2, p, st);
+            case 2: return backward ? launch_pair<2, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<2, false>(tA, tA2, tB2, tOut, p, st);
+            case 3: return backward ? launch_pair<3, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<3, false>(tA, tA2, tB2, tOut, p, st);
+            case 4: return backward ? launch_pair<4, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<4, false>(tA, tA2, tB2, tOut, p, st);
+            default: return backward ? launch_pair<8, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<8, false>(tA, tA2, tB2, tOut, p, st);
         }
     }
     const int ksplit = tc_ksplit(M, p.out_cols, p.steps_q, sm_count());

@@ -12,7 +12,8 @@
 // second ring and arrive on the LEADER's barrier (remote arrive for the second CTA); the leader's MMA
 // thread waits for the sixteen arrivals of a step, issues the MMAs and commits the ring stages back to both
 // CTAs (multicast commit).  Forward and input gradient share the code (K-major / MN-major weight operand)
-// as in the single-CTA kernel; the rank-r term is one more step whose operands come by TMA.
+// as in the single-CTA kernel; the rank-r term is one more step whose operands come by TMA; the output
+// leaves through shared memory and TMA stores.
 // Every wait is bounded; both CTAs meet at a cluster barrier before tensor memory is freed.
 #pragma once
 
@@ -87,7 +88,7 @@ template <int B> __host__ __device__ constexpr int pair_smem_bytes() {
 template <int B, bool BWD>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_pair_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA2,
-                      const __grid_constant__ CUtensorMap tmB2, const Params p) {
+                      const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmOut, const Params p) {
     constexpr int SA = pair_a_stages<B>();
     constexpr int SB = kPairBStages;
     constexpr int P_BYTES = 1024 * B;
@@ -327,37 +328,48 @@ tc_pair_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 rb.advance(); rb.advance();
             }
         }
-        // epilogue: warp reads its quarter of the 128 accumulator lanes and 64 of the 256 columns of both accumulators
+        // epilogue: a warp owns 32 accumulator lanes (rows) x 64 columns of both accumulators.  It rounds them to
+        // bf16 into a private 4 KB tile of the (now idle) activation ring, in the 128-byte-swizzled layout of a
+        // TMA box of 32 rows x 64 columns, and one lane stores the box with a bulk tensor copy, which clips at the
+        // edges of the output.
         if (ok && wait(acc_full, 0, ctl, 45)) {
             tc_fence_after();
             const int quarter = warp & 3, colq = dw >> 2;
+            const uint32_t xs = static_cast<uint32_t>(lane & 7);
+            bool stored = false;
 #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
-                const int m = m0 + h * 256 + static_cast<int>(rank) * 128 + quarter * 32 + lane;
+                uint8_t* stage = a_ring + (dw * 2 + h) * 4096;
+                uint8_t* row = stage + lane * 128;
 #pragma unroll 1
                 for (int cc = 0; cc < 2; ++cc) {
-                    const int col = colq * 64 + cc * 32;
                     uint32_t v[32];
-                    tmem_ld32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + h * BN + col, v);
+                    tmem_ld32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + h * BN + colq * 64 + cc * 32, v);
                     tmem_ld_wait();
-                    if (m < p.M) {
-                        __nv_bfloat16* dst = p.out + static_cast<size_t>(m) * p.out_cols + c0 + col;
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            if (c0 + col + i * 8 < p.out_cols) {
-                                uint32_t w[4];
+                    for (int i = 0; i < 4; ++i) {
+                        uint32_t w[4];
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[i * 8 + 2 * e]),
-                                                                                   __uint_as_float(v[i * 8 + 2 * e + 1]));
-                                    w[e] = *reinterpret_cast<const uint32_t*>(&hh);
-                                }
-                                *reinterpret_cast<uint4*>(dst + i * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-                            }
+                        for (int e = 0; e < 4; ++e) {
+                            const __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[i * 8 + 2 * e]),
+                                                                           __uint_as_float(v[i * 8 + 2 * e + 1]));
+                            w[e] = *reinterpret_cast<const uint32_t*>(&hh);
                         }
+                        *reinterpret_cast<uint4*>(row + (((cc * 4 + i) ^ xs) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
+                fence_proxy_async();
+                __syncwarp();
+                const int x = c0 + colq * 64, y = m0 + h * 256 + static_cast<int>(rank) * 128 + quarter * 32;
+                if (lane == 0 && x < p.out_cols && y < p.M) {
+                    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                                 ::"l"(reinterpret_cast<uint64_t>(&tmOut)), "r"(x), "r"(y), "r"(smem_u32(stage)) : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    stored = true;
+                }
             }
+            if (stored) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+            __syncwarp();
         }
     }
     tc_fence_before();
@@ -367,7 +379,7 @@ tc_pair_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 }
 
 template <int B, bool BWD>
-inline int launch_pair(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, Params p, cudaStream_t st) {
+inline int launch_pair(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, const CUtensorMap& tOut, Params p, cudaStream_t st) {
     constexpr int smem = pair_smem_bytes<B>();
     static_assert(smem <= kSmemLimit, "shared memory budget exceeded");
     auto kern = tc_pair_linear_kernel<B, BWD>;
@@ -391,7 +403,7 @@ inline int launch_pair(const CUtensorMap& tA, const CUtensorMap& tA2, const CUte
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = (p.steps_d > 0) ? 2 : 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA, tA2, tB2, p);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA, tA2, tB2, tOut, p);
     count_launch(1);
     if (e != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
     return LQLORA_OK;
