@@ -821,9 +821,22 @@ inline int launch_pre(const CUtensorMap& tA, const CUtensorMap& tB, PreParams p,
         }
         attr_done = true;
     }
-    kern<<<dim3(mtiles, nsplit), 192, smem, st>>>(tA, tB, p);
+    // Launched as clusters of two where possible: the CTAs then fill whole TPCs, and the CTA pairs of the linear
+    // kernel that runs beside this one find as many free TPCs as the SM count suggests.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(mtiles, nsplit);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (mtiles % 2 == 0) ? 2 : 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA, tB, p);
     count_launch(1);
-    return cudaGetLastError() == cudaSuccess ? LQLORA_OK : LQLORA_ERR_CUDA;
+    if (e != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
+    return LQLORA_OK;
 }
 
 template <int B>
