@@ -53,6 +53,34 @@ def test_linear_training_shapes(b0, B0, M):
     run_case(A, l1b, l2b, C(b0, B0, 8, 256, 32), M, seed=400 + M)
 
 
+@pytest.mark.parametrize("N,K,M", [(200, 704, 3), (200, 704, 11), (1160, 64, 16), (72, 1984, 8)])
+@pytest.mark.parametrize("b0,B0", [(3, 64), (2, 16), (8, 32)])
+def test_linear_decode_kernels_ragged_shapes(N, K, M, b0, B0):
+    """Decode kernels with a partial last tile row (N % 128 != 0), an odd number of 64-column tiles and fewer
+    tiles than cluster ranks."""
+    A = inputs.gaussian(800 + N, (N, K), 0.02)
+    l1b, l2b = inputs.lowrank_factors(801 + K, N, K, 32, 0.01)
+    run_case(A, l1b, l2b, C(b0, B0, 8, 16, 32), M, seed=900 + M)
+
+
+def test_linear_single_row_with_odd_feature_count_uses_the_fallback():
+    # N % 8 != 0 is only legal for M = 1 (no vector loads on the rows of Y): the plain kernels take it
+    N, K = 201, 192
+    A = inputs.gaussian(850, (N, K), 0.02)
+    l1b, l2b = inputs.lowrank_factors(851, N, K, 16, 0.01)
+    run_case(A, l1b, l2b, C(4, 64, 8, 16, 32), 1, seed=950)
+
+
+@pytest.mark.parametrize("N,K,M", [(640, 1088, 1000), (328, 704, 513), (896, 320, 700)])
+@pytest.mark.parametrize("b0,B0", [(3, 64), (4, 32)])
+def test_linear_pair_kernel_ragged_tiles(N, K, M, b0, B0):
+    """M > 256 (CTA-pair kernel) with M, N, K that are not multiples of the 512 x 256 pair tile: the second CTA of a
+    pair may have no weight rows / columns, the TMA stores clip, and the contraction ends inside a 128-row tile."""
+    A = inputs.gaussian(600 + N, (N, K), 0.02)
+    l1b, l2b = inputs.lowrank_factors(601 + K, N, K, 64, 0.01)
+    run_case(A, l1b, l2b, C(b0, B0, 8, 64, 32), M, seed=700 + M)
+
+
 @pytest.mark.parametrize("M", [4, 256])
 def test_linear_without_lowrank_and_with_zero_weights(M):
     N, K = 256, 512
