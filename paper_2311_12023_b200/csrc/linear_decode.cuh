@@ -31,7 +31,10 @@ constexpr int kXRowBytes = kStageTiles * kTileCols * 2 + 16;   // one token's ac
 // A ring stage: the packed tiles, then the activations of the stage's 512 columns for 8 NT token rows.
 // NT = number of 8-token groups (1: M <= 8, two CTAs per SM; 2: M <= 16, one CTA per SM)
 template <int B, int NT> __host__ __device__ constexpr int stage_bytes() { return kStageTiles * 1024 * B + 8 * NT * kXRowBytes; }
-template <int B, int NT> __host__ __device__ constexpr int num_stages() { return (B == 8) ? 2 : (NT == 2 ? (B == 4 ? 3 : 4) : 2); }
+// CTAs per SM the forward kernel is compiled for: two, except for 8-bit codes and for 4-bit codes with 16 tokens
+// (their stages and registers do not fit twice)
+template <int B, int NT> __host__ __device__ constexpr int fwd_ctas_per_sm() { return (B == 8 || (B == 4 && NT == 2)) ? 1 : 2; }
+template <int B, int NT> __host__ __device__ constexpr int num_stages() { return (B == 8) ? 2 : (fwd_ctas_per_sm<B, NT>() == 1 ? 3 : 2); }
 
 struct Params {
     QView q;
@@ -65,6 +68,13 @@ __device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank
     return v;
 }
 
+// Stores v at the shared-memory offset `local_addr` of CTA `rank` of the cluster.
+__device__ __forceinline__ void st_dsmem_f32(uint32_t local_addr, uint32_t rank, float v) {
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
+}
+
 __device__ __forceinline__ uint32_t pick(const uint4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
 __device__ __forceinline__ float pickf(const float4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
 
@@ -90,7 +100,7 @@ __device__ __forceinline__ void dequant_chunk(const uint32_t (&w)[B], int c, con
 }
 
 template <int B, int NT, bool TWO>
-__global__ void __launch_bounds__(kThreads, (NT == 1 && B != 8) ? 2 : 1)
+__global__ void __launch_bounds__(kThreads, fwd_ctas_per_sm<B, NT>())
 decode_fwd_kernel(const Params p) {
     constexpr int NS = num_stages<B, NT>();
     constexpr int STAGE = stage_bytes<B, NT>();
@@ -259,20 +269,18 @@ decode_fwd_kernel(const Params p) {
             if (active) {
                 const uint32_t* tile = reinterpret_cast<const uint32_t*>(ring + s * STAGE) + (kt_ok ? tile_in_stage : 0) * (256 * B);
                 const int kb = kt_ok ? ((col0 >> q.logB0) - kb_first) : 0;
-                // activations of this thread's 32 columns (token rows past M and missing tiles read as zero)
-                uint4 x[NT][4];
+                // activations of this thread's 32 columns (token rows past M and missing tiles read as zero): the first
+                // eight tokens stay in registers for the whole item, tokens 8..15 are re-read from the stage at each use
+                const uint8_t* xbase = ring + s * STAGE + XOFF + (tile_in_stage * kTileCols + (t & 1) * 32) * 2;
+                uint4 x0[4];
+                {
+                    const bool have = gid < p.M && kt_ok;
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const int m = nt * 8 + gid;
-                    if (m < p.M && kt_ok) {
-                        const uint4* xp = reinterpret_cast<const uint4*>(ring + s * STAGE + XOFF + m * kXRowBytes + (tile_in_stage * kTileCols + (t & 1) * 32) * 2);
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) x[nt][c] = xp[c];
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) x[nt][c] = make_uint4(0u, 0u, 0u, 0u);
-                    }
+                    for (int c = 0; c < 4; ++c)
+                        x0[c] = have ? reinterpret_cast<const uint4*>(xbase + gid * kXRowBytes)[c] : make_uint4(0u, 0u, 0u, 0u);
                 }
+                const bool have1 = NT == 2 && gid + 8 < p.M && kt_ok;
+                const uint4* xp1 = reinterpret_cast<const uint4*>(xbase + (gid + 8) * kXRowBytes);
 #pragma unroll
                 for (int sl = 0; sl < 2; ++sl) {
                     const int slab = 2 * half + sl;
@@ -303,10 +311,12 @@ decode_fwd_kernel(const Params p) {
                             uint32_t oa[4], ob[4];
                             dequant_chunk<B>(wa, c, ta, (TWO && c >= 2) ? sa_hi : sa_lo, oa, lut8);
                             dequant_chunk<B>(wb, c, tb, (TWO && c >= 2) ? sb_hi : sb_lo, ob, lut8);
-#pragma unroll
-                            for (int nt = 0; nt < NT; ++nt) {
-                                mma16816(acc[sl][set][nt], oa[0], ob[0], oa[1], ob[1], x[nt][c].x, x[nt][c].y);
-                                mma16816(acc[sl][set][nt], oa[2], ob[2], oa[3], ob[3], x[nt][c].z, x[nt][c].w);
+                            mma16816(acc[sl][set][0], oa[0], ob[0], oa[1], ob[1], x0[c].x, x0[c].y);
+                            mma16816(acc[sl][set][0], oa[2], ob[2], oa[3], ob[3], x0[c].z, x0[c].w);
+                            if constexpr (NT == 2) {
+                                const uint4 x1 = have1 ? xp1[c] : make_uint4(0u, 0u, 0u, 0u);
+                                mma16816(acc[sl][set][1], oa[0], ob[0], oa[1], ob[1], x1.x, x1.y);
+                                mma16816(acc[sl][set][1], oa[2], ob[2], oa[3], ob[3], x1.z, x1.w);
                             }
                         }
                     }
@@ -337,54 +347,87 @@ decode_fwd_kernel(const Params p) {
                         red[(warp * KF + ((sl * 2 + set) * NT + nt) * 4 + e) * 32 + lane] = acc[sl][set][nt][e];
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < 2 * KF * 32; idx += kThreads) {
-        const int half = idx / (KF * 32), rest = idx - half * (KF * 32);
-        const float* src = red + (half * 4 * KF) * 32 + rest;
-        part[idx] = (src[0] + src[KF * 32]) + (src[2 * KF * 32] + src[3 * KF * 32]);
-    }
-
-    // ---------------------------------------------------------------------- reduction over the K slices (cluster), rank-r term, store
-    // Eight lanes per output: lane `sub` fetches the partial sum of cluster rank `sub` and multiplies
-    // eight (sixteen for r > 64) elements of the rank-r term; a shuffle tree adds the eight lanes.
-    cluster_sync_all();
+    // The sum of the four warps goes straight to the CTA that owns the row: CTA `rank` of the cluster finishes rows
+    // [rank * 128 / S, (rank + 1) * 128 / S) of the tile row.  recv[(src * rows_share + rl) * MT + m] in the owner's
+    // shared memory (`part`, which nothing else uses) takes the partial sum of cluster rank `src`; remote stores
+    // need no round trip, and after the cluster barrier every CTA only reads its own shared memory.
     const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
     const int rows_share = 128 / p.S;
     const int row_lo = static_cast<int>(rank) * rows_share;
-    if (p.r > 0) pdl_wait();          // T is written by the kernel launched in front of this one
     const uint32_t part_addr = smem_u32(part);
+    for (int idx = threadIdx.x; idx < 2 * KF * 32; idx += kThreads) {
+        const int half = idx / (KF * 32), rest = idx - half * (KF * 32);
+        const float* src = red + (half * 4 * KF) * 32 + rest;
+        const float v = (src[0] + src[KF * 32]) + (src[2 * KF * 32] + src[3 * KF * 32]);
+        // fragment order -> (row, token): k = ((sl * 2 + set) * NT + nt) * 4 + e, lane = gid * 4 + t
+        const int k = rest >> 5, ln = rest & 31;
+        const int e = k & 3, nt = (k >> 2) % NT, ss = (k >> 2) / NT;
+        const int row = (2 * half + (ss >> 1)) * 32 + 4 * (ln >> 2) + 2 * (ss & 1) + (e >> 1);
+        const int m = nt * 8 + 2 * (ln & 3) + (e & 1);
+        const int owner = row / rows_share, rl = row - owner * rows_share;
+        const uint32_t dst = part_addr + static_cast<uint32_t>((static_cast<int>(rank) * rows_share + rl) * MT + m) * 4u;
+        if (m >= p.M) continue;                  // token rows that do not exist
+        if (p.S > 1) st_dsmem_f32(dst, static_cast<uint32_t>(owner), v);
+        else part[(rl) * MT + m] = v;
+    }
+    cluster_sync_all();               // all partial sums have arrived; from here on only local shared memory is read
+    if (p.r > 0) pdl_wait();          // T is written by the kernel launched in front of this one
     const int sub = threadIdx.x & 7;
-    const int n_out = rows_share * p.M;
-    for (int o0 = (threadIdx.x >> 3) & ~3; o0 < n_out; o0 += (kThreads >> 3) & ~3) {
-        const int o = o0 + ((threadIdx.x >> 3) & 3);       // a warp handles four consecutive outputs
-        const bool live = o < n_out;
-        const int m = live ? o / rows_share : 0, rl = live ? o - m * rows_share : 0;
-        const int row = row_lo + rl;
+    // T (at most 16 x 128 bf16) goes to the idle ring; eight lanes share a row n: each takes an eighth of the
+    // rank-r dot product (the row of L1 is read once for all tokens) and the partial sum of one cluster rank
+    __nv_bfloat16* tsm = reinterpret_cast<__nv_bfloat16*>(ring);
+    if (p.r > 0) {
+        for (int i = threadIdx.x; i < p.M * p.r / 8; i += kThreads)
+            reinterpret_cast<uint4*>(tsm)[i] = reinterpret_cast<const uint4*>(p.T)[i];
+    }
+    __syncthreads();
+    const int nvec = p.r / 64;                 // 16-byte vectors of a factor row per lane: 0, 1 or 2 (r <= 128, r % 16 == 0 -> tail below)
+    for (int r0 = (threadIdx.x >> 3) & ~3; r0 < rows_share; r0 += (kThreads >> 3) & ~3) {
+        const int rl = r0 + ((threadIdx.x >> 3) & 3);          // a warp handles four consecutive rows
+        const bool live = rl < rows_share;
+        const int row = row_lo + (live ? rl : 0);
         const int n = tile_row * 128 + row;
-        float sum = 0.0f;
-        if (live && sub < p.S) {
-            const int half = row >> 6, sl = (row >> 5) & 1, r32 = row & 31;
-            const int k = (((sl * 2 + ((r32 >> 1) & 1)) * NT + (m >> 3)) * 4) + (r32 & 1) * 2 + (m & 1);
-            const int ln = (r32 >> 2) * 4 + ((m & 7) >> 1);
-            sum = ld_dsmem_f32(part_addr + static_cast<uint32_t>((half * KF + k) * 32 + ln) * 4u, static_cast<uint32_t>(sub));
-        }
-        if (live && p.r > 0 && n < q.N) {
-            for (int j = sub; j < p.r / 8; j += 8) {
-                const uint4 a = __ldg(reinterpret_cast<const uint4*>(p.L1 + static_cast<size_t>(n) * p.r) + j);
-                const uint4 b = *(reinterpret_cast<const uint4*>(p.T + static_cast<size_t>(m) * p.r) + j);
-                const uint32_t aa[4] = {a.x, a.y, a.z, a.w}, bb[4] = {b.x, b.y, b.z, b.w};
+        const bool row_ok = live && n < q.N;
+        // this lane's slice of the factor row: elements [8 (sub + 8 v), +8) for v < ceil(r / 64)
+        uint4 a[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+        bool have[2] = {false, false};
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    sum = fmaf(__uint_as_float(aa[e] << 16), __uint_as_float(bb[e] << 16), sum);
-                    sum = fmaf(__uint_as_float(aa[e] & 0xffff0000u), __uint_as_float(bb[e] & 0xffff0000u), sum);
+        for (int v = 0; v < 2; ++v) {
+            have[v] = row_ok && (8 * (sub + 8 * v) < p.r);
+            if (have[v]) a[v] = __ldg(reinterpret_cast<const uint4*>(p.L1 + static_cast<size_t>(n) * p.r) + sub + 8 * v);
+        }
+        (void)nvec;
+        for (int m4 = 0; m4 < p.M; m4 += 4) {
+            float sum[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int m = m4 + u;
+                sum[u] = (live && m < p.M && sub < p.S) ? part[(sub * rows_share + rl) * MT + m] : 0.0f;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int m = m4 + u;
+                if (m < p.M) {
+#pragma unroll
+                    for (int v = 0; v < 2; ++v) {
+                        if (have[v]) {
+                            const uint4 b = *(reinterpret_cast<const uint4*>(tsm + static_cast<size_t>(m) * p.r) + sub + 8 * v);
+                            const uint32_t aa[4] = {a[v].x, a[v].y, a[v].z, a[v].w}, bb[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                sum[u] = fmaf(__uint_as_float(aa[e] << 16), __uint_as_float(bb[e] << 16), sum[u]);
+                                sum[u] = fmaf(__uint_as_float(aa[e] & 0xffff0000u), __uint_as_float(bb[e] & 0xffff0000u), sum[u]);
+                            }
+                        }
+                    }
                 }
+                sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], 1);
+                sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], 2);
+                sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], 4);
+                if (row_ok && sub == 0 && m < p.M) p.Y[static_cast<size_t>(m) * q.N + n] = __float2bfloat16_rn(sum[u]);
             }
         }
-        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-        sum += __shfl_xor_sync(0xffffffffu, sum, 4);
-        if (live && sub == 0 && n < q.N) p.Y[static_cast<size_t>(m) * q.N + n] = __float2bfloat16_rn(sum);
     }
-    cluster_sync_all();               // shared memory of this CTA may be read by its peers until here
 }
 
 // ------------------------------------------------------------------------------------ input gradient for few rows
@@ -412,12 +455,14 @@ struct BwdParams {
 constexpr int kBwdStageRows = 256;
 constexpr int kBwdYRowBytes = kBwdStageRows * 2 + 16;
 template <int B, int NT> __host__ __device__ constexpr int bwd_stage_bytes() { return 8 * 1024 * B + 8 * NT * kBwdYRowBytes; }
-template <int B> __host__ __device__ constexpr int bwd_stages() { return (B == 8) ? 2 : 3; }
+// CTAs per SM the input-gradient kernel is compiled for: two for up to 8 tokens and 2/3-bit codes
+template <int B, int NT> __host__ __device__ constexpr int bwd_ctas_per_sm() { return (NT == 1 && B <= 3) ? 2 : 1; }
+template <int B, int NT> __host__ __device__ constexpr int bwd_stages() { return (B == 8 || bwd_ctas_per_sm<B, NT>() == 2) ? 2 : 3; }
 
 template <int B, int NT, bool TWO>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, bwd_ctas_per_sm<B, NT>())
 decode_bwd_kernel(const BwdParams p) {
-    constexpr int NS = bwd_stages<B>();
+    constexpr int NS = bwd_stages<B, NT>();
     constexpr int STAGE = bwd_stage_bytes<B, NT>();
     constexpr int YOFF = 8 * 1024 * B;
     constexpr int KF = 64 * NT;            // accumulator registers per thread
@@ -631,49 +676,75 @@ decode_bwd_kernel(const BwdParams p) {
         }
         __syncthreads();
     }
+    // Warp 0 holds the CTA's sums; each value goes straight to the CTA that finishes its column: CTA `rank` owns
+    // columns [rank * 256 / S, (rank + 1) * 256 / S) of the window.  recv[(src * cols_share + cl) * MT + m] in the
+    // owner's shared memory (`part`) takes the partial sum of cluster rank `src`; after the cluster barrier every
+    // CTA only reads its own shared memory.
+    constexpr int MT = 8 * NT;
+    const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
+    const int cols_share = 256 / p.S;
+    const int col_lo = static_cast<int>(rank) * cols_share;
     if (warp == 0) {
 #pragma unroll
         for (int mm = 0; mm < 16; ++mm)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) part[((mm * NT + nt) * 4 + e) * 32 + lane] = acc[mm][nt][e];
+                for (int e = 0; e < 4; ++e) red[((mm * NT + nt) * 4 + e) * 32 + lane] = acc[mm][nt][e];
     }
     __syncthreads();
-
-    // ---------------------------------------------------------------------- sum over the row slices (cluster), rank-r term, store
-    cluster_sync_all();
-    const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
-    const int cols_share = 256 / p.S;
-    const int col_lo = static_cast<int>(rank) * cols_share;
-    if (p.r > 0) pdl_wait();
-    const uint32_t part_addr = smem_u32(part);
-    const int sub = threadIdx.x & 7;
-    const int n_out = cols_share * p.M;
-    for (int o0 = (threadIdx.x >> 3) & ~3; o0 < n_out; o0 += (kThreads >> 3) & ~3) {
-        const int o = o0 + ((threadIdx.x >> 3) & 3);
-        const bool live = o < n_out;
-        const int m = live ? o / cols_share : 0, cl = live ? o - m * cols_share : 0;
-        const int col_local = col_lo + cl;                    // 0..255 inside the window
-        const int kcol = col_first + col_local;
-        float sum = 0.0f;
-        if (live && sub < p.S) {
-            const int g8 = col_local >> 5, cc = col_local & 31;
-            const int mm = (cc >> 3) * 4 + ((cc >> 1) & 3);
-            const int e = (cc & 1) * 2 + (m & 1);
-            const int ln = g8 * 4 + ((m & 7) >> 1);
-            sum = ld_dsmem_f32(part_addr + static_cast<uint32_t>(((mm * NT + (m >> 3)) * 4 + e) * 32 + ln) * 4u, static_cast<uint32_t>(sub));
+    {
+        const uint32_t part_addr = smem_u32(part);
+        for (int idx = threadIdx.x; idx < KF * 32; idx += kThreads) {
+            // fragment order: idx = ((mm * NT + nt) * 4 + e) * 32 + lane; columns cA = 8 (mm / 4) + 2 (mm % 4) (e < 2) and
+            // cA + 1 (e >= 2) of group gid = lane / 4; token nt * 8 + 2 (lane % 4) + (e & 1)
+            const int ln = idx & 31, k = idx >> 5;
+            const int e = k & 3, nt = (k >> 2) % NT, mm = (k >> 2) / NT;
+            const int col_local = (ln >> 2) * 32 + (mm >> 2) * 8 + (mm & 3) * 2 + (e >> 1);
+            const int m = nt * 8 + 2 * (ln & 3) + (e & 1);
+            const int owner = col_local / cols_share, cl = col_local - owner * cols_share;
+            const uint32_t off = static_cast<uint32_t>((static_cast<int>(rank) * cols_share + cl) * MT + m) * 4u;
+            if (m >= p.M) continue;              // token rows that do not exist
+            if (p.S > 1) st_dsmem_f32(part_addr + off, static_cast<uint32_t>(owner), red[idx]);
+            else part[cl * MT + m] = red[idx];
         }
-        if (live && p.r > 0 && kcol < q.K) {
-            for (int jj = sub; jj < p.r; jj += 8)
-                sum = fmaf(__bfloat162float(p.T[static_cast<size_t>(m) * p.r + jj]), __bfloat162float(p.L2[static_cast<size_t>(jj) * q.K + kcol]), sum);
-        }
-        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-        sum += __shfl_xor_sync(0xffffffffu, sum, 4);
-        if (live && sub == 0 && kcol < q.K) p.dX[static_cast<size_t>(m) * q.K + kcol] = __float2bfloat16_rn(sum);
     }
-    cluster_sync_all();
+    __syncthreads();
+    cluster_sync_all();               // all partial sums have arrived
+    if (p.r > 0) pdl_wait();
+    const int sub = threadIdx.x & 7;
+    // T' (at most 16 x 128 bf16) goes to the idle ring; eight lanes share an output column: each takes an eighth of
+    // the rank-r sum (its elements of the column of L2 are read once for all tokens) and one rank's partial sum
+    __nv_bfloat16* tsm = reinterpret_cast<__nv_bfloat16*>(ring);
+    if (p.r > 0) {
+        for (int i = threadIdx.x; i < p.M * p.r / 8; i += kThreads)
+            reinterpret_cast<uint4*>(tsm)[i] = reinterpret_cast<const uint4*>(p.T)[i];
+    }
+    __syncthreads();
+    for (int c0 = (threadIdx.x >> 3) & ~3; c0 < cols_share; c0 += (kThreads >> 3) & ~3) {
+        const int cl = c0 + ((threadIdx.x >> 3) & 3);
+        const bool live = cl < cols_share;
+        const int kcol = col_first + col_lo + (live ? cl : 0);
+        const bool col_live = live && kcol < q.K;
+        float f[16];                  // L2[j][kcol] for j = sub, sub + 8, ... (r <= 128)
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int jj = sub + 8 * i;
+            f[i] = (col_live && jj < p.r) ? __bfloat162float(p.L2[static_cast<size_t>(jj) * q.K + kcol]) : 0.0f;
+        }
+        for (int m = 0; m < p.M; ++m) {
+            float sum = (live && sub < p.S) ? part[(sub * cols_share + cl) * MT + m] : 0.0f;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int jj = sub + 8 * i;
+                if (jj < p.r) sum = fmaf(__bfloat162float(tsm[static_cast<size_t>(m) * p.r + jj]), f[i], sum);
+            }
+            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+            if (col_live && sub == 0) p.dX[static_cast<size_t>(m) * q.K + kcol] = __float2bfloat16_rn(sum);
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------ rank-r pre-product for few rows
@@ -692,12 +763,12 @@ struct PreParams {
     int nranks;
 };
 
-constexpr int kPreThreads = 512;      // 16 columns j x 32 contraction phases
-constexpr int kPreJ = 16;             // columns of T per CTA
+constexpr int kPreThreads = 512;      // 8 columns j x 64 contraction phases
+constexpr int kPreJ = 8;              // columns of T per CTA
 constexpr int kPrePhases = kPreThreads / kPreJ;
 
-// Grid (ranks, r / 16), cluster (ranks, 1, 1): a cluster computes 16 columns of T, each of its CTAs over a slice
-// of the contraction.  Dynamic shared memory: [A slice: MP rows x chunk bf16][red: 32 x 16 x 16 fp32][part: 16 x 16 fp32]
+// Grid (ranks, r / 8), cluster (ranks, 1, 1): a cluster computes 8 columns of T, each of its CTAs over a slice
+// of the contraction.  Dynamic shared memory: [A slice: MP rows x chunk bf16][red: 64 x 16 x 8 fp32][part: 16 x 8 fp32]
 // MP = M rounded up to a power of two (rows staged).
 template <bool BWD, int MP>
 __global__ void __launch_bounds__(kPreThreads) decode_pre_kernel(const PreParams p) {
@@ -724,7 +795,7 @@ __global__ void __launch_bounds__(kPreThreads) decode_pre_kernel(const PreParams
     for (int m = 0; m < 16; ++m) red[(ph * 16 + m) * kPreJ + jl] = 0.0f;
     __syncthreads();
     if (j < p.r) {
-        // vectors of eight contraction elements, phase ph takes vectors ph, ph + 32, ...; four are in flight at a time
+        // vectors of eight contraction elements, phase ph takes vectors ph, ph + 64, ...; up to four are in flight at a time
 #pragma unroll 1
         for (int v0 = ph; v0 < nvec; v0 += 4 * kPrePhases) {
             float f[4][8];
@@ -749,7 +820,8 @@ __global__ void __launch_bounds__(kPreThreads) decode_pre_kernel(const PreParams
                 float acc = 0.0f;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int v = min(v0 + u * kPrePhases, nvec - 1);      // past the end: factors are zero
+                    const int v = v0 + u * kPrePhases;
+                    if (v >= nvec) break;
                     const uint4 w = *reinterpret_cast<const uint4*>(as + static_cast<size_t>(m) * p.chunk + v * 8);
                     const uint32_t vv[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
@@ -767,7 +839,7 @@ __global__ void __launch_bounds__(kPreThreads) decode_pre_kernel(const PreParams
         float sum = 0.0f;
 #pragma unroll 8
         for (int q8 = 0; q8 < kPrePhases; ++q8) sum += red[q8 * 16 * kPreJ + threadIdx.x];
-        part[threadIdx.x] = sum;          // part[m * 16 + jl]
+        part[threadIdx.x] = sum;          // part[m * kPreJ + jl]
     }
     cluster_sync_all();
     if (p.nranks == 1 || cluster_ctarank() == 0) {
@@ -816,7 +888,7 @@ inline Plan make_plan(const QView& q, int M) {
     Plan pl{};
     pl.NT = (M <= 8) ? 1 : 2;
     pl.tile_rows = q.ntiles;
-    const int per_sm = (pl.NT == 1 && B != 8) ? 2 : 1;
+    const int per_sm = (pl.NT == 1) ? fwd_ctas_per_sm<B, 1>() : fwd_ctas_per_sm<B, 2>();
     const int slots = sm_count_cached() * per_sm;
     const size_t limit = (per_sm == 2) ? 113 * 1024 : kSmemLimit;
     int S = 1;
@@ -981,7 +1053,8 @@ inline BwdPlan make_bwd_plan_s(const QView& q, int M, int S) {
     const int rows_stride = trps * 128 + 8;
     const int nkb_cap = (256 >> q.logB0) + 2;
     const size_t stage = (pl.NT == 1) ? bwd_stage_bytes<B, 1>() : bwd_stage_bytes<B, 2>();
-    const size_t smem = 128 + bwd_stages<B>() * stage + 64 * pl.NT * 32 * 4 + (B == 8 ? 1024 : 0) + (2 * bwd_stages<B>() + 2) * 8 +
+    const int ns = (pl.NT == 1) ? bwd_stages<B, 1>() : bwd_stages<B, 2>();
+    const size_t smem = 128 + ns * stage + 64 * pl.NT * 32 * 4 + (B == 8 ? 1024 : 0) + (2 * ns + 2) * 8 +
                         static_cast<size_t>(nkb_cap) * rows_stride * 4;
     pl.ok = smem <= static_cast<size_t>(kSmemLimit) && (S == 1 || q.ntiles / S >= 1);
     pl.S = S; pl.trows_per_split = trps; pl.rows_stride = rows_stride; pl.smem = smem;
