@@ -476,13 +476,19 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int row = item & 127, cg = item >> 7;
                 const int m = m0 + h * 128 + row;
                 const int col = col_lo + cg * 8;
-                float sum[8];
+                // all remote loads are requested before the first is used (a round trip costs about two thousand clocks)
+                float part[8][8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) sum[i] = 0.0f;
-                for (int rk = 0; rk < nsplit; ++rk) {
+                for (int rk = 0; rk < 8; ++rk)
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        sum[i] += dec::ld_dsmem_f32(accbuf_addr + static_cast<uint32_t>((col + i) * 128 + row) * 4u, static_cast<uint32_t>(rk));
+                        part[rk][i] = (rk < nsplit) ? dec::ld_dsmem_f32(accbuf_addr + static_cast<uint32_t>((col + i) * 128 + row) * 4u, static_cast<uint32_t>(rk)) : 0.0f;
+                float sum[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    sum[i] = 0.0f;
+#pragma unroll
+                    for (int rk = 0; rk < 8; ++rk) sum[i] += part[rk][i];
                 }
                 if (m < p.M && c0 + col < p.out_cols) {
                     uint32_t w[4];
