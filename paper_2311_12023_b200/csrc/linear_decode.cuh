@@ -334,7 +334,36 @@ decode_fwd_kernel(const Params p) {
     // which is row (2 half + sl) * 32 + 4 gid + 2 set + (e >> 1) and token nt * 8 + 2 t + (e & 1).
     constexpr int KF = 16 * NT;
     float* red = reinterpret_cast<float*>(ring);
+    // T (at most 16 x 128 bf16) is staged behind the reduction buffer
+    __nv_bfloat16* tsm = reinterpret_cast<__nv_bfloat16*>(ring + kConsumerWarps * KF * 128);
+    static_assert(kConsumerWarps * KF * 128 + 4096 <= NS * STAGE, "reduction buffer and T must fit into the ring");
+    // CTA `rank` of the cluster finishes rows [rank * 128 / S, (rank + 1) * 128 / S) of the tile row
+    const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
+    const int rows_share = 128 / p.S;
+    const int row_lo = static_cast<int>(rank) * rows_share;
+    const int sub = threadIdx.x & 7;
     __syncthreads();                      // all stages consumed: the ring is free
+    // Requested now, used after the cluster barrier (the latency of global memory is hidden behind the reduction):
+    // this thread's piece of T (written by the kernel launched in front of this one) and, for the first pass of the
+    // epilogue, its slice of the row of L1: elements [8 (sub + 8 v), +8) for v < ceil(r / 64).
+    if (p.r > 0) pdl_wait();
+    const int t_vecs = p.M * p.r / 8;
+    uint4 tv = make_uint4(0u, 0u, 0u, 0u);
+    if (static_cast<int>(threadIdx.x) < t_vecs) tv = __ldg(reinterpret_cast<const uint4*>(p.T) + threadIdx.x);
+    auto load_factor = [&](int rl, uint4 (&a)[2], bool (&have)[2]) {
+        const bool live = rl < rows_share;
+        const int n = tile_row * 128 + row_lo + (live ? rl : 0);
+#pragma unroll
+        for (int v = 0; v < 2; ++v) {
+            a[v] = make_uint4(0u, 0u, 0u, 0u);
+            have[v] = live && n < q.N && (8 * (sub + 8 * v) < p.r);
+            if (have[v]) a[v] = __ldg(reinterpret_cast<const uint4*>(p.L1 + static_cast<size_t>(n) * p.r) + sub + 8 * v);
+        }
+    };
+    uint4 a_first[2];
+    bool have_first[2];
+    load_factor(static_cast<int>(threadIdx.x >> 3), a_first, have_first);
+
     if (warp < kConsumerWarps) {
 #pragma unroll
         for (int sl = 0; sl < 2; ++sl)
@@ -347,13 +376,9 @@ decode_fwd_kernel(const Params p) {
                         red[(warp * KF + ((sl * 2 + set) * NT + nt) * 4 + e) * 32 + lane] = acc[sl][set][nt][e];
     }
     __syncthreads();
-    // The sum of the four warps goes straight to the CTA that owns the row: CTA `rank` of the cluster finishes rows
-    // [rank * 128 / S, (rank + 1) * 128 / S) of the tile row.  recv[(src * rows_share + rl) * MT + m] in the owner's
-    // shared memory (`part`, which nothing else uses) takes the partial sum of cluster rank `src`; remote stores
-    // need no round trip, and after the cluster barrier every CTA only reads its own shared memory.
-    const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
-    const int rows_share = 128 / p.S;
-    const int row_lo = static_cast<int>(rank) * rows_share;
+    // The sum of the four warps goes straight to the CTA that owns the row.  recv[(src * rows_share + rl) * MT + m] in
+    // the owner's shared memory (`part`, which nothing else uses) takes the partial sum of cluster rank `src`; remote
+    // stores need no round trip, and after the cluster barrier every CTA only reads its own shared memory.
     const uint32_t part_addr = smem_u32(part);
     for (int idx = threadIdx.x; idx < 2 * KF * 32; idx += kThreads) {
         const int half = idx / (KF * 32), rest = idx - half * (KF * 32);
@@ -370,33 +395,27 @@ decode_fwd_kernel(const Params p) {
         if (p.S > 1) st_dsmem_f32(dst, static_cast<uint32_t>(owner), v);
         else part[(rl) * MT + m] = v;
     }
-    cluster_sync_all();               // all partial sums have arrived; from here on only local shared memory is read
-    if (p.r > 0) pdl_wait();          // T is written by the kernel launched in front of this one
-    const int sub = threadIdx.x & 7;
-    // T (at most 16 x 128 bf16) goes to the idle ring; eight lanes share a row n: each takes an eighth of the
-    // rank-r dot product (the row of L1 is read once for all tokens) and the partial sum of one cluster rank
-    __nv_bfloat16* tsm = reinterpret_cast<__nv_bfloat16*>(ring);
-    if (p.r > 0) {
-        for (int i = threadIdx.x; i < p.M * p.r / 8; i += kThreads)
-            reinterpret_cast<uint4*>(tsm)[i] = reinterpret_cast<const uint4*>(p.T)[i];
-    }
-    __syncthreads();
-    const int nvec = p.r / 64;                 // 16-byte vectors of a factor row per lane: 0, 1 or 2 (r <= 128, r % 16 == 0 -> tail below)
-    for (int r0 = (threadIdx.x >> 3) & ~3; r0 < rows_share; r0 += (kThreads >> 3) & ~3) {
-        const int rl = r0 + ((threadIdx.x >> 3) & 3);          // a warp handles four consecutive rows
+    if (static_cast<int>(threadIdx.x) < t_vecs) reinterpret_cast<uint4*>(tsm)[threadIdx.x] = tv;
+    for (int i = threadIdx.x + kThreads; i < t_vecs; i += kThreads)
+        reinterpret_cast<uint4*>(tsm)[i] = __ldg(reinterpret_cast<const uint4*>(p.T) + i);
+    cluster_sync_all();               // all partial sums have arrived (and T is staged); from here on only local shared memory is read
+    // eight lanes share a row n: each takes an eighth of the rank-r dot product (the row of L1 is read once for all
+    // tokens) and the partial sum of one cluster rank
+    constexpr int kRowsPerPass = kThreads >> 3;
+    for (int r0 = 0; r0 < rows_share; r0 += kRowsPerPass) {
+        const int rl = r0 + static_cast<int>(threadIdx.x >> 3);
         const bool live = rl < rows_share;
         const int row = row_lo + (live ? rl : 0);
         const int n = tile_row * 128 + row;
         const bool row_ok = live && n < q.N;
-        // this lane's slice of the factor row: elements [8 (sub + 8 v), +8) for v < ceil(r / 64)
-        uint4 a[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
-        bool have[2] = {false, false};
+        uint4 a[2];
+        bool have[2];
+        if (r0 == 0) {
 #pragma unroll
-        for (int v = 0; v < 2; ++v) {
-            have[v] = row_ok && (8 * (sub + 8 * v) < p.r);
-            if (have[v]) a[v] = __ldg(reinterpret_cast<const uint4*>(p.L1 + static_cast<size_t>(n) * p.r) + sub + 8 * v);
+            for (int v = 0; v < 2; ++v) { a[v] = a_first[v]; have[v] = have_first[v]; }
+        } else {
+            load_factor(rl, a, have);
         }
-        (void)nvec;
         for (int m4 = 0; m4 < p.M; m4 += 4) {
             float sum[4];
 #pragma unroll
@@ -684,6 +703,10 @@ decode_bwd_kernel(const BwdParams p) {
     const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
     const int cols_share = 256 / p.S;
     const int col_lo = static_cast<int>(rank) * cols_share;
+    const int sub = threadIdx.x & 7;
+    // T' (at most 16 x 128 bf16) is staged behind the reduction buffer
+    __nv_bfloat16* tsm = reinterpret_cast<__nv_bfloat16*>(ring + 4 * KF * 128);
+    static_assert(4 * KF * 128 + 4096 <= NS * STAGE, "reduction buffer and T' must fit into the ring");
     if (warp == 0) {
 #pragma unroll
         for (int mm = 0; mm < 16; ++mm)
@@ -692,6 +715,24 @@ decode_bwd_kernel(const BwdParams p) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) red[((mm * NT + nt) * 4 + e) * 32 + lane] = acc[mm][nt][e];
     }
+    // Requested now, used after the cluster barrier: this thread's piece of T' (written by the kernel launched in
+    // front of this one) and, for the first pass of the epilogue, its elements L2[j][kcol], j = sub, sub + 8, ...
+    if (p.r > 0) pdl_wait();
+    const int t_vecs = p.M * p.r / 8;
+    uint4 tv = make_uint4(0u, 0u, 0u, 0u);
+    if (static_cast<int>(threadIdx.x) < t_vecs) tv = __ldg(reinterpret_cast<const uint4*>(p.T) + threadIdx.x);
+    auto load_factor = [&](int cl, float (&f)[16]) {
+        const bool live = cl < cols_share;
+        const int kcol = col_first + col_lo + (live ? cl : 0);
+        const bool col_live = live && kcol < q.K;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int jj = sub + 8 * i;
+            f[i] = (col_live && jj < p.r) ? __bfloat162float(p.L2[static_cast<size_t>(jj) * q.K + kcol]) : 0.0f;
+        }
+    };
+    float f_first[16];
+    load_factor(static_cast<int>(threadIdx.x >> 3), f_first);
     __syncthreads();
     {
         const uint32_t part_addr = smem_u32(part);
@@ -709,28 +750,24 @@ decode_bwd_kernel(const BwdParams p) {
             else part[cl * MT + m] = red[idx];
         }
     }
-    __syncthreads();
-    cluster_sync_all();               // all partial sums have arrived
-    if (p.r > 0) pdl_wait();
-    const int sub = threadIdx.x & 7;
-    // T' (at most 16 x 128 bf16) goes to the idle ring; eight lanes share an output column: each takes an eighth of
-    // the rank-r sum (its elements of the column of L2 are read once for all tokens) and one rank's partial sum
-    __nv_bfloat16* tsm = reinterpret_cast<__nv_bfloat16*>(ring);
-    if (p.r > 0) {
-        for (int i = threadIdx.x; i < p.M * p.r / 8; i += kThreads)
-            reinterpret_cast<uint4*>(tsm)[i] = reinterpret_cast<const uint4*>(p.T)[i];
-    }
-    __syncthreads();
-    for (int c0 = (threadIdx.x >> 3) & ~3; c0 < cols_share; c0 += (kThreads >> 3) & ~3) {
-        const int cl = c0 + ((threadIdx.x >> 3) & 3);
+    if (static_cast<int>(threadIdx.x) < t_vecs) reinterpret_cast<uint4*>(tsm)[threadIdx.x] = tv;
+    for (int i = threadIdx.x + kThreads; i < t_vecs; i += kThreads)
+        reinterpret_cast<uint4*>(tsm)[i] = __ldg(reinterpret_cast<const uint4*>(p.T) + i);
+    cluster_sync_all();               // all partial sums have arrived (and T' is staged)
+    // eight lanes share an output column: each takes an eighth of the rank-r sum (its elements of the column of L2
+    // are read once for all tokens) and one rank's partial sum
+    constexpr int kColsPerPass = kThreads >> 3;
+    for (int c0 = 0; c0 < cols_share; c0 += kColsPerPass) {
+        const int cl = c0 + static_cast<int>(threadIdx.x >> 3);
         const bool live = cl < cols_share;
         const int kcol = col_first + col_lo + (live ? cl : 0);
         const bool col_live = live && kcol < q.K;
         float f[16];                  // L2[j][kcol] for j = sub, sub + 8, ... (r <= 128)
+        if (c0 == 0) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int jj = sub + 8 * i;
-            f[i] = (col_live && jj < p.r) ? __bfloat162float(p.L2[static_cast<size_t>(jj) * q.K + kcol]) : 0.0f;
+            for (int i = 0; i < 16; ++i) f[i] = f_first[i];
+        } else {
+            load_factor(cl, f);
         }
         for (int m = 0; m < p.M; ++m) {
             float sum = (live && sub < p.S) ? part[(sub * cols_share + cl) * MT + m] : 0.0f;
