@@ -539,6 +539,48 @@ decode_bwd_kernel(const BwdParams p) {
     const int kb_first = col_first >> q.logB0;
     const int nkb = (((col_first + ncol_tiles * kTileCols - 1) >> q.logB0) - kb_first) + 1;
     const int nrows_cta = ntr_cta * 128;
+    // Fast path: the nkb scale codes of a row segment are contiguous, a power of two in number, aligned, and share
+    // one second-level group (B1 >= 16 >= nkb, both powers of two) -> one vector load per row, four rows in flight.
+    const bool seg_vec = ncol_tiles == 4 && nkb <= 16 && (nkb & (nkb - 1)) == 0 && (q.KB % nkb) == 0 && (kb_first % nkb) == 0 &&
+                         (1 << q.logB1) >= nkb;
+    if (seg_vec) {
+        for (int r0 = threadIdx.x; r0 < nrows_cta; r0 += 4 * kThreads) {
+            uint4 sc16[4];
+            float v[4];
+            int rowv[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int row = r0 + u * kThreads;
+                sc16[u] = make_uint4(0u, 0u, 0u, 0u); v[u] = 0.0f; rowv[u] = -1;
+                if (row < nrows_cta) {
+                    rowv[u] = row;
+                    const int grow = tr0 * 128 + row;
+                    if (grow < q.N) {
+                        const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first;
+                        const uint8_t* src = q.sc + blk;
+                        if (nkb == 16) sc16[u] = __ldg(reinterpret_cast<const uint4*>(src));
+                        else if (nkb == 8) { const uint2 t2 = __ldg(reinterpret_cast<const uint2*>(src)); sc16[u].x = t2.x; sc16[u].y = t2.y; }
+                        else if (nkb == 4) sc16[u].x = __ldg(reinterpret_cast<const uint32_t*>(src));
+                        else if (nkb == 2) sc16[u].x = __ldg(reinterpret_cast<const uint16_t*>(src));
+                        else sc16[u].x = __ldg(src);
+                        v[u] = __ldg(q.v + (blk >> q.logB1));
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (rowv[u] < 0) continue;
+                const uint32_t words[4] = {sc16[u].x, sc16[u].y, sc16[u].z, sc16[u].w};
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    if (i < nkb) {
+                        const uint32_t code = (words[i >> 2] >> (8 * (i & 3))) & 255u;
+                        stab[i * p.rows_stride + rowv[u]] = block_scale(static_cast<uint8_t>(code), v[u]);
+                    }
+                }
+            }
+        }
+    } else {
     for (int e0 = threadIdx.x; e0 < nkb * nrows_cta; e0 += 4 * kThreads) {
         uint32_t sc8[4];
         float v[4];
@@ -561,6 +603,7 @@ decode_bwd_kernel(const BwdParams p) {
 #pragma unroll
         for (int u = 0; u < 4; ++u)
             if (slot[u] >= 0) stab[slot[u]] = block_scale(static_cast<uint8_t>(sc8[u]), v[u]);
+    }
     }
     if constexpr (B == 8) {
         for (int i = threadIdx.x; i < 256; i += kThreads) lut8[i] = c_codebook[3][i];
