@@ -27,6 +27,40 @@ __device__ __forceinline__ uint32_t nearest_code(float x, const float* __restric
     }
 }
 
+// Fast search for 2- and 3-bit codes: binary search of x^ among the (constant) thresholds; `margin` returns the
+// distance from x^ to the nearest threshold it was compared with.  The two neighbours of the final position are
+// always among them, so when margin exceeds the error of x^ every comparison came out as it would for the exact
+// quotient and the code is the same.
+template <int B>
+__device__ __forceinline__ uint32_t search_code(float xh, float& margin) {
+    static_assert(B == 2 || B == 3, "binary search is written out for 3 and 7 thresholds");
+    const float* T = c_threshold[B == 2 ? 0 : 1];
+    if constexpr (B == 2) {
+        const bool p1 = xh > T[1];
+        const float t = p1 ? T[2] : T[0];
+        const bool p2 = xh > t;
+        margin = fminf(fabsf(xh - T[1]), fabsf(xh - t));
+        return (p1 ? 2u : 0u) + (p2 ? 1u : 0u);
+    } else {
+        const bool p1 = xh > T[3];
+        const float t2 = p1 ? T[5] : T[1];
+        const bool p2 = xh > t2;
+        const float ta = p1 ? T[4] : T[0], tb = p1 ? T[6] : T[2];
+        const float t3 = p2 ? tb : ta;
+        const bool p3 = xh > t3;
+        margin = fminf(fminf(fabsf(xh - T[3]), fabsf(xh - t2)), fabsf(xh - t3));
+        return (p1 ? 4u : 0u) + (p2 ? 2u : 0u) + (p3 ? 1u : 0u);
+    }
+}
+
+// Reciprocal used by the fast searches: 0 for an all-zero block (x^ = 0 gives the zero code), NaN for block maxima
+// whose reciprocal is not a normal number (every element then takes the exact route).
+__device__ __forceinline__ float search_reciprocal(float s) {
+    if (s == 0.0f) return 0.0f;
+    if (!(s > 1e-30f && s < 1e30f)) return __int_as_float(0x7fc00000);
+    return __fdiv_rn(1.0f, s);
+}
+
 // One CTA: 32 rows x 256 columns.  Thread (row = tid % 32, grp = tid / 32) owns 32 consecutive
 // columns of one row: it finds the block absmax (with its neighbours through shared memory when
 // B0 > 32), the 32 codes, and writes the b0 words of its group to the packed slab.
@@ -39,7 +73,8 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
     if constexpr (B == 8) {
         th8[threadIdx.x] = c_threshold[3][threadIdx.x];
     }
-    // the bin table pays off for 4- and 8-bit codes (15 / 255 thresholds); 2- and 3-bit codes compare directly
+    // 4- and 8-bit codes (15 / 255 thresholds) find their code through a bin table; 2- and 3-bit codes by a binary
+    // search among constants
     constexpr bool kUseBins = (B >= 4);
     const int nb = kUseBins ? c_nbins[bits_index(B)] : 0;
     if constexpr (kUseBins) {
@@ -98,28 +133,30 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
     uint32_t words[B];
 #pragma unroll
     for (int i = 0; i < B; ++i) words[i] = 0u;
-    // Fast search: x^ = u * fl(1/s) is within 2 ulp of the quotient fl(u/s) that defines the code; the bin of x^
-    // holds at most one threshold, and the code is the number of thresholds below the bin plus (x^ > threshold).
-    // When x^ comes within 1e-6 of that threshold (or is not a number in [-1, 1]: zero, subnormal or huge block
-    // maxima) the decision is taken exactly, with the IEEE quotient and the full search.  No threshold lies that
-    // close to a bin edge (the bin count is chosen on the host for the largest clearance), so the two routes agree.
-    const float r_lo = (s_lo != 0.0f) ? __fdiv_rn(1.0f, s_lo) : 0.0f;
-    const float r_hi = (s_hi != 0.0f) ? __fdiv_rn(1.0f, s_hi) : 0.0f;
+    // Fast search: x^ = u * fl(1/s) is within 2 ulp (2.4e-7) of the quotient fl(u/s) that defines the code.  The code
+    // is found from x^ (bin table: the bin of x^ holds at most one threshold, code = thresholds below the bin plus
+    // (x^ > threshold); 2/3-bit codes: binary search).  When x^ comes within 1e-6 of a threshold it was compared with
+    // (or is not a number in [-1, 1]) the decision is taken exactly, with the IEEE quotient and the full search.  No
+    // threshold lies that close to a bin edge (the bin count is chosen on the host for the largest clearance), so
+    // the two routes agree.
+    const float r_lo = search_reciprocal(s_lo);
+    const float r_hi = search_reciprocal(s_hi);
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
         const float s = (j < 16) ? s_lo : s_hi;
-        if constexpr (!kUseBins) {
-            uint32_t c = zero_code;
-            if (s != 0.0f) c = nearest_code<B>(__fdiv_rn(u[j], s), th8);
-            deposit_code<B>(words, j, c);
-            continue;
-        }
         const float xh = u[j] * ((j < 16) ? r_lo : r_hi);
-        int k = __float2int_rd(fmaf(xh, bin_scale, bin_scale));
-        k = min(max(k, 0), nb);
-        const float2 e = bins[k];
-        uint32_t c = static_cast<uint32_t>(__float_as_int(e.y)) + ((xh > e.x) ? 1u : 0u);
-        if (!(fabsf(xh - e.x) > 1e-6f) || !(fabsf(xh) <= 1.001f)) {
+        uint32_t c;
+        float margin;
+        if constexpr (kUseBins) {
+            int k = __float2int_rd(fmaf(xh, bin_scale, bin_scale));
+            k = min(max(k, 0), nb);
+            const float2 e = bins[k];
+            c = static_cast<uint32_t>(__float_as_int(e.y)) + ((xh > e.x) ? 1u : 0u);
+            margin = fabsf(xh - e.x);
+        } else {
+            c = search_code<B>(xh, margin);
+        }
+        if (!(margin > 1e-6f) || !(fabsf(xh) <= 1.001f)) {
             c = zero_code;
             if (s != 0.0f) c = nearest_code<B>(__fdiv_rn(u[j], s), th8);
         }
