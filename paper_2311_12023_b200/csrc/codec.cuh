@@ -68,6 +68,7 @@ template <int B>
 __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restrict__ W, uint32_t* __restrict__ codes,
                                                            float* __restrict__ absmax, int N, int K, int B0, int logB0) {
     __shared__ float red[8][33];
+    __shared__ __align__(16) float4 tile[8][32 * 8];   // per warp: 32 rows x 32 columns
     __shared__ float th8[256];
     __shared__ float2 bins[kMaxBins + 1];        // (threshold of the bin or +inf, number of thresholds below the bin)
     if constexpr (B == 8) {
@@ -90,17 +91,31 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
     const bool live = (k0 < K);
     const bool real = live && (row < N);
 
+    // A warp owns 32 rows x 32 columns.  It loads them coalesced (a load instruction covers four rows of 128 bytes),
+    // passes them through its own shared-memory tile (16-byte chunks swizzled by row, conflict-free both ways) and
+    // each lane reads back the 32 columns of one row.
     float u[32];
-    if (real) {
-        const float4* src = reinterpret_cast<const float4*>(W + static_cast<size_t>(row) * K + k0);
+    {
+        float4* mine = tile[grp];
+        const int lr = rl >> 3, ch = rl & 7;
+        float4 t[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            float4 t = __ldg(src + i);
-            u[4 * i] = t.x; u[4 * i + 1] = t.y; u[4 * i + 2] = t.z; u[4 * i + 3] = t.w;
+            const int rr = blockIdx.x * 32 + 4 * i + lr;
+            t[i] = (live && rr < N) ? __ldg(reinterpret_cast<const float4*>(W + static_cast<size_t>(rr) * K + k0) + ch)
+                                    : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         }
-    } else {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) u[i] = 0.0f;
+        for (int i = 0; i < 8; ++i) {
+            const int r = 4 * i + lr;
+            mine[r * 8 + (ch ^ (r & 7))] = t[i];
+        }
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float4 v = mine[rl * 8 + (i ^ (rl & 7))];
+            u[4 * i] = v.x; u[4 * i + 1] = v.y; u[4 * i + 2] = v.z; u[4 * i + 3] = v.w;
+        }
     }
     // absmax of each 16-wide half
     float m0 = 0.0f, m1 = 0.0f;
