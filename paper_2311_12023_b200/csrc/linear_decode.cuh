@@ -22,7 +22,7 @@ namespace dec {
 using namespace dev;
 
 constexpr int kConsumerWarps = 8;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kThreads = kConsumerWarps * 32;
 constexpr int kStageTiles = 8;              // 64-column tiles per ring stage (four windows of 128 columns)
 constexpr int kSmemLimit = 232448;
 constexpr int kStabStride = 136;            // floats per block column of the scale table (128 rows + padding against bank conflicts)
@@ -75,6 +75,14 @@ __device__ __forceinline__ void st_dsmem_f32(uint32_t local_addr, uint32_t rank,
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
 }
 
+// Counts a warp as done with a ring slot; orders the warp's reads of the slot before the count and, for the warp
+// that sees the last count, the other warps' reads before what it does next (the refill of the slot).
+__device__ __forceinline__ uint32_t slot_done(uint32_t counter_smem) {
+    uint32_t old;
+    asm volatile("atom.acq_rel.cta.shared.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(counter_smem) : "memory");
+    return old;
+}
+
 __device__ __forceinline__ uint32_t pick(const uint4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
 __device__ __forceinline__ float pickf(const float4& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
 
@@ -112,7 +120,8 @@ decode_fwd_kernel(const Params p) {
     uint8_t* ring = base;
     float* part = reinterpret_cast<float*>(ring + NS * STAGE);        // 128 x MT partial sums of this CTA, fragment order
     float* lut8 = part + 128 * MT;                                     // 256 floats (8-bit codes only)
-    uint64_t* bars = reinterpret_cast<uint64_t*>(lut8 + (B == 8 ? 256 : 0));   // full[NS], empty[NS]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(lut8 + (B == 8 ? 256 : 0));   // full[NS], then NS counters of warps done with a slot
+    uint32_t* done = reinterpret_cast<uint32_t*>(bars + NS);
     volatile int* abort_s = reinterpret_cast<volatile int*>(bars + 2 * NS);
     float* stab = reinterpret_cast<float*>(bars + 2 * NS + 2);         // [nkb][kStabStride] block scales s~
 
@@ -127,10 +136,9 @@ decode_fwd_kernel(const Params p) {
     const Ctl ctl{abort_s, p.status};
 
     auto full = [&](int s) { return smem_u32(bars + s); };
-    auto empty = [&](int s) { return smem_u32(bars + NS + s); };
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), kConsumerWarps); }
+        for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); done[s] = 0u; }
         *abort_s = 0;
         fence_barrier_init();
     }
@@ -148,7 +156,9 @@ decode_fwd_kernel(const Params p) {
         for (int m = 0; m < p.M; ++m)
             bulk_load(dst + XOFF + m * kXRowBytes, xsrc + static_cast<size_t>(m) * q.K, nt * (kTileCols * 2), full(s));
     };
-    if (warp == kConsumerWarps && lane == 0) {
+    // There is no producer warp: thread 0 fills the ring once, afterwards the warp that is last to finish a stage
+    // refills its slot (nobody waits for a free slot, and the CTA has eight warps, two per scheduler).
+    if (threadIdx.x == 0) {
         for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it);
     }
 
@@ -235,24 +245,7 @@ decode_fwd_kernel(const Params p) {
 #pragma unroll
                 for (int d = 0; d < 4; ++d) acc[a][b][c][d] = 0.0f;
 
-    if (warp == kConsumerWarps) {
-        // ------------------------------------------------------------------ producer
-        if (lane == 0) {
-            for (int it = NS; it < nstage_total; ++it) {
-                const int s = it % NS;
-                while (!mbar_try_wait(empty(s), ((it / NS) & 1) ^ 1) && !*abort_s) __nanosleep(200);   // leave the issue slots to the consumers
-                if (!wait(empty(s), ((it / NS) & 1) ^ 1, ctl, 21)) break;
-                issue_stage(it);
-            }
-            if (*abort_s) {
-                for (int s = 0; s < NS; ++s) {
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(full(s), 0) && !mbar_try_wait(full(s), 1) && clock64() - t0 < 20000000LL) {}
-                }
-            }
-        }
-        __syncwarp();
-    } else {
+    {
         // ------------------------------------------------------------------ consumers
         const int gid = lane >> 2, t = lane & 3;
         const int win_slot = warp & 3, half = warp >> 2;
@@ -269,8 +262,7 @@ decode_fwd_kernel(const Params p) {
             if (active) {
                 const uint32_t* tile = reinterpret_cast<const uint32_t*>(ring + s * STAGE) + (kt_ok ? tile_in_stage : 0) * (256 * B);
                 const int kb = kt_ok ? ((col0 >> q.logB0) - kb_first) : 0;
-                // activations of this thread's 32 columns (token rows past M and missing tiles read as zero): the first
-                // eight tokens stay in registers for the whole item, tokens 8..15 are re-read from the stage at each use
+                // activations of this thread's 32 columns (token rows past M and missing tiles read as zero)
                 const uint8_t* xbase = ring + s * STAGE + XOFF + (tile_in_stage * kTileCols + (t & 1) * 32) * 2;
                 uint4 x0[4];
                 {
@@ -279,8 +271,13 @@ decode_fwd_kernel(const Params p) {
                     for (int c = 0; c < 4; ++c)
                         x0[c] = have ? reinterpret_cast<const uint4*>(xbase + gid * kXRowBytes)[c] : make_uint4(0u, 0u, 0u, 0u);
                 }
-                const bool have1 = NT == 2 && gid + 8 < p.M && kt_ok;
-                const uint4* xp1 = reinterpret_cast<const uint4*>(xbase + (gid + 8) * kXRowBytes);
+                uint4 x1[NT == 2 ? 4 : 1];
+                if constexpr (NT == 2) {
+                    const bool have1 = gid + 8 < p.M && kt_ok;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        x1[c] = have1 ? reinterpret_cast<const uint4*>(xbase + (gid + 8) * kXRowBytes)[c] : make_uint4(0u, 0u, 0u, 0u);
+                }
 #pragma unroll
                 for (int sl = 0; sl < 2; ++sl) {
                     const int slab = 2 * half + sl;
@@ -314,16 +311,18 @@ decode_fwd_kernel(const Params p) {
                             mma16816(acc[sl][set][0], oa[0], ob[0], oa[1], ob[1], x0[c].x, x0[c].y);
                             mma16816(acc[sl][set][0], oa[2], ob[2], oa[3], ob[3], x0[c].z, x0[c].w);
                             if constexpr (NT == 2) {
-                                const uint4 x1 = have1 ? xp1[c] : make_uint4(0u, 0u, 0u, 0u);
-                                mma16816(acc[sl][set][1], oa[0], ob[0], oa[1], ob[1], x1.x, x1.y);
-                                mma16816(acc[sl][set][1], oa[2], ob[2], oa[3], ob[3], x1.z, x1.w);
+                                mma16816(acc[sl][set][1], oa[0], ob[0], oa[1], ob[1], x1[c].x, x1[c].y);
+                                mma16816(acc[sl][set][1], oa[2], ob[2], oa[3], ob[3], x1[c].z, x1[c].w);
                             }
                         }
                     }
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(empty(s));
+            if (lane == 0 && slot_done(smem_u32(done + s)) == kConsumerWarps - 1) {
+                done[s] = 0u;
+                if (it + NS < nstage_total && !*abort_s) issue_stage(it + NS);
+            }
         }
     }
 
@@ -343,6 +342,16 @@ decode_fwd_kernel(const Params p) {
     const int row_lo = static_cast<int>(rank) * rows_share;
     const int sub = threadIdx.x & 7;
     __syncthreads();                      // all stages consumed: the ring is free
+    if (*abort_s) {
+        // a wait gave up: let copies that are still in flight land before the ring is reused (bounded)
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < NS; ++s) {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(full(s), 0) && !mbar_try_wait(full(s), 1) && clock64() - t0 < 20000000LL) {}
+            }
+        }
+        __syncthreads();
+    }
     // Requested now, used after the cluster barrier (the latency of global memory is hidden behind the reduction):
     // this thread's piece of T (written by the kernel launched in front of this one) and, for the first pass of the
     // epilogue, its slice of the row of L1: elements [8 (sub + 8 v), +8) for v < ceil(r / 64).
@@ -491,7 +500,8 @@ decode_bwd_kernel(const BwdParams p) {
     uint8_t* ring = base;
     float* part = reinterpret_cast<float*>(ring + NS * STAGE);        // KF x 32 partial sums, fragment order
     float* lut8 = part + KF * 32;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(lut8 + (B == 8 ? 256 : 0));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(lut8 + (B == 8 ? 256 : 0));   // full[NS], then NS counters of warps done with a slot
+    uint32_t* done = reinterpret_cast<uint32_t*>(bars + NS);
     volatile int* abort_s = reinterpret_cast<volatile int*>(bars + 2 * NS);
     float* stab = reinterpret_cast<float*>(bars + 2 * NS + 2);         // [nkb][rows_stride] block scales s~
 
@@ -507,10 +517,9 @@ decode_bwd_kernel(const BwdParams p) {
     const Ctl ctl{abort_s, p.status};
 
     auto full = [&](int s) { return smem_u32(bars + s); };
-    auto empty = [&](int s) { return smem_u32(bars + NS + s); };
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), kConsumerWarps); }
+        for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); done[s] = 0u; }
         *abort_s = 0;
         fence_barrier_init();
     }
@@ -530,7 +539,8 @@ decode_bwd_kernel(const BwdParams p) {
         for (int m = 0; m < p.M; ++m)
             bulk_load(dst + YOFF + m * kBwdYRowBytes, p.dY + static_cast<size_t>(m) * q.N + row0, nrows * 2, full(s));
     };
-    if (warp == kConsumerWarps && lane == 0) {
+    // thread 0 fills the ring once; afterwards the warp that is last to finish a stage refills its slot
+    if (threadIdx.x == 0) {
         for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it);
     }
 
@@ -620,23 +630,7 @@ decode_bwd_kernel(const BwdParams p) {
 #pragma unroll
             for (int d = 0; d < 4; ++d) acc[a][b][d] = 0.0f;
 
-    if (warp == kConsumerWarps) {
-        if (lane == 0) {
-            for (int it = NS; it < nstage_total; ++it) {
-                const int s = it % NS;
-                while (!mbar_try_wait(empty(s), ((it / NS) & 1) ^ 1) && !*abort_s) __nanosleep(200);
-                if (!wait(empty(s), ((it / NS) & 1) ^ 1, ctl, 31)) break;
-                issue_stage(it);
-            }
-            if (*abort_s) {
-                for (int s = 0; s < NS; ++s) {
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(full(s), 0) && !mbar_try_wait(full(s), 1) && clock64() - t0 < 20000000LL) {}
-                }
-            }
-        }
-        __syncwarp();
-    } else {
+    {
         const int gid = lane >> 2, t = lane & 3;
         const int ctile = gid >> 1, grp = gid & 1;
         const bool col_ok = ctile < ncol_tiles;
@@ -708,7 +702,10 @@ decode_bwd_kernel(const BwdParams p) {
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(empty(s));
+            if (lane == 0 && slot_done(smem_u32(done + s)) == kConsumerWarps - 1) {
+                done[s] = 0u;
+                if (it + NS < nstage_total && !*abort_s) issue_stage(it + NS);
+            }
         }
     }
 
@@ -717,6 +714,16 @@ decode_bwd_kernel(const BwdParams p) {
     float* red = reinterpret_cast<float*>(ring);
     static_assert(4 * KF * 32 * 4 <= NS * STAGE, "reduction buffer must fit into the ring");
     __syncthreads();
+    if (*abort_s) {
+        // a wait gave up: let copies that are still in flight land before the ring is reused (bounded)
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < NS; ++s) {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(full(s), 0) && !mbar_try_wait(full(s), 1) && clock64() - t0 < 20000000LL) {}
+            }
+        }
+        __syncthreads();
+    }
     for (int active = kConsumerWarps; active > 1; active >>= 1) {
         const int hw = active >> 1;
         if (warp >= hw && warp < active) {
