@@ -1112,14 +1112,16 @@ inline int max_active_clusters(Kern kern, int threads, size_t smem, int cluster_
     cfg.numAttrs = 1;
     // the answer depends on (kernel, shared memory, cluster size) only: keep the last few per kernel
     struct Entry { size_t smem; int cy, n; };
-    static Entry cache[8] = {};
+    static Entry cache[32] = {};
     static int used = 0;
     for (int i = 0; i < used; ++i)
         if (cache[i].smem == smem && cache[i].cy == cluster_y) return cache[i].n;
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
-    cache[used % 8] = Entry{smem, cluster_y, n};
-    if (used < 8) ++used;
+    static int next = 0;
+    cache[next] = Entry{smem, cluster_y, n};
+    next = (next + 1) % 32;
+    if (used < 32) ++used;
     return n;
 }
 
@@ -1138,7 +1140,7 @@ inline BwdPlan make_bwd_plan_s(const QView& q, int M, int S) {
     int trps = (q.ntiles + S - 1) / S;
     trps += trps & 1;
     const int rows_stride = trps * 128 + 8;
-    const int nkb_cap = (256 >> q.logB0) + 2;
+    const int nkb_cap = (256 >> q.logB0) > 0 ? (256 >> q.logB0) : 1;      // a window is 256 aligned columns and B0 divides 256
     const size_t stage = (pl.NT == 1) ? bwd_stage_bytes<B, 1>() : bwd_stage_bytes<B, 2>();
     const int ns = (pl.NT == 1) ? bwd_stages<B, 1>() : bwd_stages<B, 2>();
     const size_t smem = 128 + ns * stage + 64 * pl.NT * 32 * 4 + (B == 8 ? 1024 : 0) + (2 * ns + 2) * 8 +
@@ -1179,13 +1181,20 @@ inline cudaError_t launch_bwd_nt(BwdParams p, const QView& q, int M, bool after_
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    // the most row slices whose clusters are all resident at once; failing that, the fewest slices that fit
+    // Number of row slices: the one with the smallest estimated time.  A wave of resident clusters takes the tile
+    // rows of a CTA times the CTAs that share an SM (a lone CTA does not fill the SM: factor 1.5 instead of 1) plus a
+    // fixed part (scale table, reduction, epilogue) worth about six tile rows.
     BwdPlan pl{};
+    long best = -1;
     for (int S = 8; S >= 1; S >>= 1) {
         const BwdPlan c = make_bwd_plan_s<B>(q, M, S);
         if (!c.ok) continue;
-        pl = c;
-        if (S == 1 || c.nwin <= max_active_clusters(kern, kThreads, c.smem, S)) break;
+        const int cap = max_active_clusters(kern, kThreads, c.smem, S);
+        if (cap <= 0) continue;
+        const long waves = (c.nwin + cap - 1) / cap;
+        const bool shared_sm = static_cast<long>(cap) * S > sm_count_cached() + sm_count_cached() / 2;
+        const long cost = waves * (static_cast<long>(c.trows_per_split) * (shared_sm ? 4 : 3) + 12);    // in half tile rows
+        if (best < 0 || cost < best) { best = cost; pl = c; }
     }
     if (!pl.ok) return cudaErrorInvalidValue;
     p.S = pl.S; p.trows_per_split = pl.trows_per_split; p.rows_stride = pl.rows_stride;
