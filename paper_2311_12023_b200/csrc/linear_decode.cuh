@@ -26,6 +26,7 @@ constexpr int kThreads = kConsumerWarps * 32;
 constexpr int kStageTiles = 8;              // 64-column tiles per ring stage (four windows of 128 columns)
 constexpr int kSmemLimit = 232448;
 constexpr int kStabStride = 136;            // floats per block column of the scale table (128 rows + padding against bank conflicts)
+constexpr int kStab8Stride = 148;           // bytes per block column of the compact scale table (8-bit codes; one sigma per 16 block columns)
 
 constexpr int kXRowBytes = kStageTiles * kTileCols * 2 + 16;   // one token's activations of a stage, padded
 // A ring stage: the packed tiles, then the activations of the stage's 512 columns for 8 NT token rows.
@@ -47,6 +48,7 @@ struct Params {
     int S;                     // K slices per tile row = cluster size
     int tiles_per_split;       // 64-column tiles per CTA (even)
     int nkb_cap;               // capacity of the scale table in blocks
+    int stab8;                 // 1: compact scale table (codes as bytes + fl(v / 127) per 16 block columns), 0: fp32 table
 };
 
 __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
@@ -123,7 +125,10 @@ decode_fwd_kernel(const Params p) {
     uint64_t* bars = reinterpret_cast<uint64_t*>(lut8 + (B == 8 ? 256 : 0));   // full[NS], then NS counters of warps done with a slot
     uint32_t* done = reinterpret_cast<uint32_t*>(bars + NS);
     volatile int* abort_s = reinterpret_cast<volatile int*>(bars + 2 * NS);
-    float* stab = reinterpret_cast<float*>(bars + 2 * NS + 2);         // [nkb][kStabStride] block scales s~
+    float* stab = reinterpret_cast<float*>(bars + 2 * NS + 2);         // [nkb][kStabStride] block scales s~ (fp32 table)
+    // compact table: s^ as bytes [nkb][kStab8Stride], then sigma = fl(v / 127) as [nkb / 16][kStabStride] floats
+    const uint8_t* stab8 = reinterpret_cast<const uint8_t*>(stab);
+    const float* sig = reinterpret_cast<const float*>(stab8 + static_cast<size_t>(p.nkb_cap) * kStab8Stride);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile_row = blockIdx.x;
@@ -166,7 +171,42 @@ decode_fwd_kernel(const Params p) {
     const int kb_first = (kt0 * kTileCols) >> q.logB0;
     const int nkb = (ntiles_cta > 0) ? (((kt1 * kTileCols - 1) >> q.logB0) - kb_first + 1) : 0;
     const bool vec16 = (q.KB % 16 == 0) && (nkb % 16 == 0) && (kb_first % 16 == 0);
-    if (vec16) {
+    if (p.stab8) {
+        // the host chose this form only where every CTA meets the conditions of the 16-code loads; the 16 codes of a
+        // load share their second-level group (aligned, B1 >= 16)
+        uint8_t* st8 = reinterpret_cast<uint8_t*>(stab);
+        float* sg = reinterpret_cast<float*>(st8 + static_cast<size_t>(p.nkb_cap) * kStab8Stride);
+        const int nvec = nkb >> 4;
+        for (int e0 = threadIdx.x; e0 < nvec * 128; e0 += 2 * kThreads) {
+            uint4 sc16[2];
+            float v0[2];
+            int rowv[2], kvv[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int e = e0 + u * kThreads;
+                sc16[u] = make_uint4(0u, 0u, 0u, 0u); v0[u] = 0.0f; rowv[u] = -1; kvv[u] = 0;
+                if (e < nvec * 128) {
+                    const int row = e / nvec, kv = e - row * nvec;
+                    const int grow = tile_row * 128 + row;
+                    rowv[u] = row; kvv[u] = kv;
+                    if (grow < q.N) {
+                        const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first + kv * 16;
+                        sc16[u] = __ldg(reinterpret_cast<const uint4*>(q.sc + blk));
+                        v0[u] = __ldg(q.v + (blk >> q.logB1));
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                if (rowv[u] < 0) continue;
+                const uint32_t words[4] = {sc16[u].x, sc16[u].y, sc16[u].z, sc16[u].w};
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    st8[(kvv[u] * 16 + i) * kStab8Stride + rowv[u]] = static_cast<uint8_t>((words[i >> 2] >> (8 * (i & 3))) & 255u);
+                sg[kvv[u] * kStabStride + rowv[u]] = __fdiv_rn(v0[u], static_cast<float>(kScaleLevels));
+            }
+        }
+    } else if (vec16) {
         // sixteen scale codes per load; they lie in at most two second-level groups (B1 >= 16)
         const int nvec = nkb >> 4;
         for (int e0 = threadIdx.x; e0 < nvec * 128; e0 += 2 * kThreads) {
@@ -285,9 +325,25 @@ decode_fwd_kernel(const Params p) {
                     uint4 w4[B];
 #pragma unroll
                     for (int i = 0; i < B; ++i) w4[i] = *reinterpret_cast<const uint4*>(sp + i * 32);
-                    float4 sc_lo = *reinterpret_cast<const float4*>(stab + kb * kStabStride + slab * 32 + 4 * gid);
-                    float4 sc_hi = sc_lo;
-                    if (TWO) sc_hi = *reinterpret_cast<const float4*>(stab + (kb + 1) * kStabStride + slab * 32 + 4 * gid);
+                    float4 sc_lo, sc_hi;
+                    if (p.stab8) {
+                        // s~ = fl32(float(s^) * fl32(v / 127)) from the compact table
+                        const float4 sg4 = *reinterpret_cast<const float4*>(sig + (kb >> 4) * kStabStride + slab * 32 + 4 * gid);
+                        const uint32_t c_lo = *reinterpret_cast<const uint32_t*>(stab8 + kb * kStab8Stride + slab * 32 + 4 * gid);
+                        sc_lo = make_float4(__fmul_rn(static_cast<float>(c_lo & 255u), sg4.x), __fmul_rn(static_cast<float>((c_lo >> 8) & 255u), sg4.y),
+                                            __fmul_rn(static_cast<float>((c_lo >> 16) & 255u), sg4.z), __fmul_rn(static_cast<float>(c_lo >> 24), sg4.w));
+                        sc_hi = sc_lo;
+                        if (TWO) {
+                            // kb is even here (two blocks of 16 columns per 32-column group), so kb + 1 has the same sigma
+                            const uint32_t c_hi = *reinterpret_cast<const uint32_t*>(stab8 + (kb + 1) * kStab8Stride + slab * 32 + 4 * gid);
+                            sc_hi = make_float4(__fmul_rn(static_cast<float>(c_hi & 255u), sg4.x), __fmul_rn(static_cast<float>((c_hi >> 8) & 255u), sg4.y),
+                                                __fmul_rn(static_cast<float>((c_hi >> 16) & 255u), sg4.z), __fmul_rn(static_cast<float>(c_hi >> 24), sg4.w));
+                        }
+                    } else {
+                        sc_lo = *reinterpret_cast<const float4*>(stab + kb * kStabStride + slab * 32 + 4 * gid);
+                        sc_hi = sc_lo;
+                        if (TWO) sc_hi = *reinterpret_cast<const float4*>(stab + (kb + 1) * kStabStride + slab * 32 + 4 * gid);
+                    }
                     if (!kt_ok) { sc_lo = make_float4(0.f, 0.f, 0.f, 0.f); sc_hi = sc_lo; }
 #pragma unroll
                     for (int set = 0; set < 2; ++set) {
@@ -948,14 +1004,16 @@ __global__ void __launch_bounds__(kPreThreads) decode_pre_kernel(const PreParams
 // ------------------------------------------------------------------------------------ host side
 struct Plan {
     bool ok;
-    int NT, S, tiles_per_split, nkb_cap, tile_rows;
+    int NT, S, tiles_per_split, nkb_cap, tile_rows, stab8;
     size_t smem;
 };
 
 template <int B, int NT>
-inline size_t smem_bytes(int nkb_cap) {
+inline size_t smem_bytes(int nkb_cap, bool stab8) {
+    const size_t table = stab8 ? static_cast<size_t>(nkb_cap) * kStab8Stride + static_cast<size_t>((nkb_cap + 15) / 16) * (kStabStride * 4)
+                               : static_cast<size_t>(nkb_cap) * (kStabStride * 4);
     return 128 + static_cast<size_t>(num_stages<B, NT>()) * stage_bytes<B, NT>() + 128 * 8 * NT * 4 + (B == 8 ? 1024 : 0) +
-           (2 * num_stages<B, NT>() + 2) * 8 + static_cast<size_t>(nkb_cap) * (kStabStride * 4);
+           (2 * num_stages<B, NT>() + 2) * 8 + table;
 }
 
 inline int sm_count_cached() {
@@ -972,27 +1030,39 @@ inline int sm_count_cached() {
 
 template <int B>
 inline Plan make_plan(const QView& q, int M) {
-    Plan pl{};
-    pl.NT = (M <= 8) ? 1 : 2;
-    pl.tile_rows = q.ntiles;
-    const int per_sm = (pl.NT == 1) ? fwd_ctas_per_sm<B, 1>() : fwd_ctas_per_sm<B, 2>();
-    const int slots = sm_count_cached() * per_sm;
-    const size_t limit = (per_sm == 2) ? 113 * 1024 : kSmemLimit;
-    int S = 1;
-    while (S < 8 && pl.tile_rows * (2 * S) <= slots && q.ktiles / (2 * S) >= 2) S *= 2;
-    for (;; S *= 2) {
+    Plan best{};
+    best.ok = false;
+    const int NT = (M <= 8) ? 1 : 2;
+    const int per_sm = (NT == 1) ? fwd_ctas_per_sm<B, 1>() : fwd_ctas_per_sm<B, 2>();
+    const int sms = sm_count_cached();
+    double best_cost = 0.0;
+    // Number of K slices: the one with the smallest estimated time.  The CTAs are spread over the SMs; an SM works
+    // through its CTAs two at a time where two fit (a lone CTA reaches about 0.65 of that rate); every round adds a
+    // fixed part (scale table, reduction, epilogue) worth about 18 tiles.
+    for (int S = 1; S <= 8; S *= 2) {
+        if (S > 1 && q.ktiles / S < 2) break;
         int tps = (q.ktiles + S - 1) / S;
         tps += tps & 1;
-        const int nkb_cap = ((tps * kTileCols) >> q.logB0) + 2;
-        const size_t smem = (pl.NT == 1) ? smem_bytes<B, 1>(nkb_cap) : smem_bytes<B, 2>(nkb_cap);
-        if (smem <= limit || (per_sm == 2 && S == 8 && smem <= static_cast<size_t>(kSmemLimit))) {
-            pl.ok = true; pl.S = S; pl.tiles_per_split = tps; pl.nkb_cap = nkb_cap; pl.smem = smem;
-            return pl;
+        // compact scale table where every CTA has the same, 16-aligned run of blocks per row
+        const int cols = tps * kTileCols;
+        const bool uniform = (q.ktiles % tps == 0) && (cols % q.B0 == 0) && (q.KB % 16 == 0) && ((cols >> q.logB0) % 16 == 0) &&
+                             (1 << q.logB1) >= 16;
+        const int nkb_cap = uniform ? (cols >> q.logB0) : ((cols >> q.logB0) + 2);
+        const size_t smem = (NT == 1) ? smem_bytes<B, 1>(nkb_cap, uniform) : smem_bytes<B, 2>(nkb_cap, uniform);
+        if (smem > static_cast<size_t>(kSmemLimit)) continue;
+        const int c = (per_sm == 2 && smem <= 113 * 1024) ? 2 : 1;
+        const long n = static_cast<long>(q.ntiles) * S;
+        const long k = (n * 10 - sms + sms * 10 - 1) / (sms * 10) > 0 ? (n * 10 - sms + sms * 10 - 1) / (sms * 10) : 1;   // ceil(n / sms - 0.1)
+        const double w = tps;
+        const double work = (c == 2) ? w * (2.0 * (k / 2) + (k % 2) / 0.65) : w * k / 0.65;
+        const double cost = work + 18.0 * ((k + c - 1) / c);
+        if (!best.ok || cost < best_cost) {
+            best.ok = true; best.NT = NT; best.tile_rows = q.ntiles; best.S = S; best.tiles_per_split = tps; best.nkb_cap = nkb_cap;
+            best.smem = smem; best.stab8 = uniform ? 1 : 0;
+            best_cost = cost;
         }
-        if (S >= 8) break;
     }
-    pl.ok = false;
-    return pl;
+    return best;
 }
 
 inline bool supported(const QView& q, int64_t M) {
@@ -1088,7 +1158,7 @@ inline cudaError_t launch_fwd(const QView& q, const void* L1, const void* L2, in
     p.L1 = static_cast<const __nv_bfloat16*>(L1);
     p.Y = static_cast<__nv_bfloat16*>(Y);
     p.status = reinterpret_cast<int*>(ws);
-    p.M = M; p.r = r; p.S = pl.S; p.tiles_per_split = pl.tiles_per_split; p.nkb_cap = pl.nkb_cap;
+    p.M = M; p.r = r; p.S = pl.S; p.tiles_per_split = pl.tiles_per_split; p.nkb_cap = pl.nkb_cap; p.stab8 = pl.stab8;
     if (r > 0) {
         cudaError_t e = launch_pre<false>(p.X, static_cast<const __nv_bfloat16*>(L2), reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes),
                                           p.status, M, q.K, r, st);
