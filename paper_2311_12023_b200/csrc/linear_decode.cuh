@@ -3,13 +3,15 @@
 //   - One CTA owns a tile row of Q (128 rows) and a slice of K; the K slices of a tile row form a
 //     thread-block cluster and are added up through distributed shared memory, so there is no
 //     workspace of partial sums and nothing to zero.
-//   - A producer thread streams the packed tiles of the CTA (they are contiguous in memory) into a
-//     shared-memory ring with bulk copies; eight consumer warps dequantize them in registers with
+//   - The packed tiles of the CTA (they are contiguous in memory) and the matching activations are streamed into a
+//     shared-memory ring with bulk copies: thread 0 fills the ring once, afterwards the warp that finishes a stage
+//     last refills its slot (no producer warp).  Eight warps dequantize them in registers with
 //     the byte-table method (bf16 bits identical to the exported dequantized weights) and feed
 //     mma.sync m16n8k16 (weights = the 16-row operand, tokens = the 8-column operand, fp32 accumulators).
 //     The contraction index is permuted so that a thread supplies 4 consecutive weights of one row per MMA
 //     and reads the matching 4 activations with one 128-bit load per 8 columns.
-//   - Block scales s~ of the CTA's rows and columns are computed once into shared memory.
+//   - Block scales of the CTA's rows and columns are staged once in shared memory: as fp32 s~, or, where the slices
+//     are uniform, as the 8-bit codes plus fl(v / 127) per 16 block columns (a quarter of the size; s~ is formed at use).
 //   - The rank-r intermediate T = X L2^T comes from a small kernel launched in front of this one; the two
 //     overlap (programmatic dependent launch) and T is only read in the epilogue, which adds T L1^T.
 #pragma once
@@ -533,7 +535,9 @@ struct BwdParams {
     int M, r;
     int S;                     // row slices per column window = cluster size
     int trows_per_split;       // tile rows (128 rows) per CTA, even
-    int rows_stride;           // floats per block column of the scale table
+    int rows_stride;           // entries per block column of the scale table
+    int stab8;                 // 1: compact scale table (codes as bytes [nkb][rows_stride] + fl(v / 127) per row), 0: fp32 table
+    int nkb_cap;               // block columns of the table
 };
 
 constexpr int kBwdStageRows = 256;
@@ -543,7 +547,8 @@ template <int B, int NT> __host__ __device__ constexpr int bwd_stage_bytes() { r
 template <int B, int NT> __host__ __device__ constexpr int bwd_ctas_per_sm() { return (NT == 1 && B <= 3) ? 2 : 1; }
 template <int B, int NT> __host__ __device__ constexpr int bwd_stages() { return (B == 8 || bwd_ctas_per_sm<B, NT>() == 2) ? 2 : 3; }
 
-template <int B, int NT, bool TWO>
+// C8: compact scale table (codes as bytes [nkb][rows_stride] + fl(v / 127) per row) instead of the fp32 table
+template <int B, int NT, bool TWO, bool C8>
 __global__ void __launch_bounds__(kThreads, bwd_ctas_per_sm<B, NT>())
 decode_bwd_kernel(const BwdParams p) {
     constexpr int NS = bwd_stages<B, NT>();
@@ -609,6 +614,9 @@ decode_bwd_kernel(const BwdParams p) {
     // one second-level group (B1 >= 16 >= nkb, both powers of two) -> one vector load per row, four rows in flight.
     const bool seg_vec = ncol_tiles == 4 && nkb <= 16 && (nkb & (nkb - 1)) == 0 && (q.KB % nkb) == 0 && (kb_first % nkb) == 0 &&
                          (1 << q.logB1) >= nkb;
+    // compact table (chosen by the host only where every CTA meets the conditions above): s^ as bytes, sigma per row
+    uint8_t* st8 = reinterpret_cast<uint8_t*>(stab);
+    float* sg = reinterpret_cast<float*>(st8 + static_cast<size_t>(p.nkb_cap) * p.rows_stride);
     if (seg_vec) {
         for (int r0 = threadIdx.x; r0 < nrows_cta; r0 += 4 * kThreads) {
             uint4 sc16[4];
@@ -641,9 +649,11 @@ decode_bwd_kernel(const BwdParams p) {
                 for (int i = 0; i < 16; ++i) {
                     if (i < nkb) {
                         const uint32_t code = (words[i >> 2] >> (8 * (i & 3))) & 255u;
-                        stab[i * p.rows_stride + rowv[u]] = block_scale(static_cast<uint8_t>(code), v[u]);
+                        if constexpr (C8) st8[i * p.rows_stride + rowv[u]] = static_cast<uint8_t>(code);
+                        else stab[i * p.rows_stride + rowv[u]] = block_scale(static_cast<uint8_t>(code), v[u]);
                     }
                 }
+                if constexpr (C8) sg[rowv[u]] = __fdiv_rn(v[u], static_cast<float>(kScaleLevels));
             }
         }
     } else {
@@ -711,9 +721,24 @@ decode_bwd_kernel(const BwdParams p) {
                 uint4 w4[B];
 #pragma unroll
                 for (int i = 0; i < B; ++i) w4[i] = *reinterpret_cast<const uint4*>(sp + i * 32);
-                float4 sc_lo = *reinterpret_cast<const float4*>(stab + kb * p.rows_stride + row_local);
-                float4 sc_hi = sc_lo;
-                if (TWO) sc_hi = *reinterpret_cast<const float4*>(stab + (kb + 1) * p.rows_stride + row_local);
+                float4 sc_lo, sc_hi;
+                if constexpr (C8) {
+                    // s~ = fl32(float(s^) * fl32(v / 127)) from the compact table
+                    const float4 sg4 = *reinterpret_cast<const float4*>(sg + row_local);
+                    const uint32_t c_lo = *reinterpret_cast<const uint32_t*>(st8 + kb * p.rows_stride + row_local);
+                    sc_lo = make_float4(__fmul_rn(static_cast<float>(c_lo & 255u), sg4.x), __fmul_rn(static_cast<float>((c_lo >> 8) & 255u), sg4.y),
+                                        __fmul_rn(static_cast<float>((c_lo >> 16) & 255u), sg4.z), __fmul_rn(static_cast<float>(c_lo >> 24), sg4.w));
+                    sc_hi = sc_lo;
+                    if (TWO) {
+                        const uint32_t c_hi = *reinterpret_cast<const uint32_t*>(st8 + (kb + 1) * p.rows_stride + row_local);
+                        sc_hi = make_float4(__fmul_rn(static_cast<float>(c_hi & 255u), sg4.x), __fmul_rn(static_cast<float>((c_hi >> 8) & 255u), sg4.y),
+                                            __fmul_rn(static_cast<float>((c_hi >> 16) & 255u), sg4.z), __fmul_rn(static_cast<float>(c_hi >> 24), sg4.w));
+                    }
+                } else {
+                    sc_lo = *reinterpret_cast<const float4*>(stab + kb * p.rows_stride + row_local);
+                    sc_hi = sc_lo;
+                    if (TWO) sc_hi = *reinterpret_cast<const float4*>(stab + (kb + 1) * p.rows_stride + row_local);
+                }
                 if (!col_ok) { sc_lo = make_float4(0.f, 0.f, 0.f, 0.f); sc_hi = sc_lo; }
                 // dY of the four rows for this lane's token(s)
                 uint32_t y0[NT], y1[NT];
@@ -1181,15 +1206,16 @@ inline int max_active_clusters(Kern kern, int threads, size_t smem, int cluster_
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     // the answer depends on (kernel, shared memory, cluster size) only: keep the last few per kernel
-    struct Entry { size_t smem; int cy, n; };
+    struct Entry { const void* kern; size_t smem; int cy, n; };
     static Entry cache[32] = {};
     static int used = 0;
+    const void* key = reinterpret_cast<const void*>(kern);
     for (int i = 0; i < used; ++i)
-        if (cache[i].smem == smem && cache[i].cy == cluster_y) return cache[i].n;
+        if (cache[i].kern == key && cache[i].smem == smem && cache[i].cy == cluster_y) return cache[i].n;
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
     static int next = 0;
-    cache[next] = Entry{smem, cluster_y, n};
+    cache[next] = Entry{key, smem, cluster_y, n};
     next = (next + 1) % 32;
     if (used < 32) ++used;
     return n;
@@ -1197,26 +1223,29 @@ inline int max_active_clusters(Kern kern, int threads, size_t smem, int cluster_
 
 struct BwdPlan {
     bool ok;
-    int NT, S, trows_per_split, rows_stride, nwin;
+    int NT, S, trows_per_split, rows_stride, nwin, stab8, nkb_cap;
     size_t smem;
 };
 
 // Plan for a given number of row slices S (a power of two <= 8); ok = false when it does not fit.
 template <int B>
-inline BwdPlan make_bwd_plan_s(const QView& q, int M, int S) {
+inline BwdPlan make_bwd_plan_s(const QView& q, int M, int S, bool allow_compact = true) {
     BwdPlan pl{};
     pl.NT = (M <= 8) ? 1 : 2;
     pl.nwin = (q.ktiles + 3) / 4;
     int trps = (q.ntiles + S - 1) / S;
     trps += trps & 1;
-    const int rows_stride = trps * 128 + 8;
     const int nkb_cap = (256 >> q.logB0) > 0 ? (256 >> q.logB0) : 1;      // a window is 256 aligned columns and B0 divides 256
+    // compact scale table where every window is whole and its blocks of a row are aligned and share a second-level group
+    const bool compact = allow_compact && (q.K % 256 == 0) && (q.KB % nkb_cap == 0) && (1 << q.logB1) >= nkb_cap;
+    const int rows_stride = trps * 128 + (compact ? 16 : 8);
     const size_t stage = (pl.NT == 1) ? bwd_stage_bytes<B, 1>() : bwd_stage_bytes<B, 2>();
     const int ns = (pl.NT == 1) ? bwd_stages<B, 1>() : bwd_stages<B, 2>();
     const size_t smem = 128 + ns * stage + 64 * pl.NT * 32 * 4 + (B == 8 ? 1024 : 0) + (2 * ns + 2) * 8 +
-                        static_cast<size_t>(nkb_cap) * rows_stride * 4;
+                        (compact ? static_cast<size_t>(nkb_cap) * rows_stride + static_cast<size_t>(rows_stride) * 4
+                                 : static_cast<size_t>(nkb_cap) * rows_stride * 4);
     pl.ok = smem <= static_cast<size_t>(kSmemLimit) && (S == 1 || q.ntiles / S >= 1);
-    pl.S = S; pl.trows_per_split = trps; pl.rows_stride = rows_stride; pl.smem = smem;
+    pl.S = S; pl.trows_per_split = trps; pl.rows_stride = rows_stride; pl.smem = smem; pl.stab8 = compact ? 1 : 0; pl.nkb_cap = nkb_cap;
     return pl;
 }
 
@@ -1244,11 +1273,13 @@ inline bool bwd_supported(const QView& q, int64_t M) {
 
 template <int B, int NT, bool TWO>
 inline cudaError_t launch_bwd_nt(BwdParams p, const QView& q, int M, bool after_pre, cudaStream_t st) {
-    auto kern = decode_bwd_kernel<B, NT, TWO>;
+    void (*kerns[2])(BwdParams) = {decode_bwd_kernel<B, NT, TWO, false>, decode_bwd_kernel<B, NT, TWO, true>};
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
-        if (e != cudaSuccess) return e;
+        for (int i = 0; i < 2; ++i) {
+            cudaError_t e = cudaFuncSetAttribute(kerns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+            if (e != cudaSuccess) return e;
+        }
         attr_done = true;
     }
     // Number of row slices: the one with the smallest estimated time.  A wave of resident clusters takes the tile
@@ -1256,18 +1287,23 @@ inline cudaError_t launch_bwd_nt(BwdParams p, const QView& q, int M, bool after_
     // fixed part (scale table, reduction, epilogue) worth about six tile rows.
     BwdPlan pl{};
     long best = -1;
-    for (int S = 8; S >= 1; S >>= 1) {
-        const BwdPlan c = make_bwd_plan_s<B>(q, M, S);
-        if (!c.ok) continue;
-        const int cap = max_active_clusters(kern, kThreads, c.smem, S);
-        if (cap <= 0) continue;
-        const long waves = (c.nwin + cap - 1) / cap;
-        const bool shared_sm = static_cast<long>(cap) * S > sm_count_cached() + sm_count_cached() / 2;
-        const long cost = waves * (static_cast<long>(c.trows_per_split) * (shared_sm ? 4 : 3) + 12);    // in half tile rows
-        if (best < 0 || cost < best) { best = cost; pl = c; }
+    // The compact scale table costs a few conversions per use (about 4 %); it wins where the fp32 table would force
+    // more slices or a single CTA per SM.
+    for (int mode = 0; mode < 2; ++mode) {
+        for (int S = 8; S >= 1; S >>= 1) {
+            const BwdPlan c = make_bwd_plan_s<B>(q, M, S, mode == 1);
+            if (!c.ok || (mode == 1 && !c.stab8)) continue;
+            const int cap = max_active_clusters(kerns[mode], kThreads, c.smem, S);
+            if (cap <= 0) continue;
+            const long waves = (c.nwin + cap - 1) / cap;
+            const bool shared_sm = static_cast<long>(cap) * S > sm_count_cached() + sm_count_cached() / 2;
+            long cost = waves * (static_cast<long>(c.trows_per_split) * (shared_sm ? 4 : 3) + 12) * 100;    // in 1/200 tile rows
+            if (mode == 1) cost += cost / 25;
+            if (best < 0 || cost < best) { best = cost; pl = c; }
+        }
     }
     if (!pl.ok) return cudaErrorInvalidValue;
-    p.S = pl.S; p.trows_per_split = pl.trows_per_split; p.rows_stride = pl.rows_stride;
+    p.S = pl.S; p.trows_per_split = pl.trows_per_split; p.rows_stride = pl.rows_stride; p.stab8 = pl.stab8; p.nkb_cap = pl.nkb_cap;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(pl.nwin, pl.S);
     cfg.blockDim = dim3(kThreads);
@@ -1281,7 +1317,7 @@ inline cudaError_t launch_bwd_nt(BwdParams p, const QView& q, int M, bool after_
     cfg.attrs = attr;
     cfg.numAttrs = after_pre ? 2 : 1;
     count_launch(1);
-    return cudaLaunchKernelEx(&cfg, kern, p);
+    return cudaLaunchKernelEx(&cfg, kerns[pl.stab8 ? 1 : 0], p);
 }
 
 // Input gradient for M <= 16.  ws: [status 256 B][T' bf16]; same status-word convention as launch_fwd.
