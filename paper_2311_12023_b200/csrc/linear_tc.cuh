@@ -758,14 +758,43 @@ inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUten
 }
 
 
+// Clusters of `ks` CTAs of the one-CTA kernel (one CTA per SM, all of its shared memory) that can be resident at the
+// same time.  A cluster lives inside one GPC, so fewer fit than SMs / ks: 15 clusters of eight on a B200, not 18.
+// Asked once per cluster size; the figures measured on a B200 stand in when there is no device to ask.
+inline int tc_max_clusters(int ks) {
+    static int cached[4] = {-1, -1, -1, -1};       // ks = 1, 2, 4, 8
+    const int idx = (ks >= 8) ? 3 : (ks >= 4) ? 2 : (ks >= 2) ? 1 : 0;
+    if (cached[idx] >= 0) return cached[idx];
+    const int fallback[4] = {148, 74, 36, 15};
+    int n = 0;
+    auto kern = tc_linear_kernel<3, false, 1>;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1, 1, ks);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemLimit;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = ks;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        n = fallback[idx];
+    }
+    cached[idx] = n;
+    return n;
+}
+
 // Splits of the contraction for the one-CTA kernel (M <= 256): few output tiles would leave most SMs idle, so
-// the contraction of a tile is divided over a cluster of up to eight CTAs (each keeps at least eight steps).
+// the contraction of a tile is divided over a cluster of up to eight CTAs (each keeps at least eight steps, and
+// all clusters must be resident at once: a second wave costs more than the finer split saves).
 inline int tc_ksplit(int64_t M, int64_t out_cols, int steps_q, int sms) {
     if (M > 256) return 1;
     const int mh = (M > 128) ? 2 : 1;
     const long long tiles = ((M + mh * 128 - 1) / (mh * 128)) * ((out_cols + BN - 1) / BN);
     int ks = 1;
-    while (ks < 8 && tiles * (2 * ks) <= sms && steps_q / (2 * ks) >= 8) ks *= 2;
+    while (ks < 8 && tiles * (2 * ks) <= sms && steps_q / (2 * ks) >= 8 && tiles <= tc_max_clusters(2 * ks)) ks *= 2;
     return ks;
 }
 
@@ -859,7 +888,7 @@ inline int launch_b(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtenso
 
 namespace lq {
 
-constexpr int kTcMinRows = 33;   // fewer rows go to the weight-streaming kernels
+constexpr int kTcMinRows = 17;   // up to 16 rows go to the weight-streaming kernels
 
 inline bool tc_supported(const QView& q, int r, int64_t M, bool backward) {
     (void)r;

@@ -36,7 +36,7 @@ def run_case(A, l1b, l2b, cfg, M, seed, rows=None, passes=("fwd", "bwd")):
 
 
 @pytest.mark.parametrize("b0,B0,B1", [(2, 16, 64), (3, 64, 256), (4, 32, 64), (4, 64, 256), (8, 128, 64), (3, 256, 256)])
-@pytest.mark.parametrize("M", [1, 5, 16, 33])
+@pytest.mark.parametrize("M", [1, 5, 16, 17, 24, 33])
 def test_linear_small_shapes(b0, B0, B1, M):
     N, K = 320, 768            # N not a multiple of 128; several column windows
     A = inputs.gaussian(100 + b0, (N, K), 0.02)
