@@ -98,7 +98,9 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 // `words` pointing at the thread's first word, the others 32 words apart -- and writes them as four
 // 16-byte chunks of the row's 128 bytes; `dst` is the row start, `goff` the byte offset of the group
 // in the row (0 or 64), `xr` is (row % 8) * 16; a chunk at byte offset o of the row lives at o ^ xr.
-template <int B>
+// 8-bit codes read the code book from shared memory.  REP: the table is stored once per bank, entry c of the copy
+// of lane l at lut8[c * 32 + l], and `lut8` already points at the lane's copy, so no look-up meets a bank conflict.
+template <int B, bool REP = false>
 __device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ words, float s_lo, float s_hi, bool two_scales,
                                               uint8_t* __restrict__ dst, uint32_t goff, uint32_t xr, const float* __restrict__ lut8) {
     uint32_t w[B];
@@ -113,7 +115,8 @@ __device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ words
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const uint32_t ww = w[2 * c + (e >> 1)] >> (16 * (e & 1));
-                const float q0 = lut8[ww & 255u], q1 = lut8[(ww >> 8) & 255u];
+                const float q0 = REP ? lut8[(ww & 255u) << 5] : lut8[ww & 255u];
+                const float q1 = REP ? lut8[((ww >> 8) & 255u) << 5] : lut8[(ww >> 8) & 255u];
                 const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(q0, s), __fmul_rn(q1, s));
                 packed[e] = *reinterpret_cast<const uint32_t*>(&h);
             }

@@ -82,7 +82,7 @@ constexpr int kPairABytes = 2 * 128 * 128;    // two activation tiles of 128 row
 constexpr int kPairBStages = 4;
 template <int B> __host__ __device__ constexpr int pair_a_stages() { return (B == 8) ? 3 : 4; }
 template <int B> __host__ __device__ constexpr int pair_smem_bytes() {
-    return 1024 + pair_a_stages<B>() * (kPairABytes + 1024 * B) + kPairBStages * kPairBBytes + 512 + (B == 8 ? 1024 : 0);
+    return 1024 + pair_a_stages<B>() * (kPairABytes + 1024 * B) + kPairBStages * kPairBBytes + 512 + (B == 8 ? 32768 : 0);   // 8-bit: code book once per bank
 }
 
 template <int B, bool BWD>
@@ -102,7 +102,7 @@ tc_pair_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     uint8_t* tail = p_ring + SA * P_BYTES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);   // full_a[4], empty_a[4], full_b[4], empty_b[4], dbar[4], acc_full, drain
     float* lut8 = reinterpret_cast<float*>(tail + 256);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 256 + (B == 8 ? 1024 : 0));
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 256 + (B == 8 ? 32768 : 0));
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -128,7 +128,7 @@ tc_pair_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         fence_barrier_init();
     }
     if constexpr (B == 8) {
-        for (int i = threadIdx.x; i < 256; i += kThreads) lut8[i] = c_codebook[3][i];
+        for (int i = threadIdx.x; i < 256 * 32; i += kThreads) lut8[i] = c_codebook[3][i >> 5];     // entry c of lane l's copy at c * 32 + l
     }
     if (warp == 1) { tmem_alloc2(smem_u32(tmem_slot), TMEM_COLS); tmem_relinquish2(); }
     tc_fence_before();
@@ -295,8 +295,8 @@ tc_pair_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     if (step + 8 < p.steps_q) slot[u] = fetch(step + 8);
                     ok = wait(full_a(sa), ra.ph, ctl, 44);
                     if (!ok) break;
-                    dequant_group<B>(slab_base + sa * (P_BYTES / 4) + ((step & 1) ? slot_odd : slot_even), s_lo, s_hi, two_scales,
-                                     my_b + sb * kPairBBytes, g << 6, xr, lut8);
+                    dequant_group<B, true>(slab_base + sa * (P_BYTES / 4) + ((step & 1) ? slot_odd : slot_even), s_lo, s_hi, two_scales,
+                                           my_b + sb * kPairBBytes, g << 6, xr, lut8 + lane);
                     fence_proxy_async();
                 } else {
                     // rank-r step: the weight-side operand of this CTA's half comes by TMA
