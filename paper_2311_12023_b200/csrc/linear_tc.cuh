@@ -149,6 +149,27 @@ __device__ __forceinline__ void make_scales(const QView& q, const RawScale& r, f
     s_hi = (q.B0 == 16) ? __fmul_rn(static_cast<float>(r.sc >> 8), sigma) : s_lo;
 }
 
+// Forward pass: the scale codes a thread needs in consecutive steps are consecutive bytes of its row, so it keeps a
+// window of 16 of them (one 128-bit load, with the second-level scale of the window: 16 aligned blocks share their
+// group since B1 >= 16) and the next window, requested one window period ahead.  `base` = block offset of the
+// window inside the row (a multiple of 16); rows need KB % 16 == 0 for the alignment.
+struct ScaleWindow { uint4 w; float v; };
+__device__ __forceinline__ ScaleWindow load_scale_window(const QView& q, uint32_t row_blk0, int base, bool row_ok) {
+    ScaleWindow s{make_uint4(0u, 0u, 0u, 0u), 0.0f};
+    if (row_ok && base < q.KB) {
+        s.w = __ldg(reinterpret_cast<const uint4*>(q.sc + row_blk0 + base));
+        s.v = __ldg(q.v + ((row_blk0 + base) >> q.logB1));
+    }
+    return s;
+}
+// scale code(s) of block offset b (and b + 1 when two blocks of 16 columns make up the thread's 32 columns)
+__device__ __forceinline__ RawScale window_scale(const ScaleWindow& s, int b, bool two) {
+    const int i = b & 15;
+    const uint32_t word = (i < 8) ? ((i < 4) ? s.w.x : s.w.y) : ((i < 12) ? s.w.z : s.w.w);
+    const uint32_t sh = word >> ((i & 3) * 8);
+    return RawScale{two ? (sh & 0xFFFFu) : (sh & 0xFFu), s.v};
+}
+
 // ------------------------------------------------------------------------------------ kernel
 // Shared memory: [activation ring: SA x A_BYTES][weight ring: 2 x 32 KB][packed ring: SA x 2048*b0]
 // [barriers][8-bit look-up table].  The activation / packed-code ring runs several steps ahead of
@@ -363,8 +384,19 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // no instruction touches a slot while its load is in flight.
         float v_cached = -1.0f, sigma = 0.0f, s_lo = 0.0f, s_hi = 0.0f;
         RawScale slot[4];
+        // forward, rows aligned to 16 blocks: windows of 16 scale codes instead of one load per step
+        const bool use_win = !BWD && (p.q.KB % 16 == 0);
+        const bool win_row_ok = !BWD && my_row < p.q.N;
+        ScaleWindow cur{make_uint4(0u, 0u, 0u, 0u), 0.0f}, nxt = cur;
+        int cur_base = 0;
+        if (use_win) {
+            cur_base = ((q_lo * BK + my_col) >> logB0) & ~15;
+            cur = load_scale_window(p.q, blk0, cur_base, win_row_ok);
+            nxt = load_scale_window(p.q, blk0, cur_base + 16, win_row_ok);
+        } else {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) slot[u] = (u < nq) ? fetch(q_lo + u) : RawScale{0u, 0.0f};
+            for (int u = 0; u < 4; ++u) slot[u] = (u < nq) ? fetch(q_lo + u) : RawScale{0u, 0.0f};
+        }
         // word plane slot of this thread's row: rotated by 8 g + 16 (tile column % 2), see slab_row_slot();
         // forward: the tile column is the step index, backward: it is fixed per thread
         const uint32_t* __restrict__ slab_base = reinterpret_cast<const uint32_t*>(p_ring) + slab_i * (64 * B) + g * (B * 32);
@@ -383,8 +415,18 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 ok = wait(empty_b(sb), rb.ph ^ 1, ctl, 6);
                 if (!ok) break;
                 if (step < nq) {
-                    make_scales(p.q, slot[u], v_cached, sigma, s_lo, s_hi);
-                    if (step + 4 < nq) slot[u] = fetch(q_lo + step + 4);
+                    if (use_win) {
+                        const int b = ((q_lo + step) * BK + my_col) >> logB0;
+                        if ((b & ~15) != cur_base) {
+                            cur = nxt;
+                            cur_base += 16;
+                            nxt = load_scale_window(p.q, blk0, cur_base + 16, win_row_ok);
+                        }
+                        make_scales(p.q, window_scale(cur, b, two_scales), v_cached, sigma, s_lo, s_hi);
+                    } else {
+                        make_scales(p.q, slot[u], v_cached, sigma, s_lo, s_hi);
+                        if (step + 4 < nq) slot[u] = fetch(q_lo + step + 4);
+                    }
                     ok = wait(full_a(sa), ra.ph, ctl, 4);
                     if (!ok) break;
                     dequant_group<B>(slab_base + sa * (P_BYTES / 4) + (((q_lo + step) & 1) ? slot_odd : slot_even), s_lo, s_hi, two_scales, my_b + sb * kBBytes, g << 6, xr, lut8);
