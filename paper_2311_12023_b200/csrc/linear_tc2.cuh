@@ -276,8 +276,19 @@ tc_pair_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         uint8_t* my_b = b_ring + b_off;
         float v_cached = -1.0f, sigma = 0.0f, s_lo = 0.0f, s_hi = 0.0f;
         RawScale slot[4];
+        // forward, rows aligned to 16 blocks: windows of 16 scale codes instead of one load per step
+        const bool use_win = !BWD && (p.q.KB % 16 == 0);
+        const bool win_row_ok = !BWD && my_row < p.q.N;
+        ScaleWindow cur{make_uint4(0u, 0u, 0u, 0u), 0.0f}, nxt = cur;
+        int cur_base = 0;
+        if (use_win) {
+            cur_base = ((par * BK + my_col) >> logB0) & ~15;
+            cur = load_scale_window(p.q, blk0, cur_base, win_row_ok);
+            nxt = load_scale_window(p.q, blk0, cur_base + 16, win_row_ok);
+        } else {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) slot[u] = (par + 2 * u < p.steps_q) ? fetch(par + 2 * u) : RawScale{0u, 0.0f};
+            for (int u = 0; u < 4; ++u) slot[u] = (par + 2 * u < p.steps_q) ? fetch(par + 2 * u) : RawScale{0u, 0.0f};
+        }
         bool ok = true;
         RingPos<SA> ra;
         RingPos<SB> rb;
@@ -291,8 +302,18 @@ tc_pair_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 ok = wait(empty_b(sb), rb.ph ^ 1, ctl, 46);
                 if (!ok) break;
                 if (step < p.steps_q) {
-                    make_scales(p.q, slot[u], v_cached, sigma, s_lo, s_hi);
-                    if (step + 8 < p.steps_q) slot[u] = fetch(step + 8);
+                    if (use_win) {
+                        const int b = (step * BK + my_col) >> logB0;
+                        if ((b & ~15) != cur_base) {
+                            cur = nxt;
+                            cur_base += 16;
+                            nxt = load_scale_window(p.q, blk0, cur_base + 16, win_row_ok);
+                        }
+                        make_scales(p.q, window_scale(cur, b, two_scales), v_cached, sigma, s_lo, s_hi);
+                    } else {
+                        make_scales(p.q, slot[u], v_cached, sigma, s_lo, s_hi);
+                        if (step + 8 < p.steps_q) slot[u] = fetch(step + 8);
+                    }
                     ok = wait(full_a(sa), ra.ph, ctl, 44);
                     if (!ok) break;
                     dequant_group<B, true>(slab_base + sa * (P_BYTES / 4) + ((step & 1) ? slot_odd : slot_even), s_lo, s_hi, two_scales,
