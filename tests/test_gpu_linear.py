@@ -63,6 +63,17 @@ def test_linear_decode_kernels_ragged_shapes(N, K, M, b0, B0):
     run_case(A, l1b, l2b, C(b0, B0, 8, 16, 32), M, seed=900 + M)
 
 
+@pytest.mark.parametrize("M", [2, 13])
+@pytest.mark.parametrize("b0,B0,B1", [(3, 64, 256), (4, 32, 64), (2, 16, 64), (8, 128, 256), (3, 16, 16)])
+def test_linear_decode_kernels_long_rows(b0, B0, B1, M):
+    """Decode kernels on long rows: slices with 16-aligned runs of blocks (the compact scale table of the forward and
+    of the input-gradient kernel, and the fp32 table where the runs are shorter)."""
+    N, K = 256, 8192
+    A = inputs.gaussian_outliers(1200 + b0, (N, K), 0.02, 0.001, 10.0)
+    l1b, l2b = inputs.lowrank_factors(1201, N, K, 64, 0.01)
+    run_case(A, l1b, l2b, C(b0, B0, 8, B1, 32), M, seed=1300 + M)
+
+
 def test_linear_single_row_with_odd_feature_count_uses_the_fallback():
     # N % 8 != 0 is only legal for M = 1 (no vector loads on the rows of Y): the plain kernels take it
     N, K = 201, 192
