@@ -42,6 +42,7 @@ def _load():
         lib.oracle_dequant.argtypes = [vp, vp, vp, c_i64, c_i64, c_int, c_int, c_int, c_int, vp, vp]
         lib.oracle_linear_fwd.argtypes = [vp, vp, vp, c_int, vp, c_i64, c_i64, c_i64, vp, c_i64, vp]
         lib.oracle_linear_bwd_input.argtypes = [vp, vp, vp, c_int, vp, c_i64, c_i64, c_i64, vp, c_i64, vp]
+        lib.oracle_lora_grads.argtypes = [vp, vp, c_int, vp, vp, c_i64, c_i64, c_i64, vp, vp]
         lib.oracle_num_threads.restype = c_int
         _lib = lib
     return _lib
@@ -145,3 +146,23 @@ def linear_bwd_input(W32: np.ndarray, L1: np.ndarray, L2: np.ndarray, dY: np.nda
     if rc != 0:
         raise ValueError("oracle_linear_bwd_input: invalid arguments")
     return dX
+
+
+def lora_grads(L1: np.ndarray, L2: np.ndarray, X: np.ndarray, dY: np.ndarray):
+    """(dL1 [N,r], dL2 [r,K]) in fp64 for Y = X W^T + (X L2^T) L1^T: dL1 = dY^T (X L2^T), dL2 = (dY L1)^T X.
+    All four inputs are bf16 bit patterns."""
+    L1 = _chk(L1, np.uint16)
+    L2 = _chk(L2, np.uint16)
+    N, r = L1.shape
+    K = L2.shape[1]
+    assert L2.shape[0] == r
+    X = _chk(X, np.uint16)
+    dY = _chk(dY, np.uint16)
+    M = X.shape[0]
+    assert X.shape[1] == K and dY.shape == (M, N)
+    dL1 = np.empty((N, r), dtype=np.float64)
+    dL2 = np.empty((r, K), dtype=np.float64)
+    rc = _load().oracle_lora_grads(_p(L1), _p(L2), r, _p(X), _p(dY), M, N, K, _p(dL1), _p(dL2))
+    if rc != 0:
+        raise ValueError("oracle_lora_grads: invalid arguments")
+    return dL1, dL2

@@ -259,6 +259,46 @@ int oracle_linear_bwd_input(const float* W /*[N,K] deq32*/, const uint16_t* L1, 
     return 0;
 }
 
+// ----------------------------------------------------------------------------------
+// Gradients of the low-rank factors of the same layer (the trained parameters, Sec. 1 and
+// Sec. 2.1).  Y = X W~^T + (X L2^T) L1^T is linear in L1 and in L2, so by the chain rule
+//     dL1[n, j] = sum_m dY[m, n] (sum_k X[m, k] L2[j, k])
+//     dL2[j, k] = sum_m (sum_n dY[m, n] L1[n, j]) X[m, k]
+// fp64 throughout, sums in ascending index order.  The quantized matrix does not enter.
+// ----------------------------------------------------------------------------------
+int oracle_lora_grads(const uint16_t* L1 /*[N,r]*/, const uint16_t* L2 /*[r,K]*/, int r, const uint16_t* X /*[M,K]*/,
+                      const uint16_t* dY /*[M,N]*/, int64_t M, int64_t N, int64_t K, double* dL1 /*[N,r]*/,
+                      double* dL2 /*[r,K]*/) {
+    if (r <= 0 || M <= 0 || N <= 0 || K <= 0) return -1;
+    std::vector<double> T(static_cast<size_t>(M) * r), Tp(static_cast<size_t>(M) * r);
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        for (int j = 0; j < r; ++j) {
+            double t = 0.0;
+            for (int64_t k = 0; k < K; ++k) t += bf16_to_double(X[m * K + k]) * bf16_to_double(L2[j * K + k]);
+            T[m * r + j] = t;
+            double tp = 0.0;
+            for (int64_t n = 0; n < N; ++n) tp += bf16_to_double(dY[m * N + n]) * bf16_to_double(L1[n * r + j]);
+            Tp[m * r + j] = tp;
+        }
+    }
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n)
+        for (int j = 0; j < r; ++j) {
+            double g = 0.0;
+            for (int64_t m = 0; m < M; ++m) g += bf16_to_double(dY[m * N + n]) * T[m * r + j];
+            dL1[n * r + j] = g;
+        }
+#pragma omp parallel for schedule(static)
+    for (int64_t k = 0; k < K; ++k)
+        for (int j = 0; j < r; ++j) {
+            double g = 0.0;
+            for (int64_t m = 0; m < M; ++m) g += Tp[m * r + j] * bf16_to_double(X[m * K + k]);
+            dL2[j * K + k] = g;
+        }
+    return 0;
+}
+
 int oracle_num_threads(void) {
 #ifdef _OPENMP
     return omp_get_max_threads();

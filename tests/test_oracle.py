@@ -325,6 +325,43 @@ def test_adjoint_identity():
     assert abs(lhs - rhs) <= 1e-10 * max(1.0, abs(lhs))
 
 
+def test_lora_grads_are_the_derivatives_of_the_forward_pass():
+    """Y is linear in L1 and in L2, so for any two factor matrices
+    <dY, Y(L1a, L2) - Y(L1b, L2)> = <dL1, L1a - L1b>  and  <dY, Y(L1, L2a) - Y(L1, L2b)> = <dL2, L2a - L2b>
+    hold exactly; the left sides come from the forward oracle, which is pinned on its own."""
+    N, K, M, r = 40, 96, 9, 16
+    W, l1a, l2a, X, dY = _layer_case(21, N, K, M, r)
+    l1b, l2b = inputs.lowrank_factors(2100, N, K, r, 0.05)
+    G = inputs.bf16_bits_to_f32(dY).astype(np.float64)
+    f = lambda b: inputs.bf16_bits_to_f32(b).astype(np.float64)
+    dL1, _ = oracle.lora_grads(l1a, l2a, X, dY)           # dL1 depends on L2 only
+    lhs = np.sum(G * (oracle.linear_fwd(W, l1a, l2a, X) - oracle.linear_fwd(W, l1b, l2a, X)))
+    rhs = np.sum(dL1 * (f(l1a) - f(l1b)))
+    assert abs(lhs - rhs) <= 1e-10 * max(1.0, abs(lhs))
+    _, dL2 = oracle.lora_grads(l1a, l2a, X, dY)           # dL2 depends on L1 only
+    lhs = np.sum(G * (oracle.linear_fwd(W, l1a, l2a, X) - oracle.linear_fwd(W, l1a, l2b, X)))
+    rhs = np.sum(dL2 * (f(l2a) - f(l2b)))
+    assert abs(lhs - rhs) <= 1e-10 * max(1.0, abs(lhs))
+    # a dropped term, a transposed operand or a swapped factor breaks the identities: dL1 must not depend on L1
+    dL1_other, dL2_other = oracle.lora_grads(l1b, l2a, X, dY)
+    assert np.array_equal(dL1_other, dL1) and not np.array_equal(dL2_other, dL2)
+
+
+def test_lora_grads_one_hot_closed_form():
+    """X = e_a (one token, one-hot), dY = e_b:  dL1[n, j] = [n == b] L2[j, a],  dL2[j, k] = L1[b, j] [k == a]."""
+    N, K, r = 24, 32, 16
+    l1, l2 = inputs.lowrank_factors(2200, N, K, r, 0.05)
+    a, b = 5, 17
+    X = np.zeros((1, K), np.float32); X[0, a] = 1.0
+    dY = np.zeros((1, N), np.float32); dY[0, b] = 1.0
+    dL1, dL2 = oracle.lora_grads(l1, l2, inputs.f32_to_bf16_bits(X), inputs.f32_to_bf16_bits(dY))
+    L1 = inputs.bf16_bits_to_f32(l1).astype(np.float64)
+    L2 = inputs.bf16_bits_to_f32(l2).astype(np.float64)
+    e1 = np.zeros((N, r)); e1[b, :] = L2[:, a]
+    e2 = np.zeros((r, K)); e2[:, a] = L1[b, :]
+    assert np.array_equal(dL1, e1) and np.array_equal(dL2, e2)
+
+
 # --------------------------------------------------------------------------- inputs
 def test_input_generators_are_seeded():
     a = inputs.gaussian(5, (8, 8), 0.02)
