@@ -164,6 +164,25 @@ int lqlora_linear_bwd_input(const lqlora_qmatrix* q, const void* L1_dev, const v
                             size_t workspace_bytes, void* stream);
 
 /*
+ * Gradients of the low-rank factors (the trained parameters: Sec. 1, Sec. 2.1; layer of Sec. 3.1).  With the layer
+ * Y = X deq(Q)^T + (X L2^T) L1^T the chain rule gives
+ *     dL1[N, r] = dY^T bf16(X L2^T)          dL2[r, K] = bf16(dY L1)^T X
+ * (the rank-r intermediates are rounded to bf16 as in the forward pass and the input gradient; products and sums in
+ * fp32 on the tensor cores).  The quantized matrix takes no part.
+ *   L1_dev [N, r], L2_dev [r, K], X_dev [M, K], dY_dev [M, N] : bf16, row-major, device, read only
+ *   dL1_dev [N, r], dL2_dev [r, K] : fp32, row-major, device, overwritten (not accumulated into)
+ *   r : multiple of 16 in [16, 128];  N, K : multiples of 8;  1 <= M <= 2^24
+ *   workspace_dev : device scratch of at least lqlora_lora_grads_workspace_bytes(N, K, r, M); it starts with the
+ *                   same status word as a linear workspace (lqlora_workspace_status)
+ * Asynchronous on `stream`; the library allocates nothing.
+ * Errors: INVALID_SHAPE, NULL_POINTER, MISALIGNED (16-byte alignment), WORKSPACE_TOO_SMALL, CUDA.
+ */
+int lqlora_lora_grads_workspace_bytes(int64_t N, int64_t K, int r, int64_t M, size_t* bytes);
+int lqlora_lora_grads(const void* L1_dev, const void* L2_dev, int r, int64_t N, int64_t K, const void* X_dev,
+                      const void* dY_dev, int64_t M, float* dL1_dev, float* dL2_dev, void* workspace_dev,
+                      size_t workspace_bytes, void* stream);
+
+/*
  * Forward pass for callers that are not allowed to allocate device memory (no counterpart in the
  * paper: this entry point exists for deployment reasons only).  Typical examples are an inference
  * server whose memory pool was carved up at start-up, or code running inside another framework's

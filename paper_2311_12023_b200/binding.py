@@ -23,6 +23,7 @@ EXPORTS = [
     "lqlora_linear_bwd_input", "lqlora_workspace_status", "lqlora_linear_path", "lqlora_launch_count",
     "lqlora_status_string", "lqlora_encode_host", "lqlora_linear_fwd_host", "lqlora_linear_bwd_input_host",
     "lqlora_static_scratch_bytes", "lqlora_linear_fwd_static", "lqlora_encode_search_clearance",
+    "lqlora_lora_grads_workspace_bytes", "lqlora_lora_grads",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20   # size of the scratch array compiled into the library (lqlora_static_scratch_bytes)
@@ -67,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.lqlora_linear_workspace_bytes.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ctypes.POINTER(sz)]
         L.lqlora_linear_fwd.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, sz, vp]
         L.lqlora_linear_bwd_input.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, sz, vp]
+        L.lqlora_lora_grads_workspace_bytes.argtypes = [i64, i64, ci, i64, ctypes.POINTER(sz)]
+        L.lqlora_lora_grads.argtypes = [vp, vp, ci, i64, i64, vp, vp, i64, vp, vp, vp, sz, vp]
         L.lqlora_encode_host.argtypes = [vp, vp, ctypes.POINTER(CQMatrix), vp, sz, vp]
         L.lqlora_linear_fwd_host.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, vp, vp, sz, vp]
         L.lqlora_linear_bwd_input_host.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, vp, vp, sz, vp]
@@ -253,6 +256,29 @@ def linear_bwd_input(q: QMatrix, L1, L2, dY: torch.Tensor, out=None, workspace=N
     """lqlora_linear_bwd_input: dX = dY deq(Q) + (dY L1) L2, bf16 [M, K]."""
     assert dY.shape[1] == q.N
     return _linear(lib().lqlora_linear_bwd_input, "lqlora_linear_bwd_input", q, L1, L2, dY, q.K, out, workspace)
+
+
+def lora_grads_workspace_bytes(N: int, K: int, r: int, M: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().lqlora_lora_grads_workspace_bytes(N, K, r, M, ctypes.byref(n)), "lqlora_lora_grads_workspace_bytes")
+    return int(n.value)
+
+
+def lora_grads(L1: torch.Tensor, L2: torch.Tensor, X: torch.Tensor, dY: torch.Tensor, out=None, workspace=None):
+    """lqlora_lora_grads: (dL1 [N, r], dL2 [r, K]) in fp32 from bf16 L1 [N, r], L2 [r, K], X [M, K], dY [M, N]."""
+    N, r = L1.shape
+    K = L2.shape[1]
+    M = X.shape[0]
+    assert L2.shape[0] == r and X.shape[1] == K and tuple(dY.shape) == (M, N)
+    for t in (L1, L2, X, dY):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    if out is None:
+        out = (torch.empty(N, r, dtype=torch.float32, device=X.device), torch.empty(r, K, dtype=torch.float32, device=X.device))
+    if workspace is None:
+        workspace = torch.empty(lora_grads_workspace_bytes(N, K, r, M), dtype=torch.uint8, device=X.device)
+    _check(lib().lqlora_lora_grads(L1.data_ptr(), L2.data_ptr(), r, N, K, X.data_ptr(), dY.data_ptr(), M, out[0].data_ptr(),
+                                   out[1].data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()), "lqlora_lora_grads")
+    return out
 
 
 def encode_host(W_host: torch.Tensor, W_stage: torch.Tensor, q: QMatrix, workspace: torch.Tensor) -> None:

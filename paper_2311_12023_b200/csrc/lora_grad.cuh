@@ -1,0 +1,289 @@
+// Gradients of the low-rank factors of the layer Y = X (Q + L1 L2) (Sec. 2.1, Sec. 3.1; nn.Linear orientation:
+// Y = X deq(Q)^T + (X L2^T) L1^T).  By the chain rule
+//     dL1 [N, r] = dY^T (X L2^T) = dY^T T,        dL2 [r, K] = (dY L1)^T X = T'^T X,
+// with T = X L2^T and T' = dY L1 the same rank-r intermediates the forward pass and the input gradient use (bf16,
+// from tc_lowrank_kernel).  Q takes no part: only the low-rank factors are trained.
+//
+// Both products have the shape  G [P, r] = sum_m A[m, P]^T T[m, r]  (A = dY, P = N  or  A = X, P = K): a long
+// contraction over the tokens and a narrow output, bound by reading A once from HBM.  tc_wgrad_kernel: one CTA per
+// 128 rows of G and slice of the tokens; A and T tiles come by TMA (boxes of 64 token rows x 64 columns, 128-byte
+// swizzle) and enter tcgen05.mma as MN-major operands (the contraction index is the slow index of both), fp32
+// accumulators in tensor memory.  The token slices of a tile form a cluster; their accumulators are added in a fixed
+// order through distributed shared memory and the CTA that owns a column writes it (fp32), transposed for dL2.
+// Every wait on an mbarrier is bounded (status word LQLORA_ERR_TIMEOUT, as in the linear kernels).
+#pragma once
+
+#include "linear_tc.cuh"
+
+namespace lq {
+namespace tc {
+
+struct WgradParams {
+    float* out;            // TRANS ? [r][P] : [P][r]
+    int* status;
+    int M, P, r, rp;       // rp = r rounded up to 64 (MMA N)
+    int steps;             // token steps of 64 in total
+    int steps_per_split;
+    int stages;
+};
+
+template <bool TRANS>
+__global__ void __launch_bounds__(192, 1)
+tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmT, const WgradParams p) {
+    constexpr int A_BYTES = 16384;                 // 64 token rows x 128 columns of A
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int b_bytes = p.rp * 128;                // 64 token rows x rp columns of T
+    const int stage_bytes = A_BYTES + b_bytes;
+    uint8_t* tail = base + static_cast<size_t>(p.stages) * stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);      // full[8], empty[8], acc_full, drain
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 160);
+    volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int p0 = blockIdx.x * 128;
+    const int split = blockIdx.y, nsplit = gridDim.y;
+    const int s_lo = min(p.steps, split * p.steps_per_split);
+    const int s_hi = min(p.steps, s_lo + p.steps_per_split);
+    const int total = s_hi - s_lo;
+    const Ctl ctl{abort_s, p.status};
+    const uint32_t tmem_cols = (p.rp <= 64) ? 64u : 128u;
+
+    auto full = [&](int s) { return smem_u32(bars + s); };
+    auto empty = [&](int s) { return smem_u32(bars + 8 + s); };
+    const uint32_t acc_full = smem_u32(bars + 16), drain = smem_u32(bars + 17);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        mbar_init(acc_full, 1);
+        mbar_init(drain, 1);
+        *abort_s = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), tmem_cols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    bool acc_ok = false;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int i = 0; i < total; ++i) {
+                const int s = i % p.stages;
+                const uint32_t ph = (i / p.stages) & 1;
+                if (!wait(empty(s), ph ^ 1, ctl, 61)) break;
+                const uint32_t a_dst = smem_u32(base + static_cast<size_t>(s) * stage_bytes), b_dst = a_dst + A_BYTES;
+                const int m = (s_lo + i) * BK;               // first token row of the step (rows past M read as zero)
+                mbar_expect_tx(full(s), A_BYTES + b_bytes);
+                for (int t = 0; t < 2; ++t) tma_load_2d(a_dst + t * 8192, &tmA, p0 + t * 64, m, full(s));
+                for (int t = 0; t < p.rp / 64; ++t) tma_load_2d(b_dst + t * 8192, &tmT, t * 64, m, full(s));
+            }
+            if (*abort_s) {
+                // let copies that are still in flight land before the CTA exits (bounded)
+                for (int s = 0; s < p.stages; ++s) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(full(s), 0) && !mbar_try_wait(full(s), 1) && clock64() - t0 < 20000000LL) {}
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // fp32 accumulators, bf16 operands, both MN-major (bits 15 and 16), N = rp, M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
+                                   (static_cast<uint32_t>(p.rp >> 3) << 17) | (static_cast<uint32_t>(128 >> 4) << 24);
+            bool ok = true;
+            for (int i = 0; i < total && ok; ++i) {
+                const int s = i % p.stages;
+                const uint32_t ph = (i / p.stages) & 1;
+                ok = wait(full(s), ph, ctl, 62);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_src = smem_u32(base + static_cast<size_t>(s) * stage_bytes), b_src = a_src + A_BYTES;
+#pragma unroll
+                for (int k16 = 0; k16 < 4; ++k16) {
+                    // 16 token rows = 2048 bytes down the tile; groups of 64 columns are 8192 bytes apart
+                    const uint64_t adesc = make_desc(a_src + k16 * 2048, 8192, 1024);
+                    const uint64_t bdesc = make_desc(b_src + k16 * 2048, 8192, 1024);
+                    tc_mma(tmem, adesc, bdesc, idesc, (i > 0 || k16 > 0) ? 1u : 0u);
+                }
+                tc_commit(empty(s));
+            }
+            if (ok) tc_commit(acc_full);
+            else {
+                tc_commit(drain);
+                const long long t0 = clock64();
+                while (!mbar_try_wait(drain, 0) && clock64() - t0 < 20000000LL) {}
+            }
+        }
+        __syncwarp();
+    } else {
+        acc_ok = (total > 0) ? wait(acc_full, 0, ctl, 63) : true;
+    }
+    // ---------------------------------------------------------------------- sum over the token slices
+    // Every CTA writes its accumulator tile ([rp columns][128 rows] fp32) over the idle ring; CTA `split` adds the
+    // rp / nsplit columns it owns from all CTAs of the cluster, in rank order, and stores them.  The barriers are
+    // executed by all threads of all CTAs whatever happened before.
+    __syncthreads();
+    float* accbuf = reinterpret_cast<float*>(base);
+    if (warp >= 2 && acc_ok) {
+        tc_fence_after();
+        const int quarter = warp & 3;
+        for (int col = 0; col < p.rp; col += 32) {
+            uint32_t v[32];
+            if (total > 0) { tmem_ld32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + col, v); tmem_ld_wait(); }
+            else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = 0u;
+            }
+#pragma unroll
+            for (int i = 0; i < 32; ++i) accbuf[(col + i) * 128 + quarter * 32 + lane] = __uint_as_float(v[i]);
+        }
+    }
+    __syncthreads();
+    if (nsplit > 1) dec::cluster_sync_all();
+    {
+        const uint32_t accbuf_addr = smem_u32(accbuf);
+        const int cols_share = p.rp / nsplit, col_lo = split * cols_share;      // nsplit divides 64
+        for (int item = threadIdx.x; item < 128 * cols_share; item += 192) {
+            const int row = item & 127, col = col_lo + (item >> 7);
+            float sum = 0.0f;
+            if (nsplit > 1) {
+                float part[8];
+#pragma unroll
+                for (int rk = 0; rk < 8; ++rk)
+                    part[rk] = (rk < nsplit) ? dec::ld_dsmem_f32(accbuf_addr + static_cast<uint32_t>(col * 128 + row) * 4u, static_cast<uint32_t>(rk)) : 0.0f;
+#pragma unroll
+                for (int rk = 0; rk < 8; ++rk) sum += part[rk];
+            } else {
+                sum = accbuf[col * 128 + row];
+            }
+            const int pr = p0 + row;
+            if (pr < p.P && col < p.r) {
+                if (TRANS) p.out[static_cast<size_t>(col) * p.P + pr] = sum;
+                else p.out[static_cast<size_t>(pr) * p.r + col] = sum;
+            }
+        }
+    }
+    if (nsplit > 1) dec::cluster_sync_all();        // the buffers of the other CTAs may be released only now
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, tmem_cols);
+}
+
+// Token slices of the weight-gradient kernel: as many as keep all CTAs resident in one wave, each with at least
+// four steps; a power of two (it divides the 64 columns of the accumulator), at most eight.
+inline int wgrad_splits(int ptiles, int steps) {
+    int ns = 1;
+    while (ns < 8 && static_cast<long long>(ptiles) * (2 * ns) <= sm_count() && steps / (2 * ns) >= 4) ns *= 2;
+    if (ns == 8 && ptiles > 15) ns = 4;      // a cluster lives in one GPC: fewer clusters of eight fit than SMs / 8
+    return ns;
+}
+
+template <bool TRANS>
+inline int launch_wgrad(const void* A, int64_t M, int64_t P, const void* T, int r, float* out, int* status, cudaStream_t st) {
+    WgradParams p;
+    p.out = out; p.status = status;
+    p.M = static_cast<int>(M); p.P = static_cast<int>(P); p.r = r; p.rp = (r <= 64) ? 64 : 128;
+    p.steps = static_cast<int>((M + BK - 1) / BK);
+    const int ptiles = static_cast<int>((P + 127) / 128);
+    const int ns = wgrad_splits(ptiles, p.steps);
+    p.steps_per_split = (p.steps + ns - 1) / ns;
+    const int stage = 16384 + p.rp * 128;
+    int stages = (kSmemLimit - 1024 - 256) / stage;
+    if (stages > 8) stages = 8;
+    p.stages = stages;
+    const int smem = 1024 + stages * stage + 256;
+    CUtensorMap tA, tT;
+    if (!make_map(&tA, A, M, P, 64) || !make_map(&tT, T, M, r, 64)) return LQLORA_ERR_CUDA;
+    auto kern = tc_wgrad_kernel<TRANS>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
+            cudaGetLastError();
+            return LQLORA_ERR_CUDA;
+        }
+        attr_done = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ptiles, ns);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = ns; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA, tT, p);
+    count_launch(1);
+    if (e != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
+    return LQLORA_OK;
+}
+
+// Plan of the two rank-r pre-products of a weight-gradient call (they have the GPU to themselves).
+struct GradPlan {
+    int mtiles, rp, steps_x, steps_y, nsplit_x, nsplit_y, sps_x, sps_y;
+    size_t counters_bytes, t_bytes, partial_bytes;
+};
+
+inline GradPlan grad_plan(int64_t N, int64_t K, int r, int64_t M) {
+    GradPlan g;
+    g.mtiles = static_cast<int>((M + 127) / 128);
+    g.rp = (r <= 64) ? 64 : 128;
+    g.steps_x = static_cast<int>((K + BK - 1) / BK);
+    g.steps_y = static_cast<int>((N + BK - 1) / BK);
+    auto splits = [&](int steps, int& nsplit, int& sps) {
+        int want = sm_count() / g.mtiles;
+        if (want > steps / 2) want = steps / 2;
+        if (want > 32) want = 32;
+        if (want < 1) want = 1;
+        sps = (steps + want - 1) / want;
+        nsplit = (steps + sps - 1) / sps;
+    };
+    splits(g.steps_x, g.nsplit_x, g.sps_x);
+    splits(g.steps_y, g.nsplit_y, g.sps_y);
+    g.counters_bytes = round_up(static_cast<size_t>(2 * g.mtiles) * 4, 256);
+    g.t_bytes = round_up(static_cast<size_t>(M) * r * 2, 256);
+    const int ns = g.nsplit_x > g.nsplit_y ? g.nsplit_x : g.nsplit_y;
+    g.partial_bytes = round_up(static_cast<size_t>(ns) * M * g.rp * 4, 256);
+    return g;
+}
+
+inline size_t lora_grads_workspace(int64_t N, int64_t K, int r, int64_t M) {
+    const GradPlan g = grad_plan(N, K, r, M);
+    return kStatusBytes + g.counters_bytes + 2 * g.t_bytes + g.partial_bytes;
+}
+
+// ws: [status][counters of T][counters of T'][T bf16][T' bf16][fp32 partial tiles, shared by the two pre-products]
+inline int lora_grads_launch(const void* L1, const void* L2, int r, int64_t N, int64_t K, const void* X, const void* dY, int64_t M,
+                             float* dL1, float* dL2, char* ws, cudaStream_t st) {
+    const GradPlan g = grad_plan(N, K, r, M);
+    if (cudaMemsetAsync(ws, 0, kStatusBytes + g.counters_bytes, st) != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
+    count_launch(1);
+    int* status = reinterpret_cast<int*>(ws);
+    int* counters = reinterpret_cast<int*>(ws + kStatusBytes);
+    __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + g.counters_bytes);
+    __nv_bfloat16* Tp = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + g.counters_bytes + g.t_bytes);
+    float* partial = reinterpret_cast<float*>(ws + kStatusBytes + g.counters_bytes + 2 * g.t_bytes);
+    CUtensorMap tA, tB;
+    PreParams pp;
+    pp.partial = partial; pp.status = status; pp.M = static_cast<int>(M); pp.r = r; pp.rp = g.rp; pp.stages = 0;
+    // T = X L2^T
+    if (!make_map(&tA, X, M, K, 128) || !make_map(&tB, L2, r, K, g.rp)) return LQLORA_ERR_CUDA;
+    pp.T = T; pp.counters = counters; pp.steps = g.steps_x; pp.steps_per_split = g.sps_x;
+    int rc = launch_pre<false>(tA, tB, pp, g.mtiles, g.nsplit_x, st);
+    if (rc != LQLORA_OK) return rc;
+    // T' = dY L1 (the partial tiles are reused: the stream orders the two kernels)
+    if (!make_map(&tA, dY, M, N, 128) || !make_map(&tB, L1, N, r, 64)) return LQLORA_ERR_CUDA;
+    pp.T = Tp; pp.counters = counters + g.mtiles; pp.steps = g.steps_y; pp.steps_per_split = g.sps_y;
+    rc = launch_pre<true>(tA, tB, pp, g.mtiles, g.nsplit_y, st);
+    if (rc != LQLORA_OK) return rc;
+    rc = launch_wgrad<false>(dY, M, N, T, r, dL1, status, st);      // dL1 = dY^T T
+    if (rc != LQLORA_OK) return rc;
+    return launch_wgrad<true>(X, M, K, Tp, r, dL2, status, st);      // dL2 = T'^T X
+}
+
+}  // namespace tc
+}  // namespace lq

@@ -8,6 +8,7 @@
 #include "linear_decode.cuh"
 #include "linear_small.cuh"
 #include "linear_tc.cuh"
+#include "lora_grad.cuh"
 
 namespace lq {
 
@@ -233,6 +234,36 @@ int lqlora_linear_fwd_static(const lqlora_qmatrix* q, const void* L1_dev, const 
     // run_linear clears the status word and the arrival counters at the head of the scratch on every
     // call, so whatever the previous call left behind is never read before it is overwritten
     return run_linear(q, L1_dev, L2_dev, r, X_dev, M, Y_dev, scratch, kStaticScratchBytes, stream, false);
+}
+
+static int check_lora_grads(int64_t N, int64_t K, int r, int64_t M) {
+    if (N <= 0 || K <= 0 || N > (int64_t(1) << 30) || K > (int64_t(1) << 30) || (N % 8) != 0 || (K % 8) != 0) return LQLORA_ERR_INVALID_SHAPE;
+    if (M <= 0 || M > (int64_t(1) << 24)) return LQLORA_ERR_INVALID_SHAPE;
+    if (r < 16 || r > 128 || (r % 16) != 0) return LQLORA_ERR_INVALID_SHAPE;
+    return LQLORA_OK;
+}
+
+int lqlora_lora_grads_workspace_bytes(int64_t N, int64_t K, int r, int64_t M, size_t* bytes) {
+    if (!bytes) return LQLORA_ERR_NULL_POINTER;
+    const int rc = check_lora_grads(N, K, r, M);
+    if (rc != LQLORA_OK) return rc;
+    *bytes = lq::tc::lora_grads_workspace(N, K, r, M);
+    return LQLORA_OK;
+}
+
+int lqlora_lora_grads(const void* L1_dev, const void* L2_dev, int r, int64_t N, int64_t K, const void* X_dev,
+                      const void* dY_dev, int64_t M, float* dL1_dev, float* dL2_dev, void* workspace_dev,
+                      size_t workspace_bytes, void* stream) {
+    using namespace lq;
+    const int rc = check_lora_grads(N, K, r, M);
+    if (rc != LQLORA_OK) return rc;
+    if (!L1_dev || !L2_dev || !X_dev || !dY_dev || !dL1_dev || !dL2_dev || !workspace_dev) return LQLORA_ERR_NULL_POINTER;
+    if (!aligned16(L1_dev) || !aligned16(L2_dev) || !aligned16(X_dev) || !aligned16(dY_dev) || !aligned16(dL1_dev) ||
+        !aligned16(dL2_dev) || !aligned16(workspace_dev))
+        return LQLORA_ERR_MISALIGNED;
+    if (workspace_bytes < tc::lora_grads_workspace(N, K, r, M)) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
+    return tc::lora_grads_launch(L1_dev, L2_dev, r, N, K, X_dev, dY_dev, M, dL1_dev, dL2_dev, static_cast<char*>(workspace_dev),
+                                 static_cast<cudaStream_t>(stream));
 }
 
 int lqlora_encode_host(const float* W_host, float* W_stage_dev, lqlora_qmatrix* out, void* workspace_dev,
