@@ -8,8 +8,9 @@
 // contraction over the tokens and a narrow output, bound by reading A once from HBM.  tc_wgrad_kernel: one CTA per
 // 128 rows of G and slice of the tokens; A and T tiles come by TMA (boxes of 64 token rows x 64 columns, 128-byte
 // swizzle) and enter tcgen05.mma as MN-major operands (the contraction index is the slow index of both), fp32
-// accumulators in tensor memory.  The token slices of a tile form a cluster; their accumulators are added in a fixed
-// order through distributed shared memory and the CTA that owns a column writes it (fp32), transposed for dL2.
+// accumulators in tensor memory.  The token slices of a tile form a cluster; their accumulators are sent to the CTA
+// that owns the column through distributed shared memory, added there in a fixed order and written (fp32),
+// transposed for dL2.
 // Every wait on an mbarrier is bounded (status word LQLORA_ERR_TIMEOUT, as in the linear kernels).
 #pragma once
 
@@ -35,7 +36,10 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int b_bytes = p.rp * 128;                // 64 token rows x rp columns of T
     const int stage_bytes = A_BYTES + b_bytes;
-    uint8_t* tail = base + static_cast<size_t>(p.stages) * stage_bytes;
+    // receive buffer of the cluster reduction: its own region (other CTAs write to it while this one may still be in
+    // its main loop), rp x 128 fp32
+    float* recv = reinterpret_cast<float*>(base + static_cast<size_t>(p.stages) * stage_bytes);
+    uint8_t* tail = reinterpret_cast<uint8_t*>(recv) + static_cast<size_t>(p.rp) * 512;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);      // full[8], empty[8], acc_full, drain
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 160);
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -122,14 +126,18 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         acc_ok = (total > 0) ? wait(acc_full, 0, ctl, 63) : true;
     }
     // ---------------------------------------------------------------------- sum over the token slices
-    // Every CTA writes its accumulator tile ([rp columns][128 rows] fp32) over the idle ring; CTA `split` adds the
-    // rp / nsplit columns it owns from all CTAs of the cluster, in rank order, and stores them.  The barriers are
-    // executed by all threads of all CTAs whatever happened before.
+    // CTA `o` of the cluster owns columns [o * rp / nsplit, (o + 1) * rp / nsplit) of the tile.  Every CTA sends its
+    // accumulators straight from tensor memory to the owners' receive buffers (remote shared-memory stores, no round
+    // trip): recv[(src * cols_share + local column) * 128 + row].  After one cluster barrier every
+    // CTA adds what it received, in rank order, and stores its columns.  The barriers are executed by all threads of
+    // all CTAs whatever happened before.
     __syncthreads();
-    float* accbuf = reinterpret_cast<float*>(base);
+    const uint32_t recv_addr = smem_u32(recv);
+    const int cols_share = p.rp / nsplit;                   // nsplit divides 64
     if (warp >= 2 && acc_ok) {
         tc_fence_after();
         const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
         for (int col = 0; col < p.rp; col += 32) {
             uint32_t v[32];
             if (total > 0) { tmem_ld32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + col, v); tmem_ld_wait(); }
@@ -138,35 +146,27 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 for (int i = 0; i < 32; ++i) v[i] = 0u;
             }
 #pragma unroll
-            for (int i = 0; i < 32; ++i) accbuf[(col + i) * 128 + quarter * 32 + lane] = __uint_as_float(v[i]);
+            for (int i = 0; i < 32; ++i) {
+                const int c = col + i;
+                const int owner = c / cols_share, cl = c - owner * cols_share;
+                const uint32_t off = static_cast<uint32_t>((split * cols_share + cl) * 128 + row) * 4u;
+                if (nsplit > 1) dec::st_dsmem_f32(recv_addr + off, static_cast<uint32_t>(owner), __uint_as_float(v[i]));
+                else recv[(cl) * 128 + row] = __uint_as_float(v[i]);
+            }
         }
     }
     __syncthreads();
-    if (nsplit > 1) dec::cluster_sync_all();
-    {
-        const uint32_t accbuf_addr = smem_u32(accbuf);
-        const int cols_share = p.rp / nsplit, col_lo = split * cols_share;      // nsplit divides 64
-        for (int item = threadIdx.x; item < 128 * cols_share; item += 192) {
-            const int row = item & 127, col = col_lo + (item >> 7);
-            float sum = 0.0f;
-            if (nsplit > 1) {
-                float part[8];
-#pragma unroll
-                for (int rk = 0; rk < 8; ++rk)
-                    part[rk] = (rk < nsplit) ? dec::ld_dsmem_f32(accbuf_addr + static_cast<uint32_t>(col * 128 + row) * 4u, static_cast<uint32_t>(rk)) : 0.0f;
-#pragma unroll
-                for (int rk = 0; rk < 8; ++rk) sum += part[rk];
-            } else {
-                sum = accbuf[col * 128 + row];
-            }
-            const int pr = p0 + row;
-            if (pr < p.P && col < p.r) {
-                if (TRANS) p.out[static_cast<size_t>(col) * p.P + pr] = sum;
-                else p.out[static_cast<size_t>(pr) * p.r + col] = sum;
-            }
+    if (nsplit > 1) dec::cluster_sync_all();                // everything has arrived; only local shared memory is read below
+    for (int item = threadIdx.x; item < 128 * cols_share; item += 192) {
+        const int row = item & 127, cl = item >> 7;
+        float sum = 0.0f;
+        for (int src = 0; src < nsplit; ++src) sum += recv[(src * cols_share + cl) * 128 + row];
+        const int pr = p0 + row, col = split * cols_share + cl;
+        if (pr < p.P && col < p.r) {
+            if (TRANS) p.out[static_cast<size_t>(col) * p.P + pr] = sum;
+            else p.out[static_cast<size_t>(pr) * p.r + col] = sum;
         }
     }
-    if (nsplit > 1) dec::cluster_sync_all();        // the buffers of the other CTAs may be released only now
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, tmem_cols);
@@ -191,10 +191,11 @@ inline int launch_wgrad(const void* A, int64_t M, int64_t P, const void* T, int 
     const int ns = wgrad_splits(ptiles, p.steps);
     p.steps_per_split = (p.steps + ns - 1) / ns;
     const int stage = 16384 + p.rp * 128;
-    int stages = (kSmemLimit - 1024 - 256) / stage;
+    const int recv_bytes = p.rp * 512;
+    int stages = (kSmemLimit - 1024 - 256 - recv_bytes) / stage;
     if (stages > 8) stages = 8;
     p.stages = stages;
-    const int smem = 1024 + stages * stage + 256;
+    const int smem = 1024 + stages * stage + recv_bytes + 256;
     CUtensorMap tA, tT;
     if (!make_map(&tA, A, M, P, 64) || !make_map(&tT, T, M, r, 64)) return LQLORA_ERR_CUDA;
     auto kern = tc_wgrad_kernel<TRANS>;
