@@ -571,9 +571,10 @@ struct PreParams {
     int stages;
 };
 
+// Body of the kernel for the CTA (row tile `tile`, split `split` of `nsplit`); the tensor maps are kernel parameters.
 template <bool BWD>
-__global__ void __launch_bounds__(192, 1)
-tc_lowrank_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const PreParams p) {
+__device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const PreParams& p, int tile, int split,
+                                             int nsplit) {
     constexpr int A_BYTES = 16384;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -587,8 +588,7 @@ tc_lowrank_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
     pdl_launch_dependents();      // the linear kernel behind this one needs T only in its last steps
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * 128;
-    const int split = blockIdx.y, nsplit = gridDim.y;
+    const int m0 = tile * 128;
     const int s_lo = split * p.steps_per_split;
     const int s_hi = min(p.steps, s_lo + p.steps_per_split);
     const int total = s_hi - s_lo;
@@ -681,7 +681,7 @@ tc_lowrank_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             __threadfence();
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (threadIdx.x == 64) {
-                const int old = atomicAdd(p.counters + blockIdx.x, 1);
+                const int old = atomicAdd(p.counters + tile, 1);
                 *last_s = (old == nsplit - 1) ? 1 : 0;
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -734,6 +734,25 @@ tc_lowrank_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, tmem_cols);
+}
+
+template <bool BWD>
+__global__ void __launch_bounds__(192, 1)
+tc_lowrank_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const PreParams p) {
+    lowrank_body<BWD>(tmA, tmB, p, blockIdx.x, blockIdx.y, gridDim.y);
+}
+
+// Both pre-products of one layer in one launch (the weight-gradient path, which has the GPU to itself): grid.z = 0
+// computes T = X L2^T with (tmA0, tmB0, p0), grid.z = 1 computes T' = dY L1 with (tmA1, tmB1, p1); grid.y covers the
+// larger number of splits, CTAs beyond their product's own number leave at once.
+__global__ void __launch_bounds__(192, 1)
+tc_lowrank_both_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0, const PreParams p0, int nsplit0,
+                       const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1, const PreParams p1, int nsplit1) {
+    if (blockIdx.z == 0) {
+        if (static_cast<int>(blockIdx.y) < nsplit0) lowrank_body<false>(tmA0, tmB0, p0, blockIdx.x, blockIdx.y, nsplit0);
+    } else {
+        if (static_cast<int>(blockIdx.y) < nsplit1) lowrank_body<true>(tmA1, tmB1, p1, blockIdx.x, blockIdx.y, nsplit1);
+    }
 }
 
 // ------------------------------------------------------------------------------------ host side

@@ -28,9 +28,10 @@ struct WgradParams {
     int stages;
 };
 
+// Body for the CTA (row tile `ptile` of G, token slice `split` of `nsplit` = cluster size); tensor maps are kernel parameters.
 template <bool TRANS>
-__global__ void __launch_bounds__(192, 1)
-tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmT, const WgradParams p) {
+__device__ __forceinline__ void wgrad_body(const CUtensorMap& tmA, const CUtensorMap& tmT, const WgradParams& p, int ptile, int split,
+                                           int nsplit) {
     constexpr int A_BYTES = 16384;                 // 64 token rows x 128 columns of A
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -45,8 +46,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int p0 = blockIdx.x * 128;
-    const int split = blockIdx.y, nsplit = gridDim.y;
+    const int p0 = ptile * 128;
     const int s_lo = min(p.steps, split * p.steps_per_split);
     const int s_hi = min(p.steps, s_lo + p.steps_per_split);
     const int total = s_hi - s_lo;
@@ -172,6 +172,19 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (warp == 1) tmem_dealloc(tmem, tmem_cols);
 }
 
+// Both weight gradients of a layer in one launch: grid.z = 0 computes dL1 = dY^T T, grid.z = 1 computes dL2 = T'^T X;
+// grid.x covers the larger number of row tiles (whole clusters beyond a product's own number leave at once), grid.y =
+// token slices = cluster size.
+__global__ void __launch_bounds__(192, 1)
+tc_wgrad_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmT0, const WgradParams p0,
+                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmT1, const WgradParams p1) {
+    if (blockIdx.z == 0) {
+        if (static_cast<int>(blockIdx.x) * 128 < p0.P) wgrad_body<false>(tmA0, tmT0, p0, blockIdx.x, blockIdx.y, gridDim.y);
+    } else {
+        if (static_cast<int>(blockIdx.x) * 128 < p1.P) wgrad_body<true>(tmA1, tmT1, p1, blockIdx.x, blockIdx.y, gridDim.y);
+    }
+}
+
 // Token slices of the weight-gradient kernel: as many as keep all CTAs resident in one wave, each with at least
 // four steps; a power of two (it divides the 64 columns of the accumulator), at most eight.
 inline int wgrad_splits(int ptiles, int steps) {
@@ -181,24 +194,27 @@ inline int wgrad_splits(int ptiles, int steps) {
     return ns;
 }
 
-template <bool TRANS>
-inline int launch_wgrad(const void* A, int64_t M, int64_t P, const void* T, int r, float* out, int* status, cudaStream_t st) {
-    WgradParams p;
-    p.out = out; p.status = status;
-    p.M = static_cast<int>(M); p.P = static_cast<int>(P); p.r = r; p.rp = (r <= 64) ? 64 : 128;
-    p.steps = static_cast<int>((M + BK - 1) / BK);
-    const int ptiles = static_cast<int>((P + 127) / 128);
-    const int ns = wgrad_splits(ptiles, p.steps);
-    p.steps_per_split = (p.steps + ns - 1) / ns;
-    const int stage = 16384 + p.rp * 128;
-    const int recv_bytes = p.rp * 512;
+// dL1 [N, r] = dY^T T and dL2 [r, K] = T'^T X in one launch.
+inline int launch_wgrad(const void* dY, const void* X, int64_t M, int64_t N, int64_t K, const void* T, const void* Tp, int r,
+                        float* dL1, float* dL2, int* status, cudaStream_t st) {
+    WgradParams p0, p1;
+    p0.out = dL1; p0.status = status; p0.M = static_cast<int>(M); p0.P = static_cast<int>(N); p0.r = r; p0.rp = (r <= 64) ? 64 : 128;
+    p0.steps = static_cast<int>((M + BK - 1) / BK);
+    const int pt0 = static_cast<int>((N + 127) / 128), pt1 = static_cast<int>((K + 127) / 128);
+    const int ns = wgrad_splits(pt0 + pt1, p0.steps);
+    p0.steps_per_split = (p0.steps + ns - 1) / ns;
+    const int stage = 16384 + p0.rp * 128;
+    const int recv_bytes = p0.rp * 512;
     int stages = (kSmemLimit - 1024 - 256 - recv_bytes) / stage;
     if (stages > 8) stages = 8;
-    p.stages = stages;
+    p0.stages = stages;
     const int smem = 1024 + stages * stage + recv_bytes + 256;
-    CUtensorMap tA, tT;
-    if (!make_map(&tA, A, M, P, 64) || !make_map(&tT, T, M, r, 64)) return LQLORA_ERR_CUDA;
-    auto kern = tc_wgrad_kernel<TRANS>;
+    p1 = p0;
+    p1.out = dL2; p1.P = static_cast<int>(K);
+    CUtensorMap tA0, tT0, tA1, tT1;
+    if (!make_map(&tA0, dY, M, N, 64) || !make_map(&tT0, T, M, r, 64) || !make_map(&tA1, X, M, K, 64) || !make_map(&tT1, Tp, M, r, 64))
+        return LQLORA_ERR_CUDA;
+    auto kern = tc_wgrad_kernel;
     static bool attr_done = false;
     if (!attr_done) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
@@ -208,7 +224,7 @@ inline int launch_wgrad(const void* A, int64_t M, int64_t P, const void* T, int 
         attr_done = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(ptiles, ns);
+    cfg.gridDim = dim3(pt0 > pt1 ? pt0 : pt1, ns, 2);
     cfg.blockDim = dim3(192);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -217,7 +233,35 @@ inline int launch_wgrad(const void* A, int64_t M, int64_t P, const void* T, int 
     attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = ns; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA, tT, p);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA0, tT0, p0, tA1, tT1, p1);
+    count_launch(1);
+    if (e != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
+    return LQLORA_OK;
+}
+
+// Both pre-products in one launch (tc_lowrank_both_kernel).
+inline int launch_pre_both(const CUtensorMap& tA0, const CUtensorMap& tB0, PreParams p0, int nsplit0, const CUtensorMap& tA1,
+                           const CUtensorMap& tB1, PreParams p1, int nsplit1, int mtiles, cudaStream_t st) {
+    const int stage = 16384 + p0.rp * 128;
+    int stages = (kSmemLimit - 1024 - 256) / stage;
+    if (stages > 8) stages = 8;
+    p0.stages = stages; p1.stages = stages;
+    const int smem = 1024 + stages * stage + 256;
+    auto kern = tc_lowrank_both_kernel;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
+            cudaGetLastError();
+            return LQLORA_ERR_CUDA;
+        }
+        attr_done = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(mtiles, nsplit0 > nsplit1 ? nsplit0 : nsplit1, 2);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA0, tB0, p0, nsplit0, tA1, tB1, p1, nsplit1);
     count_launch(1);
     if (e != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
     return LQLORA_OK;
@@ -236,7 +280,7 @@ inline GradPlan grad_plan(int64_t N, int64_t K, int r, int64_t M) {
     g.steps_x = static_cast<int>((K + BK - 1) / BK);
     g.steps_y = static_cast<int>((N + BK - 1) / BK);
     auto splits = [&](int steps, int& nsplit, int& sps) {
-        int want = sm_count() / g.mtiles;
+        int want = sm_count() / (2 * g.mtiles);       // the two pre-products share the GPU
         if (want > steps / 2) want = steps / 2;
         if (want > 32) want = 32;
         if (want < 1) want = 1;
@@ -248,16 +292,16 @@ inline GradPlan grad_plan(int64_t N, int64_t K, int r, int64_t M) {
     g.counters_bytes = round_up(static_cast<size_t>(2 * g.mtiles) * 4, 256);
     g.t_bytes = round_up(static_cast<size_t>(M) * r * 2, 256);
     const int ns = g.nsplit_x > g.nsplit_y ? g.nsplit_x : g.nsplit_y;
-    g.partial_bytes = round_up(static_cast<size_t>(ns) * M * g.rp * 4, 256);
+    g.partial_bytes = round_up(static_cast<size_t>(ns) * M * g.rp * 4, 256);      // per pre-product
     return g;
 }
 
 inline size_t lora_grads_workspace(int64_t N, int64_t K, int r, int64_t M) {
     const GradPlan g = grad_plan(N, K, r, M);
-    return kStatusBytes + g.counters_bytes + 2 * g.t_bytes + g.partial_bytes;
+    return kStatusBytes + g.counters_bytes + 2 * g.t_bytes + 2 * g.partial_bytes;
 }
 
-// ws: [status][counters of T][counters of T'][T bf16][T' bf16][fp32 partial tiles, shared by the two pre-products]
+// ws: [status][counters of T][counters of T'][T bf16][T' bf16][fp32 partial tiles of T][fp32 partial tiles of T']
 inline int lora_grads_launch(const void* L1, const void* L2, int r, int64_t N, int64_t K, const void* X, const void* dY, int64_t M,
                              float* dL1, float* dL2, char* ws, cudaStream_t st) {
     const GradPlan g = grad_plan(N, K, r, M);
@@ -268,22 +312,18 @@ inline int lora_grads_launch(const void* L1, const void* L2, int r, int64_t N, i
     __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + g.counters_bytes);
     __nv_bfloat16* Tp = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + g.counters_bytes + g.t_bytes);
     float* partial = reinterpret_cast<float*>(ws + kStatusBytes + g.counters_bytes + 2 * g.t_bytes);
-    CUtensorMap tA, tB;
-    PreParams pp;
-    pp.partial = partial; pp.status = status; pp.M = static_cast<int>(M); pp.r = r; pp.rp = g.rp; pp.stages = 0;
-    // T = X L2^T
-    if (!make_map(&tA, X, M, K, 128) || !make_map(&tB, L2, r, K, g.rp)) return LQLORA_ERR_CUDA;
-    pp.T = T; pp.counters = counters; pp.steps = g.steps_x; pp.steps_per_split = g.sps_x;
-    int rc = launch_pre<false>(tA, tB, pp, g.mtiles, g.nsplit_x, st);
+    float* partial_p = reinterpret_cast<float*>(ws + kStatusBytes + g.counters_bytes + 2 * g.t_bytes + g.partial_bytes);
+    CUtensorMap tA0, tB0, tA1, tB1;
+    if (!make_map(&tA0, X, M, K, 128) || !make_map(&tB0, L2, r, K, g.rp)) return LQLORA_ERR_CUDA;        // T = X L2^T
+    if (!make_map(&tA1, dY, M, N, 128) || !make_map(&tB1, L1, N, r, 64)) return LQLORA_ERR_CUDA;         // T' = dY L1
+    PreParams p0, p1;
+    p0.partial = partial; p0.T = T; p0.counters = counters; p0.status = status;
+    p0.M = static_cast<int>(M); p0.r = r; p0.rp = g.rp; p0.steps = g.steps_x; p0.steps_per_split = g.sps_x; p0.stages = 0;
+    p1 = p0;
+    p1.partial = partial_p; p1.T = Tp; p1.counters = counters + g.mtiles; p1.steps = g.steps_y; p1.steps_per_split = g.sps_y;
+    const int rc = launch_pre_both(tA0, tB0, p0, g.nsplit_x, tA1, tB1, p1, g.nsplit_y, g.mtiles, st);
     if (rc != LQLORA_OK) return rc;
-    // T' = dY L1 (the partial tiles are reused: the stream orders the two kernels)
-    if (!make_map(&tA, dY, M, N, 128) || !make_map(&tB, L1, N, r, 64)) return LQLORA_ERR_CUDA;
-    pp.T = Tp; pp.counters = counters + g.mtiles; pp.steps = g.steps_y; pp.steps_per_split = g.sps_y;
-    rc = launch_pre<true>(tA, tB, pp, g.mtiles, g.nsplit_y, st);
-    if (rc != LQLORA_OK) return rc;
-    rc = launch_wgrad<false>(dY, M, N, T, r, dL1, status, st);      // dL1 = dY^T T
-    if (rc != LQLORA_OK) return rc;
-    return launch_wgrad<true>(X, M, K, Tp, r, dL2, status, st);      // dL2 = T'^T X
+    return launch_wgrad(dY, X, M, N, K, T, Tp, r, dL1, dL2, status, st);
 }
 
 }  // namespace tc
