@@ -366,6 +366,26 @@ def run_device(args):
     for M in (16, 1):
         loops[f"fwd{M}"], loop_kind[f"fwd{M}"] = graph_loop(lambda c, m: binding.linear_fwd(c, L1, L2, X[m], out=Y[m], workspace=WS[m]), M)
         loops[f"bwd{M}"], loop_kind[f"bwd{M}"] = graph_loop(lambda c, m: binding.linear_bwd_input(c, L1, L2, G[m], out=DX[m], workspace=WS[m]), M)
+    # gradients of the low-rank factors at M = 2048 (the next piece of a training step; not part of the timed step):
+    # rotating activation buffers, replayed as one CUDA graph
+    dL = (torch.empty(N, r, dtype=torch.float32, device=dev), torch.empty(r, K, dtype=torch.float32, device=dev))
+    gws = torch.empty(binding.lora_grads_workspace_bytes(N, K, r, 2048), dtype=torch.uint8, device=dev)
+
+    def grads_body():
+        for i in range(reps):
+            binding.lora_grads(L1, L2, Xr[i % nrot], Gr[i % nrot], out=dL, workspace=gws)
+    try:
+        grads_body()
+        torch.cuda.synchronize()
+        gg = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gg):
+            grads_body()
+        loops["grads2048"], loop_kind["grads2048"] = timed(gg.replay, reps), "cuda graph"
+    except Exception:
+        torch.cuda.synchronize()
+        loops["grads2048"], loop_kind["grads2048"] = timed(grads_body, reps), "stream loop"
+    if binding.workspace_status(gws) != 0:
+        raise SystemExit("lora_grads reported a device-side error")
     for k in list(loops):
         loops[k] = reduce_max(loops[k], world, dev)
 
@@ -420,6 +440,14 @@ def run_device(args):
                                        "frac_of_hbm_" + pk_kind: pbytes / lms / 1e6 / pk["hbm_gbs"],
                                        "how": loop_kind[f"{ps}{M}"]}
             breakdown[f"{ps}_M{M}"] = ent
+
+    gms = loops["grads2048"]
+    gbytes = 2.0 * 2048 * (N + K)          # X and dY read once (bf16)
+    breakdown["extra_lora_grads_M2048"] = {
+        "ms": gms, "how": loop_kind["grads2048"], "in_timed_step": False,
+        "GB/s": gbytes / gms / 1e6, "frac_of_hbm_" + pk_kind: gbytes / gms / 1e6 / pk["hbm_gbs"],
+        "TFLOP/s": 8.0 * 2048 * r * (N + K) / gms / 1e9,
+        "what": "lqlora_lora_grads: dL1 = dY^T (X L2^T), dL2 = (dY L1)^T X; bytes = X and dY read once"}
 
     # dominant kernel: the tensor-core linear (forward and input gradient at M = 2048)
     tc_ms = 0.5 * (loops["fwd2048"] + loops["bwd2048"])
