@@ -73,12 +73,28 @@ __device__ __forceinline__ void wgrad_body(const CUtensorMap& tmA, const CUtenso
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int i = 0; i < total; ++i) {
+            // The kernel that writes T may still be running (programmatic dependent launch): the tiles of A of the
+            // first ring pass are requested at once, the tiles of T only after that kernel has finished.
+            const int first = min(total, p.stages);
+            for (int i = 0; i < first; ++i) {
+                const uint32_t a_dst = smem_u32(base + static_cast<size_t>(i) * stage_bytes);
+                const int m = (s_lo + i) * BK;               // first token row of the step (rows past M read as zero)
+                mbar_expect_tx(full(i), A_BYTES + b_bytes);
+                for (int t = 0; t < 2; ++t) tma_load_2d(a_dst + t * 8192, &tmA, p0 + t * 64, m, full(i));
+            }
+            pdl_wait();
+            fence_proxy_async_all();
+            for (int i = 0; i < first; ++i) {
+                const uint32_t b_dst = smem_u32(base + static_cast<size_t>(i) * stage_bytes) + A_BYTES;
+                const int m = (s_lo + i) * BK;
+                for (int t = 0; t < p.rp / 64; ++t) tma_load_2d(b_dst + t * 8192, &tmT, t * 64, m, full(i));
+            }
+            for (int i = first; i < total; ++i) {
                 const int s = i % p.stages;
                 const uint32_t ph = (i / p.stages) & 1;
                 if (!wait(empty(s), ph ^ 1, ctl, 61)) break;
                 const uint32_t a_dst = smem_u32(base + static_cast<size_t>(s) * stage_bytes), b_dst = a_dst + A_BYTES;
-                const int m = (s_lo + i) * BK;               // first token row of the step (rows past M read as zero)
+                const int m = (s_lo + i) * BK;
                 mbar_expect_tx(full(s), A_BYTES + b_bytes);
                 for (int t = 0; t < 2; ++t) tma_load_2d(a_dst + t * 8192, &tmA, p0 + t * 64, m, full(s));
                 for (int t = 0; t < p.rp / 64; ++t) tma_load_2d(b_dst + t * 8192, &tmT, t * 64, m, full(s));
@@ -228,11 +244,13 @@ inline int launch_wgrad(const void* dY, const void* X, int64_t M, int64_t N, int
     cfg.blockDim = dim3(192);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = ns; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;      // overlaps the end of the pre-product kernel
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA0, tT0, p0, tA1, tT1, p1);
     count_launch(1);
     if (e != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
