@@ -893,7 +893,7 @@ inline PrePlan pre_plan(int64_t C, int r, int64_t M, int64_t out_cols) {
     const int idle = static_cast<int>((sms - main_ctas % sms) % sms);
     int want = idle / pl.mtiles;
     if (want > pl.steps / 2) want = pl.steps / 2;
-    if (want > 32) want = 32;
+    if (want > 8) want = 8;          // the CTA that arrives last adds the partial tiles: more than eight make it the critical path
     if (want < 1) want = 1;
     pl.steps_per_split = (pl.steps + want - 1) / want;
     pl.nsplit = (pl.steps + pl.steps_per_split - 1) / pl.steps_per_split;

@@ -300,7 +300,7 @@ inline GradPlan grad_plan(int64_t N, int64_t K, int r, int64_t M) {
     auto splits = [&](int steps, int& nsplit, int& sps) {
         int want = sm_count() / (2 * g.mtiles);       // the two pre-products share the GPU
         if (want > steps / 2) want = steps / 2;
-        if (want > 32) want = 32;
+        if (want > 8) want = 8;          // more partial tiles than eight make the adding CTA the critical path
         if (want < 1) want = 1;
         sps = (steps + want - 1) / want;
         nsplit = (steps + sps - 1) / sps;
