@@ -94,6 +94,14 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 }
 
 // ------------------------------------------------------------------------------------ dequantization
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 // One thread dequantizes the 32 consecutive weights of one (row, group) -- b0 words of the slab,
 // `words` pointing at the thread's first word, the others 32 words apart -- and writes them as four
 // 16-byte chunks of the row's 128 bytes; `dst` is the row start, `goff` the byte offset of the group
@@ -101,12 +109,13 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 // 8-bit codes read the code book from shared memory.  REP: the table is stored once per bank, entry c of the copy
 // of lane l at lut8[c * 32 + l], and `lut8` already points at the lane's copy, so no look-up meets a bank conflict.
 template <int B, bool REP = false>
-__device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ words, float s_lo, float s_hi, bool two_scales,
-                                              uint8_t* __restrict__ dst, uint32_t goff, uint32_t xr, const float* __restrict__ lut8) {
+__device__ __forceinline__ void dequant_group(uint32_t words, float s_lo, float s_hi, bool two_scales,
+                                              uint32_t dst, uint32_t goff, uint32_t xr, const float* __restrict__ lut8) {
+    // `words` and `dst` are 32-bit shared-memory addresses (explicit shared-space loads and stores)
     uint32_t w[B];
 #pragma unroll
-    for (int i = 0; i < B; ++i) w[i] = words[i * 32];
-    const uint32_t x = (goff ^ xr);          // chunk c sits at this offset with bits 4, 5 flipped by c
+    for (int i = 0; i < B; ++i) w[i] = lds_u32(words + i * 128);
+    const uint32_t x = dst + (goff ^ xr);    // chunk c sits at this address with bits 4, 5 flipped by c
     if constexpr (B == 8) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -120,7 +129,7 @@ __device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ words
                 const __nv_bfloat162 h = __floats2bfloat162_rn(__fmul_rn(q0, s), __fmul_rn(q1, s));
                 packed[e] = *reinterpret_cast<const uint32_t*>(&h);
             }
-            *reinterpret_cast<uint4*>(dst + (x ^ (c << 4))) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            sts_v4(x ^ (c << 4), packed[0], packed[1], packed[2], packed[3]);
         }
     } else {
         BlockTable<B> tab;
@@ -134,7 +143,7 @@ __device__ __forceinline__ void dequant_group(const uint32_t* __restrict__ words
             uint32_t o[4];
             tab.lookup4(selA, selB, o[0], o[1]);
             tab.lookup4(selA >> 16, selB >> 16, o[2], o[3]);
-            *reinterpret_cast<uint4*>(dst + (x ^ (c << 4))) = make_uint4(o[0], o[1], o[2], o[3]);
+            sts_v4(x ^ (c << 4), o[0], o[1], o[2], o[3]);
         }
     }
 }
@@ -399,10 +408,10 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         // word plane slot of this thread's row: rotated by 8 g + 16 (tile column % 2), see slab_row_slot();
         // forward: the tile column is the step index, backward: it is fixed per thread
-        const uint32_t* __restrict__ slab_base = reinterpret_cast<const uint32_t*>(p_ring) + slab_i * (64 * B) + g * (B * 32);
+        const uint32_t slab_base = smem_u32(p_ring) + (slab_i * (64 * B) + g * (B * 32)) * 4;      // byte address in shared memory
         const int slot_even = slab_row_slot(lane, g, BWD ? ((c0 >> 6) + (slab_i >> 1)) : 0);
         const int slot_odd = BWD ? slot_even : slab_row_slot(lane, g, 1);
-        uint8_t* my_b = b_ring + b_off;
+        const uint32_t my_b = smem_u32(b_ring) + b_off;
         bool ok = true;
         RingPos<SA> ra;
         RingPos<kBStages> rb;
@@ -429,7 +438,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                     ok = wait(full_a(sa), ra.ph, ctl, 4);
                     if (!ok) break;
-                    dequant_group<B>(slab_base + sa * (P_BYTES / 4) + (((q_lo + step) & 1) ? slot_odd : slot_even), s_lo, s_hi, two_scales, my_b + sb * kBBytes, g << 6, xr, lut8);
+                    dequant_group<B>(slab_base + sa * P_BYTES + (((q_lo + step) & 1) ? slot_odd : slot_even) * 4, s_lo, s_hi, two_scales, my_b + sb * kBBytes, g << 6, xr, lut8);
                     fence_proxy_async();            // make the generic-proxy stores visible to the tensor core
                     __syncwarp();
                     if (lane == 0) mbar_arrive(full_b(sb));

@@ -270,10 +270,10 @@ tc_pair_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             }
             return r;
         };
-        const uint32_t* __restrict__ slab_base = reinterpret_cast<const uint32_t*>(p_ring) + slab_words_off;
+        const uint32_t slab_base = smem_u32(p_ring) + slab_words_off * 4;        // byte address in shared memory
         const int slot_even = slab_row_slot(lane, g, tile_col);
         const int slot_odd = BWD ? slot_even : slab_row_slot(lane, g, 1);
-        uint8_t* my_b = b_ring + b_off;
+        const uint32_t my_b = smem_u32(b_ring) + b_off;
         float v_cached = -1.0f, sigma = 0.0f, s_lo = 0.0f, s_hi = 0.0f;
         RawScale slot[4];
         // forward, rows aligned to 16 blocks: windows of 16 scale codes instead of one load per step
@@ -316,7 +316,7 @@ tc_pair_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     }
                     ok = wait(full_a(sa), ra.ph, ctl, 44);
                     if (!ok) break;
-                    dequant_group<B, true>(slab_base + sa * (P_BYTES / 4) + ((step & 1) ? slot_odd : slot_even), s_lo, s_hi, two_scales,
+                    dequant_group<B, true>(slab_base + sa * P_BYTES + ((step & 1) ? slot_odd : slot_even) * 4, s_lo, s_hi, two_scales,
                                            my_b + sb * kPairBBytes, g << 6, xr, lut8 + lane);
                     fence_proxy_async();
                 } else {
