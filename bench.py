@@ -45,7 +45,7 @@ FALLBACK = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1
 # dram__bytes_read.sum + dram__bytes_write.sum per forward launch of tc_pair_linear_kernel<3, 0> at M = 2048 on this
 # workload (profiles/kernels_c2_4096_nf3_ncu_full.txt): the operands are read once (X 16.8 MB + packed 6.6 MB +
 # factors), the output stays in L2 during the capture
-TC_TRAFFIC_BYTES = 24170752
+TC_TRAFFIC_BYTES = 24289024
 
 
 def linear_flops(M: int, N: int, K: int, r: int) -> float:
