@@ -508,7 +508,8 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // and the status word says so).
         float* accbuf = reinterpret_cast<float*>(base);
         const uint32_t accbuf_addr = smem_u32(accbuf);
-        const int cols_share = BN / nsplit, col_lo = split * cols_share;
+        // CTA `split` owns the groups of eight columns [split * 32 / nsplit, (split + 1) * 32 / nsplit) (any cluster size)
+        const int g_lo = split * (BN / 8) / nsplit, g_hi = (split + 1) * (BN / 8) / nsplit;
 #pragma unroll 1
         for (int h = 0; h < MH; ++h) {
             if (warp >= 2 && acc_ok) {
@@ -526,10 +527,10 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
             __syncthreads();
             dec::cluster_sync_all();
-            for (int item = threadIdx.x; item < 128 * (cols_share / 8); item += kThreads) {
+            for (int item = threadIdx.x; item < 128 * (g_hi - g_lo); item += kThreads) {
                 const int row = item & 127, cg = item >> 7;
                 const int m = m0 + h * 128 + row;
-                const int col = col_lo + cg * 8;
+                const int col = (g_lo + cg) * 8;
                 // all remote loads are requested before the first is used (a round trip costs about two thousand clocks)
                 float part[8][8];
 #pragma unroll
@@ -835,10 +836,10 @@ inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUten
 // same time.  A cluster lives inside one GPC, so fewer fit than SMs / ks: 15 clusters of eight on a B200, not 18.
 // Asked once per cluster size; the figures measured on a B200 stand in when there is no device to ask.
 inline int tc_max_clusters(int ks) {
-    static int cached[4] = {-1, -1, -1, -1};       // ks = 1, 2, 4, 8
-    const int idx = (ks >= 8) ? 3 : (ks >= 4) ? 2 : (ks >= 2) ? 1 : 0;
+    static int cached[8] = {-1, -1, -1, -1, -1, -1, -1, -1};       // ks = 1 .. 8
+    const int idx = (ks < 1 ? 1 : ks > 8 ? 8 : ks) - 1;
     if (cached[idx] >= 0) return cached[idx];
-    const int fallback[4] = {148, 74, 36, 15};
+    const int fallback[8] = {148, 74, 48, 36, 28, 24, 16, 15};
     int n = 0;
     auto kern = tc_linear_kernel<3, false, 1>;
     cudaLaunchConfig_t cfg = {};
@@ -860,15 +861,15 @@ inline int tc_max_clusters(int ks) {
 }
 
 // Splits of the contraction for the one-CTA kernel (M <= 256): few output tiles would leave most SMs idle, so
-// the contraction of a tile is divided over a cluster of up to eight CTAs (each keeps at least eight steps, and
+// the contraction of a tile is divided over a cluster of up to eight CTAs (any size: each keeps at least 8 steps, 16 beyond four CTAs, and
 // all clusters must be resident at once: a second wave costs more than the finer split saves).
 inline int tc_ksplit(int64_t M, int64_t out_cols, int steps_q, int sms) {
     if (M > 256) return 1;
     const int mh = (M > 128) ? 2 : 1;
     const long long tiles = ((M + mh * 128 - 1) / (mh * 128)) * ((out_cols + BN - 1) / BN);
-    int ks = 1;
-    while (ks < 8 && tiles * (2 * ks) <= sms && steps_q / (2 * ks) >= 8 && tiles <= tc_max_clusters(2 * ks)) ks *= 2;
-    return ks;
+    for (int ks = 8; ks > 1; --ks)
+        if (tiles * ks <= sms && steps_q / ks >= (ks > 4 ? 16 : 8) && tiles <= tc_max_clusters(ks)) return ks;   // the reduction grows with ks
+    return 1;
 }
 
 struct PrePlan {
