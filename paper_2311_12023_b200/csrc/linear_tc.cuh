@@ -582,7 +582,10 @@ struct PreParams {
 };
 
 // Body of the kernel for the CTA (row tile `tile`, split `split` of `nsplit`); the tensor maps are kernel parameters.
-template <bool BWD>
+// CL: the splits of a tile are the CTAs of a cluster (nsplit = cluster size <= 8, a divisor of 64); their accumulators
+// go to the CTA that owns the column through distributed shared memory (own receive buffer behind the ring, rp x 128
+// fp32), are added there in rank order and stored as bf16 -- no partial tiles in global memory, no counters.
+template <bool BWD, bool CL = false>
 __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const PreParams& p, int tile, int split,
                                              int nsplit) {
     constexpr int A_BYTES = 16384;
@@ -590,7 +593,8 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int b_bytes = p.rp * 128;
     const int stage_bytes = A_BYTES + b_bytes;
-    uint8_t* tail = base + static_cast<size_t>(p.stages) * stage_bytes;
+    float* recv = reinterpret_cast<float*>(base + static_cast<size_t>(p.stages) * stage_bytes);
+    uint8_t* tail = reinterpret_cast<uint8_t*>(recv) + (CL ? static_cast<size_t>(p.rp) * 512 : 0);
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);      // full[8], empty[8], acc_full, drain
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 160);
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -622,6 +626,7 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    bool cl_ok = false;          // CL: this thread saw the accumulators complete (epilogue warps)
 
     if (warp == 0) {
         if (lane == 0) {
@@ -671,7 +676,8 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
         const int quarter = warp & 3;
         const int m = m0 + quarter * 32 + lane;
         const bool ok = (total > 0) ? wait(acc_full, 0, ctl, 13) : true;
-        if (ok) {
+        cl_ok = ok;
+        if (ok && !CL) {
             tc_fence_after();
             for (int col = 0; col < p.rp; col += 32) {
                 uint32_t v[32];
@@ -741,6 +747,42 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
             }
         }
     }
+    if constexpr (CL) {
+        // all threads of all CTAs of the cluster pass here, whatever happened before
+        __syncthreads();
+        const uint32_t recv_addr = smem_u32(recv);
+        const int cols_share = p.rp / nsplit;
+        if (warp >= 2 && cl_ok) {
+            tc_fence_after();
+            const int quarter = warp & 3;
+            const int row = quarter * 32 + lane;
+            for (int col = 0; col < p.rp; col += 32) {
+                uint32_t v[32];
+                if (total > 0) { tmem_ld32(tmem + (static_cast<uint32_t>(quarter * 32) << 16) + col, v); tmem_ld_wait(); }
+                else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = 0u;
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int c = col + i;
+                    const int owner = c / cols_share, cl = c - owner * cols_share;
+                    const uint32_t off = static_cast<uint32_t>((split * cols_share + cl) * 128 + row) * 4u;
+                    if (nsplit > 1) dec::st_dsmem_f32(recv_addr + off, static_cast<uint32_t>(owner), __uint_as_float(v[i]));
+                    else recv[cl * 128 + row] = __uint_as_float(v[i]);
+                }
+            }
+        }
+        __syncthreads();
+        if (nsplit > 1) dec::cluster_sync_all();
+        for (int item = threadIdx.x; item < 128 * cols_share; item += 192) {
+            const int row = item & 127, cl = item >> 7;
+            float sum = 0.0f;
+            for (int src = 0; src < nsplit; ++src) sum += recv[(src * cols_share + cl) * 128 + row];
+            const int m = m0 + row, col = split * cols_share + cl;
+            if (m < p.M && col < p.r) p.T[static_cast<size_t>(m) * p.r + col] = __float2bfloat16_rn(sum);
+        }
+    }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, tmem_cols);
@@ -753,16 +795,13 @@ tc_lowrank_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 }
 
 // Both pre-products of one layer in one launch (the weight-gradient path, which has the GPU to itself): grid.z = 0
-// computes T = X L2^T with (tmA0, tmB0, p0), grid.z = 1 computes T' = dY L1 with (tmA1, tmB1, p1); grid.y covers the
-// larger number of splits, CTAs beyond their product's own number leave at once.
+// computes T = X L2^T with (tmA0, tmB0, p0), grid.z = 1 computes T' = dY L1 with (tmA1, tmB1, p1); grid.y = splits of
+// the contraction = cluster size (the same for both), reduced through distributed shared memory.
 __global__ void __launch_bounds__(192, 1)
-tc_lowrank_both_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0, const PreParams p0, int nsplit0,
-                       const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1, const PreParams p1, int nsplit1) {
-    if (blockIdx.z == 0) {
-        if (static_cast<int>(blockIdx.y) < nsplit0) lowrank_body<false>(tmA0, tmB0, p0, blockIdx.x, blockIdx.y, nsplit0);
-    } else {
-        if (static_cast<int>(blockIdx.y) < nsplit1) lowrank_body<true>(tmA1, tmB1, p1, blockIdx.x, blockIdx.y, nsplit1);
-    }
+tc_lowrank_both_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0, const PreParams p0,
+                       const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1, const PreParams p1) {
+    if (blockIdx.z == 0) lowrank_body<false, true>(tmA0, tmB0, p0, blockIdx.x, blockIdx.y, gridDim.y);
+    else lowrank_body<true, true>(tmA1, tmB1, p1, blockIdx.x, blockIdx.y, gridDim.y);
 }
 
 // ------------------------------------------------------------------------------------ host side

@@ -257,14 +257,15 @@ inline int launch_wgrad(const void* dY, const void* X, int64_t M, int64_t N, int
     return LQLORA_OK;
 }
 
-// Both pre-products in one launch (tc_lowrank_both_kernel).
-inline int launch_pre_both(const CUtensorMap& tA0, const CUtensorMap& tB0, PreParams p0, int nsplit0, const CUtensorMap& tA1,
-                           const CUtensorMap& tB1, PreParams p1, int nsplit1, int mtiles, cudaStream_t st) {
+// Both pre-products in one launch (tc_lowrank_both_kernel); `nsplit` splits of the contraction = cluster size.
+inline int launch_pre_both(const CUtensorMap& tA0, const CUtensorMap& tB0, PreParams p0, const CUtensorMap& tA1, const CUtensorMap& tB1,
+                           PreParams p1, int nsplit, int mtiles, cudaStream_t st) {
     const int stage = 16384 + p0.rp * 128;
-    int stages = (kSmemLimit - 1024 - 256) / stage;
+    const int recv_bytes = p0.rp * 512;
+    int stages = (kSmemLimit - 1024 - 256 - recv_bytes) / stage;
     if (stages > 8) stages = 8;
     p0.stages = stages; p1.stages = stages;
-    const int smem = 1024 + stages * stage + 256;
+    const int smem = 1024 + stages * stage + recv_bytes + 256;
     auto kern = tc_lowrank_both_kernel;
     static bool attr_done = false;
     if (!attr_done) {
@@ -275,11 +276,16 @@ inline int launch_pre_both(const CUtensorMap& tA0, const CUtensorMap& tB0, PrePa
         attr_done = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(mtiles, nsplit0 > nsplit1 ? nsplit0 : nsplit1, 2);
+    cfg.gridDim = dim3(mtiles, nsplit, 2);
     cfg.blockDim = dim3(192);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA0, tB0, p0, nsplit0, tA1, tB1, p1, nsplit1);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = nsplit; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA0, tB0, p0, tA1, tB1, p1);
     count_launch(1);
     if (e != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
     return LQLORA_OK;
@@ -287,8 +293,8 @@ inline int launch_pre_both(const CUtensorMap& tA0, const CUtensorMap& tB0, PrePa
 
 // Plan of the two rank-r pre-products of a weight-gradient call (they have the GPU to themselves).
 struct GradPlan {
-    int mtiles, rp, steps_x, steps_y, nsplit_x, nsplit_y, sps_x, sps_y;
-    size_t counters_bytes, t_bytes, partial_bytes;
+    int mtiles, rp, steps_x, steps_y, nsplit, sps_x, sps_y;
+    size_t t_bytes;
 };
 
 inline GradPlan grad_plan(int64_t N, int64_t K, int r, int64_t M) {
@@ -297,49 +303,42 @@ inline GradPlan grad_plan(int64_t N, int64_t K, int r, int64_t M) {
     g.rp = (r <= 64) ? 64 : 128;
     g.steps_x = static_cast<int>((K + BK - 1) / BK);
     g.steps_y = static_cast<int>((N + BK - 1) / BK);
-    auto splits = [&](int steps, int& nsplit, int& sps) {
-        int want = sm_count() / (2 * g.mtiles);       // the two pre-products share the GPU
-        if (want > steps / 2) want = steps / 2;
-        if (want > 8) want = 8;          // more partial tiles than eight make the adding CTA the critical path
-        if (want < 1) want = 1;
-        sps = (steps + want - 1) / want;
-        nsplit = (steps + sps - 1) / sps;
-    };
-    splits(g.steps_x, g.nsplit_x, g.sps_x);
-    splits(g.steps_y, g.nsplit_y, g.sps_y);
-    g.counters_bytes = round_up(static_cast<size_t>(2 * g.mtiles) * 4, 256);
+    // splits of the contraction = cluster size, the same for both products: a power of two up to eight that keeps all
+    // CTAs of both products resident at once and leaves every CTA at least two steps
+    const int steps_min = g.steps_x < g.steps_y ? g.steps_x : g.steps_y;
+    int ns = 1;
+    while (ns < 8 && 2LL * g.mtiles * (2 * ns) <= sm_count() && steps_min / (2 * ns) >= 2) ns *= 2;
+    if (ns == 8 && 2 * g.mtiles > 15) ns = 4;          // fewer clusters of eight fit than SMs / 8
+    g.nsplit = ns;
+    g.sps_x = (g.steps_x + ns - 1) / ns;
+    g.sps_y = (g.steps_y + ns - 1) / ns;
     g.t_bytes = round_up(static_cast<size_t>(M) * r * 2, 256);
-    const int ns = g.nsplit_x > g.nsplit_y ? g.nsplit_x : g.nsplit_y;
-    g.partial_bytes = round_up(static_cast<size_t>(ns) * M * g.rp * 4, 256);      // per pre-product
     return g;
 }
 
 inline size_t lora_grads_workspace(int64_t N, int64_t K, int r, int64_t M) {
     const GradPlan g = grad_plan(N, K, r, M);
-    return kStatusBytes + g.counters_bytes + 2 * g.t_bytes + 2 * g.partial_bytes;
+    return kStatusBytes + 2 * g.t_bytes;
 }
 
-// ws: [status][counters of T][counters of T'][T bf16][T' bf16][fp32 partial tiles of T][fp32 partial tiles of T']
+// ws: [status][T bf16][T' bf16]
 inline int lora_grads_launch(const void* L1, const void* L2, int r, int64_t N, int64_t K, const void* X, const void* dY, int64_t M,
                              float* dL1, float* dL2, char* ws, cudaStream_t st) {
     const GradPlan g = grad_plan(N, K, r, M);
-    if (cudaMemsetAsync(ws, 0, kStatusBytes + g.counters_bytes, st) != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
+    if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
     count_launch(1);
     int* status = reinterpret_cast<int*>(ws);
-    int* counters = reinterpret_cast<int*>(ws + kStatusBytes);
-    __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + g.counters_bytes);
-    __nv_bfloat16* Tp = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + g.counters_bytes + g.t_bytes);
-    float* partial = reinterpret_cast<float*>(ws + kStatusBytes + g.counters_bytes + 2 * g.t_bytes);
-    float* partial_p = reinterpret_cast<float*>(ws + kStatusBytes + g.counters_bytes + 2 * g.t_bytes + g.partial_bytes);
+    __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes);
+    __nv_bfloat16* Tp = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + g.t_bytes);
     CUtensorMap tA0, tB0, tA1, tB1;
     if (!make_map(&tA0, X, M, K, 128) || !make_map(&tB0, L2, r, K, g.rp)) return LQLORA_ERR_CUDA;        // T = X L2^T
     if (!make_map(&tA1, dY, M, N, 128) || !make_map(&tB1, L1, N, r, 64)) return LQLORA_ERR_CUDA;         // T' = dY L1
     PreParams p0, p1;
-    p0.partial = partial; p0.T = T; p0.counters = counters; p0.status = status;
+    p0.partial = nullptr; p0.T = T; p0.counters = nullptr; p0.status = status;
     p0.M = static_cast<int>(M); p0.r = r; p0.rp = g.rp; p0.steps = g.steps_x; p0.steps_per_split = g.sps_x; p0.stages = 0;
     p1 = p0;
-    p1.partial = partial_p; p1.T = Tp; p1.counters = counters + g.mtiles; p1.steps = g.steps_y; p1.steps_per_split = g.sps_y;
-    const int rc = launch_pre_both(tA0, tB0, p0, g.nsplit_x, tA1, tB1, p1, g.nsplit_y, g.mtiles, st);
+    p1.T = Tp; p1.steps = g.steps_y; p1.steps_per_split = g.sps_y;
+    const int rc = launch_pre_both(tA0, tB0, p0, tA1, tB1, p1, g.nsplit, g.mtiles, st);
     if (rc != LQLORA_OK) return rc;
     return launch_wgrad(dY, X, M, N, K, T, Tp, r, dL1, dL2, status, st);
 }
