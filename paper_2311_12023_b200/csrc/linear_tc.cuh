@@ -899,11 +899,20 @@ inline int tc_max_clusters(int ks) {
     return n;
 }
 
-// Splits of the contraction for the one-CTA kernel (M <= 256): few output tiles would leave most SMs idle, so
+// Splits of the contraction for the one-CTA kernel: few output tiles would leave most SMs idle, so
 // the contraction of a tile is divided over a cluster of up to eight CTAs (any size: each keeps at least 8 steps, 16 beyond four CTAs, and
 // all clusters must be resident at once: a second wave costs more than the finer split saves).
+// CTA pairs on [512, 256] tiles take over once their tiles fill more than half of the SMs; below that the one-CTA
+// kernel with its split of the contraction puts at least twice as many SMs to work (4096 x 4096 at 512 rows: 32 CTAs
+// as pairs, 128 as single CTAs in clusters of four).
+inline bool tc_use_pair(int64_t M, int64_t out_cols, int sms) {
+    if (M <= 256) return false;
+    const long long pair_ctas = 2 * ((M + 511) / 512) * ((out_cols + BN - 1) / BN);
+    return 2 * pair_ctas > sms;
+}
+
 inline int tc_ksplit(int64_t M, int64_t out_cols, int steps_q, int sms) {
-    if (M > 256) return 1;
+    if (tc_use_pair(M, out_cols, sms)) return 1;
     const int mh = (M > 128) ? 2 : 1;
     const long long tiles = ((M + mh * 128 - 1) / (mh * 128)) * ((out_cols + BN - 1) / BN);
     for (int ks = 8; ks > 1; --ks)
@@ -1030,7 +1039,7 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
     __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + pl.counters_bytes);
     float* partial = reinterpret_cast<float*>(ws + kStatusBytes + pl.counters_bytes + pl.t_bytes);
     const int mh = (M > 128) ? 2 : 1;
-    const bool pair = M > 256;            // CTA pairs (cta_group::2) on [512, 256] tiles; boxes of 128 rows
+    const bool pair = tc_use_pair(M, backward ? q.K : q.N, sm_count());      // CTA pairs (cta_group::2) on [512, 256] tiles; boxes of 128 rows
     CUtensorMap tA, tA2, tB2;
     if (!make_map(&tA, A, M, C, pair ? 128 : mh * 128)) return LQLORA_ERR_CUDA;
     if (r > 0) {

@@ -1,4 +1,4 @@
-// Tensor-core linear on CTA pairs (tcgen05 cta_group::2) for many rows of X (M > 256).
+// Tensor-core linear on CTA pairs (tcgen05 cta_group::2) for many rows of X (M > 256 and tiles on more than half of the SMs).
 //
 // A pair of CTAs (a cluster of two, on one TPC) computes a [512, 256] tile of the output: each CTA holds
 // 2 x 128 rows of the activations (two accumulators of 128 lanes x 256 fp32 columns in its tensor memory)
