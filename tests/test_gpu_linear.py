@@ -84,12 +84,25 @@ def test_linear_single_row_with_odd_feature_count_uses_the_fallback():
 
 @pytest.mark.parametrize("N,K,M", [(640, 1088, 1000), (328, 704, 513), (896, 320, 700)])
 @pytest.mark.parametrize("b0,B0", [(3, 64), (4, 32)])
-def test_linear_pair_kernel_ragged_tiles(N, K, M, b0, B0):
-    """M > 256 (CTA-pair kernel) with M, N, K that are not multiples of the 512 x 256 pair tile: the second CTA of a
-    pair may have no weight rows / columns, the TMA stores clip, and the contraction ends inside a 128-row tile."""
+def test_linear_many_rows_few_tiles(N, K, M, b0, B0):
+    """More than 256 rows on matrices whose CTA-pair tiles would fill few SMs: the one-CTA kernel with several row
+    tiles (grid.x > 1), split contraction, M, N, K not multiples of the tile."""
     A = inputs.gaussian(600 + N, (N, K), 0.02)
     l1b, l2b = inputs.lowrank_factors(601 + K, N, K, 64, 0.01)
     run_case(A, l1b, l2b, C(b0, B0, 8, 64, 32), M, seed=700 + M)
+
+
+@pytest.mark.parametrize("N,K,M", [(2504, 2368, 2100), (2184, 2496, 2561)])
+@pytest.mark.parametrize("b0,B0", [(3, 64), (4, 32)])
+def test_linear_pair_kernel_ragged_tiles(N, K, M, b0, B0):
+    """CTA-pair kernel (enough [512, 256] tiles to fill the SMs) with M, N, K that are not multiples of the pair tile:
+    the second CTA of a pair may have few weight rows / columns, the TMA stores clip, and the contraction ends inside
+    a 128-row tile.  Sampled rows (first, last, both sides of tile edges)."""
+    assert binding.linear_path(N, K, C(b0, B0, 8, 64, 32), 64, M, False) == 1
+    A = inputs.gaussian(650 + N, (N, K), 0.02)
+    l1b, l2b = inputs.lowrank_factors(651 + K, N, K, 64, 0.01)
+    rows = inputs.sample_rows(660 + M, M, count=24, tile=128)
+    run_case(A, l1b, l2b, C(b0, B0, 8, 64, 32), M, seed=750 + M, rows=rows)
 
 
 @pytest.mark.parametrize("M", [4, 256])
