@@ -579,6 +579,7 @@ struct PreParams {
     int steps;             // contraction steps of 64 in total
     int steps_per_split;
     int stages;
+    int clear_status;      // 1: this kernel is the first of a call and clears the status word (no memset in front of it)
 };
 
 // Body of the kernel for the CTA (row tile `tile`, split `split` of `nsplit`); the tensor maps are kernel parameters.
@@ -600,6 +601,8 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* last_s = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
+    // cleared before this CTA lets the dependent kernel start: that kernel is launched once all CTAs have passed here
+    if (p.clear_status && tile == 0 && split == 0 && threadIdx.x == 0) *p.status = 0;
     pdl_launch_dependents();      // the linear kernel behind this one needs T only in its last steps
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = tile * 128;
@@ -697,8 +700,8 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
             __threadfence();
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (threadIdx.x == 64) {
-                const int old = atomicAdd(p.counters + tile, 1);
-                *last_s = (old == nsplit - 1) ? 1 : 0;
+                // a single split needs no counter (and the workspace then needs no zeroing)
+                *last_s = (nsplit == 1) ? 1 : ((atomicAdd(p.counters + tile, 1) == nsplit - 1) ? 1 : 0);
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (*last_s) {
@@ -1051,6 +1054,7 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
         PreParams pp;
         pp.partial = partial; pp.T = T; pp.counters = counters; pp.status = reinterpret_cast<int*>(ws);
         pp.M = M; pp.r = r; pp.rp = pl.rp; pp.steps = pl.steps; pp.steps_per_split = pl.steps_per_split; pp.stages = 0;
+        pp.clear_status = (pl.nsplit == 1) ? 1 : 0;          // run_linear skips its memset in that case
         const int rc = backward ? launch_pre<true>(tPA, tPB, pp, pl.mtiles, pl.nsplit, st)
                                 : launch_pre<false>(tPA, tPB, pp, pl.mtiles, pl.nsplit, st);
         if (rc != LQLORA_OK) return rc;

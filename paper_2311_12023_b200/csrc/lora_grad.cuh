@@ -335,7 +335,7 @@ inline int lora_grads_launch(const void* L1, const void* L2, int r, int64_t N, i
     if (!make_map(&tA1, dY, M, N, 128) || !make_map(&tB1, L1, N, r, 64)) return LQLORA_ERR_CUDA;         // T' = dY L1
     PreParams p0, p1;
     p0.partial = nullptr; p0.T = T; p0.counters = nullptr; p0.status = status;
-    p0.M = static_cast<int>(M); p0.r = r; p0.rp = g.rp; p0.steps = g.steps_x; p0.steps_per_split = g.sps_x; p0.stages = 0;
+    p0.M = static_cast<int>(M); p0.r = r; p0.rp = g.rp; p0.steps = g.steps_x; p0.steps_per_split = g.sps_x; p0.stages = 0; p0.clear_status = 0;
     p1 = p0;
     p1.T = Tp; p1.steps = g.steps_y; p1.steps_per_split = g.sps_y;
     const int rc = launch_pre_both(tA0, tB0, p0, tA1, tB1, p1, g.nsplit, g.mtiles, st);
