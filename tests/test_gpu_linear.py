@@ -232,3 +232,32 @@ def test_workspace_status_is_clean_after_a_call():
     X = binding.bf16_from_bits(inputs.activations(2, M, K))
     binding.linear_fwd(q, None, None, X, workspace=ws)
     assert binding.workspace_status(ws) == 0
+
+
+@pytest.mark.parametrize("N,K,M", [(256, 512, 8), (512, 1024, 200), (4096, 4096, 2048), (2304, 2048, 1100), (4096, 4096, 12)])
+def test_workspace_may_hold_anything_before_a_call(N, K, M):
+    """The workspace is scratch: whatever it holds (here all ones, i.e. a non-zero status word and non-zero arrival
+    counters) a call gives the right result and leaves a clean status word -- whether the words that must start at
+    zero are cleared by a memset or by the first kernel of the call."""
+    cfg = C(3, 64, 8, 256, 32)
+    A = inputs.gaussian(1400 + N, (N, K), 0.02)
+    l1b, l2b = inputs.lowrank_factors(1401, N, K, 64, 0.01)
+    q, ref = encode_both(A, cfg)
+    L1, L2 = binding.bf16_from_bits(l1b), binding.bf16_from_bits(l2b)
+    rows = inputs.sample_rows(1402, M, count=16) if M > 512 else None
+    ws = binding.alloc_workspace(q, 64, M)
+    xb = inputs.activations(1403, M, K)
+    gb = inputs.activations(1404, M, N)
+    for _ in range(2):
+        ws.fill_(0xFF)
+        Y = binding.linear_fwd(q, L1, L2, binding.bf16_from_bits(xb), workspace=ws)
+        torch.cuda.synchronize()
+        assert binding.workspace_status(ws) == 0
+        ws.fill_(0xFF)
+        dX = binding.linear_bwd_input(q, L1, L2, binding.bf16_from_bits(gb), workspace=ws)
+        torch.cuda.synchronize()
+        assert binding.workspace_status(ws) == 0
+    got = to_np(Y) if rows is None else to_np(Y[torch.from_numpy(rows).cuda()])
+    check_close(got, oracle.linear_fwd(ref["d32"], l1b, l2b, xb, rows), "Y")
+    got = to_np(dX) if rows is None else to_np(dX[torch.from_numpy(rows).cuda()])
+    check_close(got, oracle.linear_bwd_input(ref["d32"], l1b, l2b, gb, rows), "dX")
