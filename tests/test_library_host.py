@@ -119,3 +119,15 @@ def test_product_path_never_imports_the_oracle():
                 assert "import oracle" not in txt and "from oracle" not in txt and "lqlora_oracle" not in txt, f
     src = open(os.path.join(ROOT, "oracle", "__init__.py")).read() + open(os.path.join(ROOT, "oracle", "lqlora_oracle.cpp")).read()
     assert "paper_2311_12023_b200" not in src and "liblqlora.so" not in src
+
+
+def test_dispatch_between_the_weight_streaming_and_the_tensor_core_kernels(binding):
+    """lqlora_linear_path (host only): up to 16 rows stream the packed weights; from 17 rows the tensor cores take
+    over; the input gradient of 9..16 rows goes to the tensor cores too when the matrix has at least 2048 rows."""
+    cfg = inputs.QuantConfig(3, 64, 8, 256, 32)
+    for M, want in ((1, 0), (16, 0), (17, 1), (256, 1), (2048, 1)):
+        assert binding.linear_path(4096, 4096, cfg, 64, M, False) == want
+    for M, want in ((1, 0), (8, 0), (9, 1), (16, 1), (17, 1)):
+        assert binding.linear_path(4096, 4096, cfg, 64, M, True) == want
+    for M, want in ((8, 0), (9, 0), (16, 0), (17, 1)):
+        assert binding.linear_path(1024, 8192, cfg, 64, M, True) == want
