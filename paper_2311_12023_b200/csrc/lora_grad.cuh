@@ -325,9 +325,7 @@ inline size_t lora_grads_workspace(int64_t N, int64_t K, int r, int64_t M) {
 inline int lora_grads_launch(const void* L1, const void* L2, int r, int64_t N, int64_t K, const void* X, const void* dY, int64_t M,
                              float* dL1, float* dL2, char* ws, cudaStream_t st) {
     const GradPlan g = grad_plan(N, K, r, M);
-    if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
-    count_launch(1);
-    int* status = reinterpret_cast<int*>(ws);
+    int* status = reinterpret_cast<int*>(ws);          // cleared by the first kernel of the call
     __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes);
     __nv_bfloat16* Tp = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + g.t_bytes);
     CUtensorMap tA0, tB0, tA1, tB1;
@@ -335,9 +333,9 @@ inline int lora_grads_launch(const void* L1, const void* L2, int r, int64_t N, i
     if (!make_map(&tA1, dY, M, N, 128) || !make_map(&tB1, L1, N, r, 64)) return LQLORA_ERR_CUDA;         // T' = dY L1
     PreParams p0, p1;
     p0.partial = nullptr; p0.T = T; p0.counters = nullptr; p0.status = status;
-    p0.M = static_cast<int>(M); p0.r = r; p0.rp = g.rp; p0.steps = g.steps_x; p0.steps_per_split = g.sps_x; p0.stages = 0; p0.clear_status = 0;
+    p0.M = static_cast<int>(M); p0.r = r; p0.rp = g.rp; p0.steps = g.steps_x; p0.steps_per_split = g.sps_x; p0.stages = 0; p0.clear_status = 1;
     p1 = p0;
-    p1.T = Tp; p1.steps = g.steps_y; p1.steps_per_split = g.sps_y;
+    p1.T = Tp; p1.steps = g.steps_y; p1.steps_per_split = g.sps_y; p1.clear_status = 0;
     const int rc = launch_pre_both(tA0, tB0, p0, tA1, tB1, p1, g.nsplit, g.mtiles, st);
     if (rc != LQLORA_OK) return rc;
     return launch_wgrad(dY, X, M, N, K, T, Tp, r, dL1, dL2, status, st);
