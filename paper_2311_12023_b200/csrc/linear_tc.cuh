@@ -797,6 +797,13 @@ tc_lowrank_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     lowrank_body<BWD>(tmA, tmB, p, blockIdx.x, blockIdx.y, gridDim.y);
 }
 
+// The same with the splits of a tile as the CTAs of a cluster (grid.y = cluster size, a power of two up to eight).
+template <bool BWD>
+__global__ void __launch_bounds__(192, 1)
+tc_lowrank_cl_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const PreParams p) {
+    lowrank_body<BWD, true>(tmA, tmB, p, blockIdx.x, blockIdx.y, gridDim.y);
+}
+
 // Both pre-products of one layer in one launch (the weight-gradient path, which has the GPU to itself): grid.z = 0
 // computes T = X L2^T with (tmA0, tmB0, p0), grid.z = 1 computes T' = dY L1 with (tmA1, tmB1, p1); grid.y = splits of
 // the contraction = cluster size (the same for both), reduced through distributed shared memory.
@@ -954,10 +961,17 @@ inline PrePlan pre_plan(int64_t C, int r, int64_t M, int64_t out_cols) {
     const int idle = static_cast<int>((sms - main_ctas % sms) % sms);
     int want = idle / pl.mtiles;
     if (want > pl.steps / 2) want = pl.steps / 2;
-    if (want > 8) want = 8;          // the CTA that arrives last adds the partial tiles: more than eight make it the critical path
+    if (want > 8) want = 8;          // splits of a tile form a cluster (and more than eight made the sum the critical path)
+    if (idle < 48) {
+        // beside a nearly full linear kernel (itself made of clusters) large pre-product clusters took a cluster's place
+        // from it: at most four pre-product CTAs in all
+        const int cap = (4 / pl.mtiles > 1) ? 4 / pl.mtiles : 1;
+        if (want > cap) want = cap;
+    }
     if (want < 1) want = 1;
+    while (want & (want - 1)) want &= want - 1;          // a power of two: it divides the 64 columns of the accumulator
     pl.steps_per_split = (pl.steps + want - 1) / want;
-    pl.nsplit = (pl.steps + pl.steps_per_split - 1) / pl.steps_per_split;
+    pl.nsplit = want;
     pl.rp = (r <= 64) ? 64 : 128;
     pl.counters_bytes = round_up(static_cast<size_t>(pl.mtiles) * 4, 256);
     pl.partial_bytes = round_up(static_cast<size_t>(pl.nsplit) * M * pl.rp * 4, 256);
@@ -968,21 +982,24 @@ inline PrePlan pre_plan(int64_t C, int r, int64_t M, int64_t out_cols) {
 template <bool BWD>
 inline int launch_pre(const CUtensorMap& tA, const CUtensorMap& tB, PreParams p, int mtiles, int nsplit, cudaStream_t st) {
     const int stage = 16384 + p.rp * 128;
-    int stages = (kSmemLimit - 1024 - 256) / stage;
+    const bool cl = nsplit > 1;            // several splits: reduced inside a cluster (no partial tiles, no counters)
+    const int recv_bytes = cl ? p.rp * 512 : 0;
+    int stages = (kSmemLimit - 1024 - 256 - recv_bytes) / stage;
     if (stages > 8) stages = 8;
     p.stages = stages;
-    const int smem = 1024 + stages * stage + 256;
-    auto kern = tc_lowrank_kernel<BWD>;
+    const int smem = 1024 + stages * stage + recv_bytes + 256;
+    void (*kern)(const CUtensorMap, const CUtensorMap, const PreParams) = cl ? tc_lowrank_cl_kernel<BWD> : tc_lowrank_kernel<BWD>;
     static bool attr_done = false;
     if (!attr_done) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
+        if (cudaFuncSetAttribute(tc_lowrank_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess ||
+            cudaFuncSetAttribute(tc_lowrank_cl_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess) {
             cudaGetLastError();
             return LQLORA_ERR_CUDA;
         }
         attr_done = true;
     }
-    // Launched as clusters of two where possible: the CTAs then fill whole TPCs, and the CTA pairs of the linear
-    // kernel that runs beside this one find as many free TPCs as the SM count suggests.
+    // One split: launched as clusters of two row tiles where possible (the CTAs then fill whole TPCs, and the CTA pairs
+    // of the linear kernel that runs beside this one find as many free TPCs as the SM count suggests).
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(mtiles, nsplit);
     cfg.blockDim = dim3(192);
@@ -990,7 +1007,7 @@ inline int launch_pre(const CUtensorMap& tA, const CUtensorMap& tB, PreParams p,
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (mtiles % 2 == 0) ? 2 : 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[0].val.clusterDim.x = (!cl && mtiles % 2 == 0) ? 2 : 1; attr[0].val.clusterDim.y = cl ? nsplit : 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA, tB, p);
@@ -1054,7 +1071,7 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
         PreParams pp;
         pp.partial = partial; pp.T = T; pp.counters = counters; pp.status = reinterpret_cast<int*>(ws);
         pp.M = M; pp.r = r; pp.rp = pl.rp; pp.steps = pl.steps; pp.steps_per_split = pl.steps_per_split; pp.stages = 0;
-        pp.clear_status = (pl.nsplit == 1) ? 1 : 0;          // run_linear skips its memset in that case
+        pp.clear_status = 1;           // first kernel of the call (run_linear issues no memset when there is a rank-r term)
         const int rc = backward ? launch_pre<true>(tPA, tPB, pp, pl.mtiles, pl.nsplit, st)
                                 : launch_pre<false>(tPA, tPB, pp, pl.mtiles, pl.nsplit, st);
         if (rc != LQLORA_OK) return rc;

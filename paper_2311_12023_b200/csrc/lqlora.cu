@@ -63,13 +63,11 @@ static int run_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, i
     const QView v = make_view(q);
     const bool use_tc = tc_supported(v, r, M, backward);
     const bool use_decode = !use_tc && (backward ? dec::bwd_supported(v, M) : dec::supported(v, M));
-    // With a rank-r term the first kernel of the call clears the status word itself (decode path; tensor-core path when
-    // the pre-product has a single split and so needs no arrival counters); otherwise a memset does.
-    const tc::PrePlan pre = tc::pre_plan(backward ? v.N : v.K, r, M, backward ? v.K : v.N);
-    const bool first_kernel_clears = r > 0 && (use_decode || (use_tc && pre.nsplit == 1));
+    // With a rank-r term the first kernel of the call (the pre-product) clears the status word itself and nothing else
+    // has to start at zero; otherwise a memset clears it.
+    const bool first_kernel_clears = r > 0 && (use_decode || use_tc);
     if (!first_kernel_clears) {
-        const size_t zero_bytes = kStatusBytes + (use_tc ? pre.counters_bytes : 0);
-        if (cudaMemsetAsync(ws, 0, zero_bytes, st) != cudaSuccess) return cuda_rc(cudaGetLastError());
+        if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) return cuda_rc(cudaGetLastError());
     }
     cudaError_t e = cudaSuccess;
     if (use_tc) {
