@@ -27,6 +27,8 @@
  *   - Inputs must be finite.
  *   - There is no CPU fallback: without a CUDA device every compute entry point returns
  *     LQLORA_ERR_CUDA.
+ *   - One device per process (the usual one-process-per-GPU arrangement): kernel attributes and the SM
+ *     count are looked up once, on the device that is current at the first call.
  */
 #ifndef LQLORA_H_
 #define LQLORA_H_
@@ -146,8 +148,7 @@ int lqlora_linear_workspace_bytes(int64_t N, int64_t K, const lqlora_config* cfg
  * to global memory.  r = 0 (L1 = L2 = NULL) computes the quantized part alone.
  * All of Q's arrays, L1, L2, X, Y, workspace_dev: device, 16-byte aligned.
  * The first 256 bytes of the workspace hold a status word (see lqlora_workspace_status); the rest
- * is scratch for the rank-r intermediate and split-K partial sums.  Concurrent calls must use
- * different workspaces.
+ * is scratch for the rank-r intermediate.  Concurrent calls must use different workspaces.
  * Errors: as lqlora_encode, plus UNSUPPORTED.
  */
 int lqlora_linear_fwd(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r,
@@ -197,15 +198,18 @@ int lqlora_lora_grads(const void* L1_dev, const void* L2_dev, int r, int64_t N, 
  *   - The first call on a device looks up the array's device address (a one-off set-up step);
  *     make that first call outside any stream capture.
  *   - All calls share the one array.  It still holds the previous call's data when the next call
- *     starts; the words that have to start at zero (status word, arrival counters) are cleared on
- *     the stream by each call.  Two calls whose kernels can overlap on the GPU (different streams
- *     without ordering between them) would race on it: order them, or use lqlora_linear_fwd with
- *     separate workspaces.  lqlora_workspace_status is not available for this array.
+ *     starts; the one word that has to start at zero (the status word) is cleared on the stream by
+ *     each call.  Two calls whose kernels can overlap on the GPU (different streams without ordering
+ *     between them) would race on it: order them, or use lqlora_linear_fwd with separate workspaces.
+ *   - lqlora_static_scratch_status(stream) is lqlora_workspace_status for this array: it synchronizes
+ *     `stream` and returns LQLORA_OK, or LQLORA_ERR_TIMEOUT if a kernel of the last call on the current
+ *     device gave up on a bounded wait.  It allocates nothing either.
  * Other arguments, layouts and error codes as for lqlora_linear_fwd.
  */
 size_t lqlora_static_scratch_bytes(void);
 int lqlora_linear_fwd_static(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r,
                              const void* X_dev, int64_t M, void* Y_dev, void* stream);
+int lqlora_static_scratch_status(void* stream);
 
 /*
  * Host-buffer variants (end-to-end use: activations arrive from and results return to pinned host
@@ -232,9 +236,15 @@ int lqlora_linear_bwd_input_host(const lqlora_qmatrix* q, const void* L1_dev, co
  * (its output is then undefined).  The word is cleared by every linear call before it launches. */
 int lqlora_workspace_status(const void* workspace_dev, void* stream);
 
-/* Which kernel family the last dispatch of lqlora_linear_* would use for M rows:
- * 0 = weight-streaming small-M kernel, 1 = tcgen05 tensor-core kernel.  Host only. */
-int lqlora_linear_path(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, int backward);
+/* Which kernel lqlora_linear_fwd (backward = 0) or lqlora_linear_bwd_input (backward != 0) dispatches to for M rows:
+ *   LQLORA_PATH_PLAIN    plain-FMA fall-back (shapes the vector paths do not take)
+ *   LQLORA_PATH_STREAM   weight-streaming kernel for decode-sized inputs (M <= 16)
+ *   LQLORA_PATH_TC_ONE   tcgen05 kernel, one CTA per output tile, contraction split over a cluster
+ *   LQLORA_PATH_TC_PAIR  tcgen05 kernel, CTA pairs (cta_group::2) on [512, 256] output tiles
+ * *splits (may be NULL) receives the number of CTAs that share one output tile's contraction (the cluster size; 1 for
+ * CTA pairs and the fall-back).  Returns a negative lqlora_status for invalid arguments.  Host only. */
+enum { LQLORA_PATH_PLAIN = 0, LQLORA_PATH_STREAM = 1, LQLORA_PATH_TC_ONE = 2, LQLORA_PATH_TC_PAIR = 3 };
+int lqlora_linear_path(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, int backward, int* splits);
 
 /* lqlora_encode finds the nearest code (Sec. 2.2: c_j = argmin_k |q~_k - u_j / s_i|) with a bin table over [-1, 1]:
  * every bin holds at most one decision threshold (the midpoint of two neighbouring code-book entries), and inputs

@@ -22,7 +22,8 @@ EXPORTS = [
     "lqlora_unpack", "lqlora_dequant", "lqlora_linear_workspace_bytes", "lqlora_linear_fwd",
     "lqlora_linear_bwd_input", "lqlora_workspace_status", "lqlora_linear_path", "lqlora_launch_count",
     "lqlora_status_string", "lqlora_encode_host", "lqlora_linear_fwd_host", "lqlora_linear_bwd_input_host",
-    "lqlora_static_scratch_bytes", "lqlora_linear_fwd_static", "lqlora_encode_search_clearance",
+    "lqlora_static_scratch_bytes", "lqlora_linear_fwd_static", "lqlora_static_scratch_status",
+    "lqlora_encode_search_clearance",
     "lqlora_lora_grads_workspace_bytes", "lqlora_lora_grads",
 ]
 
@@ -78,7 +79,8 @@ def lib() -> ctypes.CDLL:
         L.lqlora_encode_search_clearance.argtypes = [ci]
         L.lqlora_encode_search_clearance.restype = ctypes.c_double
         L.lqlora_linear_fwd_static.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp]
-        L.lqlora_linear_path.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ci]
+        L.lqlora_static_scratch_status.argtypes = [vp]
+        L.lqlora_linear_path.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ci, ctypes.POINTER(ci)]
         L.lqlora_launch_count.restype = i64
         L.lqlora_status_string.argtypes = [ci]
         L.lqlora_status_string.restype = ctypes.c_char_p
@@ -136,9 +138,21 @@ def linear_workspace_bytes(N: int, K: int, cfg, r: int, M: int) -> int:
     return int(out.value)
 
 
-def linear_path(N: int, K: int, cfg, r: int, M: int, backward: bool) -> int:
+PATH_PLAIN, PATH_STREAM, PATH_TC_ONE, PATH_TC_PAIR = 0, 1, 2, 3
+
+
+def linear_route(N: int, K: int, cfg, r: int, M: int, backward: bool) -> Tuple[int, int]:
+    """lqlora_linear_path: (kernel id, CTAs sharing one output tile's contraction) of the dispatch for M rows."""
     c = _cfg(cfg)
-    return int(lib().lqlora_linear_path(N, K, ctypes.byref(c), r, M, int(backward)))
+    splits = ctypes.c_int(0)
+    kernel = int(lib().lqlora_linear_path(N, K, ctypes.byref(c), r, M, int(backward), ctypes.byref(splits)))
+    if kernel < 0:
+        raise LqloraError(kernel, "lqlora_linear_path")
+    return kernel, int(splits.value)
+
+
+def linear_path(N: int, K: int, cfg, r: int, M: int, backward: bool) -> int:
+    return linear_route(N, K, cfg, r, M, backward)[0]
 
 
 def launch_count() -> int:
@@ -305,6 +319,11 @@ def linear_fwd_host(q, L1, L2, X_host, Y_host, X_stage, Y_stage, workspace) -> N
 def linear_bwd_input_host(q, L1, L2, dY_host, dX_host, dY_stage, dX_stage, workspace) -> None:
     _linear_host(lib().lqlora_linear_bwd_input_host, "lqlora_linear_bwd_input_host", q, L1, L2, dY_host, dX_host,
                  dY_stage, dX_stage, workspace)
+
+
+def static_scratch_status() -> int:
+    """lqlora_static_scratch_status: status word of the built-in scratch array after the calls on the current stream."""
+    return int(lib().lqlora_static_scratch_status(_stream()))
 
 
 def workspace_status(workspace: torch.Tensor) -> int:

@@ -164,10 +164,16 @@ decode_fwd_kernel(const Params p) {
             bulk_load(dst + XOFF + m * kXRowBytes, xsrc + static_cast<size_t>(m) * q.K, nt * (kTileCols * 2), full(s));
     };
     // There is no producer warp: thread 0 fills the ring once, afterwards the warp that is last to finish a stage
-    // refills its slot (nobody waits for a free slot, and the CTA has eight warps, two per scheduler).
-    if (threadIdx.x == 0) {
-        for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it);
-    }
+    // refills its slot (nobody waits for a free slot, and the CTA has eight warps, two per scheduler).  The first fill
+    // is issued after the first loads of the scale table below: the few bytes of the table would otherwise queue
+    // behind the ring's bulk copies of all CTAs in the memory system (measured: 4 us instead of 1).
+    bool ring_filled = false;
+    auto fill_ring = [&]() {
+        if (!ring_filled && threadIdx.x == 0) {
+            for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it);
+        }
+        ring_filled = true;
+    };
 
     // block scales of the CTA's rows and columns: s~ = fl32(float(s^) * fl32(v / 127)), 0 for rows past N
     const int kb_first = (kt0 * kTileCols) >> q.logB0;
@@ -198,6 +204,7 @@ decode_fwd_kernel(const Params p) {
                     }
                 }
             }
+            fill_ring();
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
                 if (rowv[u] < 0) continue;
@@ -231,6 +238,7 @@ decode_fwd_kernel(const Params p) {
                     }
                 }
             }
+            fill_ring();
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
                 if (rowv[u] < 0) continue;
@@ -267,11 +275,13 @@ decode_fwd_kernel(const Params p) {
                 }
             }
         }
+        fill_ring();
 #pragma unroll
         for (int u = 0; u < 4; ++u)
             if (slot[u] >= 0) stab[slot[u]] = block_scale(static_cast<uint8_t>(sc8[u]), v[u]);
     }
     }
+    fill_ring();          // (a CTA without blocks has not passed through the loops above)
     if constexpr (B == 8) {
         for (int i = threadIdx.x; i < 256; i += kThreads) lut8[i] = c_codebook[3][i];
     }
@@ -600,10 +610,15 @@ decode_bwd_kernel(const BwdParams p) {
         for (int m = 0; m < p.M; ++m)
             bulk_load(dst + YOFF + m * kBwdYRowBytes, p.dY + static_cast<size_t>(m) * q.N + row0, nrows * 2, full(s));
     };
-    // thread 0 fills the ring once; afterwards the warp that is last to finish a stage refills its slot
-    if (threadIdx.x == 0) {
-        for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it);
-    }
+    // thread 0 fills the ring once (after the first loads of the scale table below have been issued, so that they do
+    // not queue behind the bulk copies); afterwards the warp that is last to finish a stage refills its slot
+    bool ring_filled = false;
+    auto fill_ring = [&]() {
+        if (!ring_filled && threadIdx.x == 0) {
+            for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it);
+        }
+        ring_filled = true;
+    };
 
     // block scales of the CTA's rows and its (at most 256) columns
     const int col_first = kt_first * kTileCols;
@@ -641,6 +656,7 @@ decode_bwd_kernel(const BwdParams p) {
                     }
                 }
             }
+            fill_ring();
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 if (rowv[u] < 0) continue;
@@ -676,11 +692,13 @@ decode_bwd_kernel(const BwdParams p) {
                 }
             }
         }
+        fill_ring();
 #pragma unroll
         for (int u = 0; u < 4; ++u)
             if (slot[u] >= 0) stab[slot[u]] = block_scale(static_cast<uint8_t>(sc8[u]), v[u]);
     }
     }
+    fill_ring();
     if constexpr (B == 8) {
         for (int i = threadIdx.x; i < 256; i += kThreads) lut8[i] = c_codebook[3][i];
     }
@@ -1340,6 +1358,25 @@ inline cudaError_t launch_bwd(const QView& q, const void* L1, const void* L2, in
     }
     if (q.B0 == 16) return (NT == 1) ? launch_bwd_nt<B, 1, true>(p, q, M, r > 0, st) : launch_bwd_nt<B, 2, true>(p, q, M, r > 0, st);
     return (NT == 1) ? launch_bwd_nt<B, 1, false>(p, q, M, r > 0, st) : launch_bwd_nt<B, 2, false>(p, q, M, r > 0, st);
+}
+
+// Cluster sizes the two kernels would be launched with (for lqlora_linear_path; the input gradient's choice also
+// depends on the device's occupancy answer at launch time, this is the host-side default).
+inline int fwd_splits(const QView& q, int M) {
+    switch (q.b0) {
+        case 2: return make_plan<2>(q, M).S;
+        case 3: return make_plan<3>(q, M).S;
+        case 4: return make_plan<4>(q, M).S;
+        default: return make_plan<8>(q, M).S;
+    }
+}
+inline int bwd_splits(const QView& q, int M) {
+    switch (q.b0) {
+        case 2: return make_bwd_plan<2>(q, M).S;
+        case 3: return make_bwd_plan<3>(q, M).S;
+        case 4: return make_bwd_plan<4>(q, M).S;
+        default: return make_bwd_plan<8>(q, M).S;
+    }
 }
 
 }  // namespace dec

@@ -568,12 +568,10 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // ------------------------------------------------------------------------------------ rank-r pre-product
 // T = bf16(A F) with a short output width (r <= 128):  forward  T = X L2^T  (F = L2 [r, K], K-major B operand),
 // backward T = dY L1 (F = L1 [N, r], MN-major B operand).  Grid = (row tiles of 128, splits of the
-// contraction).  Each CTA accumulates its part in tensor memory and stores it as an fp32 partial tile;
-// the CTA that arrives last on the tile's counter adds the partial tiles in a fixed order and writes bf16.
+// contraction).  Each CTA accumulates its part in tensor memory; with one split it rounds its tile to bf16 and
+// stores it, with several the splits of a tile form a cluster (see CL below).
 struct PreParams {
-    float* partial;        // [nsplit][M][rp] fp32
     __nv_bfloat16* T;      // [M][r]
-    int* counters;         // one per row tile, zeroed before the launch
     int* status;
     int M, r, rp;          // rp = r rounded up to 64 (MMA N)
     int steps;             // contraction steps of 64 in total
@@ -599,7 +597,6 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);      // full[8], empty[8], acc_full, drain
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 160);
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    volatile int* last_s = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
     // cleared before this CTA lets the dependent kernel start: that kernel is launched once all CTAs have passed here
     if (p.clear_status && tile == 0 && split == 0 && threadIdx.x == 0) *p.status = 0;
@@ -621,7 +618,6 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
         mbar_init(acc_full, 1);
         mbar_init(drain, 1);
         *abort_s = 0;
-        *last_s = 0;
         fence_barrier_init();
     }
     if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), tmem_cols); tmem_relinquish(); }
@@ -681,6 +677,8 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
         const bool ok = (total > 0) ? wait(acc_full, 0, ctl, 13) : true;
         cl_ok = ok;
         if (ok && !CL) {
+            // one split: the accumulator row of this thread goes straight to T as bf16 (r is a multiple of 16, so a
+            // run of eight columns lies inside or outside of it as a whole)
             tc_fence_after();
             for (int col = 0; col < p.rp; col += 32) {
                 uint32_t v[32];
@@ -690,60 +688,16 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
                     for (int i = 0; i < 32; ++i) v[i] = 0u;
                 }
                 if (m < p.M) {
-                    float4* dst = reinterpret_cast<float4*>(p.partial + (static_cast<size_t>(split) * p.M + m) * p.rp + col);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                             __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
-                }
-            }
-            __threadfence();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (threadIdx.x == 64) {
-                // a single split needs no counter (and the workspace then needs no zeroing)
-                *last_s = (nsplit == 1) ? 1 : ((atomicAdd(p.counters + tile, 1) == nsplit - 1) ? 1 : 0);
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (*last_s) {
-                __threadfence();
-                // coalesced reduction of the nsplit partial tiles: thread -> 4 columns, rows strided
-                const int t = threadIdx.x - 64;
-                const int groups = p.rp >> 2;                 // float4 groups per row: 16 or 32
-                const int cg = t % groups, rstep = 128 / groups;
-                const size_t zstride = static_cast<size_t>(p.M) * p.rp;
-                // four rows at a time so that up to 32 loads are in flight per thread
-                for (int rr = t / groups; rr < 128; rr += 4 * rstep) {
-                    float4 acc[4];
+                    for (int i = 0; i < 4; ++i) {
+                        if (col + 8 * i < p.r) {
+                            uint32_t w[4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int z0 = 0; z0 < nsplit; z0 += 8) {
-                        float4 v[4][8];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int row = m0 + rr + u * rstep;
-                            const float* src = p.partial + static_cast<size_t>(row) * p.rp + cg * 4;
-#pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                v[u][i] = (z0 + i < nsplit && row < p.M && rr + u * rstep < 128)
-                                              ? __ldcg(reinterpret_cast<const float4*>(src + (z0 + i) * zstride))
-                                              : make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                acc[u].x += v[u][i].x; acc[u].y += v[u][i].y; acc[u].z += v[u][i].z; acc[u].w += v[u][i].w;
+                            for (int e = 0; e < 4; ++e) {
+                                const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[8 * i + 2 * e]), __uint_as_float(v[8 * i + 2 * e + 1]));
+                                w[e] = *reinterpret_cast<const uint32_t*>(&h);
                             }
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int row = m0 + rr + u * rstep;
-                        if (row < p.M && rr + u * rstep < 128 && cg * 4 < p.r) {
-                            const __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[u].x, acc[u].y), h1 = __floats2bfloat162_rn(acc[u].z, acc[u].w);
-                            uint2 o;
-                            o.x = *reinterpret_cast<const uint32_t*>(&h0);
-                            o.y = *reinterpret_cast<const uint32_t*>(&h1);
-                            *reinterpret_cast<uint2*>(p.T + static_cast<size_t>(row) * p.r + cg * 4) = o;
+                            *reinterpret_cast<uint4*>(p.T + static_cast<size_t>(m) * p.r + col + 8 * i) = make_uint4(w[0], w[1], w[2], w[3]);
                         }
                     }
                 }
@@ -932,7 +886,7 @@ inline int tc_ksplit(int64_t M, int64_t out_cols, int steps_q, int sms) {
 
 struct PrePlan {
     int mtiles, nsplit, steps, steps_per_split, rp;
-    size_t counters_bytes, partial_bytes, t_bytes;
+    size_t t_bytes;
 };
 
 // Number of SMs of the current device (148 on B200; also the answer when no device is present).
@@ -973,8 +927,6 @@ inline PrePlan pre_plan(int64_t C, int r, int64_t M, int64_t out_cols) {
     pl.steps_per_split = (pl.steps + want - 1) / want;
     pl.nsplit = want;
     pl.rp = (r <= 64) ? 64 : 128;
-    pl.counters_bytes = round_up(static_cast<size_t>(pl.mtiles) * 4, 256);
-    pl.partial_bytes = round_up(static_cast<size_t>(pl.nsplit) * M * pl.rp * 4, 256);
     pl.t_bytes = round_up(static_cast<size_t>(M) * (r > 0 ? r : 1) * 2, 256);
     return pl;
 }
@@ -982,7 +934,7 @@ inline PrePlan pre_plan(int64_t C, int r, int64_t M, int64_t out_cols) {
 template <bool BWD>
 inline int launch_pre(const CUtensorMap& tA, const CUtensorMap& tB, PreParams p, int mtiles, int nsplit, cudaStream_t st) {
     const int stage = 16384 + p.rp * 128;
-    const bool cl = nsplit > 1;            // several splits: reduced inside a cluster (no partial tiles, no counters)
+    const bool cl = nsplit > 1;            // several splits: reduced inside a cluster
     const int recv_bytes = cl ? p.rp * 512 : 0;
     int stages = (kSmemLimit - 1024 - 256 - recv_bytes) / stage;
     if (stages > 8) stages = 8;
@@ -1046,7 +998,7 @@ inline bool tc_supported(const QView& q, int r, int64_t M, bool backward) {
 
 inline size_t tc_workspace_bytes(int64_t N, int64_t K, int r, int64_t M, bool backward) {
     const tc::PrePlan pl = tc::pre_plan(backward ? N : K, r, M, backward ? K : N);
-    return kStatusBytes + pl.counters_bytes + pl.t_bytes + (r > 0 ? pl.partial_bytes : 0);
+    return kStatusBytes + pl.t_bytes;
 }
 
 inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, const void* A, int M, void* out, char* ws,
@@ -1054,10 +1006,8 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
     using namespace tc;
     const int C = backward ? q.N : q.K;              // contraction length
     const PrePlan pl = pre_plan(C, r, M, backward ? q.K : q.N);
-    // workspace: [status][row-tile counters][T bf16][fp32 partial tiles]; status and counters were zeroed by the caller
-    int* counters = reinterpret_cast<int*>(ws + kStatusBytes);
-    __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes + pl.counters_bytes);
-    float* partial = reinterpret_cast<float*>(ws + kStatusBytes + pl.counters_bytes + pl.t_bytes);
+    // workspace: [status word][T bf16]; the status word is cleared by the first kernel of the call (or the caller's memset)
+    __nv_bfloat16* T = reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes);
     const int mh = (M > 128) ? 2 : 1;
     const bool pair = tc_use_pair(M, backward ? q.K : q.N, sm_count());      // CTA pairs (cta_group::2) on [512, 256] tiles; boxes of 128 rows
     CUtensorMap tA, tA2, tB2;
@@ -1069,7 +1019,7 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
         const bool okp = backward ? make_map(&tPB, L1, q.N, r, 64) : make_map(&tPB, L2, r, q.K, pl.rp);
         if (!okp) return LQLORA_ERR_CUDA;
         PreParams pp;
-        pp.partial = partial; pp.T = T; pp.counters = counters; pp.status = reinterpret_cast<int*>(ws);
+        pp.T = T; pp.status = reinterpret_cast<int*>(ws);
         pp.M = M; pp.r = r; pp.rp = pl.rp; pp.steps = pl.steps; pp.steps_per_split = pl.steps_per_split; pp.stages = 0;
         pp.clear_status = 1;           // first kernel of the call (run_linear issues no memset when there is a rank-r term)
         const int rc = backward ? launch_pre<true>(tPA, tPB, pp, pl.mtiles, pl.nsplit, st)

@@ -332,7 +332,7 @@ inline int lora_grads_launch(const void* L1, const void* L2, int r, int64_t N, i
     if (!make_map(&tA0, X, M, K, 128) || !make_map(&tB0, L2, r, K, g.rp)) return LQLORA_ERR_CUDA;        // T = X L2^T
     if (!make_map(&tA1, dY, M, N, 128) || !make_map(&tB1, L1, N, r, 64)) return LQLORA_ERR_CUDA;         // T' = dY L1
     PreParams p0, p1;
-    p0.partial = nullptr; p0.T = T; p0.counters = nullptr; p0.status = status;
+    p0.T = T; p0.status = status;
     p0.M = static_cast<int>(M); p0.r = r; p0.rp = g.rp; p0.steps = g.steps_x; p0.steps_per_split = g.sps_x; p0.stages = 0; p0.clear_status = 1;
     p1 = p0;
     p1.T = Tp; p1.steps = g.steps_y; p1.steps_per_split = g.sps_y; p1.clear_status = 0;

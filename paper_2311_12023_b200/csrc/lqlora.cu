@@ -233,9 +233,16 @@ int lqlora_linear_fwd_static(const lqlora_qmatrix* q, const void* L1_dev, const 
     void* scratch = nullptr;
     rc = static_scratch_ptr(&scratch);
     if (rc != LQLORA_OK) return rc;
-    // run_linear clears the status word and the arrival counters at the head of the scratch on every
-    // call, so whatever the previous call left behind is never read before it is overwritten
+    // the first kernel of the call (or run_linear's memset) clears the status word at the head of the scratch;
+    // nothing else of what the previous call left behind is read before it is overwritten
     return run_linear(q, L1_dev, L2_dev, r, X_dev, M, Y_dev, scratch, kStaticScratchBytes, stream, false);
+}
+
+int lqlora_static_scratch_status(void* stream) {
+    void* scratch = nullptr;
+    const int rc = lq::static_scratch_ptr(&scratch);
+    if (rc != LQLORA_OK) return rc;
+    return lqlora_workspace_status(scratch, stream);
 }
 
 static int check_lora_grads(int64_t N, int64_t K, int r, int64_t M) {
@@ -318,13 +325,26 @@ int lqlora_workspace_status(const void* workspace_dev, void* stream) {
     return word == 0 ? LQLORA_OK : LQLORA_ERR_TIMEOUT;
 }
 
-int lqlora_linear_path(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, int backward) {
+int lqlora_linear_path(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, int backward, int* splits) {
     using namespace lq;
     if (check_config(cfg) != LQLORA_OK || check_shape(N, K, cfg) != LQLORA_OK) return LQLORA_ERR_INVALID_CONFIG;
+    if (M <= 0 || r < 0 || r > 128 || r % 16) return LQLORA_ERR_INVALID_SHAPE;
     lqlora_qmatrix q{};
     q.N = N; q.K = K; q.cfg = *cfg;
     const QView v = make_view(&q);
-    return tc_supported(v, r, M, backward != 0) ? 1 : 0;
+    const bool bwd = backward != 0;
+    int kernel = LQLORA_PATH_PLAIN, ks = 1;
+    if (tc_supported(v, r, M, bwd)) {
+        const int64_t out_cols = bwd ? K : N;
+        const int steps_q = static_cast<int>(((bwd ? N : K) + tc::BK - 1) / tc::BK);
+        if (tc::tc_use_pair(M, out_cols, tc::sm_count())) kernel = LQLORA_PATH_TC_PAIR;
+        else { kernel = LQLORA_PATH_TC_ONE; ks = tc::tc_ksplit(M, out_cols, steps_q, tc::sm_count()); }
+    } else if (bwd ? dec::bwd_supported(v, M) : dec::supported(v, M)) {
+        kernel = LQLORA_PATH_STREAM;
+        ks = bwd ? dec::bwd_splits(v, static_cast<int>(M)) : dec::fwd_splits(v, static_cast<int>(M));
+    }
+    if (splits) *splits = ks;
+    return kernel;
 }
 
 }  // extern "C"

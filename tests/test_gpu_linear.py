@@ -12,9 +12,14 @@ pytestmark = pytest.mark.gpu
 C = inputs.QuantConfig
 
 
-def run_case(A, l1b, l2b, cfg, M, seed, rows=None, passes=("fwd", "bwd")):
+def run_case(A, l1b, l2b, cfg, M, seed, rows=None, passes=("fwd", "bwd"), route=None):
+    """Encodes A on both sides (bit-exact codec parity is asserted inside encode_both for every matrix that comes
+    through here), then compares Y and dX with the fp64 oracle.  route: expected kernel id of the forward dispatch."""
     N, K = A.shape
     q, ref = encode_both(A, cfg)
+    if route is not None:
+        r = 0 if l1b is None else l1b.shape[1]
+        assert binding.linear_path(N, K, cfg, r, M, False) == route
     L1 = binding.bf16_from_bits(l1b) if l1b is not None else None
     L2 = binding.bf16_from_bits(l2b) if l2b is not None else None
     out = {}
@@ -89,6 +94,8 @@ def test_linear_many_rows_few_tiles(N, K, M, b0, B0):
     tiles (grid.x > 1), split contraction, M, N, K not multiples of the tile."""
     A = inputs.gaussian(600 + N, (N, K), 0.02)
     l1b, l2b = inputs.lowrank_factors(601 + K, N, K, 64, 0.01)
+    kernel, splits = binding.linear_route(N, K, C(b0, B0, 8, 64, 32), 64, M, False)
+    assert kernel == binding.PATH_TC_ONE and splits > 1
     run_case(A, l1b, l2b, C(b0, B0, 8, 64, 32), M, seed=700 + M)
 
 
@@ -98,7 +105,8 @@ def test_linear_pair_kernel_ragged_tiles(N, K, M, b0, B0):
     """CTA-pair kernel (enough [512, 256] tiles to fill the SMs) with M, N, K that are not multiples of the pair tile:
     the second CTA of a pair may have few weight rows / columns, the TMA stores clip, and the contraction ends inside
     a 128-row tile.  Sampled rows (first, last, both sides of tile edges)."""
-    assert binding.linear_path(N, K, C(b0, B0, 8, 64, 32), 64, M, False) == 1
+    assert binding.linear_route(N, K, C(b0, B0, 8, 64, 32), 64, M, False) == (binding.PATH_TC_PAIR, 1)
+    assert binding.linear_path(N, K, C(b0, B0, 8, 64, 32), 64, M, True) == binding.PATH_TC_PAIR
     A = inputs.gaussian(650 + N, (N, K), 0.02)
     l1b, l2b = inputs.lowrank_factors(651 + K, N, K, 64, 0.01)
     rows = inputs.sample_rows(660 + M, M, count=24, tile=128)
@@ -154,7 +162,7 @@ def test_config1_forward():
     w = inputs.workload(1)
     spec = w["matrices"][0]
     A, l1b, l2b = inputs.make_matrix(spec)
-    run_case(A, l1b, l2b, spec.cfg, 512, seed=1100, passes=("fwd",))
+    run_case(A, l1b, l2b, spec.cfg, 512, seed=1100, passes=("fwd",), route=binding.PATH_TC_ONE)
 
 
 @pytest.mark.parametrize("M", [1, 16, 2048])
@@ -162,14 +170,14 @@ def test_config2_forward_and_backward(M):
     spec = inputs.workload(2)["matrices"][0]
     A, l1b, l2b = inputs.make_matrix(spec)
     rows = inputs.sample_rows(2100 + M, M) if M > 512 else None
-    run_case(A, l1b, l2b, spec.cfg, M, seed=2200 + M, rows=rows)
+    run_case(A, l1b, l2b, spec.cfg, M, seed=2200 + M, rows=rows, route=binding.PATH_TC_PAIR if M > 16 else binding.PATH_STREAM)
 
 
 def test_config3_down_projection_sampled_rows():
     spec = inputs.workload(3)["matrices"][2]          # 4096 x 11008
     A, l1b, l2b = inputs.make_matrix(spec)
     rows = inputs.sample_rows(3100, 4096, count=16)
-    run_case(A, l1b, l2b, spec.cfg, 4096, seed=3200, rows=rows)
+    run_case(A, l1b, l2b, spec.cfg, 4096, seed=3200, rows=rows, route=binding.PATH_TC_PAIR)
 
 
 def test_config4_kv_projection_mixed_config():
@@ -184,7 +192,14 @@ def test_config3_gate_projection_sampled_rows():
     spec = inputs.workload(3)["matrices"][0]          # 11008 x 4096, Student-t, NF4
     A, l1b, l2b = inputs.make_matrix(spec)
     rows = inputs.sample_rows(3300, 4096, count=16)
-    run_case(A, l1b, l2b, spec.cfg, 4096, seed=3400, rows=rows)
+    run_case(A, l1b, l2b, spec.cfg, 4096, seed=3400, rows=rows, route=binding.PATH_TC_PAIR)
+
+
+def test_config3_up_projection_sampled_rows():
+    spec = inputs.workload(3)["matrices"][1]          # 11008 x 4096, its own seed
+    A, l1b, l2b = inputs.make_matrix(spec)
+    rows = inputs.sample_rows(3500, 4096, count=8)
+    run_case(A, l1b, l2b, spec.cfg, 4096, seed=3600, rows=rows, route=binding.PATH_TC_PAIR)
 
 
 def test_config4_query_projection_mixed_config():
@@ -203,17 +218,29 @@ def test_config4_mlp_projections_largest_shapes(name, M):
     run_case(A, l1b, l2b, spec.cfg, M, seed=4800 + M, rows=rows)
 
 
-@pytest.mark.parametrize("b0,B0", [(2, 16), (4, 128), (8, 256)])
+@pytest.mark.parametrize("name", ["v", "o", "up"])
+def test_config4_remaining_matrices(name):
+    """The other matrices of the 70B layer with their drawn configurations: bit-exact codec parity at full size (inside
+    run_case) and the decode-sized forward and input gradient."""
+    spec = [s for s in inputs.workload(4)["matrices"] if s.name == name][0]
+    A, l1b, l2b = inputs.make_matrix(spec)
+    run_case(A, l1b, l2b, spec.cfg, 1, seed=4900, route=binding.PATH_STREAM)
+
+
+@pytest.mark.parametrize("b0,B0", [(2, 16), (3, 64), (4, 128), (8, 16), (8, 256)])
 def test_config5_sweep_points(b0, B0):
-    """Points of the 8192 x 8192 sweep at every kind of M: decode kernels, one-CTA and CTA-pair tensor-core kernels."""
+    """Points of the 8192 x 8192 sweep at every M of the sweep (decode kernels, one-CTA and CTA-pair tensor-core
+    kernels; 8192 rows = 16 x 32 pair tiles), whole-height bit-exact codec parity included (encode_both)."""
     A = inputs.gaussian(5000, (8192, 8192), 0.02)
     l1b, l2b = inputs.lowrank_factors(5700, 8192, 8192, 64, 0.01)
     cfg = C(b0, B0, 8, 256, 32)
     N, K = A.shape
     q, ref = encode_both(A, cfg)
     L1, L2 = binding.bf16_from_bits(l1b), binding.bf16_from_bits(l2b)
-    for M in (1, 16, 128, 2048):
+    for M in (1, 16, 128, 2048, 8192):
         rows = inputs.sample_rows(5100 + M, M, count=8) if M > 16 else None
+        want = binding.PATH_STREAM if M <= 16 else binding.PATH_TC_ONE if M == 128 else binding.PATH_TC_PAIR
+        assert binding.linear_path(N, K, cfg, 64, M, False) == want
         xb = inputs.activations(5200 + M, M, K)
         gb = inputs.activations(5300 + M, M, N)
         Y = binding.linear_fwd(q, L1, L2, binding.bf16_from_bits(xb))

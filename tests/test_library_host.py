@@ -122,12 +122,24 @@ def test_product_path_never_imports_the_oracle():
 
 
 def test_dispatch_between_the_weight_streaming_and_the_tensor_core_kernels(binding):
-    """lqlora_linear_path (host only): up to 16 rows stream the packed weights; from 17 rows the tensor cores take
-    over; the input gradient of 9..16 rows goes to the tensor cores too when the matrix has at least 2048 rows."""
+    """lqlora_linear_path (host only) names the kernel: up to 16 rows stream the packed weights; from 17 rows the
+    one-CTA tcgen05 kernel takes over (the input gradient of 9..16 rows too when the matrix has at least 2048 rows);
+    CTA pairs run once their [512, 256] tiles fill more than half of the SMs; shapes without 16-byte rows fall back
+    to the plain kernels."""
+    S, ONE, PAIR, PLAIN = binding.PATH_STREAM, binding.PATH_TC_ONE, binding.PATH_TC_PAIR, binding.PATH_PLAIN
     cfg = inputs.QuantConfig(3, 64, 8, 256, 32)
-    for M, want in ((1, 0), (16, 0), (17, 1), (256, 1), (2048, 1)):
+    for M, want in ((1, S), (16, S), (17, ONE), (256, ONE), (512, ONE), (2048, PAIR)):
         assert binding.linear_path(4096, 4096, cfg, 64, M, False) == want
-    for M, want in ((1, 0), (8, 0), (9, 1), (16, 1), (17, 1)):
+    for M, want in ((1, S), (8, S), (9, ONE), (16, ONE), (17, ONE), (8192, PAIR)):
         assert binding.linear_path(4096, 4096, cfg, 64, M, True) == want
-    for M, want in ((8, 0), (9, 0), (16, 0), (17, 1)):
+    for M, want in ((8, S), (9, S), (16, S), (17, ONE)):
         assert binding.linear_path(1024, 8192, cfg, 64, M, True) == want
+    odd = inputs.QuantConfig(4, 64, 8, 16, 32)          # 201 rows: the rows of dY do not start on 16-byte boundaries
+    assert binding.linear_path(201, 192, odd, 16, 1, False) == S and binding.linear_path(201, 192, odd, 16, 1, True) == PLAIN
+    # the contraction of an output tile is shared by a cluster where few tiles would leave SMs idle
+    kernel, splits = binding.linear_route(8192, 8192, cfg, 64, 128, False)
+    assert kernel == ONE and 2 <= splits <= 8
+    kernel, splits = binding.linear_route(8192, 8192, cfg, 64, 2048, False)
+    assert kernel == PAIR and splits == 1
+    kernel, splits = binding.linear_route(4096, 4096, cfg, 64, 1, False)
+    assert kernel == S and 1 <= splits <= 8

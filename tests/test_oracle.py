@@ -269,6 +269,39 @@ def test_dequant_elementwise_definition():
         assert d16.reshape(-1)[idx] == inputs.f32_to_bf16_bits(np.array([w]))[0]
 
 
+def test_dequant_bf16_rounding_ties_go_to_even():
+    """The cast to bf16 (App. A) is round-to-nearest-even.  Constructed ties, with hand-written expected bit patterns:
+    scale code 1 and v = 127 t make s~ = fl32(v / 127) = t exactly; the top code (q = +1) and the bottom code
+    (q = -1) then dequantize to +-t.  t = 1 + 2^-8 lies half way between the bf16 values 1 (0x3F80, even mantissa)
+    and 1 + 2^-7 (0x3F81); t = 1 + 3 * 2^-8 half way between 0x3F81 and 0x3F82 (even).  One ulp of fp32 above or
+    below a tie must leave the tie (nearest wins)."""
+    b0, B0, B1 = 3, 16, 16
+    top, bottom = 7, 0
+    cases = [
+        (1.0 + 2.0 ** -8, 0x3F80), (1.0 + 3 * 2.0 ** -8, 0x3F82),
+        (0.5 + 2.0 ** -9, 0x3F00), (0.5 + 3 * 2.0 ** -9, 0x3F02),
+    ]
+    for t, want in cases:
+        v = np.array([127.0 * t], dtype=np.float32)
+        assert float(v[0]) == 127.0 * t                  # exactly representable
+        codes = np.full((1, B0), top, dtype=np.uint8)
+        codes[0, 1] = bottom
+        sc = np.array([1], dtype=np.uint8)
+        d32, d16 = oracle.dequant(codes, sc, v, b0, B0, 8, B1)
+        assert float(d32[0, 0]) == t and float(d32[0, 1]) == -t
+        assert d16[0, 0] == want and d16[0, 1] == (want | 0x8000)
+    # just off the tie: the nearer neighbour
+    t = np.float32(1.0 + 2.0 ** -8)
+    for tt, want in ((np.nextafter(t, np.float32(2)), 0x3F81), (np.nextafter(t, np.float32(0)), 0x3F80)):
+        # s~ = fl32(1 * fl32(v / 127)): pick v by search so that the quotient is tt
+        v = np.array([np.float32(127) * tt], dtype=np.float32)
+        if np.float32(v[0] / np.float32(127)) != tt:
+            continue
+        codes = np.full((1, B0), top, dtype=np.uint8)
+        d32, d16 = oracle.dequant(codes, np.array([1], dtype=np.uint8), v, b0, B0, 8, B1)
+        assert d32[0, 0] == tt and d16[0, 0] == want
+
+
 # --------------------------------------------------------------------------- layer
 def _layer_case(seed, N, K, M, r):
     W = inputs.gaussian(seed, (N, K), 0.02)
