@@ -1,28 +1,35 @@
 #!/usr/bin/env python
 """Benchmark of the LQ-LoRA linear hot path on B200.
 
-One step = one pass of the whole hot path on the LLaMA-2-7B attention-projection workload
-(4096x4096, NF3, B0 = 64, B1 = 256, rank 64; seeded synthetic data):
+One step = one pass of the whole hot path over the LLaMA-2-70B decoder-layer workload (seeded synthetic
+data: q, o 8192x8192; k, v 1024x8192; gate, up 28672x8192; down 8192x28672; per-matrix mixed
+configurations averaging about 2.73 bits per parameter; rank 64):
 
-    encode(R)  ->  forward + input gradient at M = 2048 (training, tensor-core kernels)
-               ->  forward + input gradient at M = 16 and M = 1 (decode, weight-streaming kernels)
+    encode of all seven matrices
+    -> forward of all seven at M = 2048, input gradient of all seven at M = 2048   (tensor-core kernels)
+    -> forward of all seven at M = 1,    input gradient of all seven at M = 1      (weight-streaming kernels)
 
-`value` is the algorithmic TFLOP/s of the whole step: 2 M (N K + r K + N r) flop per linear
-call, summed over the six calls, divided by the device time of the step (CUDA events).  The
-JSON line also carries the per-phase figures (tensor TFLOP/s at M = 2048, packed-weight GB/s
-at M = 1 / 16, encode GB/s), the roofline of the dominant kernel, the end-to-end number
-through the host-buffer C ABI, and the CPU oracle timed on the host as a baseline.
+`value` is the algorithmic TFLOP/s of the whole step: 2 M (N K + r K + N r) flop per linear call, summed
+over the 28 calls, divided by the device time of the step (CUDA events).  The JSON line also carries the
+roofline of the dominant kernel (the CTA-pair tcgen05 kernel on the 28672x8192 gate projection), per-call
+figures of the step, the other seeded workloads (RoBERTa projection, LLaMA-2-7B attention projection and MLP
+block, points of the 8192x8192 sweep) measured beside it, the end-to-end number through the host-buffer
+C ABI, and the CPU oracle timed on the host as a baseline.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py --sweep                      # the whole b0 x B0 x M table of the 8192x8192 sweep
+    python bench.py --case gate --case-m 2048    # one matrix of the layer alone (small footprint, for profilers)
 
-With N > 1 (torchrun) every rank runs the same per-GPU workload on its own tokens (data
-parallel over tokens, no collective on the data path); time is the max over ranks.
+With N > 1 every rank runs the same per-GPU workload on its own tokens (data parallel over tokens, weights
+replicated, no collective on the data path); time is the max over ranks.  Launched by torchrun the ranks
+read RANK / LOCAL_RANK / WORLD_SIZE; without them `--gpus N` starts the N ranks itself.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -38,14 +45,15 @@ if ROOT not in sys.path:
 from paper_2311_12023_b200 import inputs  # noqa: E402
 
 METRIC = "LQ-LoRA linear fwd/bwd TFLOP/s & packed-weight GB/s, % of B200 roofline"
-WORKLOAD = "llama2-7b attn-proj 4096x4096 NF3 B0=64 B1=256 r=64; encode + fwd/dX at M=2048,16,1"
-MS = (2048, 16, 1)
+WORKLOAD = ("llama2-70b decoder layer (GQA): q,o 8192x8192; k,v 1024x8192; gate,up 28672x8192; down 8192x28672; "
+            "per-matrix mixed configs (about 2.73 bits/param), r=64; encode of all seven + fwd/dX of all seven at M=2048 and M=1")
+MS = (2048, 1)
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 FALLBACK = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per forward launch of tc_pair_linear_kernel<3, 0> at M = 2048 on this
-# workload (profiles/kernels_c2_4096_nf3_ncu_full.txt): the operands are read once (X 16.8 MB + packed 6.6 MB +
-# factors), the output stays in L2 during the capture
-TC_TRAFFIC_BYTES = 24289024
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (forward of the gate projection at
+# M = 2048), from an ncu capture of `python bench.py --case gate --case-m 2048`; None while no capture of the current
+# kernel exists.
+DOMINANT_TRAFFIC_BYTES = None
 
 
 def linear_flops(M: int, N: int, K: int, r: int) -> float:
@@ -104,7 +112,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
@@ -113,36 +121,43 @@ class ClockSampler:
             try:
                 sm.append(float(f[1]))
                 mx.append(float(f[2]))
+                pw.append(float(f[3]))
             except ValueError:
                 continue
             for nm, val in zip(names, f[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(nm)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "sm_mhz_min": min(sm) if sm else None, "power_w_max": max(pw) if pw else None,
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
 # ------------------------------------------------------------------------------------- reference arm
-def oracle_sample(spec, A, l1b, l2b, rows_large: int = 24):
-    """Times the CPU oracle on a bounded sample of the step; returns (flops_done, seconds, description)."""
+def oracle_sample(names, rows_large: int):
+    """Times the CPU oracle on a bounded sample of the layer workload: the named matrices are encoded and dequantized
+    in full, then forward and input gradient run in fp64 on `rows_large` sampled rows of M = 2048 and on the M = 1 row.
+    Returns (flops_done, seconds, description)."""
     import oracle
-    cfg = spec.cfg
-    N, K, r = spec.N, spec.K, inputs.RANK
-    t0 = time.perf_counter()
-    codes, _, sc, v = oracle.encode(A, cfg.b0, cfg.B0, cfg.b1, cfg.B1)
-    d32, _ = oracle.dequant(codes, sc, v, cfg.b0, cfg.B0, cfg.b1, cfg.B1)
+    specs = [s for s in inputs.workload(4)["matrices"] if s.name in names]
+    mats = [(s,) + tuple(inputs.make_matrix(s)) for s in specs]          # generation is not timed
+    r = inputs.RANK
     flops = 0.0
-    for M in MS:
-        rows = inputs.sample_rows(900 + M, M, count=rows_large) if M > rows_large else None
-        nrows = M if rows is None else len(rows)
-        xb = inputs.activations(910 + M, M, K)
-        gb = inputs.activations(920 + M, M, N)
-        oracle.linear_fwd(d32, l1b, l2b, xb, rows)
-        oracle.linear_bwd_input(d32, l1b, l2b, gb, rows)
-        flops += 2 * linear_flops(nrows, N, K, r)
+    t0 = time.perf_counter()
+    for spec, A, l1b, l2b in mats:
+        cfg = spec.cfg
+        codes, _, sc, v = oracle.encode(A, cfg.b0, cfg.B0, cfg.b1, cfg.B1)
+        d32, _ = oracle.dequant(codes, sc, v, cfg.b0, cfg.B0, cfg.b1, cfg.B1)
+        for M in MS:
+            rows = inputs.sample_rows(900 + M, M, count=rows_large) if M > rows_large else None
+            nrows = M if rows is None else len(rows)
+            xb = inputs.activations(910 + M, M, spec.K)
+            gb = inputs.activations(920 + M, M, spec.N)
+            oracle.linear_fwd(d32, l1b, l2b, xb, rows)
+            oracle.linear_bwd_input(d32, l1b, l2b, gb, rows)
+            flops += 2 * linear_flops(nrows, spec.N, spec.K, r)
     dt = time.perf_counter() - t0
-    desc = (f"encode+dequant of the full {N}x{K} matrix, then fwd and dX in fp64 on {rows_large} sampled rows "
-            f"of M=2048 and all rows of M=16 and M=1")
+    desc = (f"matrices {'+'.join(names)} of the layer: encode+dequant in full, then fwd and dX in fp64 on {rows_large} sampled "
+            f"rows of M=2048 and on the M=1 row (input generation untimed)")
     return flops, dt, desc
 
 
@@ -151,13 +166,11 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    spec = inputs.workload(2)["matrices"][0]
-    A, l1b, l2b = inputs.make_matrix(spec)
     for _ in range(max(0, min(args.warmup, 1))):
-        oracle_sample(spec, A, l1b, l2b, rows_large=4)
-    times, flops = [], 0.0
+        oracle_sample(("k",), rows_large=4)
+    times, flops, desc = [], 0.0, ""
     for _ in range(args.steps):
-        flops, dt, desc = oracle_sample(spec, A, l1b, l2b, rows_large=64)
+        flops, dt, desc = oracle_sample(("k",), rows_large=64)
         times.append(dt)
     mean = sum(times) / len(times)
     val = flops / mean / 1e12
@@ -173,7 +186,7 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
-# ------------------------------------------------------------------------------------- device arm
+# ------------------------------------------------------------------------------------- ranks
 def shard_info():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -192,6 +205,186 @@ def reduce_max(value: float, world: int, device=None) -> float:
     return float(t.item())
 
 
+def spawn_ranks(n: int, argv) -> int:
+    """`--gpus N` without a launcher: starts N copies of this script, one per GPU, with RANK / LOCAL_RANK /
+    WORLD_SIZE / MASTER_ADDR / MASTER_PORT set, and waits for them.  Rank 0's output is this process's output."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for rank in range(n):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + list(argv), env=env,
+                                      stdout=None if rank == 0 else subprocess.DEVNULL))
+    rc = 0
+    for p in procs:
+        p.wait()
+        rc = rc or p.returncode
+    return rc
+
+
+def run_dry(args):
+    """Host logic of the multi-rank path without a device (used by the CPU tests): rendezvous over gloo, barrier,
+    max over ranks of a per-rank step time, and the one JSON line from rank 0.  No kernel runs and no throughput is
+    claimed: `value` is null."""
+    import torch.distributed as dist
+    rank, world, local = shard_info()
+    if world > 1:
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+        dist.barrier()
+    ms = reduce_max(10.0 + 5.0 * rank, world)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": None, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+                          "warmup": args.warmup, "ms_per_step": ms, "dry_run": True, "scaling": "weak",
+                          "config": {"workload": WORKLOAD}}), flush=True)
+
+
+# ------------------------------------------------------------------------------------- device helpers
+class Timer:
+    def __init__(self, torch):
+        self.torch = torch
+
+    def __call__(self, fn, count):
+        """ms per call of `fn()` (which issues `count` calls), after one untimed run."""
+        torch = self.torch
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / count
+
+
+def time_linear(binding, torch, q, L1, L2, A, M, bwd, l2_bytes, timer):
+    """ms per call of one direction of the linear at M rows.  M <= 16: the calls run over cold copies of the packed
+    matrix (together more than twice the L2) replayed as one CUDA graph; larger M: back to back over rotating
+    activation and output buffers (together larger than L2)."""
+    dev = A.device
+    N, K, r = q.N, q.K, (0 if L1 is None else L1.shape[1])
+    fn = binding.linear_bwd_input if bwd else binding.linear_fwd
+    ws = binding.alloc_workspace(q, r, M)
+    out_cols = K if bwd else N
+    if M <= 16:
+        ncopies = max(2, int(2.2 * l2_bytes / q.packed_bytes) + 1)
+        copies = [q] + [binding.QMatrix(q.codes.clone(), q.scale_codes.clone(), q.scale2.clone(), N, K, q.cfg) for _ in range(ncopies - 1)]
+        out = torch.empty((M, out_cols), dtype=torch.bfloat16, device=dev)
+
+        def body():
+            for c in copies:
+                fn(c, L1, L2, A, out=out, workspace=ws)
+        body()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            body()
+        ms = timer(g.replay, ncopies)
+        how = f"cuda graph over {ncopies} cold copies"
+    else:
+        per = M * (N + K) * 2
+        nrot = min(8, max(2, int(1.1 * l2_bytes / per) + 1))
+        As = [A] + [A.clone() for _ in range(nrot - 1)]
+        outs = [torch.empty((M, out_cols), dtype=torch.bfloat16, device=dev) for _ in range(nrot)]
+        reps = max(2, min(4 * nrot, 16))
+        ms = timer(lambda: [fn(q, L1, L2, As[i % nrot], out=outs[i % nrot], workspace=ws) for i in range(reps)], reps)
+        how = f"back to back over {nrot} rotating activation buffers"
+    if binding.workspace_status(ws) != 0:
+        raise SystemExit("a linear kernel reported a device-side error")
+    return ms, how
+
+
+def linear_entry(ms, M, N, K, r, cfg, pk, pk_kind, how=None):
+    """Figures of one linear call: tensor roofline for M > 16, HBM roofline on packed-weight bytes for M <= 16."""
+    ent = {"ms": ms, "TFLOP/s": linear_flops(M, N, K, r) / ms / 1e9}
+    if M > 16:
+        ent["frac_of_bf16_" + pk_kind] = ent["TFLOP/s"] / pk["bf16_tflops"]
+        ent["frac_of_bf16_nominal"] = ent["TFLOP/s"] / NOMINAL["bf16_tflops"]
+    else:
+        pb = packed_bytes(N, K, cfg)
+        ent["packed_GB/s"] = pb / ms / 1e6
+        ent["frac_of_hbm_" + pk_kind] = ent["packed_GB/s"] / pk["hbm_gbs"]
+        ent["frac_of_hbm_nominal"] = ent["packed_GB/s"] / NOMINAL["hbm_gbs"]
+    if how:
+        ent["how"] = how
+    return ent
+
+
+def measure_matrix(binding, torch, dev, A, l1b, l2b, cfg, Ms, passes, pk, pk_kind, l2_bytes, timer, seed=0):
+    """Encode GB/s and per-M forward / input-gradient figures of one matrix (outside the timed step)."""
+    N, K = A.shape
+    r = l1b.shape[1]
+    W = torch.from_numpy(A).to(dev)
+    L1, L2 = binding.bf16_from_bits(l1b, dev), binding.bf16_from_bits(l2b, dev)
+    q = binding.alloc_qmatrix(N, K, cfg, dev)
+    enc_ws = torch.empty(binding.packed_sizes(N, K, cfg)[3], dtype=torch.uint8, device=dev)
+    out = {"shape": [N, K], "quant": list(cfg.as_tuple())}
+    enc_ms = timer(lambda: [binding.encode(W, cfg, out=q, workspace=enc_ws) for _ in range(3)], 3)
+    gbs = encode_bytes(N, K, cfg) / enc_ms / 1e6
+    out["encode"] = {"ms": enc_ms, "GB/s": gbs, "frac_of_hbm_" + pk_kind: gbs / pk["hbm_gbs"]}
+    del W
+    for M in Ms:
+        X = binding.bf16_from_bits(inputs.activations(8000 + seed + M, M, K), dev)
+        G = binding.bf16_from_bits(inputs.activations(8500 + seed + M, M, N), dev)
+        for ps in passes:
+            if ps not in ("fwd", "bwd"):
+                continue
+            ms, how = time_linear(binding, torch, q, L1, L2, G if ps == "bwd" else X, M, ps == "bwd", l2_bytes, timer)
+            out[f"{ps}_M{M}"] = linear_entry(ms, M, N, K, r, cfg, pk, pk_kind, how)
+        del X, G
+    return out
+
+
+# ------------------------------------------------------------------------------------- device arm
+class Mat:
+    pass
+
+
+def build_layer(binding, torch, dev, rank, host_copy):
+    """Device-resident state of the seven matrices of the layer (weights replicated on every rank; every rank draws
+    its own tokens)."""
+    mats = []
+    r = inputs.RANK
+    for spec in inputs.workload(4)["matrices"]:
+        m = Mat()
+        m.spec, m.cfg, m.N, m.K = spec, spec.cfg, spec.N, spec.K
+        A, l1b, l2b = inputs.make_matrix(spec)
+        m.W_host = torch.from_numpy(A).pin_memory() if host_copy else None
+        m.W = torch.from_numpy(A).to(dev)
+        del A
+        m.L1, m.L2 = binding.bf16_from_bits(l1b, dev), binding.bf16_from_bits(l2b, dev)
+        m.q = binding.alloc_qmatrix(m.N, m.K, m.cfg, dev)
+        m.enc_ws = torch.empty(binding.packed_sizes(m.N, m.K, m.cfg)[3], dtype=torch.uint8, device=dev)
+        m.ws = {M: binding.alloc_workspace(m.q, r, M) for M in MS}
+        mats.append(m)
+    # activations: q, k, v read the same input, gate and up read the same input (as in the layer); every matrix has its
+    # own output gradient
+    groups = {"q": "attn_in", "k": "attn_in", "v": "attn_in", "o": "o_in", "gate": "mlp_in", "up": "mlp_in", "down": "down_in"}
+    XH, X = {}, {}
+    for m in mats:
+        m.X, m.XH, m.G, m.GH, m.Y, m.DX, m.YH, m.DXH = {}, {}, {}, {}, {}, {}, {}, {}
+        for M in MS:
+            key = (groups[m.spec.name], M)
+            if key not in X:
+                h = torch.from_numpy(inputs.activations(7000 + 10 * rank + M + 100 * len(X), M, m.K).view(np.int16)).view(torch.bfloat16)
+                XH[key] = h.pin_memory() if host_copy else h
+                X[key] = XH[key].to(dev)
+            m.X[M], m.XH[M] = X[key], XH[key]
+            g = torch.from_numpy(inputs.activations(7500 + 10 * rank + M + 100 * mats.index(m), M, m.N).view(np.int16)).view(torch.bfloat16)
+            m.GH[M] = g.pin_memory() if host_copy else g
+            m.G[M] = m.GH[M].to(dev)
+            m.Y[M] = torch.empty((M, m.N), dtype=torch.bfloat16, device=dev)
+            m.DX[M] = torch.empty((M, m.K), dtype=torch.bfloat16, device=dev)
+            if host_copy:
+                m.YH[M] = torch.empty((M, m.N), dtype=torch.bfloat16).pin_memory()
+                m.DXH[M] = torch.empty((M, m.K), dtype=torch.bfloat16).pin_memory()
+    return mats
+
+
 def run_device(args):
     import torch
     from paper_2311_12023_b200 import binding
@@ -205,81 +398,47 @@ def run_device(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     binding.lib()
+    timer = Timer(torch)
+    pk, pk_kind = peaks()
+    r = inputs.RANK
+    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
 
-    spec = inputs.workload(2)["matrices"][0]
-    cfg, N, K, r = spec.cfg, spec.N, spec.K, inputs.RANK
-    # every rank draws its own tokens (seed offset by rank); the weights are replicated
-    A, l1b, l2b = inputs.make_matrix(spec)
-    W_host = torch.from_numpy(A).pin_memory()
-    W = W_host.to(dev)
-    L1, L2 = binding.bf16_from_bits(l1b, dev), binding.bf16_from_bits(l2b, dev)
-    q = binding.alloc_qmatrix(N, K, cfg, dev)
-    enc_ws = torch.empty(binding.packed_sizes(N, K, cfg)[3], dtype=torch.uint8, device=dev)
-    binding.encode(W, cfg, out=q, workspace=enc_ws)
+    mats = build_layer(binding, torch, dev, rank, host_copy=True)
+    for m in mats:
+        binding.encode(m.W, m.cfg, out=m.q, workspace=m.enc_ws)
     torch.cuda.synchronize()
 
-    # cold copies of the packed matrix for the decode-sized calls: more than twice the L2 in total
-    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
-    ncopies = max(4, int(2.2 * l2_bytes / q.packed_bytes) + 1)
-    copies = [binding.QMatrix(q.codes.clone(), q.scale_codes.clone(), q.scale2.clone(), N, K, cfg) for _ in range(ncopies)]
-
-    X, G, Y, DX, WS, XH, GH, YH, DXH = {}, {}, {}, {}, {}, {}, {}, {}, {}
+    # the calls of one step, in layer order: (label, kind, matrix, M, callable)
+    calls = []
+    for m in mats:
+        calls.append((f"encode_{m.spec.name}", "encode", m, 0, lambda m=m: binding.encode(m.W, m.cfg, out=m.q, workspace=m.enc_ws)))
     for M in MS:
-        XH[M] = torch.from_numpy(inputs.activations(7000 + 10 * rank + M, M, K).view(np.int16)).view(torch.bfloat16).pin_memory()
-        GH[M] = torch.from_numpy(inputs.activations(7500 + 10 * rank + M, M, N).view(np.int16)).view(torch.bfloat16).pin_memory()
-        X[M], G[M] = XH[M].to(dev), GH[M].to(dev)
-        Y[M] = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
-        DX[M] = torch.empty((M, K), dtype=torch.bfloat16, device=dev)
-        YH[M] = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
-        DXH[M] = torch.empty((M, K), dtype=torch.bfloat16).pin_memory()
-        WS[M] = binding.alloc_workspace(q, r, M)
-    flush = torch.empty(max(256 << 20, 2 * l2_bytes), dtype=torch.uint8, device=dev)
-    flush_rd = torch.zeros(max(256 << 20, 2 * l2_bytes) // 4, dtype=torch.int32, device=dev)
+        for m in mats:
+            calls.append((f"fwd{M}_{m.spec.name}", "fwd", m, M,
+                          lambda m=m, M=M: binding.linear_fwd(m.q, m.L1, m.L2, m.X[M], out=m.Y[M], workspace=m.ws[M])))
+        for m in reversed(mats):
+            calls.append((f"bwd{M}_{m.spec.name}", "bwd", m, M,
+                          lambda m=m, M=M: binding.linear_bwd_input(m.q, m.L1, m.L2, m.G[M], out=m.DX[M], workspace=m.ws[M])))
+    ncalls = len(calls)
 
-    def flush_l2(v):
-        """Evicts L2: writes a buffer larger than L2, then reads another one so that the lines left behind are clean
-        (otherwise the first timed kernel also pays for writing the flush buffer back to HBM)."""
-        flush.fill_(v)
-        return flush_rd.max()
-
-
-    seg_names = ["encode"] + [f"{p}{M}" for M in MS for p in ("fwd", "bwd")]
-    nseg = len(seg_names)
-    copy_idx = [0]
-
-    def next_copy():
-        c = copies[copy_idx[0] % ncopies]
-        copy_idx[0] += 1
-        return c
-
-    def one_step(events=None, inner=True):
-        """The whole hot path once, device-resident inputs.  events: list of nseg+1 CUDA events; with inner=False only
-        the first and the last are recorded (the timed steps: no event records between the calls)."""
-        def mark(i):
-            if events and (inner or i == 0 or i == nseg):
-                events[i].record()
-        mark(0)
-        binding.encode(W, cfg, out=q, workspace=enc_ws)
-        i = 1
-        mark(i)
-        for M in MS:
-            qq = q if M > 64 else next_copy()
-            binding.linear_fwd(qq, L1, L2, X[M], out=Y[M], workspace=WS[M])
-            i += 1
-            mark(i)
-            qq = q if M > 64 else next_copy()
-            binding.linear_bwd_input(qq, L1, L2, G[M], out=DX[M], workspace=WS[M])
-            i += 1
-            mark(i)
+    def one_step(events=None):
+        """The whole hot path once, device-resident inputs; one CUDA event after every call."""
+        if events:
+            events[0].record()
+        for i, c in enumerate(calls):
+            c[4]()
+            if events:
+                events[i + 1].record()
 
     def one_step_host():
         """Same step through the host-buffer C ABI: H2D of W, X, dY and D2H of Y, dX inside."""
-        binding.encode_host(W_host, W, q, enc_ws)
+        for m in mats:
+            binding.encode_host(m.W_host, m.W, m.q, m.enc_ws)
         for M in MS:
-            qq = q if M > 64 else next_copy()
-            binding.linear_fwd_host(qq, L1, L2, XH[M], YH[M], X[M], Y[M], WS[M])
-            qq = q if M > 64 else next_copy()
-            binding.linear_bwd_input_host(qq, L1, L2, GH[M], DXH[M], G[M], DX[M], WS[M])
+            for m in mats:
+                binding.linear_fwd_host(m.q, m.L1, m.L2, m.XH[M], m.YH[M], m.X[M], m.Y[M], m.ws[M])
+            for m in reversed(mats):
+                binding.linear_bwd_input_host(m.q, m.L1, m.L2, m.GH[M], m.DXH[M], m.G[M], m.DX[M], m.ws[M])
 
     def barrier():
         if world > 1:
@@ -288,126 +447,40 @@ def run_device(args):
         torch.cuda.synchronize()
 
     for _ in range(args.warmup):
-        flush_l2(1)
         one_step()
     torch.cuda.synchronize()
-    for M in MS:
-        st = binding.workspace_status(WS[M])
-        if st != 0:
-            raise SystemExit(f"kernel reported {binding.status_string(st)}")
+    for m in mats:
+        for M in MS:
+            st = binding.workspace_status(m.ws[M])
+            if st != 0:
+                raise SystemExit(f"kernel reported {binding.status_string(st)}")
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nseg + 1)] for _ in range(args.steps)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(ncalls + 1)] for _ in range(args.steps)]
     launches0 = binding.launch_count()
     barrier()
     t_wall0 = time.perf_counter()
     for s in range(args.steps):
-        flush_l2(s & 0xFF)             # evict L2 between steps (untimed: outside the step's events)
-        one_step(evs[s], inner=False)
+        one_step(evs[s])
     barrier()
     t_wall = time.perf_counter() - t_wall0
     launches = binding.launch_count() - launches0
-    step_ms = [evs[s][0].elapsed_time(evs[s][nseg]) for s in range(args.steps)]
-    # per-call breakdown: the same steps once more with an event after every call (these records perturb the step a
-    # little, so they are kept out of the timed steps above)
+    step_ms = [evs[s][0].elapsed_time(evs[s][ncalls]) for s in range(args.steps)]
+    call_ms = np.zeros((args.steps, ncalls))
     for s in range(args.steps):
-        flush_l2(s & 0xFF)
-        one_step(evs[s], inner=True)
-    torch.cuda.synchronize()
-    seg_ms = np.zeros(nseg)
-    for s in range(args.steps):
-        for i in range(nseg):
-            seg_ms[i] += evs[s][i].elapsed_time(evs[s][i + 1])
-    seg_ms /= args.steps
+        for i in range(ncalls):
+            call_ms[s, i] = evs[s][i].elapsed_time(evs[s][i + 1])
     ms_step = reduce_max(sum(step_ms) / len(step_ms), world, dev)
 
-    # ---- back-to-back loops (no host gaps between launches): the tensor-core call over rotating activation
-    # buffers (together larger than L2), the decode-sized calls over the cold copies as one CUDA graph
-    loops = {}
-    nrot = max(2, int(1.1 * l2_bytes / (2048 * (N + K) * 2)) + 1)
-    Xr = [X[2048].clone() for _ in range(nrot)]
-    Gr = [G[2048].clone() for _ in range(nrot)]
-    Yr = [torch.empty_like(Y[2048]) for _ in range(nrot)]
-    DXr = [torch.empty_like(DX[2048]) for _ in range(nrot)]
-    reps = 4 * nrot
-
-    def timed(fn, count):
-        fn()
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        fn()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / count
-
-    def tc_fwd_loop():
-        for i in range(reps):
-            binding.linear_fwd(q, L1, L2, Xr[i % nrot], out=Yr[i % nrot], workspace=WS[2048])
-
-    def tc_bwd_loop():
-        for i in range(reps):
-            binding.linear_bwd_input(q, L1, L2, Gr[i % nrot], out=DXr[i % nrot], workspace=WS[2048])
-
-    loops["fwd2048"] = timed(tc_fwd_loop, reps)
-    loops["bwd2048"] = timed(tc_bwd_loop, reps)
-
-    def graph_loop(call, M):
-        """ms per call of `ncopies` calls replayed as one CUDA graph (falls back to a plain loop)."""
-        def body():
-            for c in copies:
-                call(c, M)
-        try:
-            side = torch.cuda.Stream()
-            side.wait_stream(torch.cuda.current_stream())
-            with torch.cuda.stream(side):
-                body()
-            torch.cuda.current_stream().wait_stream(side)
-            torch.cuda.synchronize()
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
-                body()
-            return timed(g.replay, ncopies), "cuda graph"
-        except Exception:
-            torch.cuda.synchronize()
-            return timed(body, ncopies), "stream loop"
-
-    loop_kind = {}
-    for M in (16, 1):
-        loops[f"fwd{M}"], loop_kind[f"fwd{M}"] = graph_loop(lambda c, m: binding.linear_fwd(c, L1, L2, X[m], out=Y[m], workspace=WS[m]), M)
-        loops[f"bwd{M}"], loop_kind[f"bwd{M}"] = graph_loop(lambda c, m: binding.linear_bwd_input(c, L1, L2, G[m], out=DX[m], workspace=WS[m]), M)
-    # gradients of the low-rank factors at M = 2048 (the next piece of a training step; not part of the timed step):
-    # rotating activation buffers, replayed as one CUDA graph
-    dL = (torch.empty(N, r, dtype=torch.float32, device=dev), torch.empty(r, K, dtype=torch.float32, device=dev))
-    gws = torch.empty(binding.lora_grads_workspace_bytes(N, K, r, 2048), dtype=torch.uint8, device=dev)
-
-    def grads_body():
-        for i in range(reps):
-            binding.lora_grads(L1, L2, Xr[i % nrot], Gr[i % nrot], out=dL, workspace=gws)
-    try:
-        grads_body()
-        torch.cuda.synchronize()
-        gg = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(gg):
-            grads_body()
-        loops["grads2048"], loop_kind["grads2048"] = timed(gg.replay, reps), "cuda graph"
-    except Exception:
-        torch.cuda.synchronize()
-        loops["grads2048"], loop_kind["grads2048"] = timed(grads_body, reps), "stream loop"
-    if binding.workspace_status(gws) != 0:
-        raise SystemExit("lora_grads reported a device-side error")
-    for k in list(loops):
-        loops[k] = reduce_max(loops[k], world, dev)
-
     # end to end through the host-buffer entry points
-    for _ in range(max(1, min(args.warmup, 3))):
+    for _ in range(2):
         one_step_host()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e2e_steps = max(3, min(args.steps, 10))
+    e2e_steps = max(3, min(args.steps, 5))
     e0.record()
     for _ in range(e2e_steps):
         one_step_host()
@@ -422,85 +495,172 @@ def run_device(args):
             dist.destroy_process_group()
         return
 
-    step_flops = sum(2 * linear_flops(M, N, K, r) for M in MS)
+    # ---- the step, call by call (mean over the timed steps of the event intervals)
+    mean_ms = call_ms.mean(axis=0)
+    step_flops = sum(linear_flops(M, m.N, m.K, r) for (_, kind, m, M, _) in calls if kind != "encode")
     value = world * step_flops / (ms_step * 1e-3) / 1e12
-    pk, pk_kind = peaks()
-    seg = dict(zip(seg_names, seg_ms.tolist()))
-    pbytes = packed_bytes(N, K, cfg)
-    small_bytes = pbytes + 2 * r * (N + K)
-    breakdown = {
-        "encode": {"ms": seg["encode"], "GB/s": encode_bytes(N, K, cfg) / seg["encode"] / 1e6,
-                   "frac_of_hbm_" + pk_kind: encode_bytes(N, K, cfg) / seg["encode"] / 1e6 / pk["hbm_gbs"]},
-    }
-    for M in MS:
-        for ps in ("fwd", "bwd"):
-            ms = seg[f"{ps}{M}"]
-            ent = {"ms": ms, "TFLOP/s": linear_flops(M, N, K, r) / ms / 1e9}
-            if M > 64:
+    layer = {}
+    for i, (label, kind, m, M, _) in enumerate(calls):
+        if kind == "encode":
+            gbs = encode_bytes(m.N, m.K, m.cfg) / mean_ms[i] / 1e6
+            layer[label] = {"ms": float(mean_ms[i]), "GB/s": gbs, "frac_of_hbm_" + pk_kind: gbs / pk["hbm_gbs"],
+                            "shape": [m.N, m.K], "quant": list(m.cfg.as_tuple())}
+        else:
+            layer[label] = linear_entry(float(mean_ms[i]), M, m.N, m.K, r, m.cfg, pk, pk_kind)
+    phases = {}
+    for ph in ("encode",) + tuple(f"{k}{M}" for M in MS for k in ("fwd", "bwd")):
+        idx = [i for i, c in enumerate(calls) if c[0].startswith(ph + "_")]
+        ms = float(mean_ms[idx].sum())
+        ent = {"ms": ms}
+        if ph == "encode":
+            b = sum(encode_bytes(m.N, m.K, m.cfg) for m in mats)
+            ent["GB/s"] = b / ms / 1e6
+            ent["frac_of_hbm_" + pk_kind] = ent["GB/s"] / pk["hbm_gbs"]
+        else:
+            M = int(ph[3:])
+            fl = sum(linear_flops(M, m.N, m.K, r) for m in mats)
+            ent["TFLOP/s"] = fl / ms / 1e9
+            if M > 16:
                 ent["frac_of_bf16_" + pk_kind] = ent["TFLOP/s"] / pk["bf16_tflops"]
+                ent["frac_of_bf16_sustained_" + pk_kind] = ent["TFLOP/s"] / pk.get("bf16_tflops_sustained", pk["bf16_tflops"])
                 ent["frac_of_bf16_nominal"] = ent["TFLOP/s"] / NOMINAL["bf16_tflops"]
             else:
-                ent["packed_GB/s"] = pbytes / ms / 1e6
+                b = sum(packed_bytes(m.N, m.K, m.cfg) for m in mats)
+                ent["packed_GB/s"] = b / ms / 1e6
                 ent["frac_of_hbm_" + pk_kind] = ent["packed_GB/s"] / pk["hbm_gbs"]
                 ent["frac_of_hbm_nominal"] = ent["packed_GB/s"] / NOMINAL["hbm_gbs"]
-                ent["all_bytes_GB/s"] = (small_bytes + 2 * M * (N + K)) / ms / 1e6
-            lms = loops[f"{ps}{M}"]
-            if M > 64:
-                ent["back_to_back"] = {"ms": lms, "TFLOP/s": linear_flops(M, N, K, r) / lms / 1e9,
-                                       "frac_of_bf16_" + pk_kind: linear_flops(M, N, K, r) / lms / 1e9 / pk["bf16_tflops"]}
-            else:
-                ent["back_to_back"] = {"ms": lms, "packed_GB/s": pbytes / lms / 1e6,
-                                       "frac_of_hbm_" + pk_kind: pbytes / lms / 1e6 / pk["hbm_gbs"],
-                                       "how": loop_kind[f"{ps}{M}"]}
-            breakdown[f"{ps}_M{M}"] = ent
+        phases[ph] = ent
 
-    gms = loops["grads2048"]
-    gbytes = 2.0 * 2048 * (N + K)          # X and dY read once (bf16)
-    breakdown["extra_lora_grads_M2048"] = {
-        "ms": gms, "how": loop_kind["grads2048"], "in_timed_step": False,
-        "GB/s": gbytes / gms / 1e6, "frac_of_hbm_" + pk_kind: gbytes / gms / 1e6 / pk["hbm_gbs"],
-        "TFLOP/s": 8.0 * 2048 * r * (N + K) / gms / 1e9,
-        "what": "lqlora_lora_grads: dL1 = dY^T (X L2^T), dL2 = (dY L1)^T X; bytes = X and dY read once"}
+    # ---- roofline of the dominant kernel: the CTA-pair tcgen05 kernel on the gate projection (forward, M = 2048),
+    # timed by the events around that call inside the timed steps
+    gi = [i for i, c in enumerate(calls) if c[0] == "fwd2048_gate"][0]
+    gate = calls[gi][2]
+    g_ms = float(mean_ms[gi])
+    achieved = linear_flops(2048, gate.N, gate.K, r) / g_ms / 1e9
+    sustained = pk.get("bf16_tflops_sustained", pk["bf16_tflops"])
+    roofline = {"bound": "tensor", "achieved": achieved, "peak": sustained, "unit": "TFLOP/s", "frac": achieved / sustained,
+                "traffic": DOMINANT_TRAFFIC_BYTES,
+                "kernel": f"tc_pair_linear_kernel<{gate.cfg.b0}, forward> on gate {gate.N}x{gate.K} at M=2048 (with the rank-r pre-product kernel "
+                          "that runs beside it); duration = mean over the timed steps of the CUDA-event interval around the call",
+                "ms_per_launch": g_ms, "ms_per_launch_median": float(np.median(call_ms[:, gi])),
+                "ms_per_launch_min_max": [float(call_ms[:, gi].min()), float(call_ms[:, gi].max())],
+                "flop_per_launch": linear_flops(2048, gate.N, gate.K, r),
+                "peak_kind": pk_kind + " cuBLAS bf16, sustained figure (the kernel is timed inside a long step)",
+                "frac_of_burst_" + pk_kind: achieved / pk["bf16_tflops"], "frac_of_nominal_2250": achieved / NOMINAL["bf16_tflops"]}
 
-    # dominant kernel: the tensor-core linear (forward and input gradient at M = 2048)
-    tc_ms = 0.5 * (loops["fwd2048"] + loops["bwd2048"])
-    achieved = linear_flops(2048, N, K, r) / tc_ms / 1e9
-    roofline = {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / pk["bf16_tflops"], "traffic": TC_TRAFFIC_BYTES,
-                "kernel": "tc_pair_linear_kernel (mean of lqlora_linear_fwd and lqlora_linear_bwd_input at M=2048, launched back to "
-                          f"back over {nrot} rotating activation buffers larger than L2; the rank-r pre-product kernel runs "
-                          "beside it on the SMs its last wave leaves idle)",
-                "ms_per_launch": tc_ms,
-                "peak_kind": pk_kind + " cuBLAS bf16 burst", "frac_of_nominal_2250": achieved / NOMINAL["bf16_tflops"]}
+    # ---- the decode-sized calls of the layer once more, each matrix alone over cold copies as one CUDA graph
+    decode = {}
+    for m in mats:
+        for ps in ("fwd", "bwd"):
+            ms, how = time_linear(binding, torch, m.q, m.L1, m.L2, m.G[1] if ps == "bwd" else m.X[1], 1, ps == "bwd", l2_bytes, timer)
+            decode[f"{ps}1_{m.spec.name}"] = linear_entry(ms, 1, m.N, m.K, r, m.cfg, pk, pk_kind, how)
+    # gradients of the low-rank factors on the gate projection at M = 2048 (the next piece of a training step; not
+    # part of the timed step)
+    gm = gate
+    dL = (torch.empty(gm.N, r, dtype=torch.float32, device=dev), torch.empty(r, gm.K, dtype=torch.float32, device=dev))
+    gws = torch.empty(binding.lora_grads_workspace_bytes(gm.N, gm.K, r, 2048), dtype=torch.uint8, device=dev)
+    g_ms2 = timer(lambda: [binding.lora_grads(gm.L1, gm.L2, gm.X[2048], gm.G[2048], out=dL, workspace=gws) for _ in range(4)], 4)
+    if binding.workspace_status(gws) != 0:
+        raise SystemExit("lora_grads reported a device-side error")
+    gbytes = 2.0 * 2048 * (gm.N + gm.K)
+    extra = {"lora_grads_gate_M2048": {"ms": g_ms2, "GB/s": gbytes / g_ms2 / 1e6, "frac_of_hbm_" + pk_kind: gbytes / g_ms2 / 1e6 / pk["hbm_gbs"],
+                                       "in_timed_step": False, "what": "lqlora_lora_grads; bytes = X and dY read once"}}
 
-    oflops, osec, odesc = oracle_sample(spec, A, l1b, l2b, rows_large=256)
+    h2d = sum(m.W_host.numel() * 4 + sum(m.XH[M].numel() * 2 + m.GH[M].numel() * 2 for M in MS) for m in mats)
+    d2h = sum(sum(m.YH[M].numel() * 2 + m.DXH[M].numel() * 2 for M in MS) for m in mats)
+    del mats, calls, gate, gm
+    torch.cuda.empty_cache()
+
+    # ---- the other seeded workloads, measured beside the step (not part of `value`)
+    other = {}
+    if not args.no_configs:
+        w1 = inputs.workload(1)
+        A, l1b, l2b = inputs.make_matrix(w1["matrices"][0])
+        other["config1_roberta_proj"] = measure_matrix(binding, torch, dev, A, l1b, l2b, w1["matrices"][0].cfg, [512], ("fwd",), pk, pk_kind, l2_bytes, timer)
+        w2 = inputs.workload(2)
+        A, l1b, l2b = inputs.make_matrix(w2["matrices"][0])
+        other["config2_llama7b_attn_proj"] = measure_matrix(binding, torch, dev, A, l1b, l2b, w2["matrices"][0].cfg, [1, 16, 2048], ("fwd", "bwd"), pk, pk_kind, l2_bytes, timer)
+        c3 = {}
+        for spec in inputs.workload(3)["matrices"]:
+            A, l1b, l2b = inputs.make_matrix(spec)
+            c3[spec.name] = measure_matrix(binding, torch, dev, A, l1b, l2b, spec.cfg, [4096], ("fwd", "bwd"), pk, pk_kind, l2_bytes, timer)
+        other["config3_llama7b_mlp"] = c3
+        A = inputs.gaussian(5000, (8192, 8192), 0.02)
+        l1b, l2b = inputs.lowrank_factors(5700, 8192, 8192, r, 0.01)
+        c5 = {}
+        for b0, B0 in ((3, 64), (2, 16), (2, 256), (8, 16), (8, 256)):
+            cfg = inputs.QuantConfig(b0, B0, 8, 256, 32)
+            c5[f"b{b0}_B{B0}"] = measure_matrix(binding, torch, dev, A, l1b, l2b, cfg, [1, 16, 128, 2048, 8192], ("fwd", "bwd"), pk, pk_kind, l2_bytes, timer)
+        other["config5_sweep_points_8192x8192"] = c5
+        del A
+
+    oflops, osec, odesc = oracle_sample(("q", "k"), rows_large=256)
     import oracle
     cpu = {"value": oflops / osec / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
            "sample": odesc, "seconds": osec}
 
-    h2d = W_host.numel() * 4 + sum(XH[M].numel() * 2 + GH[M].numel() * 2 for M in MS)
-    d2h = sum(YH[M].numel() * 2 + DXH[M].numel() * 2 for M in MS)
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": WORKLOAD, "N": N, "K": K, "rank": r, "M": list(MS), "quant": list(cfg.as_tuple()),
+        "config": {"workload": WORKLOAD, "rank": r, "M": list(MS), "calls_per_step": ncalls,
                    "parallelism": f"dp{world} over tokens, weights replicated, no collective",
-                   "l2": "flushed between steps by a 256 MiB device write followed by a 256 MiB device read (clean lines), both outside the timed events; decode-sized "
-                         f"calls rotate over {ncopies} cold copies of the packed matrix",
-                   "wall_ms_per_step_incl_flush": t_wall / args.steps * 1e3},
+                   "l2": "inputs larger than L2: a step reads 3.4 GB of fp32 weights, 0.29 GB of packed codes per pass and 0.5 GB of "
+                         "activations, and no buffer is touched twice within 126 MB of traffic except the shared inputs of q/k/v and gate/up",
+                   "ms_per_step_median": float(statistics.median(step_ms)), "ms_per_step_min_max": [min(step_ms), max(step_ms)],
+                   "wall_ms_per_step": t_wall / args.steps * 1e3},
         "clocks": clocks,
         "e2e": {"value": world * step_flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches),
         "roofline": roofline,
         "cpu_baseline": cpu,
-        "breakdown": breakdown,
+        "breakdown": {"phases": phases, "calls": layer, "decode_calls_alone": decode, "extra": extra, "other_configs": other},
     }
     print(json.dumps(line), flush=True)
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def run_case(args):
+    """One matrix of the layer alone, with random packed codes (no fp32 weights on the device): a few forward and
+    input-gradient calls at one M.  Holds well under 1 GB, so that a profiler can capture the kernels of the largest
+    shapes on their own."""
+    import torch
+    from paper_2311_12023_b200 import binding
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    spec = [s for s in inputs.workload(4)["matrices"] if s.name == args.case][0]
+    M, r = args.case_m, inputs.RANK
+    q = binding.alloc_qmatrix(spec.N, spec.K, spec.cfg, dev)
+    g = torch.Generator(device=dev)
+    g.manual_seed(1)
+    q.codes.random_(0, 256, generator=g)
+    q.scale_codes.random_(1, 128, generator=g)
+    q.scale2.fill_(0.05)
+    l1b, l2b = inputs.lowrank_factors(spec.seed + 700, spec.N, spec.K, r, 0.01)
+    L1, L2 = binding.bf16_from_bits(l1b, dev), binding.bf16_from_bits(l2b, dev)
+    X = binding.bf16_from_bits(inputs.activations(1, M, spec.K), dev)
+    G = binding.bf16_from_bits(inputs.activations(2, M, spec.N), dev)
+    ws = binding.alloc_workspace(q, r, M)
+    Y = torch.empty((M, spec.N), dtype=torch.bfloat16, device=dev)
+    DX = torch.empty((M, spec.K), dtype=torch.bfloat16, device=dev)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.case_reps + 1)]
+    evs[0].record()
+    for i in range(args.case_reps):
+        binding.linear_fwd(q, L1, L2, X, out=Y, workspace=ws)
+        evs[2 * i + 1].record()
+        binding.linear_bwd_input(q, L1, L2, G, out=DX, workspace=ws)
+        evs[2 * i + 2].record()
+    torch.cuda.synchronize()
+    if binding.workspace_status(ws) != 0:
+        raise SystemExit("a linear kernel reported a device-side error")
+    f = [evs[2 * i].elapsed_time(evs[2 * i + 1]) for i in range(args.case_reps)]
+    b = [evs[2 * i + 1].elapsed_time(evs[2 * i + 2]) for i in range(args.case_reps)]
+    print(json.dumps({"case": args.case, "shape": [spec.N, spec.K], "quant": list(spec.cfg.as_tuple()), "M": M,
+                      "fwd_ms": f, "bwd_ms": b}), flush=True)
 
 
 def run_sweep(args):
@@ -512,6 +672,7 @@ def run_sweep(args):
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     pk, pk_kind = peaks()
+    timer = Timer(torch)
     N = K = 8192
     r = inputs.RANK
     W = torch.from_numpy(inputs.gaussian(5000, (N, K), 0.02)).to(dev)
@@ -523,74 +684,55 @@ def run_sweep(args):
     print("# M <= 16: packed-weight GB/s and fraction of HBM peak (calls replayed as a CUDA graph over cold copies);")
     print("# M >= 128: algorithmic TFLOP/s and fraction of the bf16 peak (back to back over rotating activation buffers)")
     print(f"{'b0':>3} {'B0':>4} {'bits':>6} {'enc GB/s':>9} {'enc frac':>8} " + " ".join(f"{'fwd M=' + str(m):>12} {'frac':>6} {'bwd M=' + str(m):>12} {'frac':>6}" for m in Ms))
-
-    def timed(fn, count):
-        fn()
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        fn()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / count
-
     for b0 in (2, 3, 4, 8):
         for B0 in (16, 32, 64, 128, 256):
             cfg = inputs.QuantConfig(b0, B0, 8, 256, 32)
             q = binding.alloc_qmatrix(N, K, cfg, dev)
             enc_ws = torch.empty(binding.packed_sizes(N, K, cfg)[3], dtype=torch.uint8, device=dev)
-            enc_ms = timed(lambda: [binding.encode(W, cfg, out=q, workspace=enc_ws) for _ in range(3)], 3)
+            enc_ms = timer(lambda: [binding.encode(W, cfg, out=q, workspace=enc_ws) for _ in range(3)], 3)
             enc_gbs = encode_bytes(N, K, cfg) / enc_ms / 1e6
             pbytes = packed_bytes(N, K, cfg)
-            ncopies = max(2, int(2.2 * l2_bytes / q.packed_bytes) + 1)
-            copies = [binding.QMatrix(q.codes.clone(), q.scale_codes.clone(), q.scale2.clone(), N, K, cfg) for _ in range(ncopies)]
             cells = []
             for M in Ms:
                 X = binding.bf16_from_bits(inputs.activations(5200 + M, M, K), dev)
                 G = binding.bf16_from_bits(inputs.activations(5300 + M, M, N), dev)
-                ws = binding.alloc_workspace(q, r, M)
                 for bwd in (False, True):
-                    fn = binding.linear_bwd_input if bwd else binding.linear_fwd
-                    A = G if bwd else X
+                    ms, _ = time_linear(binding, torch, q, L1, L2, G if bwd else X, M, bwd, l2_bytes, timer)
                     if M <= 16:
-                        out = torch.empty((M, K if bwd else N), dtype=torch.bfloat16, device=dev)
-
-                        def body():
-                            for c in copies:
-                                fn(c, L1, L2, A, out=out, workspace=ws)
-                        body()
-                        torch.cuda.synchronize()
-                        g = torch.cuda.CUDAGraph()
-                        with torch.cuda.graph(g):
-                            body()
-                        ms = timed(g.replay, ncopies)
                         val = pbytes / ms / 1e6
                         cells.append(f"{val:9.0f}GB/s {val / pk['hbm_gbs']:6.3f}")
                     else:
-                        nrot = max(2, int(1.1 * l2_bytes / (M * (N + K) * 2)) + 1) if M < 8192 else 2
-                        As = [A.clone() for _ in range(nrot)]
-                        outs = [torch.empty((M, K if bwd else N), dtype=torch.bfloat16, device=dev) for _ in range(nrot)]
-                        reps = max(2, min(4 * nrot, 16))
-                        ms = timed(lambda: [fn(q, L1, L2, As[i % nrot], out=outs[i % nrot], workspace=ws) for i in range(reps)], reps)
                         val = linear_flops(M, N, K, r) / ms / 1e9
                         cells.append(f"{val:8.0f}TF/s {val / pk['bf16_tflops']:6.3f}")
-                        del As, outs
             bits = cfg.b0 + cfg.b1 / cfg.B0 + cfg.b2 / (cfg.B0 * cfg.B1)
             print(f"{b0:>3} {B0:>4} {bits:6.3f} {enc_gbs:9.0f} {enc_gbs / pk['hbm_gbs']:8.3f} " + " ".join(cells), flush=True)
-            del copies, q
+            del q
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-config figures measured beside the step")
+    ap.add_argument("--dry-run", action="store_true", help="host logic of the multi-rank path only (gloo, no device work)")
     ap.add_argument("--sweep", action="store_true", help="print the b0 x B0 x M table of the 8192 x 8192 sweep instead")
     ap.add_argument("--sweep-ms", default="1,16,128,2048,8192")
+    ap.add_argument("--case", default=None, help="run one matrix of the layer alone (q, k, v, o, gate, up, down)")
+    ap.add_argument("--case-m", type=int, default=2048)
+    ap.add_argument("--case-reps", type=int, default=3)
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+        return
+    if args.case:
+        run_case(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
+    if args.dry_run:
+        run_dry(args)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -25,7 +25,7 @@ using namespace dev;
 
 constexpr int kConsumerWarps = 8;
 constexpr int kThreads = kConsumerWarps * 32;
-constexpr int kStageTiles = 8;              // 64-column tiles per ring stage (four windows of 128 columns)
+constexpr int kStageTiles = 4;              // 64-column tiles per ring stage of the forward kernel (two windows of 128 columns)
 constexpr int kSmemLimit = 232448;
 constexpr int kStabStride = 136;            // floats per block column of the scale table (128 rows + padding against bank conflicts)
 constexpr int kStab8Stride = 148;           // bytes per block column of the compact scale table (8-bit codes; one sigma per 16 block columns)
@@ -34,10 +34,14 @@ constexpr int kXRowBytes = kStageTiles * kTileCols * 2 + 16;   // one token's ac
 // A ring stage: the packed tiles, then the activations of the stage's 512 columns for 8 NT token rows.
 // NT = number of 8-token groups (1: M <= 8, two CTAs per SM; 2: M <= 16, one CTA per SM)
 template <int B, int NT> __host__ __device__ constexpr int stage_bytes() { return kStageTiles * 1024 * B + 8 * NT * kXRowBytes; }
-// CTAs per SM the forward kernel is compiled for: two, except for 8-bit codes and for 4-bit codes with 16 tokens
-// (their stages and registers do not fit twice)
-template <int B, int NT> __host__ __device__ constexpr int fwd_ctas_per_sm() { return (B == 8 || (B == 4 && NT == 2)) ? 1 : 2; }
-template <int B, int NT> __host__ __device__ constexpr int num_stages() { return (B == 8) ? 2 : (fwd_ctas_per_sm<B, NT>() == 1 ? 3 : 2); }
+// CTAs per SM the forward kernel is compiled for: two (128 registers per thread), except for 8-bit codes with 16 tokens
+template <int B, int NT> __host__ __device__ constexpr int fwd_ctas_per_sm() { return (B == 8 && NT == 2) ? 1 : 2; }
+// Ring depth: what fits into about 84 KB per CTA (two CTAs per SM) or twice that, between two and eight stages
+template <int B, int NT> __host__ __device__ constexpr int num_stages() {
+    constexpr int budget = (fwd_ctas_per_sm<B, NT>() == 2 ? 84 : 168) * 1024;
+    constexpr int n = budget / stage_bytes<B, NT>();
+    return n < 2 ? 2 : n > 8 ? 8 : n;
+}
 
 struct Params {
     QView q;
@@ -64,6 +68,9 @@ __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// Split cluster barrier: arrive early, wait where the guarantee is needed.
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }
 __device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank) {
     uint32_t ra;
     float v;
@@ -122,8 +129,8 @@ decode_fwd_kernel(const Params p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
     uint8_t* ring = base;
-    float* part = reinterpret_cast<float*>(ring + NS * STAGE);        // 128 x MT partial sums of this CTA, fragment order
-    float* lut8 = part + 128 * MT;                                     // 256 floats (8-bit codes only)
+    float* recv = reinterpret_cast<float*>(ring + NS * STAGE);        // [2 S sources][128 / S rows][MT] partial sums sent to this CTA
+    float* lut8 = recv + 2 * 128 * MT;                                 // 256 floats (8-bit codes only)
     uint64_t* bars = reinterpret_cast<uint64_t*>(lut8 + (B == 8 ? 256 : 0));   // full[NS], then NS counters of warps done with a slot
     uint32_t* done = reinterpret_cast<uint32_t*>(bars + NS);
     volatile int* abort_s = reinterpret_cast<volatile int*>(bars + 2 * NS);
@@ -144,6 +151,10 @@ decode_fwd_kernel(const Params p) {
 
     auto full = [&](int s) { return smem_u32(bars + s); };
 
+    // The CTAs of a cluster write into each other's shared memory at the end; a CTA's shared memory may only be
+    // touched once it runs, which the first phase of the cluster barrier establishes (arrive here, wait before
+    // the first remote store: off the critical path).
+    if (p.S > 1) cluster_arrive_relaxed();
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); done[s] = 0u; }
         *abort_s = 0;
@@ -164,9 +175,10 @@ decode_fwd_kernel(const Params p) {
             bulk_load(dst + XOFF + m * kXRowBytes, xsrc + static_cast<size_t>(m) * q.K, nt * (kTileCols * 2), full(s));
     };
     // There is no producer warp: thread 0 fills the ring once, afterwards the warp that is last to finish a stage
-    // refills its slot (nobody waits for a free slot, and the CTA has eight warps, two per scheduler).  The first fill
-    // is issued after the first loads of the scale table below: the few bytes of the table would otherwise queue
-    // behind the ring's bulk copies of all CTAs in the memory system (measured: 4 us instead of 1).
+    // refills its slot (nobody waits for a free slot, and the CTA has eight warps, two per scheduler).  The stages are
+    // small (four tiles) so that the first one of every CTA arrives early and the dequantization, which is what
+    // binds, starts while the rest of the ring is still on its way.  The first fill is issued after the first loads
+    // of the scale table below, which are few and should not queue behind the bulk copies.
     bool ring_filled = false;
     auto fill_ring = [&]() {
         if (!ring_filled && threadIdx.x == 0) {
@@ -287,26 +299,27 @@ decode_fwd_kernel(const Params p) {
     }
     __syncthreads();
 
-    float acc[2][2][NT][4];
+    // acc[set][nt][e]: row 4 gid + 2 set + (e >> 1) of the warp's slab, token nt * 8 + 2 t + (e & 1)
+    float acc[2][NT][4];
 #pragma unroll
     for (int a = 0; a < 2; ++a)
 #pragma unroll
-        for (int b = 0; b < 2; ++b)
+        for (int c = 0; c < NT; ++c)
 #pragma unroll
-            for (int c = 0; c < NT; ++c)
-#pragma unroll
-                for (int d = 0; d < 4; ++d) acc[a][b][c][d] = 0.0f;
+            for (int d = 0; d < 4; ++d) acc[a][c][d] = 0.0f;
 
+    // ------------------------------------------------------------------ main loop
+    // A stage holds four tiles = two windows of 128 columns; warp w takes slab (w & 3) of window (w >> 2): lane
+    // (gid, t) dequantizes rows 4 gid .. 4 gid + 3 of the 32-column group (t & 1) of tile 2 (w >> 2) + (t >> 1).
+    const int gid = lane >> 2, t = lane & 3;
+    const int slab = warp & 3, window = warp >> 2;
     {
-        // ------------------------------------------------------------------ consumers
-        const int gid = lane >> 2, t = lane & 3;
-        const int win_slot = warp & 3, half = warp >> 2;
         bool ok = true;
         for (int it = 0; it < nstage_total && ok; ++it) {
             const int s = it % NS;
             const int tiles_here = min(kStageTiles, ntiles_cta - it * kStageTiles);
-            const bool active = 2 * win_slot < tiles_here;
-            const int tile_in_stage = 2 * win_slot + (t >> 1);
+            const bool active = 2 * window < tiles_here;
+            const int tile_in_stage = 2 * window + (t >> 1);
             const bool kt_ok = tile_in_stage < tiles_here;
             const int col0 = (kt0 + it * kStageTiles + tile_in_stage) * kTileCols + (t & 1) * 32;
             ok = wait(full(s), (it / NS) & 1, ctl, 22);
@@ -330,58 +343,54 @@ decode_fwd_kernel(const Params p) {
                     for (int c = 0; c < 4; ++c)
                         x1[c] = have1 ? reinterpret_cast<const uint4*>(xbase + (gid + 8) * kXRowBytes)[c] : make_uint4(0u, 0u, 0u, 0u);
                 }
+                const uint32_t* sp = tile + slab * (64 * B) + (t & 1) * (B * 32) + slab_row_slot(4 * gid, t & 1, tile_in_stage);
+                uint4 w4[B];
 #pragma unroll
-                for (int sl = 0; sl < 2; ++sl) {
-                    const int slab = 2 * half + sl;
-                    const uint32_t* sp = tile + slab * (64 * B) + (t & 1) * (B * 32) + slab_row_slot(4 * gid, t & 1, tile_in_stage);
-                    uint4 w4[B];
-#pragma unroll
-                    for (int i = 0; i < B; ++i) w4[i] = *reinterpret_cast<const uint4*>(sp + i * 32);
-                    float4 sc_lo, sc_hi;
-                    if (p.stab8) {
-                        // s~ = fl32(float(s^) * fl32(v / 127)) from the compact table
-                        const float4 sg4 = *reinterpret_cast<const float4*>(sig + (kb >> 4) * kStabStride + slab * 32 + 4 * gid);
-                        const uint32_t c_lo = *reinterpret_cast<const uint32_t*>(stab8 + kb * kStab8Stride + slab * 32 + 4 * gid);
-                        sc_lo = make_float4(__fmul_rn(static_cast<float>(c_lo & 255u), sg4.x), __fmul_rn(static_cast<float>((c_lo >> 8) & 255u), sg4.y),
-                                            __fmul_rn(static_cast<float>((c_lo >> 16) & 255u), sg4.z), __fmul_rn(static_cast<float>(c_lo >> 24), sg4.w));
-                        sc_hi = sc_lo;
-                        if (TWO) {
-                            // kb is even here (two blocks of 16 columns per 32-column group), so kb + 1 has the same sigma
-                            const uint32_t c_hi = *reinterpret_cast<const uint32_t*>(stab8 + (kb + 1) * kStab8Stride + slab * 32 + 4 * gid);
-                            sc_hi = make_float4(__fmul_rn(static_cast<float>(c_hi & 255u), sg4.x), __fmul_rn(static_cast<float>((c_hi >> 8) & 255u), sg4.y),
-                                                __fmul_rn(static_cast<float>((c_hi >> 16) & 255u), sg4.z), __fmul_rn(static_cast<float>(c_hi >> 24), sg4.w));
-                        }
-                    } else {
-                        sc_lo = *reinterpret_cast<const float4*>(stab + kb * kStabStride + slab * 32 + 4 * gid);
-                        sc_hi = sc_lo;
-                        if (TWO) sc_hi = *reinterpret_cast<const float4*>(stab + (kb + 1) * kStabStride + slab * 32 + 4 * gid);
+                for (int i = 0; i < B; ++i) w4[i] = *reinterpret_cast<const uint4*>(sp + i * 32);
+                float4 sc_lo, sc_hi;
+                if (p.stab8) {
+                    // s~ = fl32(float(s^) * fl32(v / 127)) from the compact table
+                    const float4 sg4 = *reinterpret_cast<const float4*>(sig + (kb >> 4) * kStabStride + slab * 32 + 4 * gid);
+                    const uint32_t c_lo = *reinterpret_cast<const uint32_t*>(stab8 + kb * kStab8Stride + slab * 32 + 4 * gid);
+                    sc_lo = make_float4(__fmul_rn(static_cast<float>(c_lo & 255u), sg4.x), __fmul_rn(static_cast<float>((c_lo >> 8) & 255u), sg4.y),
+                                        __fmul_rn(static_cast<float>((c_lo >> 16) & 255u), sg4.z), __fmul_rn(static_cast<float>(c_lo >> 24), sg4.w));
+                    sc_hi = sc_lo;
+                    if (TWO) {
+                        // kb is even here (two blocks of 16 columns per 32-column group), so kb + 1 has the same sigma
+                        const uint32_t c_hi = *reinterpret_cast<const uint32_t*>(stab8 + (kb + 1) * kStab8Stride + slab * 32 + 4 * gid);
+                        sc_hi = make_float4(__fmul_rn(static_cast<float>(c_hi & 255u), sg4.x), __fmul_rn(static_cast<float>((c_hi >> 8) & 255u), sg4.y),
+                                            __fmul_rn(static_cast<float>((c_hi >> 16) & 255u), sg4.z), __fmul_rn(static_cast<float>(c_hi >> 24), sg4.w));
                     }
-                    if (!kt_ok) { sc_lo = make_float4(0.f, 0.f, 0.f, 0.f); sc_hi = sc_lo; }
+                } else {
+                    sc_lo = *reinterpret_cast<const float4*>(stab + kb * kStabStride + slab * 32 + 4 * gid);
+                    sc_hi = sc_lo;
+                    if (TWO) sc_hi = *reinterpret_cast<const float4*>(stab + (kb + 1) * kStabStride + slab * 32 + 4 * gid);
+                }
+                if (!kt_ok) { sc_lo = make_float4(0.f, 0.f, 0.f, 0.f); sc_hi = sc_lo; }
 #pragma unroll
-                    for (int set = 0; set < 2; ++set) {
-                        // rows a = 2 set, b = 2 set + 1 of the thread's four; the two MMAs of a chunk are issued right
-                        // after its eight weights are ready, so consecutive MMAs on one accumulator are spaced out
-                        uint32_t wa[B], wb[B];
+                for (int set = 0; set < 2; ++set) {
+                    // rows a = 2 set, b = 2 set + 1 of the thread's four; the two MMAs of a chunk are issued right
+                    // after its eight weights are ready, so consecutive MMAs on one accumulator are spaced out
+                    uint32_t wa[B], wb[B];
 #pragma unroll
-                        for (int i = 0; i < B; ++i) { wa[i] = pick(w4[i], 2 * set); wb[i] = pick(w4[i], 2 * set + 1); }
-                        const float sa_lo = pickf(sc_lo, 2 * set), sb_lo = pickf(sc_lo, 2 * set + 1);
-                        const float sa_hi = pickf(sc_hi, 2 * set), sb_hi = pickf(sc_hi, 2 * set + 1);
-                        BlockTable<B> ta, tb;
-                        if constexpr (B != 8) { ta.build(sa_lo); tb.build(sb_lo); }
+                    for (int i = 0; i < B; ++i) { wa[i] = pick(w4[i], 2 * set); wb[i] = pick(w4[i], 2 * set + 1); }
+                    const float sa_lo = pickf(sc_lo, 2 * set), sb_lo = pickf(sc_lo, 2 * set + 1);
+                    const float sa_hi = pickf(sc_hi, 2 * set), sb_hi = pickf(sc_hi, 2 * set + 1);
+                    BlockTable<B> ta, tb;
+                    if constexpr (B != 8) { ta.build(sa_lo); tb.build(sb_lo); }
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            if constexpr (B != 8) {
-                                if (TWO && c == 2) { ta.build(sa_hi); tb.build(sb_hi); }
-                            }
-                            uint32_t oa[4], ob[4];
-                            dequant_chunk<B>(wa, c, ta, (TWO && c >= 2) ? sa_hi : sa_lo, oa, lut8);
-                            dequant_chunk<B>(wb, c, tb, (TWO && c >= 2) ? sb_hi : sb_lo, ob, lut8);
-                            mma16816(acc[sl][set][0], oa[0], ob[0], oa[1], ob[1], x0[c].x, x0[c].y);
-                            mma16816(acc[sl][set][0], oa[2], ob[2], oa[3], ob[3], x0[c].z, x0[c].w);
-                            if constexpr (NT == 2) {
-                                mma16816(acc[sl][set][1], oa[0], ob[0], oa[1], ob[1], x1[c].x, x1[c].y);
-                                mma16816(acc[sl][set][1], oa[2], ob[2], oa[3], ob[3], x1[c].z, x1[c].w);
-                            }
+                    for (int c = 0; c < 4; ++c) {
+                        if constexpr (B != 8) {
+                            if (TWO && c == 2) { ta.build(sa_hi); tb.build(sb_hi); }
+                        }
+                        uint32_t oa[4], ob[4];
+                        dequant_chunk<B>(wa, c, ta, (TWO && c >= 2) ? sa_hi : sa_lo, oa, lut8);
+                        dequant_chunk<B>(wb, c, tb, (TWO && c >= 2) ? sb_hi : sb_lo, ob, lut8);
+                        mma16816(acc[set][0], oa[0], ob[0], oa[1], ob[1], x0[c].x, x0[c].y);
+                        mma16816(acc[set][0], oa[2], ob[2], oa[3], ob[3], x0[c].z, x0[c].w);
+                        if constexpr (NT == 2) {
+                            mma16816(acc[set][1], oa[0], ob[0], oa[1], ob[1], x1[c].x, x1[c].y);
+                            mma16816(acc[set][1], oa[2], ob[2], oa[3], ob[3], x1[c].z, x1[c].w);
                         }
                     }
                 }
@@ -394,24 +403,14 @@ decode_fwd_kernel(const Params p) {
         }
     }
 
-    // ---------------------------------------------------------------------- reduction over the K windows of the CTA
-    // Every consumer warp writes its accumulators, in fragment order, to its own region of the (now
-    // idle) ring; then the four warps that cover the same rows are added into `part`, still in
-    // fragment order:  part[(half * 16 NT + k) * 32 + lane],  k = ((sl * 2 + set) * NT + nt) * 4 + e,
-    // which is row (2 half + sl) * 32 + 4 gid + 2 set + (e >> 1) and token nt * 8 + 2 t + (e & 1).
-    constexpr int KF = 16 * NT;
-    float* red = reinterpret_cast<float*>(ring);
-    // T (at most 16 x 128 bf16) is staged behind the reduction buffer
-    __nv_bfloat16* tsm = reinterpret_cast<__nv_bfloat16*>(ring + kConsumerWarps * KF * 128);
-    static_assert(kConsumerWarps * KF * 128 + 4096 <= NS * STAGE, "reduction buffer and T must fit into the ring");
+    // ---------------------------------------------------------------------- rank-r term, reduction, output
     // CTA `rank` of the cluster finishes rows [rank * 128 / S, (rank + 1) * 128 / S) of the tile row
     const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
     const int rows_share = 128 / p.S;
     const int row_lo = static_cast<int>(rank) * rows_share;
-    const int sub = threadIdx.x & 7;
-    __syncthreads();                      // all stages consumed: the ring is free
+    __syncthreads();
     if (*abort_s) {
-        // a wait gave up: let copies that are still in flight land before the ring is reused (bounded)
+        // a wait gave up: let copies that are still in flight land before the CTA exits (bounded)
         if (threadIdx.x == 0) {
             for (int s = 0; s < NS; ++s) {
                 const long long t0 = clock64();
@@ -420,109 +419,58 @@ decode_fwd_kernel(const Params p) {
         }
         __syncthreads();
     }
-    // Requested now, used after the cluster barrier (the latency of global memory is hidden behind the reduction):
-    // this thread's piece of T (written by the kernel launched in front of this one) and, for the first pass of the
-    // epilogue, its slice of the row of L1: elements [8 (sub + 8 v), +8) for v < ceil(r / 64).
-    if (p.r > 0) pdl_wait();
-    const int t_vecs = p.M * p.r / 8;
-    uint4 tv = make_uint4(0u, 0u, 0u, 0u);
-    if (static_cast<int>(threadIdx.x) < t_vecs) tv = __ldg(reinterpret_cast<const uint4*>(p.T) + threadIdx.x);
-    auto load_factor = [&](int rl, uint4 (&a)[2], bool (&have)[2]) {
-        const bool live = rl < rows_share;
-        const int n = tile_row * 128 + row_lo + (live ? rl : 0);
+    // T L1^T on the tensor cores, as more contraction steps of the same accumulators (first CTA of the cluster only):
+    // 16 columns of the factors per MMA, lane t supplies columns 4 t .. 4 t + 3 of the rows a, b of its set and of the
+    // tokens gid (gid + 8); the warps of window 0 take the even groups of 16 columns, those of window 1 the odd ones.
+    // T was written by the kernel launched in front of this one: wait for it here (plain loads, not the read-only path).
+    if (p.r > 0 && rank == 0) {
+        pdl_wait();
+        const int n0 = tile_row * 128 + slab * 32 + 4 * gid;
+        for (int ch = window; ch * 16 < p.r; ch += 2) {
+            const int j = ch * 16 + 4 * t;
+            uint2 tk0 = make_uint2(0u, 0u), tk1 = make_uint2(0u, 0u);
+            if (gid < p.M) tk0 = *reinterpret_cast<const uint2*>(p.T + static_cast<size_t>(gid) * p.r + j);
+            if (NT == 2 && gid + 8 < p.M) tk1 = *reinterpret_cast<const uint2*>(p.T + static_cast<size_t>(gid + 8) * p.r + j);
 #pragma unroll
-        for (int v = 0; v < 2; ++v) {
-            a[v] = make_uint4(0u, 0u, 0u, 0u);
-            have[v] = live && n < q.N && (8 * (sub + 8 * v) < p.r);
-            if (have[v]) a[v] = __ldg(reinterpret_cast<const uint4*>(p.L1 + static_cast<size_t>(n) * p.r) + sub + 8 * v);
-        }
-    };
-    uint4 a_first[2];
-    bool have_first[2];
-    load_factor(static_cast<int>(threadIdx.x >> 3), a_first, have_first);
-
-    if (warp < kConsumerWarps) {
-#pragma unroll
-        for (int sl = 0; sl < 2; ++sl)
-#pragma unroll
-            for (int set = 0; set < 2; ++set)
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        red[(warp * KF + ((sl * 2 + set) * NT + nt) * 4 + e) * 32 + lane] = acc[sl][set][nt][e];
-    }
-    __syncthreads();
-    // The sum of the four warps goes straight to the CTA that owns the row.  recv[(src * rows_share + rl) * MT + m] in
-    // the owner's shared memory (`part`, which nothing else uses) takes the partial sum of cluster rank `src`; remote
-    // stores need no round trip, and after the cluster barrier every CTA only reads its own shared memory.
-    const uint32_t part_addr = smem_u32(part);
-    for (int idx = threadIdx.x; idx < 2 * KF * 32; idx += kThreads) {
-        const int half = idx / (KF * 32), rest = idx - half * (KF * 32);
-        const float* src = red + (half * 4 * KF) * 32 + rest;
-        const float v = (src[0] + src[KF * 32]) + (src[2 * KF * 32] + src[3 * KF * 32]);
-        // fragment order -> (row, token): k = ((sl * 2 + set) * NT + nt) * 4 + e, lane = gid * 4 + t
-        const int k = rest >> 5, ln = rest & 31;
-        const int e = k & 3, nt = (k >> 2) % NT, ss = (k >> 2) / NT;
-        const int row = (2 * half + (ss >> 1)) * 32 + 4 * (ln >> 2) + 2 * (ss & 1) + (e >> 1);
-        const int m = nt * 8 + 2 * (ln & 3) + (e & 1);
-        const int owner = row / rows_share, rl = row - owner * rows_share;
-        const uint32_t dst = part_addr + static_cast<uint32_t>((static_cast<int>(rank) * rows_share + rl) * MT + m) * 4u;
-        if (m >= p.M) continue;                  // token rows that do not exist
-        if (p.S > 1) st_dsmem_f32(dst, static_cast<uint32_t>(owner), v);
-        else part[(rl) * MT + m] = v;
-    }
-    if (static_cast<int>(threadIdx.x) < t_vecs) reinterpret_cast<uint4*>(tsm)[threadIdx.x] = tv;
-    for (int i = threadIdx.x + kThreads; i < t_vecs; i += kThreads)
-        reinterpret_cast<uint4*>(tsm)[i] = __ldg(reinterpret_cast<const uint4*>(p.T) + i);
-    cluster_sync_all();               // all partial sums have arrived (and T is staged); from here on only local shared memory is read
-    // eight lanes share a row n: each takes an eighth of the rank-r dot product (the row of L1 is read once for all
-    // tokens) and the partial sum of one cluster rank
-    constexpr int kRowsPerPass = kThreads >> 3;
-    for (int r0 = 0; r0 < rows_share; r0 += kRowsPerPass) {
-        const int rl = r0 + static_cast<int>(threadIdx.x >> 3);
-        const bool live = rl < rows_share;
-        const int row = row_lo + (live ? rl : 0);
-        const int n = tile_row * 128 + row;
-        const bool row_ok = live && n < q.N;
-        uint4 a[2];
-        bool have[2];
-        if (r0 == 0) {
-#pragma unroll
-            for (int v = 0; v < 2; ++v) { a[v] = a_first[v]; have[v] = have_first[v]; }
-        } else {
-            load_factor(rl, a, have);
-        }
-        for (int m4 = 0; m4 < p.M; m4 += 4) {
-            float sum[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int m = m4 + u;
-                sum[u] = (live && m < p.M && sub < p.S) ? part[(sub * rows_share + rl) * MT + m] : 0.0f;
+            for (int set = 0; set < 2; ++set) {
+                const int na = n0 + 2 * set, nb = na + 1;
+                uint2 la = make_uint2(0u, 0u), lb = make_uint2(0u, 0u);
+                if (na < q.N) la = __ldg(reinterpret_cast<const uint2*>(p.L1 + static_cast<size_t>(na) * p.r + j));
+                if (nb < q.N) lb = __ldg(reinterpret_cast<const uint2*>(p.L1 + static_cast<size_t>(nb) * p.r + j));
+                mma16816(acc[set][0], la.x, lb.x, la.y, lb.y, tk0.x, tk0.y);
+                if constexpr (NT == 2) mma16816(acc[set][1], la.x, lb.x, la.y, lb.y, tk1.x, tk1.y);
             }
+        }
+    }
+    // Every warp sends its sums straight to the CTA that owns the row: recv[((src * 2 + window) * rows_share + rl) * MT + m]
+    // in the owner's shared memory takes the sum of window `window` of cluster rank `src`.  Remote stores need no round
+    // trip, and after the cluster barrier every CTA only reads its own shared memory.
+    if (p.S > 1) cluster_wait();             // every CTA of the cluster runs: its shared memory may be written
+    {
+        const uint32_t recv_addr = smem_u32(recv);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int m = m4 + u;
-                if (m < p.M) {
+        for (int set = 0; set < 2; ++set)
 #pragma unroll
-                    for (int v = 0; v < 2; ++v) {
-                        if (have[v]) {
-                            const uint4 b = *(reinterpret_cast<const uint4*>(tsm + static_cast<size_t>(m) * p.r) + sub + 8 * v);
-                            const uint32_t aa[4] = {a[v].x, a[v].y, a[v].z, a[v].w}, bb[4] = {b.x, b.y, b.z, b.w};
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                sum[u] = fmaf(__uint_as_float(aa[e] << 16), __uint_as_float(bb[e] << 16), sum[u]);
-                                sum[u] = fmaf(__uint_as_float(aa[e] & 0xffff0000u), __uint_as_float(bb[e] & 0xffff0000u), sum[u]);
-                            }
-                        }
-                    }
+                for (int e = 0; e < 4; ++e) {
+                    const int row = slab * 32 + 4 * gid + 2 * set + (e >> 1);
+                    const int m = nt * 8 + 2 * t + (e & 1);
+                    if (m >= p.M) continue;                  // token rows that do not exist
+                    const int owner = row / rows_share, rl = row - owner * rows_share;
+                    const int slot = ((static_cast<int>(rank) * 2 + window) * rows_share + rl) * MT + m;
+                    if (p.S > 1) st_dsmem_f32(recv_addr + static_cast<uint32_t>(slot) * 4u, static_cast<uint32_t>(owner), acc[set][nt][e]);
+                    else recv[slot] = acc[set][nt][e];
                 }
-                sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], 1);
-                sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], 2);
-                sum[u] += __shfl_xor_sync(0xffffffffu, sum[u], 4);
-                if (row_ok && sub == 0 && m < p.M) p.Y[static_cast<size_t>(m) * q.N + n] = __float2bfloat16_rn(sum[u]);
-            }
-        }
+    }
+    if (p.S > 1) cluster_sync_all();      // all sums have arrived
+    else __syncthreads();
+    for (int idx = threadIdx.x; idx < rows_share * p.M; idx += kThreads) {
+        const int m = idx / rows_share, rl = idx - m * rows_share;
+        const int n = tile_row * 128 + row_lo + rl;
+        float sum = 0.0f;
+        for (int src = 0; src < 2 * p.S; ++src) sum += recv[(src * rows_share + rl) * MT + m];
+        if (n < q.N) p.Y[static_cast<size_t>(m) * q.N + n] = __float2bfloat16_rn(sum);
     }
 }
 
@@ -1055,7 +1003,7 @@ template <int B, int NT>
 inline size_t smem_bytes(int nkb_cap, bool stab8) {
     const size_t table = stab8 ? static_cast<size_t>(nkb_cap) * kStab8Stride + static_cast<size_t>((nkb_cap + 15) / 16) * (kStabStride * 4)
                                : static_cast<size_t>(nkb_cap) * (kStabStride * 4);
-    return 128 + static_cast<size_t>(num_stages<B, NT>()) * stage_bytes<B, NT>() + 128 * 8 * NT * 4 + (B == 8 ? 1024 : 0) +
+    return 128 + static_cast<size_t>(num_stages<B, NT>()) * stage_bytes<B, NT>() + 2 * 128 * 8 * NT * 4 + (B == 8 ? 1024 : 0) +
            (2 * num_stages<B, NT>() + 2) * 8 + table;
 }
 

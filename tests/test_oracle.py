@@ -406,5 +406,10 @@ def test_input_generators_are_seeded():
     tot = sum(s.N * s.K for s in specs)
     avg = sum(oracle.storage_bits_per_param(s.cfg.b0, 8, 32, s.cfg.B0, s.cfg.B1) * s.N * s.K for s in specs) / tot
     assert 2.70 <= avg <= 2.80
+    # the stored table is what the committed script (which calls only the oracle) writes
+    import json
+    from oracle import make_c4_draw
+    with open(make_c4_draw.OUT) as f:
+        assert json.load(f) == make_c4_draw.table()
     rows = inputs.sample_rows(1, 2048)
     assert len(rows) <= 64 and rows[0] == 0 and rows[-1] == 2047 and 127 in rows and 128 in rows
