@@ -1,19 +1,22 @@
-// Forward pass for decode-sized inputs (M <= 16 rows of X): the packed matrix is streamed once.
+// Forward pass and input gradient for decode-sized inputs (M <= 16 rows): the packed matrix is streamed once.
 //
-//   - One CTA owns a tile row of Q (128 rows) and a slice of K; the K slices of a tile row form a
-//     thread-block cluster and are added up through distributed shared memory, so there is no
-//     workspace of partial sums and nothing to zero.
-//   - The packed tiles of the CTA (they are contiguous in memory) and the matching activations are streamed into a
-//     shared-memory ring with bulk copies: thread 0 fills the ring once, afterwards the warp that finishes a stage
-//     last refills its slot (no producer warp).  Eight warps dequantize them in registers with
-//     the byte-table method (bf16 bits identical to the exported dequantized weights) and feed
-//     mma.sync m16n8k16 (weights = the 16-row operand, tokens = the 8-column operand, fp32 accumulators).
-//     The contraction index is permuted so that a thread supplies 4 consecutive weights of one row per MMA
-//     and reads the matching 4 activations with one 128-bit load per 8 columns.
+//   - Forward: one CTA owns a tile row of Q (128 rows) and a slice of K.  The packed tiles of the CTA (they are
+//     contiguous in memory) and the matching activations are streamed into a shared-memory ring with bulk copies: warp 0
+//     fills the ring once, afterwards the warp that finishes a stage last refills its slot (no producer warp).  Eight
+//     warps dequantize in registers with the byte-table method (bf16 bits identical to the exported dequantized
+//     weights) and feed mma.sync m16n8k16 (weights = the 16-row operand, tokens = the 8-column operand, fp32
+//     accumulators).  The contraction index is permuted so that a thread supplies 4 consecutive weights of one row per
+//     MMA and reads the matching 4 activations with one 128-bit load per 8 columns.
 //   - Block scales of the CTA's rows and columns are staged once in shared memory: as fp32 s~, or, where the slices
 //     are uniform, as the 8-bit codes plus fl(v / 127) per 16 block columns (a quarter of the size; s~ is formed at use).
-//   - The rank-r intermediate T = X L2^T comes from a small kernel launched in front of this one; the two
-//     overlap (programmatic dependent launch) and T is only read in the epilogue, which adds T L1^T.
+//   - The rank-r intermediate T = X L2^T comes from a small kernel launched in front; the two overlap (programmatic
+//     dependent launch) and T L1^T is added on the tensor cores as a few more contraction steps after the main loop.
+//   - The K slices of a tile row are added through global memory: every CTA stores its fp32 sums in its own slot of
+//     the workspace and counts itself on the tile row's arrival counter; the CTA that arrives last adds the slots in
+//     slice order (the same bits on every run) and writes the bf16 output.  No clusters: the CTAs spread over all SMs,
+//     leave as soon as their sums are stored, and any number of slices is possible.  The counters are cleared by the
+//     first kernel of the call (the pre-product, or the caller's memset when there is no rank-r term).
+//   - The input gradient has the same structure with a CTA per window of 256 columns and slices of the rows.
 #pragma once
 
 #include "common.cuh"
@@ -49,9 +52,11 @@ struct Params {
     const __nv_bfloat16* T;    // [M][r], written by the kernel in front of this one (r > 0)
     const __nv_bfloat16* L1;   // [N][r]
     __nv_bfloat16* Y;          // [M][N]
+    float* partial;            // [S][M][ntiles * 128] sums of the K slices (S > 1)
+    int* counters;             // [ntiles] arrival counters, zero when the kernel starts (S > 1)
     int* status;
     int M, r;
-    int S;                     // K slices per tile row = cluster size
+    int S;                     // K slices per tile row
     int tiles_per_split;       // 64-column tiles per CTA (even)
     int nkb_cap;               // capacity of the scale table in blocks
     int stab8;                 // 1: compact scale table (codes as bytes + fl(v / 127) per 16 block columns), 0: fp32 table
@@ -118,6 +123,62 @@ __device__ __forceinline__ void dequant_chunk(const uint32_t (&w)[B], int c, con
     }
 }
 
+// Loads VW consecutive scale codes (VW = 16, 8, 4: one vector load; 1: one byte) as four words.
+template <int VW>
+__device__ __forceinline__ uint4 load_scale_codes(const uint8_t* src) {
+    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+    if constexpr (VW == 16) w = __ldg(reinterpret_cast<const uint4*>(src));
+    else if constexpr (VW == 8) { const uint2 t2 = __ldg(reinterpret_cast<const uint2*>(src)); w.x = t2.x; w.y = t2.y; }
+    else if constexpr (VW == 4) w.x = __ldg(reinterpret_cast<const uint32_t*>(src));
+    else w.x = __ldg(src);
+    return w;
+}
+
+// fp32 scale table of a forward CTA: stab[kb * kStabStride + row] = s~ of block column kb_first + kb of row
+// tile_row * 128 + row (0 for rows past N), VW codes per load (the caller has checked alignment and divisibility).
+// Two loads per thread are in flight; `after_first_loads` runs once, after the first loads have been issued.
+template <int VW, typename F>
+__device__ __forceinline__ void build_scale_table(const QView& q, int tile_row, int kb_first, int nkb, float* stab, F&& after_first_loads) {
+    const int nvec = nkb / VW;
+    const int total = nvec * 128;
+    for (int e0 = threadIdx.x; e0 < total; e0 += 2 * kThreads) {
+        uint4 sc[2];
+        float v0[2], v1[2];
+        int rowv[2], kbv[2];
+        uint32_t blkv[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int e = e0 + u * kThreads;
+            sc[u] = make_uint4(0u, 0u, 0u, 0u); v0[u] = v1[u] = 0.0f; rowv[u] = -1; kbv[u] = 0; blkv[u] = 0u;
+            if (e < total) {
+                const int row = e / nvec, kv = e - row * nvec;
+                const int grow = tile_row * 128 + row;
+                rowv[u] = row; kbv[u] = kv * VW;
+                if (grow < q.N) {
+                    const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first + kv * VW;
+                    blkv[u] = blk;
+                    sc[u] = load_scale_codes<VW>(q.sc + blk);
+                    v0[u] = __ldg(q.v + (blk >> q.logB1));
+                    v1[u] = __ldg(q.v + ((blk + VW - 1) >> q.logB1));          // B1 >= 16 >= VW: at most two groups
+                }
+            }
+        }
+        after_first_loads();
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (rowv[u] < 0) continue;
+            const uint32_t g0 = blkv[u] >> q.logB1;
+            const uint32_t words[4] = {sc[u].x, sc[u].y, sc[u].z, sc[u].w};
+#pragma unroll
+            for (int i = 0; i < VW; ++i) {
+                const uint32_t code = (words[i >> 2] >> (8 * (i & 3))) & 255u;
+                const float vv = (((blkv[u] + i) >> q.logB1) == g0) ? v0[u] : v1[u];
+                stab[(kbv[u] + i) * kStabStride + rowv[u]] = block_scale(static_cast<uint8_t>(code), vv);
+            }
+        }
+    }
+}
+
 template <int B, int NT, bool TWO>
 __global__ void __launch_bounds__(kThreads, fwd_ctas_per_sm<B, NT>())
 decode_fwd_kernel(const Params p) {
@@ -129,11 +190,12 @@ decode_fwd_kernel(const Params p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
     uint8_t* ring = base;
-    float* recv = reinterpret_cast<float*>(ring + NS * STAGE);        // [2 S sources][128 / S rows][MT] partial sums sent to this CTA
+    float* recv = reinterpret_cast<float*>(ring + NS * STAGE);        // [2 windows][MT][128 rows] sums of the two warps of a row
     float* lut8 = recv + 2 * 128 * MT;                                 // 256 floats (8-bit codes only)
     uint64_t* bars = reinterpret_cast<uint64_t*>(lut8 + (B == 8 ? 256 : 0));   // full[NS], then NS counters of warps done with a slot
     uint32_t* done = reinterpret_cast<uint32_t*>(bars + NS);
     volatile int* abort_s = reinterpret_cast<volatile int*>(bars + 2 * NS);
+    volatile int* last_s = abort_s + 1;
     float* stab = reinterpret_cast<float*>(bars + 2 * NS + 2);         // [nkb][kStabStride] block scales s~ (fp32 table)
     // compact table: s^ as bytes [nkb][kStab8Stride], then sigma = fl(v / 127) as [nkb / 16][kStabStride] floats
     const uint8_t* stab8 = reinterpret_cast<const uint8_t*>(stab);
@@ -151,38 +213,41 @@ decode_fwd_kernel(const Params p) {
 
     auto full = [&](int s) { return smem_u32(bars + s); };
 
-    // The CTAs of a cluster write into each other's shared memory at the end; a CTA's shared memory may only be
-    // touched once it runs, which the first phase of the cluster barrier establishes (arrive here, wait before
-    // the first remote store: off the critical path).
-    if (p.S > 1) cluster_arrive_relaxed();
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(full(s), 1); done[s] = 0u; }
         *abort_s = 0;
+        *last_s = 0;
         fence_barrier_init();
     }
     __syncthreads();
 
     const uint8_t* codes = reinterpret_cast<const uint8_t*>(q.codes) +
                            (static_cast<size_t>(tile_row) * q.ktiles + kt0) * (1024 * B);
-    auto issue_stage = [&](int it) {
+    // One stage by one warp: lane 0 arms the barrier and requests the packed tiles (one contiguous run), lanes
+    // 1 .. M each request one token row of the activations (a bulk copy costs its issuing thread about a hundred
+    // clocks, so the copies of a stage are issued side by side).
+    auto issue_stage = [&](int it, int ln) {
         const int s = it % NS;
         const int nt = min(kStageTiles, ntiles_cta - it * kStageTiles);
         const uint32_t dst = smem_u32(ring + s * STAGE);
-        mbar_expect_tx(full(s), nt * 1024 * B + p.M * nt * (kTileCols * 2));
-        bulk_load(dst, codes + static_cast<size_t>(it) * (kStageTiles * 1024 * B), nt * 1024 * B, full(s));
-        const __nv_bfloat16* xsrc = p.X + static_cast<size_t>(kt0 + it * kStageTiles) * kTileCols;
-        for (int m = 0; m < p.M; ++m)
-            bulk_load(dst + XOFF + m * kXRowBytes, xsrc + static_cast<size_t>(m) * q.K, nt * (kTileCols * 2), full(s));
+        if (ln == 0) {
+            mbar_expect_tx(full(s), nt * 1024 * B + p.M * nt * (kTileCols * 2));
+            bulk_load(dst, codes + static_cast<size_t>(it) * (kStageTiles * 1024 * B), nt * 1024 * B, full(s));
+        } else if (ln <= p.M) {
+            const int m = ln - 1;
+            const __nv_bfloat16* xsrc = p.X + static_cast<size_t>(kt0 + it * kStageTiles) * kTileCols + static_cast<size_t>(m) * q.K;
+            bulk_load(dst + XOFF + m * kXRowBytes, xsrc, nt * (kTileCols * 2), full(s));
+        }
     };
-    // There is no producer warp: thread 0 fills the ring once, afterwards the warp that is last to finish a stage
+    // There is no producer warp: warp 0 fills the ring once, afterwards the warp that is last to finish a stage
     // refills its slot (nobody waits for a free slot, and the CTA has eight warps, two per scheduler).  The stages are
     // small (four tiles) so that the first one of every CTA arrives early and the dequantization, which is what
-    // binds, starts while the rest of the ring is still on its way.  The first fill is issued after the first loads
-    // of the scale table below, which are few and should not queue behind the bulk copies.
+    // binds, starts while the rest of the ring is still on its way.  The first fill is issued right after the first
+    // loads of the scale table below, which are few and should not queue behind the bulk copies.
     bool ring_filled = false;
     auto fill_ring = [&]() {
-        if (!ring_filled && threadIdx.x == 0) {
-            for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it);
+        if (!ring_filled && warp == 0) {
+            for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it, lane);
         }
         ring_filled = true;
     };
@@ -190,7 +255,6 @@ decode_fwd_kernel(const Params p) {
     // block scales of the CTA's rows and columns: s~ = fl32(float(s^) * fl32(v / 127)), 0 for rows past N
     const int kb_first = (kt0 * kTileCols) >> q.logB0;
     const int nkb = (ntiles_cta > 0) ? (((kt1 * kTileCols - 1) >> q.logB0) - kb_first + 1) : 0;
-    const bool vec16 = (q.KB % 16 == 0) && (nkb % 16 == 0) && (kb_first % 16 == 0);
     if (p.stab8) {
         // the host chose this form only where every CTA meets the conditions of the 16-code loads; the 16 codes of a
         // load share their second-level group (aligned, B1 >= 16)
@@ -227,71 +291,13 @@ decode_fwd_kernel(const Params p) {
                 sg[kvv[u] * kStabStride + rowv[u]] = __fdiv_rn(v0[u], static_cast<float>(kScaleLevels));
             }
         }
-    } else if (vec16) {
-        // sixteen scale codes per load; they lie in at most two second-level groups (B1 >= 16)
-        const int nvec = nkb >> 4;
-        for (int e0 = threadIdx.x; e0 < nvec * 128; e0 += 2 * kThreads) {
-            uint4 sc16[2];
-            float v0[2], v1[2];
-            int rowv[2], kbv[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const int e = e0 + u * kThreads;
-                sc16[u] = make_uint4(0u, 0u, 0u, 0u); v0[u] = v1[u] = 0.0f; rowv[u] = -1; kbv[u] = 0;
-                if (e < nvec * 128) {
-                    const int row = e / nvec, kv = e - row * nvec;
-                    const int grow = tile_row * 128 + row;
-                    rowv[u] = row; kbv[u] = kv * 16;
-                    if (grow < q.N) {
-                        const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first + kv * 16;
-                        sc16[u] = __ldg(reinterpret_cast<const uint4*>(q.sc + blk));
-                        v0[u] = __ldg(q.v + (blk >> q.logB1));
-                        v1[u] = __ldg(q.v + ((blk + 15) >> q.logB1));
-                    }
-                }
-            }
-            fill_ring();
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                if (rowv[u] < 0) continue;
-                const int grow = tile_row * 128 + rowv[u];
-                const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first + kbv[u];
-                const uint32_t g0 = blk >> q.logB1;
-                const uint32_t words[4] = {sc16[u].x, sc16[u].y, sc16[u].z, sc16[u].w};
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const uint32_t code = (words[i >> 2] >> (8 * (i & 3))) & 255u;
-                    const float vv = (((blk + i) >> q.logB1) == g0) ? v0[u] : v1[u];
-                    stab[(kbv[u] + i) * kStabStride + rowv[u]] = block_scale(static_cast<uint8_t>(code), vv);
-                }
-            }
-        }
     } else {
-    // (four elements per thread and pass, all loads requested before the first is used)
-    for (int e0 = threadIdx.x; e0 < nkb * 128; e0 += 4 * kThreads) {
-        uint32_t sc8[4];
-        float v[4];
-        int slot[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int e = e0 + u * kThreads;
-            sc8[u] = 0u; v[u] = 0.0f; slot[u] = -1;
-            if (e < nkb * 128) {
-                const int row = e / nkb, kb = e - row * nkb;
-                const int grow = tile_row * 128 + row;
-                slot[u] = kb * kStabStride + row;
-                if (grow < q.N) {
-                    const uint32_t blk = static_cast<uint32_t>(grow) * q.KB + kb_first + kb;
-                    sc8[u] = __ldg(q.sc + blk);
-                    v[u] = __ldg(q.v + (blk >> q.logB1));
-                }
-            }
-        }
-        fill_ring();
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-            if (slot[u] >= 0) stab[slot[u]] = block_scale(static_cast<uint8_t>(sc8[u]), v[u]);
-    }
+        // as many codes per load as the alignment of the CTA's run of blocks allows
+        const int al = q.KB | nkb | kb_first;
+        if ((al & 15) == 0) build_scale_table<16>(q, tile_row, kb_first, nkb, stab, fill_ring);
+        else if ((al & 7) == 0) build_scale_table<8>(q, tile_row, kb_first, nkb, stab, fill_ring);
+        else if ((al & 3) == 0) build_scale_table<4>(q, tile_row, kb_first, nkb, stab, fill_ring);
+        else build_scale_table<1>(q, tile_row, kb_first, nkb, stab, fill_ring);
     }
     fill_ring();          // (a CTA without blocks has not passed through the loops above)
     if constexpr (B == 8) {
@@ -396,18 +402,18 @@ decode_fwd_kernel(const Params p) {
                 }
             }
             __syncwarp();
-            if (lane == 0 && slot_done(smem_u32(done + s)) == kConsumerWarps - 1) {
-                done[s] = 0u;
-                if (it + NS < nstage_total && !*abort_s) issue_stage(it + NS);
+            uint32_t last = 0u;
+            if (lane == 0) last = (slot_done(smem_u32(done + s)) == kConsumerWarps - 1) ? 1u : 0u;
+            last = __shfl_sync(0xffffffffu, last, 0);
+            if (last) {
+                // this warp is the last one done with the slot: it refills it
+                if (lane == 0) done[s] = 0u;
+                if (it + NS < nstage_total && !*abort_s) issue_stage(it + NS, lane);
             }
         }
     }
 
     // ---------------------------------------------------------------------- rank-r term, reduction, output
-    // CTA `rank` of the cluster finishes rows [rank * 128 / S, (rank + 1) * 128 / S) of the tile row
-    const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
-    const int rows_share = 128 / p.S;
-    const int row_lo = static_cast<int>(rank) * rows_share;
     __syncthreads();
     if (*abort_s) {
         // a wait gave up: let copies that are still in flight land before the CTA exits (bounded)
@@ -419,18 +425,18 @@ decode_fwd_kernel(const Params p) {
         }
         __syncthreads();
     }
-    // T L1^T on the tensor cores, as more contraction steps of the same accumulators (first CTA of the cluster only):
-    // 16 columns of the factors per MMA, lane t supplies columns 4 t .. 4 t + 3 of the rows a, b of its set and of the
-    // tokens gid (gid + 8); the warps of window 0 take the even groups of 16 columns, those of window 1 the odd ones.
-    // T was written by the kernel launched in front of this one: wait for it here (plain loads, not the read-only path).
-    if (p.r > 0 && rank == 0) {
-        pdl_wait();
+    // The kernel launched in front of this one has written T and cleared the arrival counters: wait for it here.
+    if (p.r > 0) pdl_wait();
+    // T L1^T on the tensor cores, as more contraction steps of the same accumulators (first K slice only): 16 columns
+    // of the factors per MMA, lane t supplies columns 4 t .. 4 t + 3 of the rows a, b of its set and of the tokens
+    // gid (gid + 8); the warps of window 0 take the even groups of 16 columns, those of window 1 the odd ones.
+    if (p.r > 0 && split == 0) {
         const int n0 = tile_row * 128 + slab * 32 + 4 * gid;
         for (int ch = window; ch * 16 < p.r; ch += 2) {
             const int j = ch * 16 + 4 * t;
             uint2 tk0 = make_uint2(0u, 0u), tk1 = make_uint2(0u, 0u);
-            if (gid < p.M) tk0 = *reinterpret_cast<const uint2*>(p.T + static_cast<size_t>(gid) * p.r + j);
-            if (NT == 2 && gid + 8 < p.M) tk1 = *reinterpret_cast<const uint2*>(p.T + static_cast<size_t>(gid + 8) * p.r + j);
+            if (gid < p.M) tk0 = __ldcg(reinterpret_cast<const uint2*>(p.T + static_cast<size_t>(gid) * p.r + j));
+            if (NT == 2 && gid + 8 < p.M) tk1 = __ldcg(reinterpret_cast<const uint2*>(p.T + static_cast<size_t>(gid + 8) * p.r + j));
 #pragma unroll
             for (int set = 0; set < 2; ++set) {
                 const int na = n0 + 2 * set, nb = na + 1;
@@ -442,34 +448,44 @@ decode_fwd_kernel(const Params p) {
             }
         }
     }
-    // Every warp sends its sums straight to the CTA that owns the row: recv[((src * 2 + window) * rows_share + rl) * MT + m]
-    // in the owner's shared memory takes the sum of window `window` of cluster rank `src`.  Remote stores need no round
-    // trip, and after the cluster barrier every CTA only reads its own shared memory.
-    if (p.S > 1) cluster_wait();             // every CTA of the cluster runs: its shared memory may be written
-    {
-        const uint32_t recv_addr = smem_u32(recv);
+    // the two warps that cover the same rows (windows 0 and 1) meet in shared memory: recv[(window * MT + m) * 128 + row]
 #pragma unroll
-        for (int set = 0; set < 2; ++set)
+    for (int set = 0; set < 2; ++set)
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
+        for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int row = slab * 32 + 4 * gid + 2 * set + (e >> 1);
-                    const int m = nt * 8 + 2 * t + (e & 1);
-                    if (m >= p.M) continue;                  // token rows that do not exist
-                    const int owner = row / rows_share, rl = row - owner * rows_share;
-                    const int slot = ((static_cast<int>(rank) * 2 + window) * rows_share + rl) * MT + m;
-                    if (p.S > 1) st_dsmem_f32(recv_addr + static_cast<uint32_t>(slot) * 4u, static_cast<uint32_t>(owner), acc[set][nt][e]);
-                    else recv[slot] = acc[set][nt][e];
-                }
+            for (int e = 0; e < 4; ++e) {
+                const int row = slab * 32 + 4 * gid + 2 * set + (e >> 1);
+                const int m = nt * 8 + 2 * t + (e & 1);
+                if (m < p.M) recv[(window * MT + m) * 128 + row] = acc[set][nt][e];
+            }
+    __syncthreads();
+    const int npad = q.ntiles * 128;
+    if (p.S == 1) {
+        for (int idx = threadIdx.x; idx < 128 * p.M; idx += kThreads) {
+            const int m = idx >> 7, row = idx & 127;
+            const int n = tile_row * 128 + row;
+            if (n < q.N) p.Y[static_cast<size_t>(m) * q.N + n] = __float2bfloat16_rn(recv[m * 128 + row] + recv[(MT + m) * 128 + row]);
+        }
+        return;
     }
-    if (p.S > 1) cluster_sync_all();      // all sums have arrived
-    else __syncthreads();
-    for (int idx = threadIdx.x; idx < rows_share * p.M; idx += kThreads) {
-        const int m = idx / rows_share, rl = idx - m * rows_share;
-        const int n = tile_row * 128 + row_lo + rl;
+    // several K slices: store this CTA's sums in its slot, count it on the tile row's counter; the last one adds up
+    for (int idx = threadIdx.x; idx < 128 * p.M; idx += kThreads) {
+        const int m = idx >> 7, row = idx & 127;
+        __stcg(p.partial + (static_cast<size_t>(split) * p.M + m) * npad + tile_row * 128 + row, recv[m * 128 + row] + recv[(MT + m) * 128 + row]);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) *last_s = (atomicAdd(p.counters + tile_row, 1) == p.S - 1) ? 1 : 0;
+    __syncthreads();
+    if (!*last_s) return;
+    __threadfence();
+    for (int idx = threadIdx.x; idx < 128 * p.M; idx += kThreads) {
+        const int m = idx >> 7, row = idx & 127;
+        const int n = tile_row * 128 + row;
+        const float* src = p.partial + static_cast<size_t>(m) * npad + n;
         float sum = 0.0f;
-        for (int src = 0; src < 2 * p.S; ++src) sum += recv[(src * rows_share + rl) * MT + m];
+        for (int sp = 0; sp < p.S; ++sp) sum += __ldcg(src + static_cast<size_t>(sp) * p.M * npad);
         if (n < q.N) p.Y[static_cast<size_t>(m) * q.N + n] = __float2bfloat16_rn(sum);
     }
 }
@@ -489,9 +505,11 @@ struct BwdParams {
     const __nv_bfloat16* T;    // [M][r] = dY L1, written by the kernel in front of this one (r > 0)
     const __nv_bfloat16* L2;   // [r][K]
     __nv_bfloat16* dX;         // [M][K]
+    float* partial;            // [S][M][nwin * 256] sums of the row slices (S > 1)
+    int* counters;             // [nwin] arrival counters, zero when the kernel starts (S > 1)
     int* status;
     int M, r;
-    int S;                     // row slices per column window = cluster size
+    int S;                     // row slices per column window
     int trows_per_split;       // tile rows (128 rows) per CTA, even
     int rows_stride;           // entries per block column of the scale table
     int stab8;                 // 1: compact scale table (codes as bytes [nkb][rows_stride] + fl(v / 127) per row), 0: fp32 table
@@ -517,11 +535,12 @@ decode_bwd_kernel(const BwdParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
     uint8_t* ring = base;
-    float* part = reinterpret_cast<float*>(ring + NS * STAGE);        // KF x 32 partial sums, fragment order
-    float* lut8 = part + KF * 32;
+    float* outs = reinterpret_cast<float*>(ring + NS * STAGE);        // [8 NT tokens][256 columns] sums of the CTA
+    float* lut8 = outs + KF * 32;
     uint64_t* bars = reinterpret_cast<uint64_t*>(lut8 + (B == 8 ? 256 : 0));   // full[NS], then NS counters of warps done with a slot
     uint32_t* done = reinterpret_cast<uint32_t*>(bars + NS);
     volatile int* abort_s = reinterpret_cast<volatile int*>(bars + 2 * NS);
+    volatile int* last_s = abort_s + 1;
     float* stab = reinterpret_cast<float*>(bars + 2 * NS + 2);         // [nkb][rows_stride] block scales s~
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -545,25 +564,29 @@ decode_bwd_kernel(const BwdParams p) {
     __syncthreads();
 
     const uint8_t* codes = reinterpret_cast<const uint8_t*>(q.codes);
-    auto issue_stage = [&](int it) {
+    // One stage by one warp: lane 0 arms the barrier, lanes 0 and 1 request the two runs of packed tiles, lanes
+    // 2 .. M + 1 one row of dY each (the copies of a stage are issued side by side).
+    auto issue_stage = [&](int it, int ln) {
         const int s = it % NS;
         const int ntr = min(2, ntr_cta - 2 * it);
         const uint32_t dst = smem_u32(ring + s * STAGE);
         const int row0 = (tr0 + 2 * it) * 128;
         const int nrows = min(ntr * 128, q.N - row0);             // entries of dY that exist (a multiple of 8)
-        mbar_expect_tx(full(s), ntr * ncol_tiles * 1024 * B + p.M * nrows * 2);
-        for (int j = 0; j < ntr; ++j)
-            bulk_load(dst + j * (4 * 1024 * B), codes + (static_cast<size_t>(tr0 + 2 * it + j) * q.ktiles + kt_first) * (1024 * B),
+        if (ln == 0) mbar_expect_tx(full(s), ntr * ncol_tiles * 1024 * B + p.M * nrows * 2);
+        if (ln < ntr)
+            bulk_load(dst + ln * (4 * 1024 * B), codes + (static_cast<size_t>(tr0 + 2 * it + ln) * q.ktiles + kt_first) * (1024 * B),
                       ncol_tiles * 1024 * B, full(s));
-        for (int m = 0; m < p.M; ++m)
+        else if (ln >= 2 && ln < 2 + p.M) {
+            const int m = ln - 2;
             bulk_load(dst + YOFF + m * kBwdYRowBytes, p.dY + static_cast<size_t>(m) * q.N + row0, nrows * 2, full(s));
+        }
     };
-    // thread 0 fills the ring once (after the first loads of the scale table below have been issued, so that they do
+    // warp 0 fills the ring once (after the first loads of the scale table below have been issued, so that they do
     // not queue behind the bulk copies); afterwards the warp that is last to finish a stage refills its slot
     bool ring_filled = false;
     auto fill_ring = [&]() {
-        if (!ring_filled && threadIdx.x == 0) {
-            for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it);
+        if (!ring_filled && warp == 0) {
+            for (int it = 0; it < NS && it < nstage_total; ++it) issue_stage(it, lane);
         }
         ring_filled = true;
     };
@@ -749,9 +772,12 @@ decode_bwd_kernel(const BwdParams p) {
                 }
             }
             __syncwarp();
-            if (lane == 0 && slot_done(smem_u32(done + s)) == kConsumerWarps - 1) {
-                done[s] = 0u;
-                if (it + NS < nstage_total && !*abort_s) issue_stage(it + NS);
+            uint32_t last = 0u;
+            if (lane == 0) last = (slot_done(smem_u32(done + s)) == kConsumerWarps - 1) ? 1u : 0u;
+            last = __shfl_sync(0xffffffffu, last, 0);
+            if (last) {
+                if (lane == 0) done[s] = 0u;
+                if (it + NS < nstage_total && !*abort_s) issue_stage(it + NS, lane);
             }
         }
     }
@@ -792,91 +818,78 @@ decode_bwd_kernel(const BwdParams p) {
         }
         __syncthreads();
     }
-    // Warp 0 holds the CTA's sums; each value goes straight to the CTA that finishes its column: CTA `rank` owns
-    // columns [rank * 256 / S, (rank + 1) * 256 / S) of the window.  recv[(src * cols_share + cl) * MT + m] in the
-    // owner's shared memory (`part`) takes the partial sum of cluster rank `src`; after the cluster barrier every
-    // CTA only reads its own shared memory.
+    // Warp 0 holds the CTA's sums of the quantized part, in fragment order: idx = ((mm * NT + nt) * 4 + e) * 32 + lane is
+    // column 32 (lane / 4) + 8 (mm / 4) + 2 (mm % 4) + (e >> 1) of the window and token nt * 8 + 2 (lane % 4) + (e & 1).
+    // They are laid out as out[m][column] in shared memory; the first row slice adds T' L2; then the slices of a window
+    // meet in global memory (own slot per slice, arrival counter per window, the last CTA adds them in slice order).
     constexpr int MT = 8 * NT;
-    const uint32_t rank = (p.S > 1) ? cluster_ctarank() : 0u;
-    const int cols_share = 256 / p.S;
-    const int col_lo = static_cast<int>(rank) * cols_share;
-    const int sub = threadIdx.x & 7;
-    // T' (at most 16 x 128 bf16) is staged behind the reduction buffer
-    __nv_bfloat16* tsm = reinterpret_cast<__nv_bfloat16*>(ring + 4 * KF * 128);
-    static_assert(4 * KF * 128 + 4096 <= NS * STAGE, "reduction buffer and T' must fit into the ring");
     if (warp == 0) {
 #pragma unroll
         for (int mm = 0; mm < 16; ++mm)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) red[((mm * NT + nt) * 4 + e) * 32 + lane] = acc[mm][nt][e];
+                for (int e = 0; e < 4; ++e) {
+                    const int col_local = (lane >> 2) * 32 + (mm >> 2) * 8 + (mm & 3) * 2 + (e >> 1);
+                    const int m = nt * 8 + 2 * (lane & 3) + (e & 1);
+                    outs[m * 256 + col_local] = acc[mm][nt][e];
+                }
     }
-    // Requested now, used after the cluster barrier: this thread's piece of T' (written by the kernel launched in
-    // front of this one) and, for the first pass of the epilogue, its elements L2[j][kcol], j = sub, sub + 8, ...
+    // the kernel launched in front of this one has written T' and cleared the arrival counters
     if (p.r > 0) pdl_wait();
-    const int t_vecs = p.M * p.r / 8;
-    uint4 tv = make_uint4(0u, 0u, 0u, 0u);
-    if (static_cast<int>(threadIdx.x) < t_vecs) tv = __ldg(reinterpret_cast<const uint4*>(p.T) + threadIdx.x);
-    auto load_factor = [&](int cl, float (&f)[16]) {
-        const bool live = cl < cols_share;
-        const int kcol = col_first + col_lo + (live ? cl : 0);
-        const bool col_live = live && kcol < q.K;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int jj = sub + 8 * i;
-            f[i] = (col_live && jj < p.r) ? __bfloat162float(p.L2[static_cast<size_t>(jj) * q.K + kcol]) : 0.0f;
-        }
-    };
-    float f_first[16];
-    load_factor(static_cast<int>(threadIdx.x >> 3), f_first);
     __syncthreads();
+    const int split_id = split;
+    // thread = one column of the window; the rank-r term (first row slice only): sum_j T'[m][j] L2[j][col]
     {
-        const uint32_t part_addr = smem_u32(part);
-        for (int idx = threadIdx.x; idx < KF * 32; idx += kThreads) {
-            // fragment order: idx = ((mm * NT + nt) * 4 + e) * 32 + lane; columns cA = 8 (mm / 4) + 2 (mm % 4) (e < 2) and
-            // cA + 1 (e >= 2) of group gid = lane / 4; token nt * 8 + 2 (lane % 4) + (e & 1)
-            const int ln = idx & 31, k = idx >> 5;
-            const int e = k & 3, nt = (k >> 2) % NT, mm = (k >> 2) / NT;
-            const int col_local = (ln >> 2) * 32 + (mm >> 2) * 8 + (mm & 3) * 2 + (e >> 1);
-            const int m = nt * 8 + 2 * (ln & 3) + (e & 1);
-            const int owner = col_local / cols_share, cl = col_local - owner * cols_share;
-            const uint32_t off = static_cast<uint32_t>((static_cast<int>(rank) * cols_share + cl) * MT + m) * 4u;
-            if (m >= p.M) continue;              // token rows that do not exist
-            if (p.S > 1) st_dsmem_f32(part_addr + off, static_cast<uint32_t>(owner), red[idx]);
-            else part[cl * MT + m] = red[idx];
-        }
-    }
-    if (static_cast<int>(threadIdx.x) < t_vecs) reinterpret_cast<uint4*>(tsm)[threadIdx.x] = tv;
-    for (int i = threadIdx.x + kThreads; i < t_vecs; i += kThreads)
-        reinterpret_cast<uint4*>(tsm)[i] = __ldg(reinterpret_cast<const uint4*>(p.T) + i);
-    cluster_sync_all();               // all partial sums have arrived (and T' is staged)
-    // eight lanes share an output column: each takes an eighth of the rank-r sum (its elements of the column of L2
-    // are read once for all tokens) and one rank's partial sum
-    constexpr int kColsPerPass = kThreads >> 3;
-    for (int c0 = 0; c0 < cols_share; c0 += kColsPerPass) {
-        const int cl = c0 + static_cast<int>(threadIdx.x >> 3);
-        const bool live = cl < cols_share;
-        const int kcol = col_first + col_lo + (live ? cl : 0);
-        const bool col_live = live && kcol < q.K;
-        float f[16];                  // L2[j][kcol] for j = sub, sub + 8, ... (r <= 128)
-        if (c0 == 0) {
+        const int cl = threadIdx.x;              // kThreads == 256 columns
+        const int kcol = col_first + cl;
+        const bool col_live = kcol < q.K;
+        float add[MT];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) f[i] = f_first[i];
-        } else {
-            load_factor(cl, f);
-        }
-        for (int m = 0; m < p.M; ++m) {
-            float sum = (live && sub < p.S) ? part[(sub * cols_share + cl) * MT + m] : 0.0f;
+        for (int m = 0; m < MT; ++m) add[m] = 0.0f;
+        if (p.r > 0 && split_id == 0 && col_live) {
+            for (int j0 = 0; j0 < p.r; j0 += 8) {
+                float f[8];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int jj = sub + 8 * i;
-                if (jj < p.r) sum = fmaf(__bfloat162float(tsm[static_cast<size_t>(m) * p.r + jj]), f[i], sum);
+                for (int jj = 0; jj < 8; ++jj) f[jj] = __bfloat162float(p.L2[static_cast<size_t>(j0 + jj) * q.K + kcol]);
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    if (m < p.M) {
+                        const uint4 tv = __ldcg(reinterpret_cast<const uint4*>(p.T + static_cast<size_t>(m) * p.r + j0));
+                        const uint32_t tw[4] = {tv.x, tv.y, tv.z, tv.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            add[m] = fmaf(__uint_as_float(tw[e] << 16), f[2 * e], add[m]);
+                            add[m] = fmaf(__uint_as_float(tw[e] & 0xffff0000u), f[2 * e + 1], add[m]);
+                        }
+                    }
+                }
             }
-            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 4);
-            if (col_live && sub == 0) p.dX[static_cast<size_t>(m) * q.K + kcol] = __float2bfloat16_rn(sum);
+        }
+        const int kpad = gridDim.x * 256;
+        if (p.S == 1) {
+#pragma unroll
+            for (int m = 0; m < MT; ++m)
+                if (m < p.M && col_live) p.dX[static_cast<size_t>(m) * q.K + kcol] = __float2bfloat16_rn(outs[m * 256 + cl] + add[m]);
+            return;
+        }
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+            if (m < p.M) __stcg(p.partial + (static_cast<size_t>(split_id) * p.M + m) * kpad + cw * 256 + cl, outs[m * 256 + cl] + add[m]);
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) *last_s = (atomicAdd(p.counters + cw, 1) == p.S - 1) ? 1 : 0;
+        __syncthreads();
+        if (!*last_s) return;
+        __threadfence();
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            if (m < p.M && col_live) {
+                const float* src = p.partial + static_cast<size_t>(m) * kpad + cw * 256 + cl;
+                float sum = 0.0f;
+                for (int sp = 0; sp < p.S; ++sp) sum += __ldcg(src + static_cast<size_t>(sp) * p.M * kpad);
+                p.dX[static_cast<size_t>(m) * q.K + kcol] = __float2bfloat16_rn(sum);
+            }
         }
     }
 }
@@ -892,6 +905,8 @@ struct PreParams {
     const __nv_bfloat16* F;
     __nv_bfloat16* T;
     int* status;       // cleared here: this kernel is the first of a call
+    int* counters;     // arrival counters of the linear kernel behind this one, cleared here too
+    int ncounters;
     int M, C, r;
     int chunk;         // contraction elements per CTA (multiple of 8)
     int nranks;
@@ -911,7 +926,10 @@ __global__ void __launch_bounds__(kPreThreads) decode_pre_kernel(const PreParams
     float* red = reinterpret_cast<float*>(pre_smem + static_cast<size_t>(MP) * p.chunk * 2);
     float* part = red + kPrePhases * 16 * kPreJ;
     pdl_launch_dependents();
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.status = 0;
+    if (blockIdx.x == 0 && blockIdx.y == 0) {
+        if (threadIdx.x == 0) *p.status = 0;
+        for (int i = threadIdx.x; i < p.ncounters; i += kPreThreads) p.counters[i] = 0;
+    }
     const int jl = threadIdx.x & (kPreJ - 1), ph = threadIdx.x / kPreJ;
     const int j = blockIdx.y * kPreJ + jl;
     const int c_lo = blockIdx.x * p.chunk;
@@ -993,6 +1011,34 @@ __global__ void __launch_bounds__(kPreThreads) decode_pre_kernel(const PreParams
 }
 
 // ------------------------------------------------------------------------------------ host side
+inline size_t round_up_ws(size_t x) { return (x + 255) / 256 * 256; }
+
+inline int sm_count_cached() {
+    static const int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+            cudaGetLastError();
+            v = 148;
+        }
+        return v;
+    }();
+    return n;
+}
+
+// Workspace of a decode-sized call: [status word 256 B][arrival counters][T bf16 [M][r]][slots of the slices, fp32]
+struct WsLayout {
+    size_t counters_off, counters_bytes, t_off, partial_off, total;
+};
+inline WsLayout ws_layout(int ncounters, int M, int r, int S, int out_pad) {
+    WsLayout w;
+    w.counters_off = kStatusBytes;
+    w.counters_bytes = round_up_ws(static_cast<size_t>(ncounters) * 4);
+    w.t_off = w.counters_off + w.counters_bytes;
+    w.partial_off = w.t_off + round_up_ws(static_cast<size_t>(M) * (r > 0 ? r : 1) * 2);
+    w.total = w.partial_off + (S > 1 ? round_up_ws(static_cast<size_t>(S) * M * out_pad * 4) : 0);
+    return w;
+}
+
 struct Plan {
     bool ok;
     int NT, S, tiles_per_split, nkb_cap, tile_rows, stab8;
@@ -1007,16 +1053,14 @@ inline size_t smem_bytes(int nkb_cap, bool stab8) {
            (2 * num_stages<B, NT>() + 2) * 8 + table;
 }
 
-inline int sm_count_cached() {
-    static const int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
-            cudaGetLastError();
-            v = 148;
-        }
-        return v;
-    }();
-    return n;
+// Estimated time of a grid of `n` equal CTAs of `work` units each (a unit = one 128 x 64 tile of dequantization, which
+// is what binds): the busiest SM runs ceil(n / sms) of them one after the other at full rate (CTAs that share an SM
+// share its ALU pipe), and each round of `per_sm` resident CTAs pays a fixed part (first bytes from HBM, scale table,
+// reduction) worth about `fixed` units.
+inline double grid_cost(long n, double work, int per_sm, int sms, double fixed) {
+    const long on_sm = (n + sms - 1) / sms;
+    const long rounds = (on_sm + per_sm - 1) / per_sm;
+    return static_cast<double>(on_sm) * work + fixed * static_cast<double>(rounds);
 }
 
 template <int B>
@@ -1027,13 +1071,16 @@ inline Plan make_plan(const QView& q, int M) {
     const int per_sm = (NT == 1) ? fwd_ctas_per_sm<B, 1>() : fwd_ctas_per_sm<B, 2>();
     const int sms = sm_count_cached();
     double best_cost = 0.0;
-    // Number of K slices: the one with the smallest estimated time.  The CTAs are spread over the SMs; an SM works
-    // through its CTAs two at a time where two fit (a lone CTA reaches about 0.65 of that rate); every round adds a
-    // fixed part (scale table, reduction, epilogue) worth about 18 tiles.
-    for (int S = 1; S <= 8; S *= 2) {
+    int last_tps = -1;
+    // Number of K slices: the one with the smallest estimated time (any number up to 16; more slices mean more
+    // slots to add up at the end, hence the small penalty per slice).
+    for (int S = 1; S <= 16; ++S) {
         if (S > 1 && q.ktiles / S < 2) break;
         int tps = (q.ktiles + S - 1) / S;
         tps += tps & 1;
+        if (tps == last_tps) continue;
+        last_tps = tps;
+        const int splits = (q.ktiles + tps - 1) / tps;
         // compact scale table where every CTA has the same, 16-aligned run of blocks per row
         const int cols = tps * kTileCols;
         const bool uniform = (q.ktiles % tps == 0) && (cols % q.B0 == 0) && (q.KB % 16 == 0) && ((cols >> q.logB0) % 16 == 0) &&
@@ -1042,18 +1089,20 @@ inline Plan make_plan(const QView& q, int M) {
         const size_t smem = (NT == 1) ? smem_bytes<B, 1>(nkb_cap, uniform) : smem_bytes<B, 2>(nkb_cap, uniform);
         if (smem > static_cast<size_t>(kSmemLimit)) continue;
         const int c = (per_sm == 2 && smem <= 113 * 1024) ? 2 : 1;
-        const long n = static_cast<long>(q.ntiles) * S;
-        const long k = (n * 10 - sms + sms * 10 - 1) / (sms * 10) > 0 ? (n * 10 - sms + sms * 10 - 1) / (sms * 10) : 1;   // ceil(n / sms - 0.1)
-        const double w = tps;
-        const double work = (c == 2) ? w * (2.0 * (k / 2) + (k % 2) / 0.65) : w * k / 0.65;
-        const double cost = work + 18.0 * ((k + c - 1) / c);
+        const double cost = grid_cost(static_cast<long>(q.ntiles) * splits, tps, c, sms, 12.0) + 0.25 * splits;
         if (!best.ok || cost < best_cost) {
-            best.ok = true; best.NT = NT; best.tile_rows = q.ntiles; best.S = S; best.tiles_per_split = tps; best.nkb_cap = nkb_cap;
+            best.ok = true; best.NT = NT; best.tile_rows = q.ntiles; best.S = splits; best.tiles_per_split = tps; best.nkb_cap = nkb_cap;
             best.smem = smem; best.stab8 = uniform ? 1 : 0;
             best_cost = cost;
         }
     }
     return best;
+}
+
+template <int B>
+inline size_t fwd_workspace(const QView& q, int r, int M) {
+    const Plan pl = make_plan<B>(q, M);
+    return ws_layout(q.ntiles, M, r, pl.ok ? pl.S : 1, q.ntiles * 128).total;
 }
 
 inline bool supported(const QView& q, int64_t M) {
@@ -1067,12 +1116,13 @@ inline bool supported(const QView& q, int64_t M) {
     }
 }
 
-// Launches the pre-product kernel for few rows (both directions use it).
+// Launches the pre-product kernel for few rows (both directions use it).  It is the first kernel of the call: it clears
+// the status word and the arrival counters of the linear kernel behind it.
 template <bool BWD>
-inline cudaError_t launch_pre(const __nv_bfloat16* A, const __nv_bfloat16* F, __nv_bfloat16* T, int* status, int M, int C, int r,
-                              cudaStream_t st) {
+inline cudaError_t launch_pre(const __nv_bfloat16* A, const __nv_bfloat16* F, __nv_bfloat16* T, int* status, int* counters,
+                              int ncounters, int M, int C, int r, cudaStream_t st) {
     PreParams pp;
-    pp.A = A; pp.F = F; pp.T = T; pp.status = status; pp.M = M; pp.C = C; pp.r = r;
+    pp.A = A; pp.F = F; pp.T = T; pp.status = status; pp.counters = counters; pp.ncounters = ncounters; pp.M = M; pp.C = C; pp.r = r;
     int nranks = 8;
     while (nranks > 1 && C / nranks < 512) nranks >>= 1;
     int chunk = (C + nranks - 1) / nranks;
@@ -1111,6 +1161,23 @@ inline cudaError_t launch_pre(const __nv_bfloat16* A, const __nv_bfloat16* F, __
     return cudaLaunchKernelEx(&cfg, kern, pp);
 }
 
+// Launch of a linear kernel behind the pre-product: programmatic dependent launch lets the two overlap.
+template <typename Kern, typename P>
+inline cudaError_t launch_stream_kernel(Kern kern, const P& p, dim3 grid, size_t smem, bool after_pre, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_pre ? 1 : 0;
+    count_launch(1);
+    return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
 template <int B, int NT, bool TWO>
 inline cudaError_t launch_fwd_nt(const Params& p, const Plan& pl, bool after_pre, cudaStream_t st) {
     auto kern = decode_fwd_kernel<B, NT, TWO>;
@@ -1120,71 +1187,33 @@ inline cudaError_t launch_fwd_nt(const Params& p, const Plan& pl, bool after_pre
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(pl.tile_rows, pl.S);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = pl.smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = pl.S; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = after_pre ? 2 : 1;
-    count_launch(1);
-    return cudaLaunchKernelEx(&cfg, kern, p);
+    return launch_stream_kernel(kern, p, dim3(pl.tile_rows, pl.S), pl.smem, after_pre, st);
 }
 
-// Forward for M <= 16.  ws: [status 256 B][T bf16].  When r > 0 the pre-product kernel clears the status
-// word; otherwise the caller has cleared it.
+// Forward for M <= 16.  When r > 0 the pre-product kernel clears the status word and the arrival counters; otherwise the
+// caller has cleared them (clear_bytes of the workspace).
 template <int B>
 inline cudaError_t launch_fwd(const QView& q, const void* L1, const void* L2, int r, const void* X, int M, void* Y, char* ws,
                               cudaStream_t st) {
     const Plan pl = make_plan<B>(q, M);
+    const WsLayout w = ws_layout(q.ntiles, M, r, pl.S, q.ntiles * 128);
     Params p;
     p.q = q;
     p.X = static_cast<const __nv_bfloat16*>(X);
-    p.T = reinterpret_cast<const __nv_bfloat16*>(ws + kStatusBytes);
+    p.T = reinterpret_cast<const __nv_bfloat16*>(ws + w.t_off);
     p.L1 = static_cast<const __nv_bfloat16*>(L1);
     p.Y = static_cast<__nv_bfloat16*>(Y);
+    p.partial = reinterpret_cast<float*>(ws + w.partial_off);
+    p.counters = reinterpret_cast<int*>(ws + w.counters_off);
     p.status = reinterpret_cast<int*>(ws);
     p.M = M; p.r = r; p.S = pl.S; p.tiles_per_split = pl.tiles_per_split; p.nkb_cap = pl.nkb_cap; p.stab8 = pl.stab8;
     if (r > 0) {
-        cudaError_t e = launch_pre<false>(p.X, static_cast<const __nv_bfloat16*>(L2), reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes),
-                                          p.status, M, q.K, r, st);
+        cudaError_t e = launch_pre<false>(p.X, static_cast<const __nv_bfloat16*>(L2), reinterpret_cast<__nv_bfloat16*>(ws + w.t_off),
+                                          p.status, p.counters, q.ntiles, M, q.K, r, st);
         if (e != cudaSuccess) return e;
     }
     if (q.B0 == 16) return (pl.NT == 1) ? launch_fwd_nt<B, 1, true>(p, pl, r > 0, st) : launch_fwd_nt<B, 2, true>(p, pl, r > 0, st);
     return (pl.NT == 1) ? launch_fwd_nt<B, 1, false>(p, pl, r > 0, st) : launch_fwd_nt<B, 2, false>(p, pl, r > 0, st);
-}
-
-// Number of clusters of the given launch configuration that can be resident at the same time (0 on error).
-template <typename Kern>
-inline int max_active_clusters(Kern kern, int threads, size_t smem, int cluster_y) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(1, cluster_y);
-    cfg.blockDim = dim3(threads);
-    cfg.dynamicSmemBytes = smem;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = cluster_y; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    // the answer depends on (kernel, shared memory, cluster size) only: keep the last few per kernel
-    struct Entry { const void* kern; size_t smem; int cy, n; };
-    static Entry cache[32] = {};
-    static int used = 0;
-    const void* key = reinterpret_cast<const void*>(kern);
-    for (int i = 0; i < used; ++i)
-        if (cache[i].kern == key && cache[i].smem == smem && cache[i].cy == cluster_y) return cache[i].n;
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
-    static int next = 0;
-    cache[next] = Entry{key, smem, cluster_y, n};
-    next = (next + 1) % 32;
-    if (used < 32) ++used;
-    return n;
 }
 
 struct BwdPlan {
@@ -1193,14 +1222,12 @@ struct BwdPlan {
     size_t smem;
 };
 
-// Plan for a given number of row slices S (a power of two <= 8); ok = false when it does not fit.
+// Plan for `trps` tile rows per CTA; ok = false when the scale table does not fit.
 template <int B>
-inline BwdPlan make_bwd_plan_s(const QView& q, int M, int S, bool allow_compact = true) {
+inline BwdPlan make_bwd_plan_t(const QView& q, int M, int trps, bool allow_compact) {
     BwdPlan pl{};
     pl.NT = (M <= 8) ? 1 : 2;
     pl.nwin = (q.ktiles + 3) / 4;
-    int trps = (q.ntiles + S - 1) / S;
-    trps += trps & 1;
     const int nkb_cap = (256 >> q.logB0) > 0 ? (256 >> q.logB0) : 1;      // a window is 256 aligned columns and B0 divides 256
     // compact scale table where every window is whole and its blocks of a row are aligned and share a second-level group
     const bool compact = allow_compact && (q.K % 256 == 0) && (q.KB % nkb_cap == 0) && (1 << q.logB1) >= nkb_cap;
@@ -1210,20 +1237,46 @@ inline BwdPlan make_bwd_plan_s(const QView& q, int M, int S, bool allow_compact 
     const size_t smem = 128 + ns * stage + 64 * pl.NT * 32 * 4 + (B == 8 ? 1024 : 0) + (2 * ns + 2) * 8 +
                         (compact ? static_cast<size_t>(nkb_cap) * rows_stride + static_cast<size_t>(rows_stride) * 4
                                  : static_cast<size_t>(nkb_cap) * rows_stride * 4);
-    pl.ok = smem <= static_cast<size_t>(kSmemLimit) && (S == 1 || q.ntiles / S >= 1);
-    pl.S = S; pl.trows_per_split = trps; pl.rows_stride = rows_stride; pl.smem = smem; pl.stab8 = compact ? 1 : 0; pl.nkb_cap = nkb_cap;
+    pl.ok = smem <= static_cast<size_t>(kSmemLimit);
+    pl.S = (q.ntiles + trps - 1) / trps;
+    pl.trows_per_split = trps; pl.rows_stride = rows_stride; pl.smem = smem; pl.stab8 = compact ? 1 : 0; pl.nkb_cap = nkb_cap;
     return pl;
 }
 
-// Default plan (used for the support check): the largest S that fits.
+// Number of row slices and form of the scale table: the pair with the smallest estimated time (host arithmetic only).
+// A unit of work is one tile row of the window (128 x 256 weights); the compact table costs a few conversions per use
+// (about 4 %) and wins where the fp32 table would force more slices or a single CTA per SM.
 template <int B>
 inline BwdPlan make_bwd_plan(const QView& q, int M) {
-    for (int S = 8; S >= 1; S >>= 1) {
-        const BwdPlan pl = make_bwd_plan_s<B>(q, M, S);
-        if (pl.ok) return pl;
+    BwdPlan best{};
+    double best_cost = 0.0;
+    const int NT = (M <= 8) ? 1 : 2;
+    const int per_sm = (NT == 1) ? bwd_ctas_per_sm<B, 1>() : bwd_ctas_per_sm<B, 2>();
+    const int sms = sm_count_cached();
+    for (int mode = 0; mode < 2; ++mode) {
+        int last_trps = -1;
+        for (int S = 1; S <= 32; ++S) {
+            if (S > 1 && q.ntiles / S < 1) break;
+            int trps = (q.ntiles + S - 1) / S;
+            trps += trps & 1;
+            if (trps == last_trps) continue;
+            last_trps = trps;
+            const BwdPlan c = make_bwd_plan_t<B>(q, M, trps, mode == 1);
+            if (!c.ok || (mode == 1 && !c.stab8)) continue;
+            const int on = (per_sm == 2 && c.smem <= 113 * 1024) ? 2 : 1;
+            double cost = grid_cost(static_cast<long>(c.nwin) * c.S, 4.0 * trps, on, sms, 14.0) + 0.25 * c.S;
+            if (mode == 1) cost *= 1.04;
+            if (!best.ok || cost < best_cost) { best = c; best_cost = cost; }
+        }
     }
-    BwdPlan none{};
-    return none;
+    return best;
+}
+
+template <int B>
+inline size_t bwd_workspace(const QView& q, int r, int M) {
+    const BwdPlan pl = make_bwd_plan<B>(q, M);
+    const int nwin = (q.ktiles + 3) / 4;
+    return ws_layout(nwin, M, r, pl.ok ? pl.S : 1, nwin * 256).total;
 }
 
 inline bool bwd_supported(const QView& q, int64_t M) {
@@ -1238,7 +1291,7 @@ inline bool bwd_supported(const QView& q, int64_t M) {
 }
 
 template <int B, int NT, bool TWO>
-inline cudaError_t launch_bwd_nt(BwdParams p, const QView& q, int M, bool after_pre, cudaStream_t st) {
+inline cudaError_t launch_bwd_nt(BwdParams p, const BwdPlan& pl, bool after_pre, cudaStream_t st) {
     void (*kerns[2])(BwdParams) = {decode_bwd_kernel<B, NT, TWO, false>, decode_bwd_kernel<B, NT, TWO, true>};
     static bool attr_done = false;
     if (!attr_done) {
@@ -1248,68 +1301,49 @@ inline cudaError_t launch_bwd_nt(BwdParams p, const QView& q, int M, bool after_
         }
         attr_done = true;
     }
-    // Number of row slices: the one with the smallest estimated time.  A wave of resident clusters takes the tile
-    // rows of a CTA times the CTAs that share an SM (a lone CTA does not fill the SM: factor 1.5 instead of 1) plus a
-    // fixed part (scale table, reduction, epilogue) worth about six tile rows.
-    BwdPlan pl{};
-    long best = -1;
-    // The compact scale table costs a few conversions per use (about 4 %); it wins where the fp32 table would force
-    // more slices or a single CTA per SM.
-    for (int mode = 0; mode < 2; ++mode) {
-        for (int S = 8; S >= 1; S >>= 1) {
-            const BwdPlan c = make_bwd_plan_s<B>(q, M, S, mode == 1);
-            if (!c.ok || (mode == 1 && !c.stab8)) continue;
-            const int cap = max_active_clusters(kerns[mode], kThreads, c.smem, S);
-            if (cap <= 0) continue;
-            const long waves = (c.nwin + cap - 1) / cap;
-            const bool shared_sm = static_cast<long>(cap) * S > sm_count_cached() + sm_count_cached() / 2;
-            long cost = waves * (static_cast<long>(c.trows_per_split) * (shared_sm ? 4 : 3) + 12) * 100;    // in 1/200 tile rows
-            if (mode == 1) cost += cost / 25;
-            if (best < 0 || cost < best) { best = cost; pl = c; }
-        }
-    }
-    if (!pl.ok) return cudaErrorInvalidValue;
     p.S = pl.S; p.trows_per_split = pl.trows_per_split; p.rows_stride = pl.rows_stride; p.stab8 = pl.stab8; p.nkb_cap = pl.nkb_cap;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(pl.nwin, pl.S);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = pl.smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = pl.S; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = after_pre ? 2 : 1;
-    count_launch(1);
-    return cudaLaunchKernelEx(&cfg, kerns[pl.stab8 ? 1 : 0], p);
+    return launch_stream_kernel(kerns[pl.stab8 ? 1 : 0], p, dim3(pl.nwin, pl.S), pl.smem, after_pre, st);
 }
 
-// Input gradient for M <= 16.  ws: [status 256 B][T' bf16]; same status-word convention as launch_fwd.
+// Input gradient for M <= 16; same conventions as launch_fwd.
 template <int B>
 inline cudaError_t launch_bwd(const QView& q, const void* L1, const void* L2, int r, const void* dY, int M, void* dX, char* ws,
                               cudaStream_t st) {
+    const BwdPlan pl = make_bwd_plan<B>(q, M);
+    if (!pl.ok) return cudaErrorInvalidValue;
+    const WsLayout w = ws_layout(pl.nwin, M, r, pl.S, pl.nwin * 256);
     BwdParams p;
     p.q = q;
     p.dY = static_cast<const __nv_bfloat16*>(dY);
-    p.T = reinterpret_cast<const __nv_bfloat16*>(ws + kStatusBytes);
+    p.T = reinterpret_cast<const __nv_bfloat16*>(ws + w.t_off);
     p.L2 = static_cast<const __nv_bfloat16*>(L2);
     p.dX = static_cast<__nv_bfloat16*>(dX);
+    p.partial = reinterpret_cast<float*>(ws + w.partial_off);
+    p.counters = reinterpret_cast<int*>(ws + w.counters_off);
     p.status = reinterpret_cast<int*>(ws);
-    p.M = M; p.r = r; p.S = 1; p.trows_per_split = 0; p.rows_stride = 0;
-    const int NT = (M <= 8) ? 1 : 2;
+    p.M = M; p.r = r;
     if (r > 0) {
-        cudaError_t e = launch_pre<true>(p.dY, static_cast<const __nv_bfloat16*>(L1), reinterpret_cast<__nv_bfloat16*>(ws + kStatusBytes),
-                                         p.status, M, q.N, r, st);
+        cudaError_t e = launch_pre<true>(p.dY, static_cast<const __nv_bfloat16*>(L1), reinterpret_cast<__nv_bfloat16*>(ws + w.t_off),
+                                         p.status, p.counters, pl.nwin, M, q.N, r, st);
         if (e != cudaSuccess) return e;
     }
-    if (q.B0 == 16) return (NT == 1) ? launch_bwd_nt<B, 1, true>(p, q, M, r > 0, st) : launch_bwd_nt<B, 2, true>(p, q, M, r > 0, st);
-    return (NT == 1) ? launch_bwd_nt<B, 1, false>(p, q, M, r > 0, st) : launch_bwd_nt<B, 2, false>(p, q, M, r > 0, st);
+    if (q.B0 == 16) return (pl.NT == 1) ? launch_bwd_nt<B, 1, true>(p, pl, r > 0, st) : launch_bwd_nt<B, 2, true>(p, pl, r > 0, st);
+    return (pl.NT == 1) ? launch_bwd_nt<B, 1, false>(p, pl, r > 0, st) : launch_bwd_nt<B, 2, false>(p, pl, r > 0, st);
 }
 
-// Cluster sizes the two kernels would be launched with (for lqlora_linear_path; the input gradient's choice also
-// depends on the device's occupancy answer at launch time, this is the host-side default).
+// Bytes at the head of the workspace that must be zero when the linear kernel starts (status word and arrival counters)
+// and workspace need of a decode-sized call; slices per output tile (for lqlora_linear_path).
+inline size_t clear_bytes(const QView& q, bool backward) {
+    return kStatusBytes + round_up_ws(static_cast<size_t>(backward ? (q.ktiles + 3) / 4 : q.ntiles) * 4);
+}
+inline size_t workspace_bytes(const QView& q, int r, int M, bool backward) {
+    switch (q.b0) {
+        case 2: return backward ? bwd_workspace<2>(q, r, M) : fwd_workspace<2>(q, r, M);
+        case 3: return backward ? bwd_workspace<3>(q, r, M) : fwd_workspace<3>(q, r, M);
+        case 4: return backward ? bwd_workspace<4>(q, r, M) : fwd_workspace<4>(q, r, M);
+        default: return backward ? bwd_workspace<8>(q, r, M) : fwd_workspace<8>(q, r, M);
+    }
+}
 inline int fwd_splits(const QView& q, int M) {
     switch (q.b0) {
         case 2: return make_plan<2>(q, M).S;

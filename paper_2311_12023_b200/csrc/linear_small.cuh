@@ -262,7 +262,7 @@ inline cudaError_t launch_small(const QView& q, const void* L1, const void* L2, 
     } else {
         if (r > 0) {
             if (M <= 16 && q.N % 8 == 0 && q.N <= 40960) {
-                const cudaError_t e = dec::launch_pre<true>(a, l1, T, reinterpret_cast<int*>(ws), M, q.N, r, st);
+                const cudaError_t e = dec::launch_pre<true>(a, l1, T, reinterpret_cast<int*>(ws), nullptr, 0, M, q.N, r, st);
                 if (e != cudaSuccess) return e;
             } else {
                 lowrank_pre_kernel<<<M, 256, 0, st>>>(a, l1, T, q.N, r, 1, r);

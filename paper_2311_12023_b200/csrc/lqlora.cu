@@ -32,6 +32,7 @@ static int cuda_rc(cudaError_t e) {
 // Scratch bytes one direction of the linear needs for M rows, for the kernel family it dispatches to.
 static size_t linear_need(const QView& v, int r, int64_t M, bool backward) {
     if (tc_supported(v, r, M, backward)) return tc_workspace_bytes(v.N, v.K, r, M, backward);
+    if (backward ? dec::bwd_supported(v, M) : dec::supported(v, M)) return dec::workspace_bytes(v, r, static_cast<int>(M), backward);
     const SmallPlan p = small_plan(v.N, v.K, r, M, backward);
     return kStatusBytes + p.t_bytes + p.p_bytes;
 }
@@ -63,11 +64,12 @@ static int run_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, i
     const QView v = make_view(q);
     const bool use_tc = tc_supported(v, r, M, backward);
     const bool use_decode = !use_tc && (backward ? dec::bwd_supported(v, M) : dec::supported(v, M));
-    // With a rank-r term the first kernel of the call (the pre-product) clears the status word itself and nothing else
-    // has to start at zero; otherwise a memset clears it.
+    // With a rank-r term the first kernel of the call (the pre-product) clears what has to start at zero (the status
+    // word, and the arrival counters of the weight-streaming kernels); otherwise a memset does.
     const bool first_kernel_clears = r > 0 && (use_decode || use_tc);
     if (!first_kernel_clears) {
-        if (cudaMemsetAsync(ws, 0, kStatusBytes, st) != cudaSuccess) return cuda_rc(cudaGetLastError());
+        const size_t n = use_decode ? dec::clear_bytes(v, backward) : static_cast<size_t>(kStatusBytes);
+        if (cudaMemsetAsync(ws, 0, n, st) != cudaSuccess) return cuda_rc(cudaGetLastError());
     }
     cudaError_t e = cudaSuccess;
     if (use_tc) {
