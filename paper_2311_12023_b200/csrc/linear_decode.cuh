@@ -1054,13 +1054,17 @@ inline size_t smem_bytes(int nkb_cap, bool stab8) {
 }
 
 // Estimated time of a grid of `n` equal CTAs of `work` units each (a unit = one 128 x 64 tile of dequantization, which
-// is what binds): the busiest SM runs ceil(n / sms) of them one after the other at full rate (CTAs that share an SM
-// share its ALU pipe), and each round of `per_sm` resident CTAs pays a fixed part (first bytes from HBM, scale table,
-// reduction) worth about `fixed` units.
+// is what binds).  The grid runs in waves of sms * per_sm resident CTAs; CTAs that share an SM share its ALU pipe (a
+// wave of pairs takes 2 * work), a lone CTA per SM reaches about 0.65 of the SM's rate.  The first bytes from HBM, the
+// scale table and the reduction cost about `fixed` units once, and a little per further wave (the waves overlap).
 inline double grid_cost(long n, double work, int per_sm, int sms, double fixed) {
-    const long on_sm = (n + sms - 1) / sms;
-    const long rounds = (on_sm + per_sm - 1) / per_sm;
-    return static_cast<double>(on_sm) * work + fixed * static_cast<double>(rounds);
+    const long slots = static_cast<long>(sms) * per_sm;
+    const long waves = n / slots, rem = n - waves * slots;
+    const double full = (per_sm == 2) ? 2.0 * work : work / 0.65;
+    double t = static_cast<double>(waves) * full;
+    if (rem > 0) t += (per_sm == 2 && rem > sms) ? 2.0 * work : work / 0.65;
+    const long nw = waves + (rem > 0 ? 1 : 0);
+    return t + fixed + 0.25 * fixed * static_cast<double>(nw - 1);
 }
 
 template <int B>
@@ -1089,7 +1093,9 @@ inline Plan make_plan(const QView& q, int M) {
         const size_t smem = (NT == 1) ? smem_bytes<B, 1>(nkb_cap, uniform) : smem_bytes<B, 2>(nkb_cap, uniform);
         if (smem > static_cast<size_t>(kSmemLimit)) continue;
         const int c = (per_sm == 2 && smem <= 113 * 1024) ? 2 : 1;
-        const double cost = grid_cost(static_cast<long>(q.ntiles) * splits, tps, c, sms, 12.0) + 0.25 * splits;
+        // (slices that are not whole stages, or that rule out the compact table, measured 20-40 % slower)
+        const double cost = (grid_cost(static_cast<long>(q.ntiles) * splits, tps, c, sms, 12.0) + 0.1 * splits) *
+                            ((tps % kStageTiles == 0 && q.ktiles % tps == 0) ? (uniform ? 1.0 : 1.05) : 1.3);
         if (!best.ok || cost < best_cost) {
             best.ok = true; best.NT = NT; best.tile_rows = q.ntiles; best.S = splits; best.tiles_per_split = tps; best.nkb_cap = nkb_cap;
             best.smem = smem; best.stab8 = uniform ? 1 : 0;
@@ -1264,7 +1270,8 @@ inline BwdPlan make_bwd_plan(const QView& q, int M) {
             const BwdPlan c = make_bwd_plan_t<B>(q, M, trps, mode == 1);
             if (!c.ok || (mode == 1 && !c.stab8)) continue;
             const int on = (per_sm == 2 && c.smem <= 113 * 1024) ? 2 : 1;
-            double cost = grid_cost(static_cast<long>(c.nwin) * c.S, 4.0 * trps, on, sms, 14.0) + 0.25 * c.S;
+            double cost = grid_cost(static_cast<long>(c.nwin) * c.S, 4.0 * trps, on, sms, 14.0) + 0.1 * c.S;
+            if (q.ntiles % trps != 0) cost *= 1.15;              // uneven slices
             if (mode == 1) cost *= 1.04;
             if (!best.ok || cost < best_cost) { best = c; best_cost = cost; }
         }
