@@ -184,6 +184,45 @@ int lqlora_lora_grads(const void* L1_dev, const void* L2_dev, int r, int64_t N, 
                       size_t workspace_bytes, void* stream);
 
 /*
+ * The low-rank plus quantized decomposition of Sec. 3.1 (Eq. (1)-(2), Algorithm 2), with Factorize of Sec. 3.3
+ * (Eq. (4), Algorithm 4), in nn.Linear orientation:  W [N, K] ~ deq(Q) + L1 [N, r] L2 [r, K].
+ *     Q <- 0;  repeat  L1, L2 <- Factorize(W - Q, F, r);  Q <- Quantize(W - L1 L2, c);  e_t <- error
+ *     until e_t > e_(t-1) or max_steps steps are done.
+ * error = || W - (Q + L1 L2) ||_F, or || sqrt(F) o (W - (Q + L1 L2)) ||_F when F is given (Eq. (3)); with F, Factorize
+ * takes the SVD of D_row A D_col (D_row, D_col = row / column means of sqrt(F)) and divides the factors by D_row, D_col.
+ * Factorize is a randomized SVD (footnote to Eq. (2)): range finder with the caller's test matrix Omega, `power_iters`
+ * power iterations, exact SVD of the projected (r + oversample) x K matrix; L1 = U sqrt(S), L2 = sqrt(S) V^T.
+ * The iterate before the error rose is returned (Sec. 3.1: the algorithm terminates if the error increases).
+ *   W_dev, F_dev (may be NULL) : fp32 [N, K], device, read only
+ *   out                        : N, K, cfg filled in and the three arrays allocated by the caller (as for lqlora_encode)
+ *   L1_dev [N, r], L2_dev [r, K] : fp32, device, written
+ *   omega_dev                  : fp32 [K, r + oversample] standard-normal entries, device (the random numbers of the
+ *                                method are an input); 1 <= r <= 128, 0 <= oversample <= 64
+ *   errors_host [max_steps], steps_taken : host memory; errors_host[t] = e_(t+1) for the steps that ran (the last one
+ *                                is the rejected step when the loop ended on a rise)
+ *   workspace_dev              : at least lqlora_lq_workspace_bytes (two fp32 copies of the matrix and the factors)
+ * Synchronous: the stopping rule needs the error of every step on the host; the small (r + oversample)^2
+ * factorizations run on the host between the launches.  Preparation work, not the layer's hot path.
+ * Errors: INVALID_CONFIG, INVALID_SHAPE, NULL_POINTER, MISALIGNED, WORKSPACE_TOO_SMALL, CUDA.
+ */
+int lqlora_lq_workspace_bytes(int64_t N, int64_t K, const lqlora_config* cfg, int r, int oversample, size_t* bytes);
+int lqlora_lq_decompose(const float* W_dev, const float* F_dev, lqlora_qmatrix* out, float* L1_dev, float* L2_dev, int r,
+                        int max_steps, const float* omega_dev, int oversample, int power_iters, double* errors_host,
+                        int* steps_taken, void* workspace_dev, size_t workspace_bytes, void* stream);
+/* y = bf16(x), n elements, device (the trained factors are kept in bf16 by the layer: Sec. 4, App. A). */
+int lqlora_to_bf16(const float* x_dev, void* y_dev, int64_t n, void* stream);
+
+/*
+ * The budgeted assignment of Sec. 3.2 (Algorithm 3, ILPSolve): errors[i * n_configs + c] = error(A_i, c)^2 and
+ * storage[i * n_configs + c] = storage(A_i, c) (Eq. (2) times the matrix size); picks one configuration per matrix so
+ * that the summed storage is <= budget and the summed error is minimal.  Exact dynamic programming over the Pareto
+ * frontier of (storage, error) prefixes (thinned beyond 32768 points).  Host only.  assignment: [n_matrices];
+ * total_error / total_storage may be NULL.  Returns LQLORA_ERR_UNSUPPORTED when no assignment fits the budget.
+ */
+int lqlora_assign_configs(const double* errors, const double* storage, int n_matrices, int n_configs, double budget,
+                          int* assignment, double* total_error, double* total_storage);
+
+/*
  * Forward pass for callers that are not allowed to allocate device memory (no counterpart in the
  * paper: this entry point exists for deployment reasons only).  Typical examples are an inference
  * server whose memory pool was carved up at start-up, or code running inside another framework's

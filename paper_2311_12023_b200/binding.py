@@ -25,6 +25,7 @@ EXPORTS = [
     "lqlora_static_scratch_bytes", "lqlora_linear_fwd_static", "lqlora_static_scratch_status",
     "lqlora_encode_search_clearance",
     "lqlora_lora_grads_workspace_bytes", "lqlora_lora_grads",
+    "lqlora_lq_workspace_bytes", "lqlora_lq_decompose", "lqlora_to_bf16", "lqlora_assign_configs",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20   # size of the scratch array compiled into the library (lqlora_static_scratch_bytes)
@@ -80,6 +81,10 @@ def lib() -> ctypes.CDLL:
         L.lqlora_encode_search_clearance.restype = ctypes.c_double
         L.lqlora_linear_fwd_static.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp]
         L.lqlora_static_scratch_status.argtypes = [vp]
+        L.lqlora_lq_workspace_bytes.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, ci, ctypes.POINTER(sz)]
+        L.lqlora_lq_decompose.argtypes = [vp, vp, ctypes.POINTER(CQMatrix), vp, vp, ci, ci, vp, ci, ci, vp, ctypes.POINTER(ci), vp, sz, vp]
+        L.lqlora_to_bf16.argtypes = [vp, vp, i64, vp]
+        L.lqlora_assign_configs.argtypes = [vp, vp, ci, ci, ctypes.c_double, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
         L.lqlora_linear_path.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ci, ctypes.POINTER(ci)]
         L.lqlora_launch_count.restype = i64
         L.lqlora_status_string.argtypes = [ci]
@@ -319,6 +324,52 @@ def linear_fwd_host(q, L1, L2, X_host, Y_host, X_stage, Y_stage, workspace) -> N
 def linear_bwd_input_host(q, L1, L2, dY_host, dX_host, dY_stage, dX_stage, workspace) -> None:
     _linear_host(lib().lqlora_linear_bwd_input_host, "lqlora_linear_bwd_input_host", q, L1, L2, dY_host, dX_host,
                  dY_stage, dX_stage, workspace)
+
+
+def lq_decompose(W: torch.Tensor, cfg, r: int, omega: torch.Tensor, F: Optional[torch.Tensor] = None, max_steps: int = 20,
+                 power_iters: int = 4):
+    """lqlora_lq_decompose: W fp32 [N, K] -> (QMatrix, L1 fp32 [N, r], L2 fp32 [r, K], errors of the steps that ran)."""
+    assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous() and W.dim() == 2
+    N, K = W.shape
+    assert omega.is_cuda and omega.dtype == torch.float32 and omega.is_contiguous() and omega.shape[0] == K and omega.shape[1] >= r
+    p = omega.shape[1] - r
+    q = alloc_qmatrix(N, K, cfg, W.device)
+    L1 = torch.empty((N, r), dtype=torch.float32, device=W.device)
+    L2 = torch.empty((r, K), dtype=torch.float32, device=W.device)
+    c = _cfg(cfg)
+    need = ctypes.c_size_t(0)
+    _check(lib().lqlora_lq_workspace_bytes(N, K, ctypes.byref(c), r, p, ctypes.byref(need)), "lqlora_lq_workspace_bytes")
+    ws = torch.empty(int(need.value), dtype=torch.uint8, device=W.device)
+    errs = np.zeros(max_steps, dtype=np.float64)
+    steps = ctypes.c_int(0)
+    cs = q.cstruct()
+    _check(lib().lqlora_lq_decompose(W.data_ptr(), _ptr(F), ctypes.byref(cs), L1.data_ptr(), L2.data_ptr(), r, max_steps,
+                                     omega.data_ptr(), p, power_iters, errs.ctypes.data, ctypes.byref(steps), ws.data_ptr(),
+                                     ws.numel(), _stream()), "lqlora_lq_decompose")
+    return q, L1, L2, errs[:steps.value].copy()
+
+
+def to_bf16(x: torch.Tensor) -> torch.Tensor:
+    """lqlora_to_bf16."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    y = torch.empty(x.shape, dtype=torch.bfloat16, device=x.device)
+    _check(lib().lqlora_to_bf16(x.data_ptr(), y.data_ptr(), x.numel(), _stream()), "lqlora_to_bf16")
+    return y
+
+
+def assign_configs(errors: np.ndarray, storage: np.ndarray, budget: float):
+    """lqlora_assign_configs: errors, storage [n_matrices, n_configs] -> (assignment, total error, total storage) or None."""
+    E = np.ascontiguousarray(errors, dtype=np.float64)
+    S = np.ascontiguousarray(storage, dtype=np.float64)
+    assert E.shape == S.shape and E.ndim == 2
+    out = np.zeros(E.shape[0], dtype=np.int32)
+    te, ts = ctypes.c_double(0), ctypes.c_double(0)
+    rc = lib().lqlora_assign_configs(E.ctypes.data, S.ctypes.data, E.shape[0], E.shape[1], float(budget), out.ctypes.data,
+                                     ctypes.byref(te), ctypes.byref(ts))
+    if rc == -8:
+        return None
+    _check(rc, "lqlora_assign_configs")
+    return [int(a) for a in out], float(te.value), float(ts.value)
 
 
 def static_scratch_status() -> int:

@@ -9,6 +9,8 @@
 #include "linear_small.cuh"
 #include "linear_tc.cuh"
 #include "lora_grad.cuh"
+#include "lq_decompose.cuh"
+#include "config_search.cuh"
 
 namespace lq {
 
@@ -275,6 +277,61 @@ int lqlora_lora_grads(const void* L1_dev, const void* L2_dev, int r, int64_t N, 
     if (workspace_bytes < tc::lora_grads_workspace(N, K, r, M)) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
     return tc::lora_grads_launch(L1_dev, L2_dev, r, N, K, X_dev, dY_dev, M, dL1_dev, dL2_dev, static_cast<char*>(workspace_dev),
                                  static_cast<cudaStream_t>(stream));
+}
+
+int lqlora_lq_workspace_bytes(int64_t N, int64_t K, const lqlora_config* cfg, int r, int oversample, size_t* bytes) {
+    using namespace lq;
+    int rc = check_config(cfg);
+    if (rc != LQLORA_OK) return rc;
+    rc = check_shape(N, K, cfg);
+    if (rc != LQLORA_OK) return rc;
+    if (r < 1 || r > 128 || oversample < 0 || oversample > 64 || r + oversample > N || r + oversample > K) return LQLORA_ERR_INVALID_SHAPE;
+    if (!bytes) return LQLORA_ERR_NULL_POINTER;
+    *bytes = lqd::workspace_bytes(N, K, cfg, r, oversample);
+    return LQLORA_OK;
+}
+
+int lqlora_lq_decompose(const float* W_dev, const float* F_dev, lqlora_qmatrix* out, float* L1_dev, float* L2_dev, int r,
+                        int max_steps, const float* omega_dev, int oversample, int power_iters, double* errors_host,
+                        int* steps_taken, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    using namespace lq;
+    if (!W_dev || !L1_dev || !L2_dev || !omega_dev || !errors_host || !steps_taken || !workspace_dev) return LQLORA_ERR_NULL_POINTER;
+    int rc = check_qmatrix(out);
+    if (rc != LQLORA_OK) return rc;
+    if (r < 1 || r > 128 || oversample < 0 || oversample > 64 || r + oversample > out->N || r + oversample > out->K) return LQLORA_ERR_INVALID_SHAPE;
+    if (max_steps < 1 || max_steps > 1000 || power_iters < 0 || power_iters > 16) return LQLORA_ERR_INVALID_SHAPE;
+    if (!aligned16(W_dev) || !aligned16(L1_dev) || !aligned16(L2_dev) || !aligned16(omega_dev) || !aligned16(workspace_dev) ||
+        (F_dev && !aligned16(F_dev)))
+        return LQLORA_ERR_MISALIGNED;
+    if (workspace_bytes < lqd::workspace_bytes(out->N, out->K, &out->cfg, r, oversample)) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
+    rc = ensure_tables();
+    if (rc != LQLORA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace_dev);
+    *steps_taken = 0;
+    switch (out->cfg.b0) {
+        case 2: return lqd::run<2>(W_dev, F_dev, out, L1_dev, L2_dev, r, max_steps, omega_dev, oversample, power_iters, errors_host, steps_taken, ws, st);
+        case 3: return lqd::run<3>(W_dev, F_dev, out, L1_dev, L2_dev, r, max_steps, omega_dev, oversample, power_iters, errors_host, steps_taken, ws, st);
+        case 4: return lqd::run<4>(W_dev, F_dev, out, L1_dev, L2_dev, r, max_steps, omega_dev, oversample, power_iters, errors_host, steps_taken, ws, st);
+        default: return lqd::run<8>(W_dev, F_dev, out, L1_dev, L2_dev, r, max_steps, omega_dev, oversample, power_iters, errors_host, steps_taken, ws, st);
+    }
+}
+
+int lqlora_to_bf16(const float* x_dev, void* y_dev, int64_t n, void* stream) {
+    if (!x_dev || !y_dev) return LQLORA_ERR_NULL_POINTER;
+    if (n <= 0) return LQLORA_ERR_INVALID_SHAPE;
+    lq::lqd::to_bf16_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        x_dev, static_cast<__nv_bfloat16*>(y_dev), n);
+    lq::count_launch(1);
+    return lq::cuda_rc(cudaGetLastError());
+}
+
+int lqlora_assign_configs(const double* errors, const double* storage, int n_matrices, int n_configs, double budget,
+                          int* assignment, double* total_error, double* total_storage) {
+    if (!errors || !storage || !assignment) return LQLORA_ERR_NULL_POINTER;
+    if (n_matrices < 1 || n_configs < 1) return LQLORA_ERR_INVALID_SHAPE;
+    return lq::cfgsearch::assign(errors, storage, n_matrices, n_configs, budget, assignment, total_error, total_storage) == 0
+               ? LQLORA_OK : LQLORA_ERR_UNSUPPORTED;
 }
 
 int lqlora_encode_host(const float* W_host, float* W_stage_dev, lqlora_qmatrix* out, void* workspace_dev,

@@ -143,3 +143,27 @@ def test_dispatch_between_the_weight_streaming_and_the_tensor_core_kernels(bindi
     assert kernel == PAIR and splits == 1
     kernel, splits = binding.linear_route(4096, 4096, cfg, 64, 1, False)
     assert kernel == S and 1 <= splits <= 8
+
+
+def test_budgeted_assignment_matches_exhaustive_search(binding):
+    """lqlora_assign_configs (Sec. 3.2, Algorithm 3) against the oracle's enumeration on random small instances."""
+    from oracle import lq
+    g = inputs.rng(123)
+    for trial in range(30):
+        n, m = int(g.integers(1, 6)), int(g.integers(1, 5))
+        S = np.sort(g.uniform(1.0, 10.0, (n, m)), axis=1)
+        E = -np.sort(-g.uniform(0.0, 5.0, (n, m)), axis=1)          # more storage, less error
+        budget = float(g.uniform(S[:, 0].sum() * 0.9, S[:, -1].sum() * 1.1))
+        want = lq.ilp_solve(S, E, budget)
+        got = binding.assign_configs(E, S, budget)
+        if want is None:
+            assert got is None
+            continue
+        assert got is not None and got[2] <= budget + 1e-12
+        assert abs(got[1] - want[1]) < 1e-12                          # same optimal error (the argmin may tie)
+        assert abs(sum(E[i, a] for i, a in enumerate(got[0])) - got[1]) < 1e-12
+    # non-monotone tables are handled too (a configuration that is worse in both respects is never chosen)
+    S = np.array([[1.0, 2.0, 3.0]])
+    E = np.array([[5.0, 7.0, 1.0]])
+    assert binding.assign_configs(E, S, 2.5)[0] == [0]
+    assert binding.assign_configs(E, S, 3.0)[0] == [2]
