@@ -39,6 +39,7 @@ def _load():
         lib.oracle_storage_bits_per_param.argtypes = [c_int] * 5
         lib.oracle_storage_bits_per_param.restype = ctypes.c_double
         lib.oracle_encode.argtypes = [vp, c_i64, c_i64, c_int, c_int, c_int, c_int, vp, vp, vp, vp]
+        lib.oracle_cast_scale2.argtypes = [vp, c_i64, c_int, vp]
         lib.oracle_dequant.argtypes = [vp, vp, vp, c_i64, c_i64, c_int, c_int, c_int, c_int, vp, vp]
         lib.oracle_linear_fwd.argtypes = [vp, vp, vp, c_int, vp, c_i64, c_i64, c_i64, vp, c_i64, vp]
         lib.oracle_linear_bwd_input.argtypes = [vp, vp, vp, c_int, vp, c_i64, c_i64, c_i64, vp, c_i64, vp]
@@ -89,6 +90,15 @@ def encode(A: np.ndarray, b0: int, B0: int, b1: int = 8, B1: int = 256):
     if rc != 0:
         raise ValueError("oracle_encode: invalid arguments")
     return codes, absmax, sc, v
+
+
+def cast_scale2(v: np.ndarray, b2: int) -> np.ndarray:
+    """cast(v, b2): 32 = fp32, 16 = fp16, -16 = bf16; returns the fp32 values the stored numbers decode to."""
+    v = _chk(v, np.float32)
+    out = np.empty_like(v)
+    if _load().oracle_cast_scale2(_p(v), v.size, b2, _p(out)) != 0:
+        raise ValueError("oracle_cast_scale2: invalid kind")
+    return out
 
 
 def dequant(codes: np.ndarray, scale_codes: np.ndarray, scale2: np.ndarray, b0: int, B0: int,

@@ -63,9 +63,42 @@ inline uint16_t f32_to_bf16_rne(float f) {
     return static_cast<uint16_t>(u >> 16);
 }
 
+// fp32 -> IEEE binary16 -> fp32, round to nearest, ties to even, written from the format's definition: 5 exponent bits
+// (bias 15), 10 fraction bits, subnormals down to 2^-24, overflow to infinity beyond 65504 + half an ulp.
+inline float round_through_fp16(float f) {
+    if (std::isnan(f) || std::isinf(f) || f == 0.0f) return f;
+    const double a = std::fabs(static_cast<double>(f));
+    int e;
+    std::frexp(a, &e);                    // a = m * 2^e, 0.5 <= m < 1  ->  a in [2^(e-1), 2^e)
+    int ex = e - 1;                       // binade exponent
+    if (ex < -14) ex = -14;               // subnormal range shares the spacing of the lowest binade
+    const double ulp = std::ldexp(1.0, ex - 10);
+    double qd = a / ulp;                  // exact (power-of-two scaling)
+    double fl = std::floor(qd);
+    const double frac = qd - fl;
+    if (frac > 0.5 || (frac == 0.5 && std::fmod(fl, 2.0) == 1.0)) fl += 1.0;
+    double r = fl * ulp;
+    if (r > 65504.0) r = INFINITY;
+    return static_cast<float>(f < 0 ? -r : r);
+}
+
 }  // namespace
 
 extern "C" {
+
+// ----------------------------------------------------------------------------------
+// cast(v, b2) of Sec. 3.2 for the second-level scales: kind 32 = fp32 (identity), 16 = IEEE fp16, -16 = bfloat16;
+// round to nearest even, result returned as the fp32 value the stored number decodes to.
+// ----------------------------------------------------------------------------------
+int oracle_cast_scale2(const float* v, int64_t n, int kind, float* out) {
+    if (kind != 32 && kind != 16 && kind != -16) return -1;
+    for (int64_t i = 0; i < n; ++i) {
+        if (kind == 32) out[i] = v[i];
+        else if (kind == 16) out[i] = round_through_fp16(v[i]);
+        else out[i] = static_cast<float>(bf16_to_double(f32_to_bf16_rne(v[i])));
+    }
+    return 0;
+}
 
 // ----------------------------------------------------------------------------------
 // NF codebook, Sec. 2.2: 2^(b-1) evenly spaced probabilities on [delta, 1/2] and

@@ -302,6 +302,45 @@ def test_dequant_bf16_rounding_ties_go_to_even():
         assert d32[0, 0] == tt and d16[0, 0] == want
 
 
+def test_cast_of_second_level_scales():
+    """cast(v, b2) (Sec. 3.2, Table 1: bf16 / fp16 / fp32) against numpy's own half-precision conversion, on random
+    values, exact ties, subnormals and the overflow edge; bf16 against hand-written ties; fp32 is the identity."""
+    g = inputs.rng(31)
+    v = np.concatenate([
+        np.abs(g.standard_normal(4000)).astype(np.float32) * np.float32(0.05),
+        (10.0 ** g.uniform(-9, 4.8, 4000)).astype(np.float32),
+        np.array([0.0, 1.0, 1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 2.0 ** -24, 2.0 ** -25, 3 * 2.0 ** -25, 65504.0, 65519.9, 65520.0,
+                  6.1e-5, 5.9e-8], dtype=np.float32)])
+    with np.errstate(over="ignore"):
+        want = v.astype(np.float16).astype(np.float32)
+    assert np.array_equal(oracle.cast_scale2(v, 16), want)
+    assert np.array_equal(oracle.cast_scale2(v, 32), v)
+    b = oracle.cast_scale2(np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 0.3], dtype=np.float32), -16)
+    assert b[0] == 1.0 and b[1] == 1.0 + 2.0 ** -6 and b[2] == inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(np.array([0.3])))[0]
+    with pytest.raises(ValueError):
+        oracle.cast_scale2(v, 8)
+
+
+@pytest.mark.parametrize("b1", [2, 3, 4])
+def test_scale_quantization_with_fewer_bits(b1):
+    """Quantize-INT with b1 bits (Table 1): levels 2^(b1-1) - 1; multiples of v / levels are stored exactly, the block
+    that holds the group maximum gets the top level, everything else rounds to the nearest level."""
+    levels = 2 ** (b1 - 1) - 1
+    B0, B1 = 16, 16
+    v = np.float32(0.75)
+    step = np.float32(v / np.float32(levels))
+    A = np.zeros((1, B0 * B1), dtype=np.float32)
+    want = [(i % (levels + 1)) for i in range(B1)]
+    want[0] = levels
+    for i, lv in enumerate(want):
+        A[0, i * B0] = np.float32(lv) * step
+    _, absmax, sc, v2 = oracle.encode(A, 3, B0, b1, B1)
+    assert v2[0] == absmax.max() and list(sc) == want
+    codes = np.full((1, B0 * B1), 7, dtype=np.uint8)                 # q = +1 everywhere: w~ = s~
+    d32, _ = oracle.dequant(codes, sc, v2, 3, B0, b1, B1)
+    assert np.array_equal(d32[0, ::B0], np.array(want, dtype=np.float32) * np.float32(v2[0] / np.float32(levels)))
+
+
 # --------------------------------------------------------------------------- layer
 def _layer_case(seed, N, K, M, r):
     W = inputs.gaussian(seed, (N, K), 0.02)
