@@ -61,7 +61,7 @@ def linear_flops(M: int, N: int, K: int, r: int) -> float:
 
 
 def packed_bytes(N: int, K: int, cfg) -> float:
-    return N * K * (cfg.b0 + cfg.b1 / cfg.B0 + cfg.b2 / (cfg.B0 * cfg.B1)) / 8.0
+    return N * K * (cfg.b0 + cfg.b1 / cfg.B0 + abs(cfg.b2) / (cfg.B0 * cfg.B1)) / 8.0
 
 
 def encode_bytes(N: int, K: int, cfg) -> float:

@@ -43,7 +43,8 @@ extern "C" {
 typedef enum {
     LQLORA_OK = 0,
     LQLORA_ERR_INVALID_CONFIG = -1,   /* b0 not in {2,3,4,8}; B0 not a power of two in [16,256];
-                                         B1 not a power of two in [16,4096]; b1 != 8; b2 != 32     */
+                                         B1 not a power of two in [16,4096]; b1 not in {2,3,4,8};
+                                         b2 not one of LQLORA_B2_*                                  */
     LQLORA_ERR_INVALID_SHAPE = -2,    /* N, K, M <= 0; K % 64 != 0; K % B0 != 0; r % 16 != 0; r > 128 */
     LQLORA_ERR_NULL_POINTER = -3,
     LQLORA_ERR_MISALIGNED = -4,       /* a device pointer is not 16-byte aligned                    */
@@ -53,22 +54,26 @@ typedef enum {
     LQLORA_ERR_UNSUPPORTED = -8       /* valid arguments that this build has no kernel for          */
 } lqlora_status;
 
-/* Configuration tuple c = (b0, b1, b2, B0, B1) of Sec. 3.2. */
+/* Configuration tuple c = (b0, b1, b2, B0, B1) of Sec. 3.2 (search space: Table 1). */
+enum { LQLORA_B2_FP32 = 32, LQLORA_B2_FP16 = 16, LQLORA_B2_BF16 = -16 };
 typedef struct {
     int b0;   /* bits of a NormalFloat code: 2, 3, 4 or 8                         */
     int B0;   /* weights per first-level block (along K): 16, 32, 64, 128, 256    */
-    int b1;   /* bits of a quantized block scale: 8                               */
+    int b1;   /* bits of a quantized block scale: 2, 3, 4 or 8                    */
     int B1;   /* blocks per second-level group (flattened row-major block order)  */
-    int b2;   /* bits of a second-level scale: 32 (fp32; cast(v, fp32) = v)       */
+    int b2;   /* format of a second-level scale, cast(v, b2): LQLORA_B2_FP32, _FP16 (IEEE half) or _BF16;
+                 the storage formula counts |b2| bits                              */
 } lqlora_config;
 
 /*
  * A quantized matrix.  All three arrays are device memory owned by the caller, each 16-byte
  * aligned, of the sizes lqlora_packed_sizes reports.
  *
- *   scale_codes  uint8 [N * K / B0]      s^_i, flattened row-major block order (block i covers
- *                                        elements [i*B0, (i+1)*B0) of the row-major matrix)
- *   scale2       fp32  [ceil(nblk / B1)] v_g = absmax of the block scales of group g
+ *   scale_codes  s^_i in flattened row-major block order (block i covers elements [i*B0, (i+1)*B0) of the
+ *                row-major matrix): one byte each for b1 = 8; for b1 < 8 a bit stream of b1 bits each, code i in
+ *                bits [i*b1, (i+1)*b1) of the little-endian byte stream (eight codes take b1 bytes)
+ *   scale2       v_g = absmax of the block scales of group g, [ceil(nblk / B1)] numbers in the format b2 names
+ *                (lqlora_unpack_scales returns both arrays as one byte per code and fp32)
  *   codes        packed b0-bit codes, exactly b0 bits per weight when N % 128 == 0 (rows are
  *                padded to a multiple of 128 otherwise).  Layout ("tile-interleaved bitstream"):
  *                  - the matrix is cut into tiles of 128 rows x 64 columns, stored one after the
@@ -121,7 +126,10 @@ int lqlora_nf_codebook(int b0, float* out_host);
  *   v_g  = max s_i over group g (B1 consecutive blocks; the last group may be short);
  *   s^_i = clamp(round_half_even(fl32(s_i / fl32(v_g / 127))), 0, 127); 0 if v_g = 0.
  * out->N, K, cfg must be filled in and its three arrays allocated by the caller.
- * workspace_dev: device scratch of at least encode_workspace_bytes (block absmax values in fp32).
+ * With b1 < 8 the codes use the 2^(b1-1) - 1 levels of the b1-bit quantizer (127 above becomes that number); the
+ * stored second-level scale is cast(v_g, b2), computed after the scale codes (which use the uncast v_g).
+ * workspace_dev: device scratch of at least encode_workspace_bytes (block absmax values in fp32, and the unpacked
+ * scales before packing when b1 < 8 or b2 is a 16-bit format).
  * Errors: INVALID_CONFIG, INVALID_SHAPE, NULL_POINTER, MISALIGNED, WORKSPACE_TOO_SMALL, CUDA.
  */
 int lqlora_encode(const float* W_dev, lqlora_qmatrix* out, void* workspace_dev,
@@ -135,6 +143,9 @@ int lqlora_encode(const float* W_dev, lqlora_qmatrix* out, void* workspace_dev,
  *   Either output may be NULL. */
 int lqlora_unpack(const lqlora_qmatrix* q, uint8_t* codes_dev, void* stream);
 int lqlora_dequant(const lqlora_qmatrix* q, float* deq32_dev, void* deq16_dev, void* stream);
+/* The scales in plain form: scale_codes_dev uint8 [N*K/B0] (one code per byte), scale2_dev fp32 [ngrp] (the value each
+ * stored second-level scale decodes to), whatever b1 and b2 are (Sec. 3.2: s^ and cast(v, b2)). */
+int lqlora_unpack_scales(const lqlora_qmatrix* q, uint8_t* scale_codes_dev, float* scale2_dev, void* stream);
 
 /* Bytes of device scratch lqlora_linear_fwd / lqlora_linear_bwd_input need for M rows.
  * Returns 0 (and sets *bytes) or an error.  Host only. */
@@ -163,6 +174,20 @@ int lqlora_linear_fwd(const lqlora_qmatrix* q, const void* L1_dev, const void* L
 int lqlora_linear_bwd_input(const lqlora_qmatrix* q, const void* L1_dev, const void* L2_dev, int r,
                             const void* dY_dev, int64_t M, void* dX_dev, void* workspace_dev,
                             size_t workspace_bytes, void* stream);
+
+/*
+ * The layer with quantized factors (compression setting of Sec. 4.2: after training, L1 and L2 are themselves stored in
+ * NF-8, i.e. Quantize with b0 = 8): qL1 is the [N, r] factor and qL2 the [r, K] factor as quantized matrices (any
+ * configuration; r a multiple of 64 so that qL1's rows satisfy the K % 64 rule).  Computes what lqlora_linear_fwd /
+ * lqlora_linear_bwd_input compute with L1 = deq16(qL1), L2 = deq16(qL2); the factors are dequantized to bf16 inside the
+ * workspace (lqlora_linear_qfactors_workspace_bytes).  Errors as for lqlora_linear_fwd.
+ */
+int lqlora_linear_qfactors_workspace_bytes(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, size_t* bytes);
+int lqlora_linear_fwd_qfactors(const lqlora_qmatrix* q, const lqlora_qmatrix* qL1, const lqlora_qmatrix* qL2, const void* X_dev,
+                               int64_t M, void* Y_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
+int lqlora_linear_bwd_input_qfactors(const lqlora_qmatrix* q, const lqlora_qmatrix* qL1, const lqlora_qmatrix* qL2,
+                                     const void* dY_dev, int64_t M, void* dX_dev, void* workspace_dev, size_t workspace_bytes,
+                                     void* stream);
 
 /*
  * Gradients of the low-rank factors (the trained parameters: Sec. 1, Sec. 2.1; layer of Sec. 3.1).  With the layer

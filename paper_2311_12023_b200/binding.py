@@ -26,6 +26,8 @@ EXPORTS = [
     "lqlora_encode_search_clearance",
     "lqlora_lora_grads_workspace_bytes", "lqlora_lora_grads",
     "lqlora_lq_workspace_bytes", "lqlora_lq_decompose", "lqlora_to_bf16", "lqlora_assign_configs",
+    "lqlora_unpack_scales", "lqlora_linear_qfactors_workspace_bytes", "lqlora_linear_fwd_qfactors",
+    "lqlora_linear_bwd_input_qfactors",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20   # size of the scratch array compiled into the library (lqlora_static_scratch_bytes)
@@ -81,6 +83,10 @@ def lib() -> ctypes.CDLL:
         L.lqlora_encode_search_clearance.restype = ctypes.c_double
         L.lqlora_linear_fwd_static.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp]
         L.lqlora_static_scratch_status.argtypes = [vp]
+        L.lqlora_unpack_scales.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, vp]
+        L.lqlora_linear_qfactors_workspace_bytes.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ctypes.POINTER(sz)]
+        L.lqlora_linear_fwd_qfactors.argtypes = [ctypes.POINTER(CQMatrix)] * 3 + [vp, i64, vp, vp, sz, vp]
+        L.lqlora_linear_bwd_input_qfactors.argtypes = [ctypes.POINTER(CQMatrix)] * 3 + [vp, i64, vp, vp, sz, vp]
         L.lqlora_lq_workspace_bytes.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, ci, ctypes.POINTER(sz)]
         L.lqlora_lq_decompose.argtypes = [vp, vp, ctypes.POINTER(CQMatrix), vp, vp, ci, ci, vp, ci, ci, vp, ctypes.POINTER(ci), vp, sz, vp]
         L.lqlora_to_bf16.argtypes = [vp, vp, i64, vp]
@@ -169,8 +175,8 @@ def launch_count() -> int:
 class QMatrix:
     """Device arrays of one quantized matrix (owned here, as torch tensors)."""
     codes: torch.Tensor        # uint8 buffer holding the packed code words
-    scale_codes: torch.Tensor  # uint8 [nblk]
-    scale2: torch.Tensor       # float32 [ngrp]
+    scale_codes: torch.Tensor  # uint8: one code per byte (b1 = 8) or the packed bit stream (b1 < 8)
+    scale2: torch.Tensor       # float32 [ngrp] (b2 = fp32) or a byte buffer holding fp16 / bf16 numbers
     N: int
     K: int
     cfg: object
@@ -181,14 +187,18 @@ class QMatrix:
 
     @property
     def packed_bytes(self) -> int:
-        return self.codes.numel() + self.scale_codes.numel() + 4 * self.scale2.numel()
+        return self.codes.numel() + self.scale_codes.numel() + self.scale2.numel() * self.scale2.element_size()
 
 
 def alloc_qmatrix(N: int, K: int, cfg, device="cuda") -> QMatrix:
     cb, sb, s2b, _ = packed_sizes(N, K, cfg)
+    if int(cfg.b2) == 32:
+        s2 = torch.empty(s2b // 4, dtype=torch.float32, device=device)
+    else:
+        s2 = torch.zeros((s2b + 15) // 16 * 16, dtype=torch.uint8, device=device)
     return QMatrix(torch.empty(cb, dtype=torch.uint8, device=device),
-                   torch.empty(sb, dtype=torch.uint8, device=device),
-                   torch.empty(s2b // 4, dtype=torch.float32, device=device), N, K, cfg)
+                   torch.zeros((sb + 15) // 16 * 16, dtype=torch.uint8, device=device) if int(cfg.b1) != 8 else
+                   torch.empty(sb, dtype=torch.uint8, device=device), s2, N, K, cfg)
 
 
 def encode(W: torch.Tensor, cfg, out: Optional[QMatrix] = None, workspace: Optional[torch.Tensor] = None) -> QMatrix:
@@ -219,6 +229,33 @@ def dequant(q: QMatrix, want32: bool = True, want16: bool = True):
     cs = q.cstruct()
     _check(lib().lqlora_dequant(ctypes.byref(cs), _ptr(d32), _ptr(d16), _stream()), "lqlora_dequant")
     return d32, d16
+
+
+def unpack_scales(q: QMatrix):
+    """lqlora_unpack_scales: (scale codes uint8 [nblk], second-level scales fp32 [ngrp]) in plain form."""
+    nblk = q.N * q.K // q.cfg.B0
+    ngrp = (nblk + q.cfg.B1 - 1) // q.cfg.B1
+    sc = torch.empty(nblk, dtype=torch.uint8, device=q.codes.device)
+    v = torch.empty(ngrp, dtype=torch.float32, device=q.codes.device)
+    cs = q.cstruct()
+    _check(lib().lqlora_unpack_scales(ctypes.byref(cs), sc.data_ptr(), v.data_ptr(), _stream()), "lqlora_unpack_scales")
+    return sc, v
+
+
+def linear_qfactors(q: QMatrix, qL1: QMatrix, qL2: QMatrix, A: torch.Tensor, backward: bool = False) -> torch.Tensor:
+    """lqlora_linear_fwd_qfactors / lqlora_linear_bwd_input_qfactors: the layer with quantized (NF-8) factors."""
+    assert A.is_cuda and A.dtype == torch.bfloat16 and A.is_contiguous() and A.dim() == 2
+    M, r = A.shape[0], qL1.K
+    c = _cfg(q.cfg)
+    need = ctypes.c_size_t(0)
+    _check(lib().lqlora_linear_qfactors_workspace_bytes(q.N, q.K, ctypes.byref(c), r, M, ctypes.byref(need)), "qfactors workspace")
+    ws = torch.empty(int(need.value), dtype=torch.uint8, device=A.device)
+    out = torch.empty((M, q.K if backward else q.N), dtype=torch.bfloat16, device=A.device)
+    fn = lib().lqlora_linear_bwd_input_qfactors if backward else lib().lqlora_linear_fwd_qfactors
+    a, b, cc = q.cstruct(), qL1.cstruct(), qL2.cstruct()
+    _check(fn(ctypes.byref(a), ctypes.byref(b), ctypes.byref(cc), A.data_ptr(), M, out.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+           "lqlora_linear_qfactors")
+    return out
 
 
 def alloc_workspace(q: QMatrix, r: int, M: int) -> torch.Tensor:

@@ -3,6 +3,8 @@
 // exports used for parity checks.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace lq {
@@ -183,9 +185,9 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
     for (int w = 0; w < B; ++w) dst[slab_word_offset(row, g, w, B, k0 >> 6)] = words[w];
 }
 
-// One CTA per second-level group: v_g = max s_i, s^_i = clamp(rint(s_i / (v_g / 127)), 0, 127).
+// One CTA per second-level group: v_g = max s_i, s^_i = clamp(rint(s_i / (v_g / levels)), 0, levels).
 __global__ void __launch_bounds__(256) encode_scales_kernel(const float* __restrict__ absmax, uint8_t* __restrict__ sc,
-                                                            float* __restrict__ v, long long nblk, int B1) {
+                                                            float* __restrict__ v, long long nblk, int B1, float levels) {
     __shared__ float red[8];
     __shared__ float vmax;
     const long long lo = static_cast<long long>(blockIdx.x) * B1;
@@ -204,18 +206,99 @@ __global__ void __launch_bounds__(256) encode_scales_kernel(const float* __restr
     }
     __syncthreads();
     const float vg = vmax;
-    const float sigma = __fdiv_rn(vg, static_cast<float>(kScaleLevels));
+    const float sigma = __fdiv_rn(vg, levels);
     for (long long i = lo + threadIdx.x; i < hi; i += blockDim.x) {
         float c = 0.0f;
         if (vg != 0.0f) {
             c = rintf(__fdiv_rn(absmax[i], sigma));
-            c = fminf(fmaxf(c, 0.0f), static_cast<float>(kScaleLevels));
+            c = fminf(fmaxf(c, 0.0f), levels);
         }
         sc[i] = static_cast<uint8_t>(c);
     }
 }
 
-// Thread per (row, 32-column group): unpack to one code per byte and / or dequantize.
+// Storage forms of the scales (Table 1 of Sec. 3.2).  b1 < 8: the codes form a bit stream of b1 bits each, code i in
+// bits [i b1, (i + 1) b1) of the little-endian byte stream (eight codes = b1 bytes); cast(v, b2): fp16 or bf16 numbers
+// (round to nearest even).  One thread packs / expands eight codes; the second-level scales go one per thread.
+__global__ void pack_scales_kernel(const uint8_t* __restrict__ sc8, const float* __restrict__ v32, uint8_t* __restrict__ sc_out,
+                                   void* __restrict__ v_out, long long nblk, long long ngrp, int b1, int b2) {
+    const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (t * 8 < nblk) {
+        if (b1 == 8) {
+            for (int i = 0; i < 8 && t * 8 + i < nblk; ++i) sc_out[t * 8 + i] = sc8[t * 8 + i];
+        } else {
+            unsigned long long word = 0ull;
+            for (int i = 0; i < 8; ++i)
+                if (t * 8 + i < nblk) word |= static_cast<unsigned long long>(sc8[t * 8 + i]) << (i * b1);
+            for (int j = 0; j < b1; ++j) sc_out[t * b1 + j] = static_cast<uint8_t>(word >> (8 * j));
+        }
+    }
+    if (t < ngrp) {
+        if (b2 == kB2Fp32) static_cast<float*>(v_out)[t] = v32[t];
+        else if (b2 == kB2Fp16) static_cast<__half*>(v_out)[t] = __float2half_rn(v32[t]);
+        else static_cast<__nv_bfloat16*>(v_out)[t] = __float2bfloat16_rn(v32[t]);
+    }
+}
+__global__ void expand_scales_kernel(const uint8_t* __restrict__ sc_in, const void* __restrict__ v_in, uint8_t* __restrict__ sc8,
+                                     float* __restrict__ v32, long long nblk, long long ngrp, int b1, int b2) {
+    const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (t * 8 < nblk) {
+        if (b1 == 8) {
+            for (int i = 0; i < 8 && t * 8 + i < nblk; ++i) sc8[t * 8 + i] = sc_in[t * 8 + i];
+        } else {
+            unsigned long long word = 0ull;
+            for (int j = 0; j < b1; ++j) word |= static_cast<unsigned long long>(sc_in[t * b1 + j]) << (8 * j);
+            for (int i = 0; i < 8; ++i)
+                if (t * 8 + i < nblk) sc8[t * 8 + i] = static_cast<uint8_t>((word >> (i * b1)) & ((1u << b1) - 1u));
+        }
+    }
+    if (t < ngrp) {
+        if (b2 == kB2Fp32) v32[t] = static_cast<const float*>(v_in)[t];
+        else if (b2 == kB2Fp16) v32[t] = __half2float(static_cast<const __half*>(v_in)[t]);
+        else v32[t] = __bfloat162float(static_cast<const __nv_bfloat16*>(v_in)[t]);
+    }
+}
+
+// Bytes of scratch an expanded copy of the scales takes, and the expansion itself: returns the view the kernels read.
+inline size_t expanded_scale_bytes(int64_t N, int64_t K, const lqlora_config* c) {
+    if (!packed_scales(c)) return 0;
+    const int64_t nblk = N * K / c->B0, ngrp = (nblk + c->B1 - 1) / c->B1;
+    return (static_cast<size_t>(nblk) + 255) / 256 * 256 + (static_cast<size_t>(ngrp) * 4 + 255) / 256 * 256;
+}
+inline cudaError_t expand_scales(const lqlora_qmatrix* q, QView* view, char* scratch, cudaStream_t st) {
+    *view = make_view(q);
+    if (!packed_scales(&q->cfg)) return cudaSuccess;
+    const long long nblk = static_cast<long long>(q->N) * q->K / q->cfg.B0, ngrp = (nblk + q->cfg.B1 - 1) / q->cfg.B1;
+    uint8_t* sc8 = reinterpret_cast<uint8_t*>(scratch);
+    float* v32 = reinterpret_cast<float*>(scratch + (static_cast<size_t>(nblk) + 255) / 256 * 256);
+    const long long threads = (nblk + 7) / 8 > ngrp ? (nblk + 7) / 8 : ngrp;
+    expand_scales_kernel<<<static_cast<unsigned>((threads + 255) / 256), 256, 0, st>>>(q->scale_codes, q->scale2, sc8, v32, nblk, ngrp,
+                                                                                   q->cfg.b1, q->cfg.b2);
+    count_launch(1);
+    view->sc = sc8;
+    view->v = v32;
+    view->b1 = 8;
+    view->b2 = kB2Fp32;
+    return cudaGetLastError();
+}
+
+// Scale code of block `blk` and second-level scale of group `g` in whatever form the view holds them.
+__device__ __forceinline__ uint32_t load_scale_code(const QView& q, long long blk) {
+    if (q.b1 == 8) return q.sc[blk];
+    const long long bit = blk * q.b1;
+    const long long byte = bit >> 3;
+    const int sh = static_cast<int>(bit & 7);
+    uint32_t w = q.sc[byte];
+    if (sh + q.b1 > 8) w |= static_cast<uint32_t>(q.sc[byte + 1]) << 8;
+    return (w >> sh) & ((1u << q.b1) - 1u);
+}
+__device__ __forceinline__ float load_scale2(const QView& q, long long g) {
+    if (q.b2 == kB2Fp32) return q.v[g];
+    if (q.b2 == kB2Fp16) return __half2float(reinterpret_cast<const __half*>(q.v)[g]);
+    return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(q.v)[g]);
+}
+
+// Thread per (row, 32-column group): unpack to one code per byte and / or dequantize (any storage form of the scales).
 template <int B>
 __global__ void __launch_bounds__(256) export_kernel(QView q, uint8_t* __restrict__ codes_out, float* __restrict__ deq32,
                                                      __nv_bfloat16* __restrict__ deq16) {
@@ -240,7 +323,7 @@ __global__ void __launch_bounds__(256) export_kernel(QView q, uint8_t* __restric
         if (codes_out) codes_out[out + j] = static_cast<uint8_t>(c);
         if (deq32 || deq16) {
             const long long blk = static_cast<long long>(row) * q.KB + ((k0 + j) >> q.logB0);
-            const float st = block_scale(q.sc[blk], q.v[blk >> q.logB1]);
+            const float st = block_scale(static_cast<uint8_t>(load_scale_code(q, blk)), load_scale2(q, blk >> q.logB1), q.levels);
             const float wv = __fmul_rn(cb[c], st);
             if (deq32) deq32[out + j] = wv;
             if (deq16) deq16[out + j] = __float2bfloat16_rn(wv);
@@ -257,8 +340,21 @@ inline cudaError_t launch_encode(const float* W, const lqlora_qmatrix* out, floa
                                                  ilog2(out->cfg.B0));
     const long long nblk = static_cast<long long>(N) * K / out->cfg.B0;
     const long long ngrp = (nblk + out->cfg.B1 - 1) / out->cfg.B1;
-    encode_scales_kernel<<<static_cast<unsigned>(ngrp), 256, 0, st>>>(absmax, out->scale_codes, out->scale2, nblk, out->cfg.B1);
-    count_launch(2);
+    const float levels = static_cast<float>(scale_levels(out->cfg.b1));
+    if (!packed_scales(&out->cfg)) {
+        encode_scales_kernel<<<static_cast<unsigned>(ngrp), 256, 0, st>>>(absmax, out->scale_codes, out->scale2, nblk, out->cfg.B1, levels);
+        count_launch(2);
+        return cudaGetLastError();
+    }
+    // other storage forms: byte codes and fp32 scales into the scratch behind the absmax values, then packed / cast
+    char* tail = reinterpret_cast<char*>(absmax) + (static_cast<size_t>(nblk) * sizeof(float) + 255) / 256 * 256;
+    uint8_t* sc8 = reinterpret_cast<uint8_t*>(tail);
+    float* v32 = reinterpret_cast<float*>(tail + (static_cast<size_t>(nblk) + 255) / 256 * 256);
+    encode_scales_kernel<<<static_cast<unsigned>(ngrp), 256, 0, st>>>(absmax, sc8, v32, nblk, out->cfg.B1, levels);
+    const long long threads = (nblk + 7) / 8 > ngrp ? (nblk + 7) / 8 : ngrp;
+    pack_scales_kernel<<<static_cast<unsigned>((threads + 255) / 256), 256, 0, st>>>(sc8, v32, out->scale_codes, out->scale2, nblk, ngrp,
+                                                                                 out->cfg.b1, out->cfg.b2);
+    count_launch(3);
     return cudaGetLastError();
 }
 

@@ -14,7 +14,10 @@ namespace lq {
 constexpr int kTileRows = 128;   // rows of a packed tile
 constexpr int kTileCols = 64;    // columns of a packed tile
 constexpr int kSlabRows = 32;    // rows of a slab (one warp's worth)
-constexpr int kScaleLevels = 127;  // 2^(b1-1) - 1 positive levels of the 8-bit RTN scale quantizer (Sec. 2.2)
+// 2^(b1-1) - 1 positive levels of the b1-bit round-to-nearest quantizer of the block scales (Sec. 2.2, Sec. 3.2)
+__host__ __device__ inline int scale_levels(int b1) { return (1 << (b1 - 1)) - 1; }
+// Second-level scale formats (the b2 field): 32 = fp32, 16 = IEEE fp16, -16 = bfloat16 (Table 1 of Sec. 3.2)
+constexpr int kB2Fp32 = 32, kB2Fp16 = 16, kB2Bf16 = -16;
 constexpr int kStatusBytes = 256;  // status word area at the start of a linear workspace
 
 // Index of a code width in the table arrays.
@@ -28,7 +31,8 @@ inline int check_config(const lqlora_config* c) {
     if (!(c->b0 == 2 || c->b0 == 3 || c->b0 == 4 || c->b0 == 8)) return LQLORA_ERR_INVALID_CONFIG;
     if (!is_pow2(c->B0) || c->B0 < 16 || c->B0 > 256) return LQLORA_ERR_INVALID_CONFIG;
     if (!is_pow2(c->B1) || c->B1 < 16 || c->B1 > 4096) return LQLORA_ERR_INVALID_CONFIG;
-    if (c->b1 != 8 || c->b2 != 32) return LQLORA_ERR_INVALID_CONFIG;
+    if (!(c->b1 == 2 || c->b1 == 3 || c->b1 == 4 || c->b1 == 8)) return LQLORA_ERR_INVALID_CONFIG;
+    if (!(c->b2 == kB2Fp32 || c->b2 == kB2Fp16 || c->b2 == kB2Bf16)) return LQLORA_ERR_INVALID_CONFIG;
     return LQLORA_OK;
 }
 
@@ -39,13 +43,20 @@ inline int check_shape(int64_t N, int64_t K, const lqlora_config* c) {
     return LQLORA_OK;
 }
 
+// The kernels read one scale code per byte and fp32 second-level scales; any other storage form (b1 < 8, 16-bit v) is
+// expanded into scratch first.
+inline bool packed_scales(const lqlora_config* c) { return c->b1 != 8 || c->b2 != kB2Fp32; }
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Device-side view of a quantized matrix.
+// Device-side view of a quantized matrix.  sc / v are the arrays the kernels read: one code per byte and fp32 (the
+// matrix's own arrays for b1 = 8, b2 = fp32; expanded copies otherwise, see expand_scales).
 struct QView {
     const uint32_t* codes;
     const uint8_t* sc;     // s^ [N * KB]
     const float* v;        // v  [ngrp]
+    float levels;          // 2^(b1-1) - 1
+    int b1, b2;            // storage form of sc / v as this view holds them (8 / fp32 once expanded)
     int N, K;
     int b0, B0, B1;
     int logB0, logB1;
@@ -62,6 +73,8 @@ inline QView make_view(const lqlora_qmatrix* q) {
     v.N = static_cast<int>(q->N);
     v.K = static_cast<int>(q->K);
     v.b0 = q->cfg.b0; v.B0 = q->cfg.B0; v.B1 = q->cfg.B1;
+    v.levels = static_cast<float>(scale_levels(q->cfg.b1));
+    v.b1 = q->cfg.b1; v.b2 = q->cfg.b2;
     v.logB0 = ilog2(v.B0); v.logB1 = ilog2(v.B1);
     v.KB = v.K / v.B0;
     v.ktiles = v.K / kTileCols;
@@ -121,9 +134,9 @@ __host__ __device__ __forceinline__ uint32_t extract_code(const uint32_t* w, int
     }
 }
 
-// s~ = fl32(float(s^) * fl32(v / 127))
-__device__ __forceinline__ float block_scale(uint8_t sc, float v) {
-    return __fmul_rn(static_cast<float>(sc), __fdiv_rn(v, static_cast<float>(kScaleLevels)));
+// s~ = fl32(float(s^) * fl32(v / levels)),  levels = 2^(b1-1) - 1 (127 for 8-bit scale codes)
+__device__ __forceinline__ float block_scale(uint8_t sc, float v, float levels) {
+    return __fmul_rn(static_cast<float>(sc), __fdiv_rn(v, levels));
 }
 
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }

@@ -173,7 +173,7 @@ __device__ __forceinline__ void build_scale_table(const QView& q, int tile_row, 
             for (int i = 0; i < VW; ++i) {
                 const uint32_t code = (words[i >> 2] >> (8 * (i & 3))) & 255u;
                 const float vv = (((blkv[u] + i) >> q.logB1) == g0) ? v0[u] : v1[u];
-                stab[(kbv[u] + i) * kStabStride + rowv[u]] = block_scale(static_cast<uint8_t>(code), vv);
+                stab[(kbv[u] + i) * kStabStride + rowv[u]] = block_scale(static_cast<uint8_t>(code), vv, q.levels);
             }
         }
     }
@@ -288,7 +288,7 @@ decode_fwd_kernel(const Params p) {
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
                     st8[(kvv[u] * 16 + i) * kStab8Stride + rowv[u]] = static_cast<uint8_t>((words[i >> 2] >> (8 * (i & 3))) & 255u);
-                sg[kvv[u] * kStabStride + rowv[u]] = __fdiv_rn(v0[u], static_cast<float>(kScaleLevels));
+                sg[kvv[u] * kStabStride + rowv[u]] = __fdiv_rn(v0[u], q.levels);
             }
         }
     } else {
@@ -637,10 +637,10 @@ decode_bwd_kernel(const BwdParams p) {
                     if (i < nkb) {
                         const uint32_t code = (words[i >> 2] >> (8 * (i & 3))) & 255u;
                         if constexpr (C8) st8[i * p.rows_stride + rowv[u]] = static_cast<uint8_t>(code);
-                        else stab[i * p.rows_stride + rowv[u]] = block_scale(static_cast<uint8_t>(code), v[u]);
+                        else stab[i * p.rows_stride + rowv[u]] = block_scale(static_cast<uint8_t>(code), v[u], q.levels);
                     }
                 }
-                if constexpr (C8) sg[rowv[u]] = __fdiv_rn(v[u], static_cast<float>(kScaleLevels));
+                if constexpr (C8) sg[rowv[u]] = __fdiv_rn(v[u], q.levels);
             }
         }
     } else {
@@ -666,7 +666,7 @@ decode_bwd_kernel(const BwdParams p) {
         fill_ring();
 #pragma unroll
         for (int u = 0; u < 4; ++u)
-            if (slot[u] >= 0) stab[slot[u]] = block_scale(static_cast<uint8_t>(sc8[u]), v[u]);
+            if (slot[u] >= 0) stab[slot[u]] = block_scale(static_cast<uint8_t>(sc8[u]), v[u], q.levels);
     }
     }
     fill_ring();

@@ -117,9 +117,9 @@ __global__ void __launch_bounds__(128) small_fwd_kernel(QView q, const __nv_bflo
             float s_lo = 0.0f, s_hi = 0.0f;
             if (row < q.N) {
                 const long long blk = static_cast<long long>(row) * q.KB + (kbase >> q.logB0);
-                s_lo = block_scale(q.sc[blk], q.v[blk >> q.logB1]);
+                s_lo = block_scale(q.sc[blk], q.v[blk >> q.logB1], q.levels);
                 s_hi = s_lo;
-                if (q.B0 == 16) s_hi = block_scale(q.sc[blk + 1], q.v[(blk + 1) >> q.logB1]);
+                if (q.B0 == 16) s_hi = block_scale(q.sc[blk + 1], q.v[(blk + 1) >> q.logB1], q.levels);
             }
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
@@ -179,9 +179,9 @@ __global__ void __launch_bounds__(128) small_bwd_kernel(QView q, const __nv_bflo
             uint32_t rw[B + 1];
             row_words<B>(w, r, rw);
             const long long blk = static_cast<long long>(row) * q.KB + (kbase >> q.logB0);
-            const float s_lo = block_scale(q.sc[blk], q.v[blk >> q.logB1]);
+            const float s_lo = block_scale(q.sc[blk], q.v[blk >> q.logB1], q.levels);
             float s_hi = s_lo;
-            if (q.B0 == 16) s_hi = block_scale(q.sc[blk + 1], q.v[(blk + 1) >> q.logB1]);
+            if (q.B0 == 16) s_hi = block_scale(q.sc[blk + 1], q.v[(blk + 1) >> q.logB1], q.levels);
             float g[MT];
 #pragma unroll
             for (int m = 0; m < MT; ++m)

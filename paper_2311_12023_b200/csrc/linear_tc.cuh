@@ -153,7 +153,7 @@ __device__ __forceinline__ void dequant_group(uint32_t words, float s_lo, float 
 struct RawScale { uint32_t sc; float v; };
 // s~ = fl32(float(s^) * fl32(v / 127)); the quotient is recomputed only when v changes.
 __device__ __forceinline__ void make_scales(const QView& q, const RawScale& r, float& v_cached, float& sigma, float& s_lo, float& s_hi) {
-    if (r.v != v_cached) { v_cached = r.v; sigma = __fdiv_rn(r.v, static_cast<float>(kScaleLevels)); }
+    if (r.v != v_cached) { v_cached = r.v; sigma = __fdiv_rn(r.v, q.levels); }
     s_lo = __fmul_rn(static_cast<float>(r.sc & 0xFFu), sigma);
     s_hi = (q.B0 == 16) ? __fmul_rn(static_cast<float>(r.sc >> 8), sigma) : s_lo;
 }

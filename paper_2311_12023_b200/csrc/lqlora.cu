@@ -32,11 +32,16 @@ static int cuda_rc(cudaError_t e) {
 }
 
 // Scratch bytes one direction of the linear needs for M rows, for the kernel family it dispatches to.
-static size_t linear_need(const QView& v, int r, int64_t M, bool backward) {
+static size_t linear_need_base(const QView& v, int r, int64_t M, bool backward) {
     if (tc_supported(v, r, M, backward)) return tc_workspace_bytes(v.N, v.K, r, M, backward);
     if (backward ? dec::bwd_supported(v, M) : dec::supported(v, M)) return dec::workspace_bytes(v, r, static_cast<int>(M), backward);
     const SmallPlan p = small_plan(v.N, v.K, r, M, backward);
     return kStatusBytes + p.t_bytes + p.p_bytes;
+}
+// ... plus, for matrices whose scales are stored packed (b1 < 8) or in 16 bits, room for their expanded copy
+static size_t linear_need(const lqlora_qmatrix* q, int r, int64_t M, bool backward) {
+    const size_t base = (linear_need_base(make_view(q), r, M, backward) + 255) / 256 * 256;
+    return base + expanded_scale_bytes(q->N, q->K, &q->cfg);
 }
 
 static int check_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, int r, const void* A, int64_t M,
@@ -52,7 +57,7 @@ static int check_linear(const lqlora_qmatrix* q, const void* L1, const void* L2,
         // rows of X / Y must start on 16-byte boundaries for the vector loads and TMA
         if (M > 1) return LQLORA_ERR_INVALID_SHAPE;
     }
-    if (ws_bytes < linear_need(make_view(q), r, M, backward)) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
+    if (ws_bytes < linear_need(q, r, M, backward)) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
     return LQLORA_OK;
 }
 
@@ -63,7 +68,12 @@ static int run_linear(const lqlora_qmatrix* q, const void* L1, const void* L2, i
     rc = ensure_tables();
     if (rc != LQLORA_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const QView v = make_view(q);
+    QView v = make_view(q);
+    if (packed_scales(&q->cfg)) {
+        // scales stored packed or in 16 bits: the kernels read an expanded copy behind the call's own scratch
+        const size_t base = (linear_need_base(v, r, M, backward) + 255) / 256 * 256;
+        if (expand_scales(q, &v, static_cast<char*>(ws) + base, st) != cudaSuccess) return cuda_rc(cudaGetLastError());
+    }
     const bool use_tc = tc_supported(v, r, M, backward);
     const bool use_decode = !use_tc && (backward ? dec::bwd_supported(v, M) : dec::supported(v, M));
     // With a rank-r term the first kernel of the call (the pre-product) clears what has to start at zero (the status
@@ -196,6 +206,75 @@ int lqlora_dequant(const lqlora_qmatrix* q, float* deq32_dev, void* deq16_dev, v
     return cuda_rc(e);
 }
 
+int lqlora_unpack_scales(const lqlora_qmatrix* q, uint8_t* scale_codes_dev, float* scale2_dev, void* stream) {
+    using namespace lq;
+    int rc = check_qmatrix(q);
+    if (rc != LQLORA_OK) return rc;
+    if (!scale_codes_dev || !scale2_dev) return LQLORA_ERR_NULL_POINTER;
+    const long long nblk = static_cast<long long>(q->N) * q->K / q->cfg.B0, ngrp = (nblk + q->cfg.B1 - 1) / q->cfg.B1;
+    const long long threads = (nblk + 7) / 8 > ngrp ? (nblk + 7) / 8 : ngrp;
+    expand_scales_kernel<<<static_cast<unsigned>((threads + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        q->scale_codes, q->scale2, scale_codes_dev, scale2_dev, nblk, ngrp, q->cfg.b1, q->cfg.b2);
+    count_launch(1);
+    return cuda_rc(cudaGetLastError());
+}
+
+// Layer with quantized factors (the compression setting of Sec. 4.2: L1, L2 stored in NF-8 after training): the two
+// factors are dequantized to bf16 into the tail of the workspace, then the ordinary path runs.
+static int run_linear_qfactors(const lqlora_qmatrix* q, const lqlora_qmatrix* qL1, const lqlora_qmatrix* qL2, const void* A,
+                               int64_t M, void* out, void* ws, size_t ws_bytes, void* stream, bool backward) {
+    using namespace lq;
+    int rc = check_qmatrix(q);
+    if (rc == LQLORA_OK) rc = check_qmatrix(qL1);
+    if (rc == LQLORA_OK) rc = check_qmatrix(qL2);
+    if (rc != LQLORA_OK) return rc;
+    const int64_t r = qL1->K;
+    if (qL1->N != q->N || qL2->N != r || qL2->K != q->K || r > 128 || r % 16 != 0) return LQLORA_ERR_INVALID_SHAPE;
+    if (!ws || !aligned16(ws)) return ws ? LQLORA_ERR_MISALIGNED : LQLORA_ERR_NULL_POINTER;
+    if (M <= 0 || M > (int64_t(1) << 24)) return LQLORA_ERR_INVALID_SHAPE;
+    const size_t base = (linear_need(q, static_cast<int>(r), M, backward) + 255) / 256 * 256;
+    const size_t l1_bytes = (static_cast<size_t>(q->N) * r * 2 + 255) / 256 * 256, l2_bytes = (static_cast<size_t>(r) * q->K * 2 + 255) / 256 * 256;
+    if (ws_bytes < base + l1_bytes + l2_bytes) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
+    rc = ensure_tables();
+    if (rc != LQLORA_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* w = static_cast<char*>(ws);
+    void* L1 = w + base;
+    void* L2 = w + base + l1_bytes;
+    const lqlora_qmatrix* fs[2] = {qL1, qL2};
+    void* dst[2] = {L1, L2};
+    for (int i = 0; i < 2; ++i) {
+        const QView v = make_view(fs[i]);
+        cudaError_t e;
+        switch (v.b0) {
+            case 2: e = launch_export<2>(v, nullptr, nullptr, dst[i], st); break;
+            case 3: e = launch_export<3>(v, nullptr, nullptr, dst[i], st); break;
+            case 4: e = launch_export<4>(v, nullptr, nullptr, dst[i], st); break;
+            default: e = launch_export<8>(v, nullptr, nullptr, dst[i], st); break;
+        }
+        if (e != cudaSuccess) return cuda_rc(e);
+    }
+    return run_linear(q, L1, L2, static_cast<int>(r), A, M, out, ws, base, stream, backward);
+}
+
+int lqlora_linear_qfactors_workspace_bytes(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, size_t* bytes) {
+    size_t base = 0;
+    const int rc = lqlora_linear_workspace_bytes(N, K, cfg, r, M, &base);
+    if (rc != LQLORA_OK) return rc;
+    *bytes = (base + 255) / 256 * 256 + (static_cast<size_t>(N) * r * 2 + 255) / 256 * 256 + (static_cast<size_t>(r) * K * 2 + 255) / 256 * 256;
+    return LQLORA_OK;
+}
+
+int lqlora_linear_fwd_qfactors(const lqlora_qmatrix* q, const lqlora_qmatrix* qL1, const lqlora_qmatrix* qL2, const void* X_dev,
+                               int64_t M, void* Y_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    return run_linear_qfactors(q, qL1, qL2, X_dev, M, Y_dev, workspace_dev, workspace_bytes, stream, false);
+}
+
+int lqlora_linear_bwd_input_qfactors(const lqlora_qmatrix* q, const lqlora_qmatrix* qL1, const lqlora_qmatrix* qL2, const void* dY_dev,
+                                     int64_t M, void* dX_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    return run_linear_qfactors(q, qL1, qL2, dY_dev, M, dX_dev, workspace_dev, workspace_bytes, stream, true);
+}
+
 int lqlora_linear_workspace_bytes(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, size_t* bytes) {
     using namespace lq;
     int rc = check_config(cfg);
@@ -207,8 +286,7 @@ int lqlora_linear_workspace_bytes(int64_t N, int64_t K, const lqlora_config* cfg
     // the same workspace must serve the forward and the input gradient
     lqlora_qmatrix q{};
     q.N = N; q.K = K; q.cfg = *cfg;
-    const QView v = make_view(&q);
-    const size_t f = linear_need(v, r, M, false), b = linear_need(v, r, M, true);
+    const size_t f = linear_need(&q, r, M, false), b = linear_need(&q, r, M, true);
     const size_t need = f > b ? f : b;
     *bytes = need;
     return LQLORA_OK;
@@ -233,7 +311,7 @@ int lqlora_linear_fwd_static(const lqlora_qmatrix* q, const void* L1_dev, const 
     int rc = check_qmatrix(q);
     if (rc != LQLORA_OK) return rc;
     if (M <= 0 || M > (int64_t(1) << 24) || r < 0 || r > 128 || (r % 16) != 0) return LQLORA_ERR_INVALID_SHAPE;
-    if (linear_need(make_view(q), r, M, false) > kStaticScratchBytes) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
+    if (linear_need(q, r, M, false) > kStaticScratchBytes) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
     void* scratch = nullptr;
     rc = static_scratch_ptr(&scratch);
     if (rc != LQLORA_OK) return rc;

@@ -135,8 +135,9 @@ extern "C" {
 
 double lqlora_storage_bits_per_param(const lqlora_config* cfg) {
     if (lq::check_config(cfg) != LQLORA_OK) return -1.0;
+    const int b2 = cfg->b2 < 0 ? -cfg->b2 : cfg->b2;
     return static_cast<double>(cfg->b0) + static_cast<double>(cfg->b1) / cfg->B0 +
-           static_cast<double>(cfg->b2) / (static_cast<double>(cfg->B0) * cfg->B1);
+           static_cast<double>(b2) / (static_cast<double>(cfg->B0) * cfg->B1);
 }
 
 int lqlora_packed_sizes(int64_t N, int64_t K, const lqlora_config* cfg, size_t* code_bytes,
@@ -149,9 +150,13 @@ int lqlora_packed_sizes(int64_t N, int64_t K, const lqlora_config* cfg, size_t* 
     const int64_t nblk = N * K / cfg->B0;
     const int64_t ngrp = (nblk + cfg->B1 - 1) / cfg->B1;
     if (code_bytes) *code_bytes = static_cast<size_t>(Np) * K * cfg->b0 / 8;
-    if (scale_bytes) *scale_bytes = static_cast<size_t>(nblk);
-    if (scale2_bytes) *scale2_bytes = static_cast<size_t>(ngrp) * sizeof(float);
-    if (encode_workspace_bytes) *encode_workspace_bytes = static_cast<size_t>(nblk) * sizeof(float);
+    // scale codes: a bit stream of b1 bits each (eight codes take b1 bytes); second-level scales: 4 or 2 bytes each
+    if (scale_bytes) *scale_bytes = (cfg->b1 == 8) ? static_cast<size_t>(nblk) : static_cast<size_t>((nblk + 7) / 8) * cfg->b1;
+    if (scale2_bytes) *scale2_bytes = static_cast<size_t>(ngrp) * (cfg->b2 == lq::kB2Fp32 ? 4 : 2);
+    // encoder scratch: the block absmax values, plus byte codes and fp32 scales before packing
+    if (encode_workspace_bytes)
+        *encode_workspace_bytes = (static_cast<size_t>(nblk) * sizeof(float) + 255) / 256 * 256 +
+                                  (lq::packed_scales(cfg) ? (static_cast<size_t>(nblk) + 255) / 256 * 256 + static_cast<size_t>(ngrp) * 4 : 0);
     return LQLORA_OK;
 }
 

@@ -76,8 +76,11 @@ def test_invalid_arguments_are_rejected_before_any_launch(binding):
     assert sizes(128, 128, good) == 0
     assert sizes(128, 128, inputs.QuantConfig(5, 64, 8, 256, 32)) == -1      # b0
     assert sizes(128, 128, inputs.QuantConfig(3, 48, 8, 256, 32)) == -1      # B0 not a power of two
-    assert sizes(128, 128, inputs.QuantConfig(3, 64, 4, 256, 32)) == -1      # b1
-    assert sizes(128, 128, inputs.QuantConfig(3, 64, 8, 256, 16)) == -1      # b2
+    assert sizes(128, 128, inputs.QuantConfig(3, 64, 5, 256, 32)) == -1      # b1 not in {2, 3, 4, 8}
+    assert sizes(128, 128, inputs.QuantConfig(3, 64, 8, 256, 8)) == -1       # b2 not fp32 / fp16 / bf16
+    for b1 in (2, 3, 4, 8):
+        for b2 in (32, 16, -16):
+            assert sizes(128, 128, inputs.QuantConfig(3, 64, b1, 256, b2)) == 0
     assert sizes(128, 100, good) == -2                                       # K % 64
     assert sizes(128, 128, inputs.QuantConfig(3, 256, 8, 256, 32)) == -2     # K % B0
     assert sizes(0, 128, good) == -2
