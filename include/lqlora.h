@@ -300,6 +300,13 @@ int lqlora_linear_bwd_input_host(const lqlora_qmatrix* q, const void* L1_dev, co
  * (its output is then undefined).  The word is cleared by every linear call before it launches. */
 int lqlora_workspace_status(const void* workspace_dev, void* stream);
 
+/* Self-test of the bounded device-side waits: enqueues a one-CTA kernel that holds a tensor-memory allocation and waits,
+ * with the helper and status word the linear kernels use, on an mbarrier armed for bytes that nothing delivers.  After
+ * budget_cycles SM clocks (1e3 .. 2e9) the wait is abandoned: the kernel records the time-out in the status word at the
+ * head of workspace_dev (at least 256 bytes), frees its tensor memory and returns, so lqlora_workspace_status then
+ * reports LQLORA_ERR_TIMEOUT while the context stays usable.  Nothing traps, faults or spins without bound. */
+int lqlora_selftest_bounded_wait(void* workspace_dev, int64_t budget_cycles, void* stream);
+
 /* Which kernel lqlora_linear_fwd (backward = 0) or lqlora_linear_bwd_input (backward != 0) dispatches to for M rows:
  *   LQLORA_PATH_PLAIN    plain-FMA fall-back (shapes the vector paths do not take)
  *   LQLORA_PATH_STREAM   weight-streaming kernel for decode-sized inputs (M <= 16)

@@ -27,7 +27,7 @@ EXPORTS = [
     "lqlora_lora_grads_workspace_bytes", "lqlora_lora_grads",
     "lqlora_lq_workspace_bytes", "lqlora_lq_decompose", "lqlora_to_bf16", "lqlora_assign_configs",
     "lqlora_unpack_scales", "lqlora_linear_qfactors_workspace_bytes", "lqlora_linear_fwd_qfactors",
-    "lqlora_linear_bwd_input_qfactors",
+    "lqlora_linear_bwd_input_qfactors", "lqlora_selftest_bounded_wait",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20   # size of the scratch array compiled into the library (lqlora_static_scratch_bytes)
@@ -83,6 +83,7 @@ def lib() -> ctypes.CDLL:
         L.lqlora_encode_search_clearance.restype = ctypes.c_double
         L.lqlora_linear_fwd_static.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp]
         L.lqlora_static_scratch_status.argtypes = [vp]
+        L.lqlora_selftest_bounded_wait.argtypes = [vp, i64, vp]
         L.lqlora_unpack_scales.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, vp]
         L.lqlora_linear_qfactors_workspace_bytes.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ctypes.POINTER(sz)]
         L.lqlora_linear_fwd_qfactors.argtypes = [ctypes.POINTER(CQMatrix)] * 3 + [vp, i64, vp, vp, sz, vp]
@@ -407,6 +408,11 @@ def assign_configs(errors: np.ndarray, storage: np.ndarray, budget: float):
         return None
     _check(rc, "lqlora_assign_configs")
     return [int(a) for a in out], float(te.value), float(ts.value)
+
+
+def selftest_bounded_wait(workspace: torch.Tensor, budget_cycles: int) -> None:
+    """lqlora_selftest_bounded_wait: a wait that nothing satisfies, abandoned after budget_cycles."""
+    _check(lib().lqlora_selftest_bounded_wait(workspace.data_ptr(), int(budget_cycles), _stream()), "lqlora_selftest_bounded_wait")
 
 
 def static_scratch_status() -> int:

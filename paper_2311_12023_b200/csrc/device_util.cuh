@@ -55,6 +55,7 @@ constexpr long long kWaitCycles = 4000000000LL;   // about two seconds
 struct Ctl {
     volatile int* abort_s;
     int* status_g;
+    long long budget = kWaitCycles;      // clock cycles a wait may take before it is abandoned
 };
 __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const Ctl& c, int where) {
     const long long t0 = clock64();
@@ -62,7 +63,7 @@ __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, const Ctl&
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63) == 63) {
             if (*c.abort_s) return false;
-            if (clock64() - t0 > kWaitCycles) {
+            if (clock64() - t0 > c.budget) {
                 *c.abort_s = 1;
                 atomicCAS(c.status_g, 0, where);
                 return false;

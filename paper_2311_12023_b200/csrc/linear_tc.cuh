@@ -598,6 +598,9 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 160);
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
+    // The CTAs of a cluster write into each other's shared memory at the end; that is allowed once every CTA of the
+    // cluster runs, which the first phase of the cluster barrier establishes: arrive here, wait before the first store.
+    if (CL && nsplit > 1) dec::cluster_arrive_relaxed();
     // cleared before this CTA lets the dependent kernel start: that kernel is launched once all CTAs have passed here
     if (p.clear_status && tile == 0 && split == 0 && threadIdx.x == 0) *p.status = 0;
     pdl_launch_dependents();      // the linear kernel behind this one needs T only in its last steps
@@ -707,6 +710,7 @@ __device__ __forceinline__ void lowrank_body(const CUtensorMap& tmA, const CUten
     if constexpr (CL) {
         // all threads of all CTAs of the cluster pass here, whatever happened before
         __syncthreads();
+        if (nsplit > 1) dec::cluster_wait();           // every CTA of the cluster has started
         const uint32_t recv_addr = smem_u32(recv);
         const int cols_share = p.rp / nsplit;
         if (warp >= 2 && cl_ok) {

@@ -57,6 +57,8 @@ __device__ __forceinline__ void wgrad_body(const CUtensorMap& tmA, const CUtenso
     auto empty = [&](int s) { return smem_u32(bars + 8 + s); };
     const uint32_t acc_full = smem_u32(bars + 16), drain = smem_u32(bars + 17);
 
+    // first phase of the cluster barrier: every CTA of the cluster runs before its shared memory is written remotely
+    if (nsplit > 1) dec::cluster_arrive_relaxed();
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
         mbar_init(acc_full, 1);
@@ -148,6 +150,7 @@ __device__ __forceinline__ void wgrad_body(const CUtensorMap& tmA, const CUtenso
     // CTA adds what it received, in rank order, and stores its columns.  The barriers are executed by all threads of
     // all CTAs whatever happened before.
     __syncthreads();
+    if (nsplit > 1) dec::cluster_wait();                    // every CTA of the cluster has started (arrival at kernel entry)
     const uint32_t recv_addr = smem_u32(recv);
     const int cols_share = p.rp / nsplit;                   // nsplit divides 64
     if (warp >= 2 && acc_ok) {

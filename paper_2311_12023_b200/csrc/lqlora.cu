@@ -141,9 +141,47 @@ static int static_scratch_ptr(void** out) {
     return LQLORA_OK;
 }
 
+// Self-test of the bounded waits: a CTA arms an mbarrier for bytes that nobody delivers and waits on it with the same
+// helper (and the same status word) as the linear kernels, holding a tensor-memory allocation meanwhile; when the
+// budget runs out the wait is abandoned, the status word is set, tensor memory is freed and the kernel returns.
+__global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(int* status, long long budget) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_s;
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        dev::mbar_init(dev::smem_u32(&bar), 1);
+        abort_s = 0;
+        dev::fence_barrier_init();
+    }
+    if (warp == 1) { tc::tmem_alloc(dev::smem_u32(&tmem_slot), 32); tc::tmem_relinquish(); }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+    if (threadIdx.x == 0) {
+        dev::Ctl ctl{&abort_s, status, budget};
+        dev::mbar_expect_tx(dev::smem_u32(&bar), 128);           // 128 bytes that never arrive
+        dev::wait(dev::smem_u32(&bar), 0, ctl, 99);
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tc::tmem_dealloc(tmem, 32);
+}
+
 }  // namespace lq
 
 extern "C" {
+
+int lqlora_selftest_bounded_wait(void* workspace_dev, int64_t budget_cycles, void* stream) {
+    if (!workspace_dev) return LQLORA_ERR_NULL_POINTER;
+    if (budget_cycles < 1000 || budget_cycles > 2000000000LL) return LQLORA_ERR_INVALID_SHAPE;     // at most about a second
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(workspace_dev, 0, lq::kStatusBytes, st) != cudaSuccess) return lq::cuda_rc(cudaGetLastError());
+    lq::bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(static_cast<int*>(workspace_dev), budget_cycles);
+    lq::count_launch(1);
+    return lq::cuda_rc(cudaGetLastError());
+}
 
 int lqlora_encode(const float* W_dev, lqlora_qmatrix* out, void* workspace_dev, size_t workspace_bytes, void* stream) {
     using namespace lq;

@@ -288,3 +288,28 @@ def test_workspace_may_hold_anything_before_a_call(N, K, M):
     check_close(got, oracle.linear_fwd(ref["d32"], l1b, l2b, xb, rows), "Y")
     got = to_np(dX) if rows is None else to_np(dX[torch.from_numpy(rows).cuda()])
     check_close(got, oracle.linear_bwd_input(ref["d32"], l1b, l2b, gb, rows), "dX")
+
+
+def test_a_bounded_wait_that_runs_out_sets_the_status_and_leaves_the_device_usable():
+    """A wait on bytes that never arrive is abandoned after its budget (about a millisecond here): the status word says
+    LQLORA_ERR_TIMEOUT, tensor memory was freed (the tcgen05 kernels that follow allocate all of it on every SM) and
+    the same workspace serves correct calls afterwards.  Also the host-side reading of a non-zero status word."""
+    N, K, M = 2560, 2304, 2100
+    cfg = C(3, 64, 8, 256, 32)
+    A = inputs.gaussian(1500, (N, K), 0.02)
+    l1b, l2b = inputs.lowrank_factors(1501, N, K, 64, 0.01)
+    q, ref = encode_both(A, cfg, check=False)
+    L1, L2 = binding.bf16_from_bits(l1b), binding.bf16_from_bits(l2b)
+    ws = binding.alloc_workspace(q, 64, M)
+    for _ in range(3):
+        binding.selftest_bounded_wait(ws, 2_000_000)
+        assert binding.workspace_status(ws) == -7
+        assert binding.status_string(-7) == "device-side wait timed out"
+    # a status word written by anyone reads as a time-out until the next call clears it
+    ws[:4] = torch.tensor([5, 0, 0, 0], dtype=torch.uint8, device="cuda")
+    assert binding.workspace_status(ws) == -7
+    rows = inputs.sample_rows(1502, M, count=8)
+    xb = inputs.activations(1503, M, K)
+    Y = binding.linear_fwd(q, L1, L2, binding.bf16_from_bits(xb), workspace=ws)
+    assert binding.workspace_status(ws) == 0
+    check_close(to_np(Y[torch.from_numpy(rows).cuda()]), oracle.linear_fwd(ref["d32"], l1b, l2b, xb, rows), "Y after the time-outs")
