@@ -47,6 +47,8 @@ struct Params {
     int steps_q;       // steps whose weights are dequantized
     int steps_d;       // steps of the rank-r term
     int stages;
+    int c_base;        // first output column of this launch (a call may be split over two launches by output columns)
+    int c_tiles;       // number of 256-column output tiles of this launch
 };
 
 // ------------------------------------------------------------------------------------ PTX (tensor memory, tcgen05)
@@ -232,7 +234,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * (MH * 128);
-    const int c0 = blockIdx.y * BN;          // first output column: n0 (forward) or k0 (backward)
+    const int c0 = p.c_base + blockIdx.y * BN;          // first output column: n0 (forward) or k0 (backward)
     // split of the contraction over the CTAs of a cluster (gridDim.z of them); the rank-r steps go to split 0
     const int nsplit = gridDim.z, split = blockIdx.z;
     const int per_split = (p.steps_q + nsplit - 1) / nsplit;
@@ -805,7 +807,8 @@ inline bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t 
 }
 
 template <int B, bool BWD, int MH>
-inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, Params p, int ksplit, cudaStream_t st) {
+inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, Params p, int ksplit, cudaStream_t st,
+                      bool after_pre = true) {
     constexpr int stages = ring_stages<B, MH>();
     static_assert(stages >= 2, "activation ring too shallow");
     p.stages = stages;
@@ -821,7 +824,7 @@ inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUten
         attr_done = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((p.M + MH * 128 - 1) / (MH * 128), (p.out_cols + BN - 1) / BN, ksplit);
+    cfg.gridDim = dim3((p.M + MH * 128 - 1) / (MH * 128), p.c_tiles, ksplit);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -831,7 +834,7 @@ inline int launch_one(const CUtensorMap& tA, const CUtensorMap& tA2, const CUten
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = (p.steps_d > 0) ? 2 : 1;      // overlap with the rank-r pre-product kernel in front of it
+    cfg.numAttrs = (p.steps_d > 0 && after_pre) ? 2 : 1;      // overlap with the rank-r pre-product kernel in front of it
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA, tA2, tB2, p);
     count_launch(1);
     if (e != cudaSuccess) { cudaGetLastError(); return LQLORA_ERR_CUDA; }
@@ -879,13 +882,15 @@ inline bool tc_use_pair(int64_t M, int64_t out_cols, int sms) {
     return 2 * pair_ctas > sms;
 }
 
-inline int tc_ksplit(int64_t M, int64_t out_cols, int steps_q, int sms) {
-    if (tc_use_pair(M, out_cols, sms)) return 1;
-    const int mh = (M > 128) ? 2 : 1;
-    const long long tiles = ((M + mh * 128 - 1) / (mh * 128)) * ((out_cols + BN - 1) / BN);
+inline int tc_ksplit_tiles(long long tiles, int steps_q, int sms) {
     for (int ks = 8; ks > 1; --ks)
         if (tiles * ks <= sms && steps_q / ks >= (ks > 4 ? 16 : 8) && tiles <= tc_max_clusters(ks)) return ks;   // the reduction grows with ks
     return 1;
+}
+inline int tc_ksplit(int64_t M, int64_t out_cols, int steps_q, int sms) {
+    if (tc_use_pair(M, out_cols, sms)) return 1;
+    const int mh = (M > 128) ? 2 : 1;
+    return tc_ksplit_tiles(((M + mh * 128 - 1) / (mh * 128)) * ((out_cols + BN - 1) / BN), steps_q, sms);
 }
 
 struct PrePlan {
@@ -974,9 +979,9 @@ inline int launch_pre(const CUtensorMap& tA, const CUtensorMap& tB, PreParams p,
 
 template <int B>
 inline int launch_b(const CUtensorMap& tA, const CUtensorMap& tA2, const CUtensorMap& tB2, const Params& p, bool bwd, int mh,
-                    int ksplit, cudaStream_t st) {
-    if (!bwd) return mh == 2 ? launch_one<B, false, 2>(tA, tA2, tB2, p, ksplit, st) : launch_one<B, false, 1>(tA, tA2, tB2, p, ksplit, st);
-    return mh == 2 ? launch_one<B, true, 2>(tA, tA2, tB2, p, ksplit, st) : launch_one<B, true, 1>(tA, tA2, tB2, p, ksplit, st);
+                    int ksplit, cudaStream_t st, bool after_pre = true) {
+    if (!bwd) return mh == 2 ? launch_one<B, false, 2>(tA, tA2, tB2, p, ksplit, st, after_pre) : launch_one<B, false, 1>(tA, tA2, tB2, p, ksplit, st, after_pre);
+    return mh == 2 ? launch_one<B, true, 2>(tA, tA2, tB2, p, ksplit, st, after_pre) : launch_one<B, true, 1>(tA, tA2, tB2, p, ksplit, st, after_pre);
 }
 
 }  // namespace tc
@@ -1044,14 +1049,50 @@ inline int tc_launch(const QView& q, const void* L1, const void* L2, int r, cons
     p.steps_q = (C + BK - 1) / BK;
     p.steps_d = (r + BK - 1) / BK;
     p.stages = 0;
+    p.c_base = 0;
+    p.c_tiles = static_cast<int>((p.out_cols + BN - 1) / BN);
     if (pair) {
+        // Wave quantisation: the pair tiles run in waves of sms / 2 clusters.  When the last wave would hold only a few
+        // tiles (at most a quarter of a wave), the output columns it would cover are peeled off and computed by the
+        // one-CTA kernel with the contraction split over clusters, which spreads that small remainder over many SMs
+        // (28672 x 8192 at 2048 rows: 448 pair tiles = 6 waves + 4 tiles, 817 -> 740 us).  Larger remainders stay with
+        // the pairs: the one-CTA kernel needs about 1.6 pair-tile times for three quarters of a wave (measured).
+        const int mt = (M + 511) / 512, pairs = sm_count() / 2;
+        const int tiles = mt * p.c_tiles, rem = tiles % pairs;
+        int peel = 0;
+        if (tiles > pairs && rem > 0 && 4 * rem <= pairs) peel = (rem + mt - 1) / mt;
+        if (peel >= p.c_tiles) peel = 0;
         CUtensorMap tOut;         // output as boxes of 32 rows x 64 columns
         if (!make_map(&tOut, out, M, p.out_cols, 32)) return LQLORA_ERR_CUDA;
+        p.c_tiles -= peel;
+        int rc;
         switch (q.b0) {
-            case 2: return backward ? launch_pair<2, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<2, false>(tA, tA2, tB2, tOut, p, st);
-            case 3: return backward ? launch_pair<3, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<3, false>(tA, tA2, tB2, tOut, p, st);
-            case 4: return backward ? launch_pair<4, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<4, false>(tA, tA2, tB2, tOut, p, st);
-            default: return backward ? launch_pair<8, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<8, false>(tA, tA2, tB2, tOut, p, st);
+            case 2: rc = backward ? launch_pair<2, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<2, false>(tA, tA2, tB2, tOut, p, st); break;
+            case 3: rc = backward ? launch_pair<3, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<3, false>(tA, tA2, tB2, tOut, p, st); break;
+            case 4: rc = backward ? launch_pair<4, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<4, false>(tA, tA2, tB2, tOut, p, st); break;
+            default: rc = backward ? launch_pair<8, true>(tA, tA2, tB2, tOut, p, st) : launch_pair<8, false>(tA, tA2, tB2, tOut, p, st); break;
+        }
+        if (rc != LQLORA_OK || peel == 0) return rc;
+        // the peeled columns: boxes of 256 rows for the one-CTA kernel; it runs behind the pair kernel (which has waited
+        // for the rank-r intermediate), so it needs no programmatic dependency of its own
+        CUtensorMap uA, uA2, uB2;
+        if (!make_map(&uA, A, M, C, 256)) return LQLORA_ERR_CUDA;
+        if (r > 0) {
+            if (!make_map(&uA2, T, M, r, 256)) return LQLORA_ERR_CUDA;
+            const bool okb = backward ? make_map(&uB2, L2, r, q.K, 64) : make_map(&uB2, L1, q.N, r, 256);
+            if (!okb) return LQLORA_ERR_CUDA;
+        } else {
+            uA2 = uA; uB2 = uA;
+        }
+        Params p2 = p;
+        p2.c_base = p.c_tiles * BN;
+        p2.c_tiles = peel;
+        const int ks2 = tc_ksplit_tiles(static_cast<long long>(peel) * ((M + 255) / 256), p.steps_q, sm_count());
+        switch (q.b0) {
+            case 2: return launch_b<2>(uA, uA2, uB2, p2, backward, 2, ks2, st, false);
+            case 3: return launch_b<3>(uA, uA2, uB2, p2, backward, 2, ks2, st, false);
+            case 4: return launch_b<4>(uA, uA2, uB2, p2, backward, 2, ks2, st, false);
+            default: return launch_b<8>(uA, uA2, uB2, p2, backward, 2, ks2, st, false);
         }
     }
     const int ksplit = tc_ksplit(M, p.out_cols, p.steps_q, sm_count());

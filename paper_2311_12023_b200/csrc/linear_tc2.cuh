@@ -108,7 +108,7 @@ tc_pair_linear_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_rank();                 // 0 = leader
     const int m0 = (blockIdx.x >> 1) * 512;               // first token row of the pair
-    const int c0 = blockIdx.y * BN;                       // first output column of the pair
+    const int c0 = p.c_base + blockIdx.y * BN;            // first output column of the pair
     const int total = p.steps_q + p.steps_d;
     const Ctl ctl{abort_s, p.status};
 
@@ -413,7 +413,7 @@ inline int launch_pair(const CUtensorMap& tA, const CUtensorMap& tA2, const CUte
         attr_done = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * ((p.M + 511) / 512), (p.out_cols + BN - 1) / BN);
+    cfg.gridDim = dim3(2 * ((p.M + 511) / 512), p.c_tiles);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;

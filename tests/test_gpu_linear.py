@@ -113,6 +113,18 @@ def test_linear_pair_kernel_ragged_tiles(N, K, M, b0, B0):
     run_case(A, l1b, l2b, C(b0, B0, 8, 64, 32), M, seed=750 + M, rows=rows)
 
 
+@pytest.mark.parametrize("b0,B0,r", [(3, 64, 64), (8, 32, 0)])
+def test_linear_pair_kernel_with_peeled_last_wave(b0, B0, r):
+    """80 pair tiles on 74 CTA pairs: the six tiles of the second wave are peeled off as two output column tiles and run
+    on the one-CTA kernel (forward: N = 4096 at 2560 rows; the input gradient of the transposed shape likewise)."""
+    M = 2560
+    for N, K in ((4096, 512), (512, 4096)):
+        A = inputs.gaussian(670 + N, (N, K), 0.02)
+        l1b, l2b = inputs.lowrank_factors(671 + K, N, K, r, 0.01) if r else (None, None)
+        rows = inputs.sample_rows(672, M, count=16, tile=256)
+        run_case(A, l1b, l2b, C(b0, B0, 8, 64, 32), M, seed=760 + N, rows=rows, route=binding.PATH_TC_PAIR if N == 4096 else None)
+
+
 @pytest.mark.parametrize("M", [4, 256])
 def test_linear_without_lowrank_and_with_zero_weights(M):
     N, K = 256, 512
@@ -210,7 +222,7 @@ def test_config4_query_projection_mixed_config():
     run_case(A, l1b, l2b, spec.cfg, 2048, seed=4600, rows=rows)
 
 
-@pytest.mark.parametrize("name,M", [("gate", 1), ("down", 2048)])
+@pytest.mark.parametrize("name,M", [("gate", 1), ("down", 2048), ("gate", 2048)])
 def test_config4_mlp_projections_largest_shapes(name, M):
     spec = [s for s in inputs.workload(4)["matrices"] if s.name == name][0]   # 28672 x 8192 / 8192 x 28672
     A, l1b, l2b = inputs.make_matrix(spec)
