@@ -50,10 +50,11 @@ WORKLOAD = ("llama2-70b decoder layer (GQA): q,o 8192x8192; k,v 1024x8192; gate,
 MS = (2048, 1)
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 FALLBACK = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (forward of the gate projection at
-# M = 2048), from an ncu capture of `python bench.py --case gate --case-m 2048`; None while no capture of the current
-# kernel exists.
-DOMINANT_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (tc_pair_linear_kernel<3, forward> on
+# the gate projection at M = 2048: 231.5 MB read + 101.4 MB written), from an ncu capture of
+# `python bench.py --case gate --case-m 2048 --case-reps 2` (profiles/tc_pair_linear_gate_28672x8192_m2048_ncu_full.txt);
+# algorithmic bytes: X 33.6 MB + packed codes and scales 107 MB + Y 117 MB.  Set to None when that kernel changes.
+DOMINANT_TRAFFIC_BYTES = 332832512
 
 
 def linear_flops(M: int, N: int, K: int, r: int) -> float:
