@@ -185,29 +185,22 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
     for (int w = 0; w < B; ++w) dst[slab_word_offset(row, g, w, B, k0 >> 6)] = words[w];
 }
 
-// One CTA per second-level group: v_g = max s_i, s^_i = clamp(rint(s_i / (v_g / levels)), 0, levels).
+// One warp per second-level group (eight groups per CTA): v_g = max s_i, s^_i = clamp(rint(s_i / (v_g / levels)), 0, levels).
 __global__ void __launch_bounds__(256) encode_scales_kernel(const float* __restrict__ absmax, uint8_t* __restrict__ sc,
-                                                            float* __restrict__ v, long long nblk, int B1, float levels) {
-    __shared__ float red[8];
-    __shared__ float vmax;
-    const long long lo = static_cast<long long>(blockIdx.x) * B1;
+                                                            float* __restrict__ v, long long nblk, long long ngrp, int B1, float levels) {
+    const long long g = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+    if (g >= ngrp) return;
+    const int lane = threadIdx.x & 31;
+    const long long lo = g * B1;
     const long long hi = (lo + B1 < nblk) ? lo + B1 : nblk;
     float m = 0.0f;
-    for (long long i = lo + threadIdx.x; i < hi; i += blockDim.x) m = fmaxf(m, absmax[i]);
+    for (long long i = lo + lane; i < hi; i += 32) m = fmaxf(m, absmax[i]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float t = red[0];
-        for (int i = 1; i < 8; ++i) t = fmaxf(t, red[i]);
-        vmax = t;
-        v[blockIdx.x] = t;
-    }
-    __syncthreads();
-    const float vg = vmax;
+    const float vg = m;
+    if (lane == 0) v[g] = vg;
     const float sigma = __fdiv_rn(vg, levels);
-    for (long long i = lo + threadIdx.x; i < hi; i += blockDim.x) {
+    for (long long i = lo + lane; i < hi; i += 32) {
         float c = 0.0f;
         if (vg != 0.0f) {
             c = rintf(__fdiv_rn(absmax[i], sigma));
@@ -342,7 +335,7 @@ inline cudaError_t launch_encode(const float* W, const lqlora_qmatrix* out, floa
     const long long ngrp = (nblk + out->cfg.B1 - 1) / out->cfg.B1;
     const float levels = static_cast<float>(scale_levels(out->cfg.b1));
     if (!packed_scales(&out->cfg)) {
-        encode_scales_kernel<<<static_cast<unsigned>(ngrp), 256, 0, st>>>(absmax, out->scale_codes, out->scale2, nblk, out->cfg.B1, levels);
+        encode_scales_kernel<<<static_cast<unsigned>((ngrp + 7) / 8), 256, 0, st>>>(absmax, out->scale_codes, out->scale2, nblk, ngrp, out->cfg.B1, levels);
         count_launch(2);
         return cudaGetLastError();
     }
@@ -350,7 +343,7 @@ inline cudaError_t launch_encode(const float* W, const lqlora_qmatrix* out, floa
     char* tail = reinterpret_cast<char*>(absmax) + (static_cast<size_t>(nblk) * sizeof(float) + 255) / 256 * 256;
     uint8_t* sc8 = reinterpret_cast<uint8_t*>(tail);
     float* v32 = reinterpret_cast<float*>(tail + (static_cast<size_t>(nblk) + 255) / 256 * 256);
-    encode_scales_kernel<<<static_cast<unsigned>(ngrp), 256, 0, st>>>(absmax, sc8, v32, nblk, out->cfg.B1, levels);
+    encode_scales_kernel<<<static_cast<unsigned>((ngrp + 7) / 8), 256, 0, st>>>(absmax, sc8, v32, nblk, ngrp, out->cfg.B1, levels);
     const long long threads = (nblk + 7) / 8 > ngrp ? (nblk + 7) / 8 : ngrp;
     pack_scales_kernel<<<static_cast<unsigned>((threads + 255) / 256), 256, 0, st>>>(sc8, v32, out->scale_codes, out->scale2, nblk, ngrp,
                                                                                  out->cfg.b1, out->cfg.b2);

@@ -90,3 +90,21 @@ def test_reference_arm_prints_one_json_line_and_other_ranks_stay_silent():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0"],
                          env=env, capture_output=True, text=True, timeout=600)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_gpus_flag_starts_the_ranks_itself_and_reports_their_number():
+    """`bench.py --gpus 2` without a launcher's environment starts two ranks (RANK / LOCAL_RANK / WORLD_SIZE /
+    MASTER_* set per rank); they meet over gloo (--dry-run: the host logic of the multi-rank path, no device work), take
+    the max over ranks of their step times (10 ms on rank 0, 15 ms on rank 1) and rank 0 alone prints the JSON line."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run", "--steps", "2", "--warmup", "3"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr
+    lines = [ln for ln in out.stdout.strip().splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["dry_run"] is True and line["ms_per_step"] == 15.0 and line["scaling"] == "weak"
+    # one process when one GPU is asked for
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "1", "--dry-run"], env=env, capture_output=True,
+                         text=True, timeout=300)
+    assert out.returncode == 0 and json.loads(out.stdout.strip().splitlines()[-1])["n_gpus"] == 1
