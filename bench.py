@@ -638,6 +638,21 @@ def run_case(args):
     q = binding.alloc_qmatrix(spec.N, spec.K, spec.cfg, dev)
     g = torch.Generator(device=dev)
     g.manual_seed(1)
+    if args.case_encode:
+        # the encoder alone: seeded Gaussian weights made on the device (no host copy of the largest matrices)
+        W = torch.empty((spec.N, spec.K), dtype=torch.float32, device=dev).normal_(0.0, 0.02, generator=g)
+        enc_ws = torch.empty(binding.packed_sizes(spec.N, spec.K, spec.cfg)[3], dtype=torch.uint8, device=dev)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.case_reps + 1)]
+        evs[0].record()
+        for i in range(args.case_reps):
+            binding.encode(W, spec.cfg, out=q, workspace=enc_ws)
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.case_reps)]
+        gbs = [encode_bytes(spec.N, spec.K, spec.cfg) / t / 1e6 for t in ms]
+        print(json.dumps({"case": args.case, "shape": [spec.N, spec.K], "quant": list(spec.cfg.as_tuple()),
+                          "encode_ms": ms, "encode_GB/s": gbs}), flush=True)
+        return
     q.codes.random_(0, 256, generator=g)
     q.scale_codes.random_(1, 128, generator=g)
     q.scale2.fill_(0.05)
@@ -723,6 +738,7 @@ def main():
     ap.add_argument("--case", default=None, help="run one matrix of the layer alone (q, k, v, o, gate, up, down)")
     ap.add_argument("--case-m", type=int, default=2048)
     ap.add_argument("--case-reps", type=int, default=3)
+    ap.add_argument("--case-encode", action="store_true", help="with --case: time lqlora_encode of that matrix instead of the linear calls")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)

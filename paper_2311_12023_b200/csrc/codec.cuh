@@ -55,6 +55,68 @@ __device__ __forceinline__ uint32_t search_code(float xh, float& margin) {
     }
 }
 
+// Fast search for 2- and 3-bit codes without compares or selects (the compare / select pipe is the encoder's
+// bottleneck; this runs on the fused-multiply-add pipe).  For x^ and threshold T_k, f_k = saturate(x^ * S + b_k) with
+// S = kSatScale, b_k = fl(0.5 - T_k S) is exactly 0 when x^ < T_k - 0.5/S, exactly 1 when x^ > T_k + 0.5/S, so the code
+// is f_1 + ... + f_n whenever x^ is not that close to a threshold.  The sum starts from a power of two chosen so that
+// the code lands in the mantissa bits that are the code's field of the packed word, seven bits above the bottom of the
+// word's 16-bit half: all bits below the field are zero unless some f_k was fractional (to 2^-8), i.e. unless x^ lies
+// within (0.5 - 2^-8 - 2^-5) / S = 8.9e-7 of a threshold (2^-5 bounds the rounding of b_k) -- more than the 2.4e-7 that x^ can
+// differ from the quotient.  Those bits are collected in `danger`; the caller then decides every code of the thread
+// exactly.  field_bits: position p (0, 2, .. 14) of the field in its half-word.
+template <int B>
+__device__ __forceinline__ uint32_t sat_count(float xh, float start) {
+    float acc = start;
+#pragma unroll
+    for (int k = 0; k < (1 << B) - 1; ++k) acc += __saturatef(fmaf(xh, kSatScale, c_satbias[B - 2][k]));
+    return __float_as_uint(acc);
+}
+// The B words of 32 codes from u * (r_lo | r_hi), layout of deposit_code<B>.
+template <int B>
+__device__ __forceinline__ void sat_encode(const float (&u)[32], float r_lo, float r_hi, uint32_t (&words)[B], uint32_t& danger) {
+    static_assert(B == 2 || B == 3, "2- and 3-bit codes");
+    constexpr uint32_t cmask = (1u << B) - 1u;
+    if constexpr (B == 3) {
+        uint32_t V = 0;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            uint32_t H[2] = {0u, 0u};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = 8 * w + 4 * h + jj, p = 4 * jj;
+                    const uint32_t bits = sat_count<3>(u[j] * ((j < 16) ? r_lo : r_hi), static_cast<float>(1u << (16 - p)));
+                    H[h] |= bits & (cmask << (7 + p));
+                    danger |= bits & ((1u << (7 + p)) - 1u);
+                }
+            }
+            const uint32_t word = (H[0] >> 7) | (H[1] << 9);
+            if (w < 3) words[w] = word;
+            else V = word;                 // codes 24..31 as 4-bit fields: their bits go to the spare fourth bits
+        }
+        words[0] |= (V & 0x11111111u) << 3;
+        words[1] |= ((V >> 1) & 0x11111111u) << 3;
+        words[2] |= ((V >> 2) & 0x11111111u) << 3;
+    } else {
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            uint32_t H[2] = {0u, 0u};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                for (int t2 = 0; t2 < 8; ++t2) {
+                    const int j = 16 * w + (t2 >> 2) * 8 + 4 * h + (t2 & 3), p = 4 * (t2 & 3) + 2 * (t2 >> 2);
+                    const uint32_t bits = sat_count<2>(u[j] * ((j < 16) ? r_lo : r_hi), static_cast<float>(1u << (16 - p)));
+                    H[h] |= bits & (cmask << (7 + p));
+                    danger |= bits & ((1u << (7 + p)) - 1u);
+                }
+            }
+            words[w] = (H[0] >> 7) | (H[1] << 9);
+        }
+    }
+}
+
 // Reciprocal used by the fast searches: 0 for an all-zero block (x^ = 0 gives the zero code), NaN for block maxima
 // whose reciprocal is not a normal number (every element then takes the exact route).
 __device__ __forceinline__ float search_reciprocal(float s) {
@@ -158,6 +220,23 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
     // the two routes agree.
     const float r_lo = search_reciprocal(s_lo);
     const float r_hi = search_reciprocal(s_hi);
+    if constexpr (B <= 3) {
+        // codes by saturating arithmetic; exact route for the whole thread when some x^ came close to a threshold or a
+        // reciprocal is not a normal number
+        uint32_t danger = (r_lo == r_lo && r_hi == r_hi) ? 0u : 1u;
+        if (danger == 0u) sat_encode<B>(u, r_lo, r_hi, words, danger);
+        if (danger != 0u) {
+#pragma unroll
+            for (int i = 0; i < B; ++i) words[i] = 0u;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float s = (j < 16) ? s_lo : s_hi;
+                uint32_t c = zero_code;
+                if (s != 0.0f) c = nearest_code<B>(__fdiv_rn(u[j], s), th8);
+                deposit_code<B>(words, j, c);
+            }
+        }
+    } else {
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
         const float s = (j < 16) ? s_lo : s_hi;
@@ -178,6 +257,7 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
             if (s != 0.0f) c = nearest_code<B>(__fdiv_rn(u[j], s), th8);
         }
         deposit_code<B>(words, j, c);
+    }
     }
     uint32_t* dst = codes + slab_word_base(row, k0 >> 6, K >> 6, B);
     const int g = (k0 >> 5) & 1;

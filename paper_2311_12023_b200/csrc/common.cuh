@@ -145,6 +145,10 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_
 // neighbouring code-book entries (x > midpoint  <=>  x > threshold for fp32 x).
 __constant__ float c_codebook[4][256];
 __constant__ float c_threshold[4][256];
+// 2- and 3-bit encoder: fl(0.5 - threshold * kSatScale) per threshold; saturate(x * kSatScale + bias) is 0 below the
+// threshold, 1 above it and in between only within 0.5 / kSatScale = 9.5e-7 of it.
+constexpr float kSatScale = 524288.0f;
+__constant__ float c_satbias[2][8];
 
 // Bin table for the nearest-code search of the encoder: [-1, 1] is cut into `nb` equal bins chosen so that every
 // bin holds at most one threshold and no threshold lies near a bin edge.  Entry k = (threshold in the bin or +inf,

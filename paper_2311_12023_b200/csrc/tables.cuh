@@ -35,6 +35,7 @@ struct HostTables {
     float threshold[4][256];
     BinEntry bins[4][kMaxBins + 1];
     int nbins[4];
+    float satbias[2][8];
     // Bin count for `n - 1` thresholds: the candidate with the largest distance between any threshold and any
     // bin edge among those with at most one threshold per bin.
     void build_bins(int t, int n) {
@@ -95,6 +96,9 @@ struct HostTables {
             }
             build_bins(t, n);
         }
+        for (int t = 0; t < 2; ++t)
+            for (int i = 0; i < 8; ++i)
+                satbias[t][i] = (i + 1 < (4 << t)) ? static_cast<float>(0.5 - static_cast<double>(threshold[t][i]) * static_cast<double>(kSatScale)) : 0.0f;
     }
 };
 
@@ -117,6 +121,7 @@ int ensure_tables() {
     const detail::HostTables& t = detail::host_tables();
     if (cudaMemcpyToSymbol(c_codebook, t.codebook, sizeof(t.codebook)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_threshold, t.threshold, sizeof(t.threshold)) != cudaSuccess ||
+        cudaMemcpyToSymbol(c_satbias, t.satbias, sizeof(t.satbias)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_bins, t.bins, sizeof(t.bins)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_nbins, t.nbins, sizeof(t.nbins)) != cudaSuccess) {
         cudaGetLastError();

@@ -57,6 +57,33 @@ def test_codec_degenerate_inputs():
     assert_codec_parity(q, ref)
 
 
+@pytest.mark.parametrize("b0,B0", [(2, 16), (2, 64), (3, 16), (3, 128)])
+def test_codec_values_next_to_thresholds(b0, B0):
+    """2- and 3-bit codes are found with saturating arithmetic and re-decided exactly when the scaled value comes
+    within a micro-unit of a midpoint: elements u = fl((mid + d) s) for every midpoint, offsets d from 0 to 3e-6 on both
+    sides and random block maxima s (so that the rounding of u / s matters), plus block maxima whose reciprocal is not
+    a normal number.  Codes must equal the oracle's bit for bit."""
+    g = inputs.rng(40 + b0 + B0)
+    cb = binding.nf_codebook(b0).astype(np.float64)
+    mids = 0.5 * (cb[:-1] + cb[1:])
+    offs = np.array([0.0, 1e-9, 3e-8, 6e-8, 1.2e-7, 2.4e-7, 5e-7, 8.5e-7, 9.6e-7, 1.5e-6, 3e-6])
+    offs = np.concatenate([offs, -offs[1:]])
+    vals = (mids[:, None] + offs[None, :]).ravel()
+    rows = []
+    for rep in range(96):
+        s = np.float32(10.0 ** g.uniform(-3.0, 1.0))
+        row = np.zeros(1024, dtype=np.float32)
+        pick = g.choice(vals, size=1024)
+        row[:] = (pick * np.float64(s)).astype(np.float32)
+        row[::B0] = s * np.float32(1.0 if rep % 2 else -1.0)       # the block maximum itself
+        rows.append(row)
+    A = np.stack(rows)
+    A[5, :B0] *= np.float32(1e-38)        # subnormal block maximum: no usable reciprocal
+    A[6, :B0] = 0.0
+    q, ref = encode_both(A, C(b0, B0, 8, 64, 32), check=False)
+    assert_codec_parity(q, ref)
+
+
 def test_codec_config1_roberta_proj():
     spec = inputs.workload(1)["matrices"][0]
     A, _, _ = inputs.make_matrix(spec)
