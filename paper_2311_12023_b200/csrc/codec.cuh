@@ -68,7 +68,11 @@ template <int B>
 __device__ __forceinline__ uint32_t sat_count(float xh, float start) {
     float acc = start;
 #pragma unroll
-    for (int k = 0; k < (1 << B) - 1; ++k) acc += __saturatef(fmaf(xh, kSatScale, c_satbias[B - 2][k]));
+    for (int k = 0; k < (1 << B) - 1; ++k) {
+        float f;
+        asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(f) : "f"(xh), "f"(kSatScale), "f"(c_satbias[B - 2][k]));
+        acc += f;
+    }
     return __float_as_uint(acc);
 }
 // The B words of 32 codes from u * (r_lo | r_hi), layout of deposit_code<B>.
@@ -266,28 +270,104 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
 }
 
 // One warp per second-level group (eight groups per CTA): v_g = max s_i, s^_i = clamp(rint(s_i / (v_g / levels)), 0, levels).
+// The quotient is found without a division where that is safe: t = fl(s_i * fl(1 / sigma) + 3072) holds the quotient in
+// fixed point with 12 fraction bits (s_i <= v_g, so it is at most levels <= 127 and t stays in [2048, 4096)); its error
+// against fl(s_i / sigma) is below 2^-13 + 1.2e-5, so rounding the fixed-point value half up gives rint of the IEEE
+// quotient unless the fraction lies within 2^-12 of one half; those elements (0.07 %) take the IEEE division.
+__device__ __forceinline__ uint32_t scale_code_exact(float a, float sigma, float levels) {
+    return static_cast<uint32_t>(fminf(fmaxf(rintf(__fdiv_rn(a, sigma)), 0.0f), levels));
+}
+__device__ __forceinline__ uint32_t scale_code(float a, float sigma, float rsigma, float levels, bool fast) {
+    if (fast) {
+        const uint32_t bits = __float_as_uint(fmaf(a, rsigma, 3072.0f));
+        if ((bits & 0xFFFu) - 0x7FFu > 2u) return ((bits + 0x800u) >> 12) & 0xFFu;
+    }
+    return scale_code_exact(a, sigma, levels);
+}
+// Groups of up to 256 blocks: a warp owns a span of 256 consecutive blocks (whole groups: spans and groups are aligned),
+// four pairs of blocks per lane, all loaded before anything else happens (the kernel is bound by memory latency: the
+// maxima, the quotients and the stores come from registers).  A group is a run of lanes of one load (B1 <= 64), two loads
+// (128) or all four (256).
+__global__ void __launch_bounds__(256) encode_scales_span_kernel(const float* __restrict__ absmax, uint8_t* __restrict__ sc,
+                                                                 float* __restrict__ v, long long nblk, long long ngrp, int B1, int logB1,
+                                                                 float levels) {
+    const long long base = (static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5)) * 256;
+    if (base >= nblk) return;
+    const int lane = threadIdx.x & 31;
+    float2 a[4];
+    float m[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const long long blk = base + 2 * (e * 32 + lane);
+        a[e] = make_float2(0.0f, 0.0f);
+        if (blk + 1 < nblk) a[e] = *reinterpret_cast<const float2*>(absmax + blk);
+        else if (blk < nblk) a[e].x = absmax[blk];
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) m[e] = fmaxf(a[e].x, a[e].y);
+    const int seg = (B1 >= 64) ? 32 : (B1 >> 1);           // lanes of one load that share a group
+    for (int o = seg >> 1; o > 0; o >>= 1) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) m[e] = fmaxf(m[e], __shfl_xor_sync(0xffffffffu, m[e], o));
+    }
+    if (B1 >= 128) {
+        m[0] = m[1] = fmaxf(m[0], m[1]);
+        m[2] = m[3] = fmaxf(m[2], m[3]);
+    }
+    if (B1 == 256) m[0] = m[1] = m[2] = m[3] = fmaxf(m[0], m[2]);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const long long blk = base + 2 * (e * 32 + lane);
+        const float vg = m[e];
+        if ((blk & (B1 - 1)) == 0 && blk < nblk) v[blk >> logB1] = vg;
+        uint32_t c0 = 0u, c1 = 0u;
+        if (vg != 0.0f) {
+            const float sigma = __fdiv_rn(vg, levels);
+            const bool fast = sigma > 1e-30f && sigma < 1e30f;
+            const float rsigma = fast ? __fdiv_rn(1.0f, sigma) : 0.0f;
+            c0 = scale_code(a[e].x, sigma, rsigma, levels, fast);
+            c1 = scale_code(a[e].y, sigma, rsigma, levels, fast);
+        }
+        if (blk + 1 < nblk) *reinterpret_cast<uint16_t*>(sc + blk) = static_cast<uint16_t>(c0 | (c1 << 8));
+        else if (blk < nblk) sc[blk] = static_cast<uint8_t>(c0);
+    }
+    (void)ngrp;
+}
+
+// Larger groups: one warp per group.
 __global__ void __launch_bounds__(256) encode_scales_kernel(const float* __restrict__ absmax, uint8_t* __restrict__ sc,
                                                             float* __restrict__ v, long long nblk, long long ngrp, int B1, float levels) {
     const long long g = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
     if (g >= ngrp) return;
     const int lane = threadIdx.x & 31;
-    const long long lo = g * B1;
-    const long long hi = (lo + B1 < nblk) ? lo + B1 : nblk;
+    const long long lo = g * B1;                          // a multiple of 16: pairs of blocks are 8-byte aligned
+    const int n = static_cast<int>((lo + B1 < nblk) ? B1 : nblk - lo);
+    const float2* __restrict__ a2 = reinterpret_cast<const float2*>(absmax + lo);
     float m = 0.0f;
-    for (long long i = lo + lane; i < hi; i += 32) m = fmaxf(m, absmax[i]);
+    for (int i = lane; 2 * i + 1 < n; i += 32) {
+        const float2 a = a2[i];
+        m = fmaxf(m, fmaxf(a.x, a.y));
+    }
+    if ((n & 1) && lane == 0) m = fmaxf(m, absmax[lo + n - 1]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     const float vg = m;
     if (lane == 0) v[g] = vg;
-    const float sigma = __fdiv_rn(vg, levels);
-    for (long long i = lo + lane; i < hi; i += 32) {
-        float c = 0.0f;
-        if (vg != 0.0f) {
-            c = rintf(__fdiv_rn(absmax[i], sigma));
-            c = fminf(fmaxf(c, 0.0f), levels);
-        }
-        sc[i] = static_cast<uint8_t>(c);
+    uint16_t* __restrict__ sc2 = reinterpret_cast<uint16_t*>(sc + lo);
+    if (vg == 0.0f) {
+        for (int i = lane; 2 * i + 1 < n; i += 32) sc2[i] = 0;
+        if ((n & 1) && lane == 0) sc[lo + n - 1] = 0;
+        return;
     }
+    const float sigma = __fdiv_rn(vg, levels);
+    const bool fast = sigma > 1e-30f && sigma < 1e30f;
+    const float rsigma = fast ? __fdiv_rn(1.0f, sigma) : 0.0f;
+    for (int i = lane; 2 * i + 1 < n; i += 32) {
+        const float2 a = a2[i];
+        const uint32_t c0 = scale_code(a.x, sigma, rsigma, levels, fast), c1 = scale_code(a.y, sigma, rsigma, levels, fast);
+        sc2[i] = static_cast<uint16_t>(c0 | (c1 << 8));
+    }
+    if ((n & 1) && lane == 0) sc[lo + n - 1] = static_cast<uint8_t>(scale_code_exact(absmax[lo + n - 1], sigma, levels));
 }
 
 // Storage forms of the scales (Table 1 of Sec. 3.2).  b1 < 8: the codes form a bit stream of b1 bits each, code i in
@@ -404,6 +484,15 @@ __global__ void __launch_bounds__(256) export_kernel(QView q, uint8_t* __restric
     }
 }
 
+inline void launch_encode_scales(const float* absmax, uint8_t* sc, float* v, long long nblk, long long ngrp, int B1, float levels, cudaStream_t st) {
+    if (B1 <= 256) {
+        const long long spans = (nblk + 255) / 256;
+        encode_scales_span_kernel<<<static_cast<unsigned>((spans + 7) / 8), 256, 0, st>>>(absmax, sc, v, nblk, ngrp, B1, ilog2(B1), levels);
+    } else {
+        encode_scales_kernel<<<static_cast<unsigned>((ngrp + 7) / 8), 256, 0, st>>>(absmax, sc, v, nblk, ngrp, B1, levels);
+    }
+}
+
 template <int B>
 inline cudaError_t launch_encode(const float* W, const lqlora_qmatrix* out, float* absmax, cudaStream_t st) {
     const int N = static_cast<int>(out->N), K = static_cast<int>(out->K);
@@ -415,7 +504,7 @@ inline cudaError_t launch_encode(const float* W, const lqlora_qmatrix* out, floa
     const long long ngrp = (nblk + out->cfg.B1 - 1) / out->cfg.B1;
     const float levels = static_cast<float>(scale_levels(out->cfg.b1));
     if (!packed_scales(&out->cfg)) {
-        encode_scales_kernel<<<static_cast<unsigned>((ngrp + 7) / 8), 256, 0, st>>>(absmax, out->scale_codes, out->scale2, nblk, ngrp, out->cfg.B1, levels);
+        launch_encode_scales(absmax, out->scale_codes, out->scale2, nblk, ngrp, out->cfg.B1, levels, st);
         count_launch(2);
         return cudaGetLastError();
     }
@@ -423,7 +512,7 @@ inline cudaError_t launch_encode(const float* W, const lqlora_qmatrix* out, floa
     char* tail = reinterpret_cast<char*>(absmax) + (static_cast<size_t>(nblk) * sizeof(float) + 255) / 256 * 256;
     uint8_t* sc8 = reinterpret_cast<uint8_t*>(tail);
     float* v32 = reinterpret_cast<float*>(tail + (static_cast<size_t>(nblk) + 255) / 256 * 256);
-    encode_scales_kernel<<<static_cast<unsigned>((ngrp + 7) / 8), 256, 0, st>>>(absmax, sc8, v32, nblk, ngrp, out->cfg.B1, levels);
+    launch_encode_scales(absmax, sc8, v32, nblk, ngrp, out->cfg.B1, levels, st);
     const long long threads = (nblk + 7) / 8 > ngrp ? (nblk + 7) / 8 : ngrp;
     pack_scales_kernel<<<static_cast<unsigned>((threads + 255) / 256), 256, 0, st>>>(sc8, v32, out->scale_codes, out->scale2, nblk, ngrp,
                                                                                  out->cfg.b1, out->cfg.b2);

@@ -29,6 +29,22 @@ def test_codec_groups_straddle_rows_and_ragged_tail():
     assert_codec_parity(q, ref)
 
 
+@pytest.mark.parametrize("B1", [16, 32, 128, 256, 512, 4096])
+def test_codec_second_level_group_sizes(B1):
+    """Every group size class of the scale quantization: runs of lanes (16, 32), two and four loads per lane (128, 256),
+    one warp per group beyond that; 131 x 3 = 393 and 77 x 25 = 1925 blocks (odd counts, short last group), 3200 blocks, and
+    a matrix with zero groups and huge / tiny magnitudes."""
+    for shape, B0 in (((131, 192), 64), ((77, 1600), 64), ((50, 1024), 16)):
+        A = inputs.gaussian_outliers(60 + B1, shape, 0.02, 0.01, 8.0)
+        q, ref = encode_both(A, C(3, B0, 8, B1, 32), check=False)
+        assert_codec_parity(q, ref)
+    g = inputs.rng(61 + B1)
+    A = (g.standard_normal((64, 1024)) * 10.0 ** g.integers(-40, 30, size=(64, 1))).astype(np.float32)
+    A[7:23] = 0.0
+    q, ref = encode_both(A, C(2, 16, 8, B1, 32), check=False)
+    assert_codec_parity(q, ref)
+
+
 def test_codec_degenerate_inputs():
     cfg = C(4, 64, 8, 256, 32)
     zero = np.zeros((64, 128), dtype=np.float32)
