@@ -167,11 +167,19 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
         float4* mine = tile[grp];
         const int lr = rl >> 3, ch = rl & 7;
         float4 t[8];
+        if (live && blockIdx.x * 32 + 32 <= N) {
+            // all 32 rows exist: one pointer, constant strides
+            const float4* src = reinterpret_cast<const float4*>(W + static_cast<size_t>(blockIdx.x * 32 + lr) * K + k0) + ch;
+            const size_t stride = static_cast<size_t>(K);            // four rows, in float4
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int rr = blockIdx.x * 32 + 4 * i + lr;
-            t[i] = (live && rr < N) ? __ldg(reinterpret_cast<const float4*>(W + static_cast<size_t>(rr) * K + k0) + ch)
-                                    : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            for (int i = 0; i < 8; ++i) t[i] = __ldg(src + i * stride);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int rr = blockIdx.x * 32 + 4 * i + lr;
+                t[i] = (live && rr < N) ? __ldg(reinterpret_cast<const float4*>(W + static_cast<size_t>(rr) * K + k0) + ch)
+                                        : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            }
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -189,13 +197,14 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
     float m0 = 0.0f, m1 = 0.0f;
 #pragma unroll
     for (int i = 0; i < 16; ++i) { m0 = fmaxf(m0, fabsf(u[i])); m1 = fmaxf(m1, fabsf(u[16 + i])); }
-    red[grp][rl] = fmaxf(m0, m1);
-    __syncthreads();
-
+    if constexpr (B >= 4) __syncthreads();       // the search tables in shared memory are complete
     float s_lo, s_hi;   // block absmax for columns 0..15 and 16..31 of this thread's group
     if (B0 == 16) { s_lo = m0; s_hi = m1; }
     else if (B0 == 32) { s_lo = s_hi = fmaxf(m0, m1); }
     else {
+        // blocks wider than a thread's 32 columns: the maxima of the neighbouring groups come through shared memory
+        red[grp][rl] = fmaxf(m0, m1);
+        __syncthreads();
         const int span = B0 >> 5, g0 = grp & ~(span - 1);
         float m = 0.0f;
         for (int i = 0; i < span; ++i) m = fmaxf(m, red[g0 + i][rl]);
@@ -204,8 +213,7 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
     if (real) {
         const int KB = K >> logB0;
         if (B0 == 16) {
-            absmax[static_cast<size_t>(row) * KB + (k0 >> 4)] = s_lo;
-            absmax[static_cast<size_t>(row) * KB + (k0 >> 4) + 1] = s_hi;
+            *reinterpret_cast<float2*>(absmax + static_cast<size_t>(row) * KB + (k0 >> 4)) = make_float2(s_lo, s_hi);   // KB, k0 / 16 even
         } else if ((k0 & (B0 - 1)) == 0) {
             absmax[static_cast<size_t>(row) * KB + (k0 >> logB0)] = s_lo;
         }
