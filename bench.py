@@ -634,6 +634,9 @@ def run_case(args):
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     spec = [s for s in inputs.workload(4)["matrices"] if s.name == args.case][0]
+    if args.case_cfg:
+        import dataclasses
+        spec = dataclasses.replace(spec, cfg=inputs.QuantConfig(*[int(x) for x in args.case_cfg.split(",")]))
     M, r = args.case_m, inputs.RANK
     q = binding.alloc_qmatrix(spec.N, spec.K, spec.cfg, dev)
     g = torch.Generator(device=dev)
@@ -738,6 +741,7 @@ def main():
     ap.add_argument("--case", default=None, help="run one matrix of the layer alone (q, k, v, o, gate, up, down)")
     ap.add_argument("--case-m", type=int, default=2048)
     ap.add_argument("--case-reps", type=int, default=3)
+    ap.add_argument("--case-cfg", default=None, help="with --case: another configuration b0,B0,b1,B1,b2 for that matrix's shape")
     ap.add_argument("--case-encode", action="store_true", help="with --case: time lqlora_encode of that matrix instead of the linear calls")
     args = ap.parse_args()
     if args.sweep:

@@ -29,32 +29,6 @@ __device__ __forceinline__ uint32_t nearest_code(float x, const float* __restric
     }
 }
 
-// Fast search for 2- and 3-bit codes: binary search of x^ among the (constant) thresholds; `margin` returns the
-// distance from x^ to the nearest threshold it was compared with.  The two neighbours of the final position are
-// always among them, so when margin exceeds the error of x^ every comparison came out as it would for the exact
-// quotient and the code is the same.
-template <int B>
-__device__ __forceinline__ uint32_t search_code(float xh, float& margin) {
-    static_assert(B == 2 || B == 3, "binary search is written out for 3 and 7 thresholds");
-    const float* T = c_threshold[B == 2 ? 0 : 1];
-    if constexpr (B == 2) {
-        const bool p1 = xh > T[1];
-        const float t = p1 ? T[2] : T[0];
-        const bool p2 = xh > t;
-        margin = fminf(fabsf(xh - T[1]), fabsf(xh - t));
-        return (p1 ? 2u : 0u) + (p2 ? 1u : 0u);
-    } else {
-        const bool p1 = xh > T[3];
-        const float t2 = p1 ? T[5] : T[1];
-        const bool p2 = xh > t2;
-        const float ta = p1 ? T[4] : T[0], tb = p1 ? T[6] : T[2];
-        const float t3 = p2 ? tb : ta;
-        const bool p3 = xh > t3;
-        margin = fminf(fminf(fabsf(xh - T[3]), fabsf(xh - t2)), fabsf(xh - t3));
-        return (p1 ? 4u : 0u) + (p2 ? 2u : 0u) + (p3 ? 1u : 0u);
-    }
-}
-
 // Fast search for 2- and 3-bit codes without compares or selects (the compare / select pipe is the encoder's
 // bottleneck; this runs on the fused-multiply-add pipe).  For x^ and threshold T_k, f_k = saturate(x^ * S + b_k) with
 // S = kSatScale, b_k = fl(0.5 - T_k S) is exactly 0 when x^ < T_k - 0.5/S, exactly 1 when x^ > T_k + 0.5/S, so the code
@@ -148,7 +122,7 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
     const int nb = kUseBins ? c_nbins[bits_index(B)] : 0;
     if constexpr (kUseBins) {
         for (int i = threadIdx.x; i <= nb; i += 256) {
-            const BinEntry e = c_bins[bits_index(B)][i];
+            const BinEntry e = g_bins[bits_index(B)][i];       // global memory: coalesced (the constant bank would serialize the lanes)
             bins[i] = make_float2(e.thr, __int_as_float(e.base));
         }
     }
@@ -249,27 +223,38 @@ __global__ void __launch_bounds__(256) encode_codes_kernel(const float* __restri
             }
         }
     } else {
+        // Bin table: the bin of x^ holds at most one threshold, code = thresholds below the bin plus (x^ > threshold).
+        // First all 32 codes without a branch (32 independent chains for the scheduler), keeping the smallest distance
+        // between an x^ and the threshold it was compared with; only a thread where that distance is within 1e-6 (or a
+        // reciprocal is not a normal number) goes through its elements again and decides the close ones exactly.
+        float margin = (r_lo == r_lo && r_hi == r_hi) ? 1.0f : 0.0f;
+        if (margin != 0.0f) {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        const float s = (j < 16) ? s_lo : s_hi;
-        const float xh = u[j] * ((j < 16) ? r_lo : r_hi);
-        uint32_t c;
-        float margin;
-        if constexpr (kUseBins) {
-            int k = __float2int_rd(fmaf(xh, bin_scale, bin_scale));
-            k = min(max(k, 0), nb);
-            const float2 e = bins[k];
-            c = static_cast<uint32_t>(__float_as_int(e.y)) + ((xh > e.x) ? 1u : 0u);
-            margin = fabsf(xh - e.x);
-        } else {
-            c = search_code<B>(xh, margin);
+            for (int j = 0; j < 32; ++j) {
+                const float xh = u[j] * ((j < 16) ? r_lo : r_hi);
+                const uint32_t k = min(__float2uint_rd(fmaf(xh, bin_scale, bin_scale)), static_cast<uint32_t>(nb));
+                const float2 e = bins[k];
+                deposit_code<B>(words, j, static_cast<uint32_t>(__float_as_int(e.y)) + ((xh > e.x) ? 1u : 0u));
+                margin = fminf(margin, fabsf(xh - e.x));
+            }
         }
-        if (!(margin > 1e-6f) || !(fabsf(xh) <= 1.001f)) {
-            c = zero_code;
-            if (s != 0.0f) c = nearest_code<B>(__fdiv_rn(u[j], s), th8);
+        if (!(margin > 1e-6f)) {
+#pragma unroll
+            for (int i = 0; i < B; ++i) words[i] = 0u;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float s = (j < 16) ? s_lo : s_hi, r = (j < 16) ? r_lo : r_hi;
+                const float xh = u[j] * r;
+                const uint32_t k = min(__float2uint_rd(fmaf(xh, bin_scale, bin_scale)), static_cast<uint32_t>(nb));
+                const float2 e = bins[k];
+                uint32_t c = static_cast<uint32_t>(__float_as_int(e.y)) + ((xh > e.x) ? 1u : 0u);
+                if (!(fabsf(xh - e.x) > 1e-6f) || !(r == r)) {
+                    c = zero_code;
+                    if (s != 0.0f) c = nearest_code<B>(__fdiv_rn(u[j], s), th8);
+                }
+                deposit_code<B>(words, j, c);
+            }
         }
-        deposit_code<B>(words, j, c);
-    }
     }
     uint32_t* dst = codes + slab_word_base(row, k0 >> 6, K >> 6, B);
     const int g = (k0 >> 5) & 1;

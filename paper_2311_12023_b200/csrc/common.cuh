@@ -155,7 +155,7 @@ __constant__ float c_satbias[2][8];
 // number of thresholds below the bin); entry nb serves x slightly above 1.
 constexpr int kMaxBins = 1280;
 struct BinEntry { float thr; int base; };
-__constant__ BinEntry c_bins[4][kMaxBins + 1];
+__device__ BinEntry g_bins[4][kMaxBins + 1];
 __constant__ int c_nbins[4];
 
 int ensure_tables();                 // uploads the tables to the current device once; LQLORA_OK or error

@@ -122,7 +122,7 @@ int ensure_tables() {
     if (cudaMemcpyToSymbol(c_codebook, t.codebook, sizeof(t.codebook)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_threshold, t.threshold, sizeof(t.threshold)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_satbias, t.satbias, sizeof(t.satbias)) != cudaSuccess ||
-        cudaMemcpyToSymbol(c_bins, t.bins, sizeof(t.bins)) != cudaSuccess ||
+        cudaMemcpyToSymbol(g_bins, t.bins, sizeof(t.bins)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_nbins, t.nbins, sizeof(t.nbins)) != cudaSuccess) {
         cudaGetLastError();
         return LQLORA_ERR_CUDA;

@@ -73,10 +73,10 @@ def test_codec_degenerate_inputs():
     assert_codec_parity(q, ref)
 
 
-@pytest.mark.parametrize("b0,B0", [(2, 16), (2, 64), (3, 16), (3, 128)])
+@pytest.mark.parametrize("b0,B0", [(2, 16), (2, 64), (3, 16), (3, 128), (4, 64), (8, 32)])
 def test_codec_values_next_to_thresholds(b0, B0):
-    """2- and 3-bit codes are found with saturating arithmetic and re-decided exactly when the scaled value comes
-    within a micro-unit of a midpoint: elements u = fl((mid + d) s) for every midpoint, offsets d from 0 to 3e-6 on both
+    """The fast searches (saturating arithmetic for 2- and 3-bit codes, a bin table for 4 and 8 bits) decide from
+    u * fl(1/s) and fall back to the exact quotient when that comes within a micro-unit of a midpoint: elements u = fl((mid + d) s) for every midpoint, offsets d from 0 to 3e-6 on both
     sides and random block maxima s (so that the rounding of u / s matters), plus block maxima whose reciprocal is not
     a normal number.  Codes must equal the oracle's bit for bit."""
     g = inputs.rng(40 + b0 + B0)
