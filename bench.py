@@ -566,6 +566,19 @@ def run_device(args):
     gbytes = 2.0 * 2048 * (gm.N + gm.K)
     extra = {"lora_grads_gate_M2048": {"ms": g_ms2, "GB/s": gbytes / g_ms2 / 1e6, "frac_of_hbm_" + pk_kind: gbytes / g_ms2 / 1e6 / pk["hbm_gbs"],
                                        "in_timed_step": False, "what": "lqlora_lora_grads; bytes = X and dY read once"}}
+    # the same gradients from the intermediates that the forward and the input-gradient call left in their workspaces
+    ws_f, ws_b = binding.alloc_workspace(gm.q, r, 2048), binding.alloc_workspace(gm.q, r, 2048)
+    binding.linear_fwd(gm.q, gm.L1, gm.L2, gm.X[2048], workspace=ws_f)
+    binding.linear_bwd_input(gm.q, gm.L1, gm.L2, gm.G[2048], workspace=ws_b)
+    T = binding.linear_intermediate(ws_f, gm.N, gm.K, gm.cfg, r, 2048, False)
+    Tp = binding.linear_intermediate(ws_b, gm.N, gm.K, gm.cfg, r, 2048, True)
+    sws = torch.empty(256, dtype=torch.uint8, device=dev)
+    g_ms3 = timer(lambda: [binding.lora_grads_from(T, Tp, gm.N, gm.K, gm.X[2048], gm.G[2048], out=dL, workspace=sws) for _ in range(4)], 4)
+    if binding.workspace_status(sws) != 0:
+        raise SystemExit("lora_grads_from reported a device-side error")
+    extra["lora_grads_from_gate_M2048"] = {"ms": g_ms3, "GB/s": gbytes / g_ms3 / 1e6, "frac_of_hbm_" + pk_kind: gbytes / g_ms3 / 1e6 / pk["hbm_gbs"],
+                                           "in_timed_step": False, "what": "lqlora_lora_grads_from (T, T' reused); bytes = X and dY read once"}
+    del ws_f, ws_b
 
     h2d = sum(m.W_host.numel() * 4 + sum(m.XH[M].numel() * 2 + m.GH[M].numel() * 2 for M in MS) for m in mats)
     d2h = sum(sum(m.YH[M].numel() * 2 + m.DXH[M].numel() * 2 for M in MS) for m in mats)

@@ -209,6 +209,22 @@ int lqlora_lora_grads(const void* L1_dev, const void* L2_dev, int r, int64_t N, 
                       size_t workspace_bytes, void* stream);
 
 /*
+ * The same gradients from the rank-r intermediates that the other two passes have already computed (the trained layer of
+ * Sec. 2.1 runs forward, input gradient and factor gradients on the same X and dY): T = bf16(X L2^T) is what
+ * lqlora_linear_fwd leaves in its workspace, T' = bf16(dY L1) what lqlora_linear_bwd_input leaves in its own, each at the
+ * byte offset lqlora_linear_intermediate_offset reports for that call's (N, K, cfg, r, M, direction), as [M, r] bf16
+ * row-major, valid until that workspace is used again.  X and dY are then read once instead of twice.
+ *   T_dev, Tp_dev [M, r] : bf16, device, 16-byte aligned, read only;  the other arguments as for lqlora_lora_grads
+ *   workspace_dev : at least 256 bytes (the status word only); it must not be one of the workspaces that hold T or T'
+ * Asynchronous on `stream`; the library allocates nothing.  Errors as for lqlora_lora_grads.
+ */
+int lqlora_linear_intermediate_offset(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, int backward,
+                                      size_t* offset);
+int lqlora_lora_grads_from(const void* T_dev, const void* Tp_dev, int r, int64_t N, int64_t K, const void* X_dev,
+                           const void* dY_dev, int64_t M, float* dL1_dev, float* dL2_dev, void* workspace_dev,
+                           size_t workspace_bytes, void* stream);
+
+/*
  * The low-rank plus quantized decomposition of Sec. 3.1 (Eq. (1)-(2), Algorithm 2), with Factorize of Sec. 3.3
  * (Eq. (4), Algorithm 4), in nn.Linear orientation:  W [N, K] ~ deq(Q) + L1 [N, r] L2 [r, K].
  *     Q <- 0;  repeat  L1, L2 <- Factorize(W - Q, F, r);  Q <- Quantize(W - L1 L2, c);  e_t <- error

@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.lqlora_linear_bwd_input.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, sz, vp]
         L.lqlora_lora_grads_workspace_bytes.argtypes = [i64, i64, ci, i64, ctypes.POINTER(sz)]
         L.lqlora_lora_grads.argtypes = [vp, vp, ci, i64, i64, vp, vp, i64, vp, vp, vp, sz, vp]
+        L.lqlora_linear_intermediate_offset.argtypes = [i64, i64, ctypes.POINTER(CConfig), ci, i64, ci, ctypes.POINTER(sz)]
+        L.lqlora_lora_grads_from.argtypes = [vp, vp, ci, i64, i64, vp, vp, i64, vp, vp, vp, sz, vp]
         L.lqlora_encode_host.argtypes = [vp, vp, ctypes.POINTER(CQMatrix), vp, sz, vp]
         L.lqlora_linear_fwd_host.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, vp, vp, sz, vp]
         L.lqlora_linear_bwd_input_host.argtypes = [ctypes.POINTER(CQMatrix), vp, vp, ci, vp, i64, vp, vp, vp, vp, sz, vp]
@@ -335,6 +337,31 @@ def lora_grads(L1: torch.Tensor, L2: torch.Tensor, X: torch.Tensor, dY: torch.Te
         workspace = torch.empty(lora_grads_workspace_bytes(N, K, r, M), dtype=torch.uint8, device=X.device)
     _check(lib().lqlora_lora_grads(L1.data_ptr(), L2.data_ptr(), r, N, K, X.data_ptr(), dY.data_ptr(), M, out[0].data_ptr(),
                                    out[1].data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()), "lqlora_lora_grads")
+    return out
+
+
+def linear_intermediate(workspace: torch.Tensor, N: int, K: int, cfg, r: int, M: int, backward: bool) -> torch.Tensor:
+    """View of the bf16 [M, r] intermediate (X L2^T or dY L1) that the last linear call left in `workspace`
+    (lqlora_linear_intermediate_offset)."""
+    off = ctypes.c_size_t(0)
+    c = _cfg(cfg)
+    _check(lib().lqlora_linear_intermediate_offset(N, K, ctypes.byref(c), r, M, 1 if backward else 0, ctypes.byref(off)),
+           "lqlora_linear_intermediate_offset")
+    return workspace[off.value:off.value + M * r * 2].view(torch.bfloat16).view(M, r)
+
+
+def lora_grads_from(T: torch.Tensor, Tp: torch.Tensor, N: int, K: int, X: torch.Tensor, dY: torch.Tensor, out=None, workspace=None):
+    """lqlora_lora_grads_from: (dL1 [N, r], dL2 [r, K]) in fp32 from the intermediates T = bf16(X L2^T), T' = bf16(dY L1)."""
+    M, r = T.shape
+    assert tuple(Tp.shape) == (M, r) and tuple(X.shape) == (M, K) and tuple(dY.shape) == (M, N)
+    for t in (T, Tp, X, dY):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    if out is None:
+        out = (torch.empty(N, r, dtype=torch.float32, device=X.device), torch.empty(r, K, dtype=torch.float32, device=X.device))
+    if workspace is None:
+        workspace = torch.empty(256, dtype=torch.uint8, device=X.device)
+    _check(lib().lqlora_lora_grads_from(T.data_ptr(), Tp.data_ptr(), r, N, K, X.data_ptr(), dY.data_ptr(), M, out[0].data_ptr(),
+                                        out[1].data_ptr(), workspace.data_ptr(), workspace.numel(), _stream()), "lqlora_lora_grads_from")
     return out
 
 

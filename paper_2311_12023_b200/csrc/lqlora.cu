@@ -395,6 +395,38 @@ int lqlora_lora_grads(const void* L1_dev, const void* L2_dev, int r, int64_t N, 
                                  static_cast<cudaStream_t>(stream));
 }
 
+int lqlora_linear_intermediate_offset(int64_t N, int64_t K, const lqlora_config* cfg, int r, int64_t M, int backward, size_t* offset) {
+    using namespace lq;
+    if (!offset) return LQLORA_ERR_NULL_POINTER;
+    if (check_config(cfg) != LQLORA_OK || check_shape(N, K, cfg) != LQLORA_OK) return LQLORA_ERR_INVALID_CONFIG;
+    if (M <= 0 || r <= 0 || r > 128 || r % 16) return LQLORA_ERR_INVALID_SHAPE;
+    lqlora_qmatrix q{};
+    q.N = N; q.K = K; q.cfg = *cfg;
+    const QView v = make_view(&q);
+    const bool bwd = backward != 0;
+    // the tensor-core and the plain kernels keep [status][T]; the weight-streaming kernels [status][arrival counters][T]
+    size_t off = kStatusBytes;
+    if (!tc_supported(v, r, M, bwd) && (bwd ? dec::bwd_supported(v, M) : dec::supported(v, M))) off = dec::clear_bytes(v, bwd);
+    *offset = off;
+    return LQLORA_OK;
+}
+
+int lqlora_lora_grads_from(const void* T_dev, const void* Tp_dev, int r, int64_t N, int64_t K, const void* X_dev,
+                           const void* dY_dev, int64_t M, float* dL1_dev, float* dL2_dev, void* workspace_dev,
+                           size_t workspace_bytes, void* stream) {
+    using namespace lq;
+    const int rc = check_lora_grads(N, K, r, M);
+    if (rc != LQLORA_OK) return rc;
+    if (!T_dev || !Tp_dev || !X_dev || !dY_dev || !dL1_dev || !dL2_dev || !workspace_dev) return LQLORA_ERR_NULL_POINTER;
+    if (!aligned16(T_dev) || !aligned16(Tp_dev) || !aligned16(X_dev) || !aligned16(dY_dev) || !aligned16(dL1_dev) ||
+        !aligned16(dL2_dev) || !aligned16(workspace_dev))
+        return LQLORA_ERR_MISALIGNED;
+    if (workspace_bytes < static_cast<size_t>(kStatusBytes)) return LQLORA_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(workspace_dev, 0, kStatusBytes, st) != cudaSuccess) return cuda_rc(cudaGetLastError());
+    return tc::launch_wgrad(dY_dev, X_dev, M, N, K, T_dev, Tp_dev, r, dL1_dev, dL2_dev, static_cast<int*>(workspace_dev), st);
+}
+
 int lqlora_lq_workspace_bytes(int64_t N, int64_t K, const lqlora_config* cfg, int r, int oversample, size_t* bytes) {
     using namespace lq;
     int rc = check_config(cfg);

@@ -44,6 +44,34 @@ def test_lora_grads_training_shape_and_repeatability():
     assert torch.equal(a1, dL1) and torch.equal(a2, dL2)
 
 
+@pytest.mark.parametrize("N,K,M,r,b0,B0", [(2304, 2560, 2100, 64, 3, 64), (512, 1024, 200, 64, 2, 16), (320, 768, 8, 32, 4, 32),
+                                           (384, 640, 1000, 128, 3, 32)])
+def test_lora_grads_from_the_intermediates_of_the_other_passes(N, K, M, r, b0, B0):
+    """The layer's three passes on the same X and dY: forward, input gradient, then lqlora_lora_grads_from with the
+    intermediates T, T' the first two left in their workspaces (CTA-pair kernel, one-CTA kernel, weight-streaming
+    kernel, rank padded to 128).  Same tolerance against the fp64 oracle as lqlora_lora_grads."""
+    from gpu_util import encode_both
+    cfg = inputs.QuantConfig(b0, B0, 8, 64, 32)
+    q, _ = encode_both(inputs.gaussian(5100 + N, (N, K), 0.02), cfg)
+    l1b, l2b = inputs.lowrank_factors(5101 + N, N, K, r, 0.05)
+    xb = inputs.activations(5102 + N, M, K)
+    gb = inputs.activations(5103 + N, M, N)
+    L1, L2 = binding.bf16_from_bits(l1b), binding.bf16_from_bits(l2b)
+    X, dY = binding.bf16_from_bits(xb), binding.bf16_from_bits(gb)
+    ws_f, ws_b = binding.alloc_workspace(q, r, M), binding.alloc_workspace(q, r, M)
+    binding.linear_fwd(q, L1, L2, X, workspace=ws_f)
+    binding.linear_bwd_input(q, L1, L2, dY, workspace=ws_b)
+    T = binding.linear_intermediate(ws_f, N, K, cfg, r, M, False)
+    Tp = binding.linear_intermediate(ws_b, N, K, cfg, r, M, True)
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    dL1, dL2 = binding.lora_grads_from(T, Tp, N, K, X, dY, workspace=ws)
+    torch.cuda.synchronize()
+    assert binding.workspace_status(ws) == 0
+    o1, o2 = oracle.lora_grads(l1b, l2b, xb, gb)
+    check_close(to_np(dL1), o1, f"dL1 from T N={N} K={K} M={M} r={r}")
+    check_close(to_np(dL2), o2, f"dL2 from T' N={N} K={K} M={M} r={r}")
+
+
 def test_lora_grads_one_hot_tokens():
     """One-hot X and dY rows pick single entries of the factors: exact in any arithmetic."""
     N, K, r, M = 256, 384, 64, 3
