@@ -650,7 +650,7 @@ def run_case(args):
     if args.case_cfg:
         import dataclasses
         spec = dataclasses.replace(spec, cfg=inputs.QuantConfig(*[int(x) for x in args.case_cfg.split(",")]))
-    M, r = args.case_m, inputs.RANK
+    M, r = args.case_m, (inputs.RANK if args.case_r is None else args.case_r)
     q = binding.alloc_qmatrix(spec.N, spec.K, spec.cfg, dev)
     g = torch.Generator(device=dev)
     g.manual_seed(1)
@@ -672,8 +672,10 @@ def run_case(args):
     q.codes.random_(0, 256, generator=g)
     q.scale_codes.random_(1, 128, generator=g)
     q.scale2.fill_(0.05)
-    l1b, l2b = inputs.lowrank_factors(spec.seed + 700, spec.N, spec.K, r, 0.01)
-    L1, L2 = binding.bf16_from_bits(l1b, dev), binding.bf16_from_bits(l2b, dev)
+    L1 = L2 = None
+    if r > 0:
+        l1b, l2b = inputs.lowrank_factors(spec.seed + 700, spec.N, spec.K, r, 0.01)
+        L1, L2 = binding.bf16_from_bits(l1b, dev), binding.bf16_from_bits(l2b, dev)
     X = binding.bf16_from_bits(inputs.activations(1, M, spec.K), dev)
     G = binding.bf16_from_bits(inputs.activations(2, M, spec.N), dev)
     ws = binding.alloc_workspace(q, r, M)
@@ -755,6 +757,7 @@ def main():
     ap.add_argument("--case-m", type=int, default=2048)
     ap.add_argument("--case-reps", type=int, default=3)
     ap.add_argument("--case-cfg", default=None, help="with --case: another configuration b0,B0,b1,B1,b2 for that matrix's shape")
+    ap.add_argument("--case-r", type=int, default=None, help="with --case: rank of the low-rank term (0 = none; default 64)")
     ap.add_argument("--case-encode", action="store_true", help="with --case: time lqlora_encode of that matrix instead of the linear calls")
     args = ap.parse_args()
     if args.sweep:

@@ -794,16 +794,28 @@ inline EncodeTiledFn encode_tiled_fn() {
 }
 
 // bf16 row-major [rows, cols] matrix, box of 64 columns x box_rows rows, 128-byte swizzle, zero fill.
+// A descriptor depends only on (pointer, rows, columns, box rows); a training step issues the same few over and over, so
+// the last ones built by this thread are kept (a call needs four to six of them).
 inline bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    struct Entry { const void* ptr; uint64_t rows, cols; uint32_t box_rows; bool valid; CUtensorMap map; };
+    constexpr int kEntries = 64;
+    thread_local Entry cache[kEntries] = {};
+    uint64_t h = reinterpret_cast<uintptr_t>(ptr) >> 4;
+    h = (h ^ (h >> 17)) * 0x9E3779B97F4A7C15ull + rows * 31u + cols * 131u + box_rows;
+    Entry& e = cache[(h >> 20) % kEntries];
+    if (e.valid && e.ptr == ptr && e.rows == rows && e.cols == cols && e.box_rows == box_rows) { *map = e.map; return true; }
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {cols * 2};
     const cuuint32_t box[2] = {64, box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    e.ptr = ptr; e.rows = rows; e.cols = cols; e.box_rows = box_rows; e.map = *map; e.valid = true;
+    return true;
 }
 
 template <int B, bool BWD, int MH>
